@@ -1,0 +1,370 @@
+#!/usr/bin/env python
+"""Benchmark of the SPMM / SDDMM / FusedMM hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl b200|reference]
+
+One *step* = one pass of the whole hot path over one synthetic problem: SPMM, SDDMM and FusedMM
+once each on the same CSR pattern (row extents, work assignment, index staging, sampled dot
+products, their store, the gather-AXPY sweep, the output store and the fused pass).
+Metric: GFLOP/s with 2*nnz*width flop per stage (FusedMM = its two stages), whole job.
+
+Default workload `sweep_d30_n128`: S 8192 x 8192, power-law row lengths at 30% mean density,
+Kd = N = 128 -- the size, width and density of the paper's headline case (8k/8k/128/70%).
+
+Prints ONE JSON line (rank 0).  `value` has all inputs resident in HBM; `e2e` goes through the
+host-buffer C-ABI entry points with the copies inside the timed region.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2311_00368_b200 import replicas  # noqa: E402
+from paper_2311_00368_b200 import workloads as W  # noqa: E402
+
+OPS = ("spmm", "sddmm", "fusedmm")
+SM_COUNT, FP32_LANES_PER_SM = 148, 128
+L2_FLUSH_BYTES = 256 << 20
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel,
+# from the ncu captures summarised under profiles/; None where no capture exists yet.
+MEASURED_TRAFFIC_BYTES = {}
+
+
+def make_workload(name: str, rank: int = 0) -> W.Problem:
+    if name.startswith("sweep_d"):
+        d, n = name[len("sweep_d"):].split("_n")
+        return W.sweep_case(int(d) / 100.0, int(n), seed=replicas.instance_seed(4, rank))
+    if name == "tiny":
+        return W.tiny(replicas.instance_seed(0, rank))
+    if name == "spmm":
+        p = W.spmm_case(replicas.instance_seed(1, rank))
+        rng = np.random.default_rng(99)
+        p.Kd, p.A, p.B = 128, W.dense_normal(rng, p.M, 128), W.dense_normal(rng, p.K, 128)
+        return p
+    if name == "sddmm":
+        p = W.sddmm_case(replicas.instance_seed(2, rank))
+        rng = np.random.default_rng(99)
+        p.N, p.D = 128, W.dense_normal(rng, p.K, 128)
+        return p
+    if name.startswith("attn"):
+        return W.attention_case(int(name[4:] or 0) + 8 * rank)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        m = json.load(open(path))
+        return float(m["hbm_gbs"]), float(m.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid):
+        self.rows, self.proc, self.uuid = [], None, uuid
+
+    def start(self):
+        try:
+            cmd = ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"]
+            if self.uuid:
+                cmd += ["-i", self.uuid]
+            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.t.join(timeout=2)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for r in self.rows:
+            if len(r) < 7:
+                continue
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def oracle_sample(p: W.Problem, budget_s: float):
+    """Times the CPU oracle (as it stands) on a bounded sample of the workload: the first R rows of
+    S for all three ops, R sized from a short calibration so the sample costs about budget_s."""
+    import oracle
+    M = p.M
+
+    def run(r1):
+        t0 = time.perf_counter()
+        oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D, rows=(0, r1))
+        oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, rows=(0, r1))
+        oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D, rows=(0, r1))
+        return time.perf_counter() - t0
+
+    r_cal = min(M, max(oracle.num_threads() * 16, 64))
+    run(min(M, 8))  # load the library, touch the pages
+    t_cal = run(r_cal)
+    nnz_cal = int(p.row_ptr[r_cal])
+    if r_cal >= M or t_cal >= budget_s:
+        rows, t, nnz_s = r_cal, t_cal, nnz_cal
+    else:
+        want_nnz = nnz_cal * budget_s / max(t_cal, 1e-6)
+        rows = int(np.searchsorted(p.row_ptr, min(want_nnz, p.nnz), side="left"))
+        rows = max(r_cal, min(M, rows))
+        t = run(rows)
+        nnz_s = int(p.row_ptr[rows])
+    fl = sum(W.flops(op, nnz_s, p.Kd, p.N) for op in OPS)
+    return {"value": fl / t / 1e9, "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"rows 0..{rows} of {M} ({nnz_s} of {p.nnz} nonzeros), spmm+sddmm+fusedmm once, "
+                      f"{t:.1f} s"}, t
+
+
+def run_reference(args):
+    rank, _, world = replicas.env_world()
+    if rank != 0:
+        return 0
+    p = make_workload(args.workload)
+    total = args.steps + args.warmup
+    budget = min(20.0, 150.0 / max(total, 1))
+    vals, secs = [], []
+    for s in range(total):
+        cb, t = oracle_sample(p, budget)
+        if s >= args.warmup:
+            vals.append(cb["value"]); secs.append(t)
+    v = float(np.mean(vals))
+    cb["value"] = v
+    line = {"impl": "reference", "metric": "SPMM+SDDMM+FusedMM GFLOP/s (2*nnz*width per stage)",
+            "value": v, "unit": "GFLOP/s", "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": float(np.mean(secs)) * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(p, args.workload),
+            "cpu_baseline": cb,
+            "e2e": {"value": v, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+    return 0
+
+
+def workload_config(p, name):
+    lens = np.diff(p.row_ptr)
+    return {"workload": name, "M": p.M, "K": p.K, "Kd": p.Kd, "N": p.N, "nnz": p.nnz,
+            "density": round(p.nnz / (p.M * p.K), 4),
+            "row_len_min_med_max": [int(lens.min()), int(np.median(lens)), int(lens.max())],
+            "step": "spmm + sddmm + fusedmm, once each",
+            "l2": "flushed between steps (256 MiB write, untimed)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="sweep_d30_n128")
+    ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
+    ap.add_argument("--algo", type=int, default=0, help="B2SP_ALGO_* (0 = auto)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--min-warmup", type=int, default=3,
+                    help="lower bound on warm-up steps (only profiler captures go below 3)")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    from paper_2311_00368_b200 import binding as b  # raises if libb2sp.so is missing
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    rank, local_rank, world = replicas.env_world()
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    replicas.init("nccl", device)
+    hbm_gbs, sm_max_mhz, peak_src = peaks()
+    fp32_peak_gflops = SM_COUNT * FP32_LANES_PER_SM * 2 * sm_max_mhz / 1e3
+
+    p = make_workload(args.workload, rank)
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(device)
+    rp, ci, v, A, B, D = map(dev, (p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D))
+    O = torch.empty((p.M, p.N), dtype=torch.float32, device=device)
+    O2 = torch.empty_like(O)
+    C = torch.empty(p.nnz, dtype=torch.float32, device=device)
+    ws_bytes = max(b.workspace_bytes(op, p.M, p.K, p.Kd, p.N, p.nnz) for op in range(3))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream()
+
+    calls = {
+        "spmm": lambda: b.spmm(rp, ci, v, D, K=p.K, out=O2, workspace=ws, algo=args.algo),
+        "sddmm": lambda: b.sddmm(rp, ci, v, A, B, out=C, workspace=ws, algo=args.algo),
+        "fusedmm": lambda: b.fusedmm(rp, ci, v, A, B, D, out=O, workspace=ws, algo=args.algo),
+    }
+    fl = {op: W.flops(op, p.nnz, p.Kd, p.N) for op in OPS}
+    by = {op: W.compulsory_bytes(op, p.M, p.K, p.nnz, p.Kd, p.N) for op in OPS}
+
+    def step(events=None):
+        for op in OPS:
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            calls[op]()
+            if events is not None:
+                e1.record(stream)
+                events.append((op, e0, e1))
+
+    for _ in range(max(args.warmup, args.min_warmup)):
+        flush.fill_(1)
+        step()
+    torch.cuda.synchronize()
+    launches = {op: b.last_launches(i) for i, op in enumerate(OPS)}
+    algos = {op: b.ALGO_NAMES[b.last_algo(i)] for i, op in enumerate(OPS)}
+
+    sampler = ClockSampler(str(torch.cuda.get_device_properties(device).uuid) if rank == 0 else None)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    if rank == 0:
+        sampler.start()
+    events, step_events = [], []
+    for _ in range(args.steps):
+        flush.fill_(1)  # evict the operands from L2 (untimed)
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        step(events)
+        s1.record(stream)
+        step_events.append((s0, s1))
+    torch.cuda.synchronize()
+    replicas.barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    step_ms = [a.elapsed_time(z) for a, z in step_events]
+    total_ms_local = float(np.sum(step_ms))
+    total_ms = replicas.max_over_ranks(total_ms_local, device)
+    flops_all = replicas.sum_over_ranks(float(sum(fl.values())), device)
+    ms_per_step = total_ms / args.steps
+    value = flops_all / (ms_per_step * 1e-3) / 1e9
+
+    per_op = {}
+    for op in OPS:
+        ms = [a.elapsed_time(z) for (o, a, z) in events if o == op]
+        mean_ms, min_ms = float(np.mean(ms)), float(np.min(ms))
+        t_alu = fl[op] / (fp32_peak_gflops * 1e9)
+        t_hbm = by[op] / (hbm_gbs * 1e9)
+        per_op[op] = {"ms": round(mean_ms, 4), "ms_min": round(min_ms, 4),
+                      "gflops": round(fl[op] / mean_ms / 1e6, 1),
+                      "gflops_at_min": round(fl[op] / min_ms / 1e6, 1),
+                      "compulsory_gbs": round(by[op] / mean_ms / 1e6, 1),
+                      "roofline_bound": "alu" if t_alu >= t_hbm else "hbm",
+                      "roofline_frac": round(max(t_alu, t_hbm) / (mean_ms * 1e-3), 4),
+                      "launches": launches[op], "algo": algos[op]}
+    sep_ms = per_op["sddmm"]["ms"] + per_op["spmm"]["ms"]
+    fused_vs_separate = sep_ms / per_op["fusedmm"]["ms"]
+
+    # roofline object for the dominant kernel (FusedMM): FP32-FMA bound on this workload
+    dom = "fusedmm"
+    dom_ms = per_op[dom]["ms"]
+    t_alu = fl[dom] / (fp32_peak_gflops * 1e9)
+    t_hbm = by[dom] / (hbm_gbs * 1e9)
+    if t_alu >= t_hbm:
+        roof = {"bound": "alu", "achieved": fl[dom] / dom_ms / 1e9, "peak": fp32_peak_gflops / 1e3,
+                "unit": "TFLOP/s"}
+        roof["peak_source"] = (f"{SM_COUNT} SMs x {FP32_LANES_PER_SM} FP32 lanes x 2 flop x "
+                               f"{sm_max_mhz:.0f} MHz (clocks.max.sm, {peak_src})")
+    else:
+        roof = {"bound": "hbm", "achieved": by[dom] / dom_ms / 1e6, "peak": hbm_gbs, "unit": "GB/s",
+                "peak_source": f"hbm_gbs of {peak_src}"}
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["kernel"] = dom
+    roof["traffic"] = MEASURED_TRAFFIC_BYTES.get(args.workload)
+    roof["algorithmic_bytes"] = by[dom]
+    roof["algorithmic_flops"] = fl[dom]
+
+    # end to end: host buffers through the C ABI, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        pin = lambda x: torch.from_numpy(np.ascontiguousarray(x)).pin_memory()
+        h = {k: pin(x) for k, x in (("rp", p.row_ptr), ("ci", p.col_idx), ("v", p.values), ("A", p.A),
+                                    ("B", p.B), ("D", p.D))}
+        hO = torch.empty((p.M, p.N), dtype=torch.float32).pin_memory()
+        hC = torch.empty(p.nnz, dtype=torch.float32).pin_memory()
+        nb = lambda *ts: int(sum(t.numel() * t.element_size() for t in ts))
+        h2d = (nb(h["rp"], h["ci"], h["v"], h["D"]) + nb(h["rp"], h["ci"], h["v"], h["A"], h["B"]) +
+               nb(h["rp"], h["ci"], h["v"], h["A"], h["B"], h["D"]))
+        d2h = nb(hO) + nb(hC) + nb(hO)
+
+        def host_step():
+            b.spmm_host(h["rp"], h["ci"], h["v"], h["D"], hO)
+            b.sddmm_host(h["rp"], h["ci"], h["v"], h["A"], h["B"], hC)
+            b.fusedmm_host(h["rp"], h["ci"], h["v"], h["A"], h["B"], h["D"], hO)
+
+        e2e_steps = max(3, min(args.steps, 10))
+        for _ in range(2):
+            host_step()
+        replicas.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            host_step()  # each call synchronises its stream before returning
+        torch.cuda.synchronize()
+        t_local = (time.perf_counter() - t0) / e2e_steps
+        t_e2e = replicas.max_over_ranks(t_local, device)
+        e2e = {"value": flops_all / t_e2e / 1e9, "unit": "GFLOP/s", "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": e2e_steps,
+               "timer": "host wall clock around synchronous C-ABI calls"}
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline, _ = oracle_sample(p, 15.0)
+
+    if rank == 0:
+        line = {"metric": "SPMM+SDDMM+FusedMM GFLOP/s (2*nnz*width per stage)", "value": value,
+                "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, args.min_warmup),
+                "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": workload_config(p, args.workload), "roofline": roof, "cpu_baseline": cpu_baseline,
+                "e2e": e2e, "gpu_launches": int(sum(launches.values()) * args.steps),
+                "clocks": clocks, "ops": per_op,
+                "fused_speedup_over_separate_launches": round(fused_vs_separate, 3),
+                "paper_context": "Intel Max 1550 (1 stack), 8k/8k/128/70%: SDDMM 9732, SPMM 11482, "
+                                 "FusedMM 12647 GFLOP/s (other hardware; context only)"}
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,161 @@
+/*
+ * b2sp -- SPMM, SDDMM and FusedMM over a CSR sparsity pattern S on NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only; `stream` is a cudaStream_t passed as void*
+ * (NULL = the legacy default stream).
+ *
+ * Storage (paper, section "Matrix Storage Layout", Fig. 1):
+ *   S  is M x K in compressed sparse row form: row_ptr[M+1], col_idx[nnz], values[nnz];
+ *      int32, 0-based; row i owns positions row_ptr[i] <= p < row_ptr[i+1].  Any valid CSR is
+ *      accepted: rows may be empty, and the column indices of a row need be neither sorted
+ *      nor unique (each stored entry is its own term and its own SDDMM output slot).
+ *   Dense operands are fp32, row-major, with a leading dimension counted in elements
+ *      (ld >= number of columns).
+ *   Names: the paper's (A, I_A; C; B; D; E) are here (S; A; B; D; O); its single letter N is
+ *      split into Kd (length of the sampled dot product) and N (width of D and O).
+ *
+ * Conventions for the device entry points (b2sp_spmm, b2sp_sddmm, b2sp_fusedmm):
+ *   - every data pointer is a DEVICE pointer on the current device; the caller owns all of
+ *     them, including the workspace; the library allocates nothing;
+ *   - inputs are read-only; outputs are fully overwritten (never accumulated into; an empty
+ *     row gives a zero output row, Alg. 2 line 1);
+ *   - the call enqueues kernels on `stream` and returns without synchronising;
+ *   - `workspace` is scratch of at least b2sp_workspace_bytes(...) bytes, 256-byte aligned;
+ *     its contents are overwritten by every call, so two calls that may overlap in time on
+ *     the GPU (different streams) need different workspaces;
+ *   - argument errors are reported synchronously with no kernel launched; a launch failure
+ *     is reported as B2SP_ERR_CUDA; nothing traps, asserts or exits.
+ *   - M = 0, nnz = 0 and zero widths are valid (outputs of the stated size are zero-filled).
+ *
+ * `algo` selects the kernel family:
+ *   B2SP_ALGO_AUTO     the library chooses (fastest family whose preconditions hold);
+ *   B2SP_ALGO_ROW      CUDA-core row kernels, rows taken longest-first (binned by length);
+ *   B2SP_ALGO_ROW_NAT  the same kernels, rows in natural order (no binning pass);
+ *   B2SP_ALGO_TILE     dense-tile tensor-core kernels (tcgen05, 3xTF32 split).  They need
+ *                      column indices sorted within each row; if an explicit request cannot be
+ *                      met the call returns B2SP_ERR_UNSUPPORTED.
+ * Floating-point results of the families differ in summation order only; all stay within
+ * |x - exact| <= 1e-5 * sum|terms| + 1e-6.
+ */
+#ifndef B2SP_H
+#define B2SP_H
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    B2SP_OK = 0,
+    B2SP_ERR_INVALID_ARG = 1, /* negative size, NULL required pointer, ld < width, nnz > 2^31-1 */
+    B2SP_ERR_UNSUPPORTED = 2, /* explicit algo whose preconditions do not hold */
+    B2SP_ERR_BAD_CSR = 3,     /* b2sp_validate_csr: row_ptr not monotone / col_idx out of range */
+    B2SP_ERR_CUDA = 4,        /* a CUDA runtime call or a kernel launch failed */
+    B2SP_ERR_WORKSPACE = 5,   /* workspace NULL, misaligned or too small */
+    B2SP_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by b2sp_device_status) */
+} b2sp_status;
+
+enum { B2SP_ALGO_AUTO = 0, B2SP_ALGO_ROW = 1, B2SP_ALGO_ROW_NAT = 2, B2SP_ALGO_TILE = 3 };
+enum { B2SP_OP_SPMM = 0, B2SP_OP_SDDMM = 1, B2SP_OP_FUSEDMM = 2 };
+
+/* Library version (major*10000 + minor*100 + patch). */
+int b2sp_version(void);
+
+/* Static, human-readable name of a status code. */
+const char *b2sp_status_string(b2sp_status s);
+
+/*
+ * Bytes of device workspace an op needs for the given sizes (an upper bound over all algo
+ * values; always a multiple of 256, never 0).  `op` is one of B2SP_OP_*.  Unused sizes
+ * (Kd for SPMM, N for SDDMM) may be 0.  Returns 0 on invalid arguments.
+ */
+size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz);
+
+/*
+ * SPMM, Eq. 2 / Alg. 2 (SPMM-ROW):  O[i, :] = sum over stored entries (s, k) of row i of
+ * s * D[k, :].
+ *   M, K, N     S is M x K, D is K x N, O is M x N
+ *   nnz         number of stored entries (= row_ptr[M])
+ *   row_ptr, col_idx, values   CSR of S (device, read-only)
+ *   D, ldd      dense K x N (device, read-only), leading dimension >= N
+ *   O, ldo      dense M x N (device, written), leading dimension >= N; must not alias an input
+ */
+b2sp_status b2sp_spmm(int M, int K, int N, long long nnz,
+                      const int *row_ptr, const int *col_idx, const float *values,
+                      const float *D, long long ldd, float *O, long long ldo,
+                      void *workspace, size_t workspace_bytes, int algo, void *stream);
+
+/*
+ * SDDMM, Eq. 1 / Alg. 1 (SDDMM-ROW), with the sampled value scaled by the stored one:
+ *   out_values[p] = s_p * sum_{l < Kd} A[i, l] * B[j, l]   for the p-th stored entry (i, j).
+ * The paper samples with an all-ones pattern; pass s_values = NULL for that (s_p = 1).
+ * The result's sparsity pattern is S's: row_ptr and col_idx are not modified and out_values
+ * follows the order of col_idx.
+ *   A, lda      dense M x Kd (device, read-only);  B, ldb  dense K x Kd (device, read-only)
+ *   out_values  nnz floats (device, written); may be the same pointer as s_values
+ *               (in-place, as the paper overwrites its avalues array)
+ */
+b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz,
+                       const int *row_ptr, const int *col_idx, const float *s_values,
+                       const float *A, long long lda, const float *B, long long ldb,
+                       float *out_values,
+                       void *workspace, size_t workspace_bytes, int algo, void *stream);
+
+/*
+ * FusedMM, Eq. 3 / Alg. 3 (FusedMM-ROW):  O = (S .* (A * B^T)) * D, i.e. the SDDMM values of a
+ * row are consumed by the SPMM sweep of the same row without ever being written to global
+ * memory.  s_values may be NULL (all ones).  Arguments as in the two ops above.
+ */
+b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz,
+                         const int *row_ptr, const int *col_idx, const float *s_values,
+                         const float *A, long long lda, const float *B, long long ldb,
+                         const float *D, long long ldd, float *O, long long ldo,
+                         void *workspace, size_t workspace_bytes, int algo, void *stream);
+
+/*
+ * Host-buffer forms of the three ops: every data pointer is a HOST pointer (pinned memory
+ * makes the copies asynchronous and faster, pageable memory also works).  Each call copies
+ * its inputs to the device, runs the device entry point above with algo = B2SP_ALGO_AUTO,
+ * copies the result back and synchronises `stream` before returning.  Device memory comes
+ * from the stream-ordered CUDA memory pool (cudaMallocAsync) and is returned to it before the
+ * call ends.  Dense operands are contiguous (ld = number of columns).
+ */
+b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz,
+                           const int *row_ptr, const int *col_idx, const float *values,
+                           const float *D, float *O, void *stream);
+b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz,
+                            const int *row_ptr, const int *col_idx, const float *s_values,
+                            const float *A, const float *B, float *out_values, void *stream);
+b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz,
+                              const int *row_ptr, const int *col_idx, const float *s_values,
+                              const float *A, const float *B, const float *D, float *O,
+                              void *stream);
+
+/*
+ * Debug helper: checks on the device that row_ptr[0] = 0, row_ptr is non-decreasing,
+ * row_ptr[M] = nnz and 0 <= col_idx[p] < K.  Synchronises `stream`.  `workspace` needs 256
+ * bytes.  Returns B2SP_OK or B2SP_ERR_BAD_CSR.
+ */
+b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Reads back (synchronising `stream`) the status word device code left in `workspace` during
+ * the most recent op that used it: B2SP_OK, or B2SP_ERR_TIMEOUT if a bounded wait inside a
+ * kernel gave up (the outputs of that call are then undefined).
+ */
+b2sp_status b2sp_device_status(const void *workspace, void *stream);
+
+/*
+ * Which kernel family the most recent call of the given op on this host thread resolved
+ * B2SP_ALGO_AUTO (or its explicit request) to: one of B2SP_ALGO_ROW, _ROW_NAT, _TILE; -1 if the
+ * op has not been called.  Number of kernels that call enqueued: b2sp_last_launches(op).
+ */
+int b2sp_last_algo(int op);
+int b2sp_last_launches(int op);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B2SP_H */

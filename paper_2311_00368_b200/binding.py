@@ -1,0 +1,232 @@
+"""Thin Python binding over the C-ABI library ``libb2sp.so``: argument marshalling only.
+
+Every step of the three ops runs inside the CUDA library; this module turns torch tensors
+into raw device pointers + sizes, supplies a workspace and the current CUDA stream, and
+raises on a non-zero status.  There is no CPU fallback: importing this module raises
+``ImportError`` if the library has not been built, and calling an op without a CUDA device
+fails in the library.
+
+Function names and argument order follow ``include/b2sp.h``.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libb2sp.so")
+
+ALGO_AUTO, ALGO_ROW, ALGO_ROW_NAT, ALGO_TILE = 0, 1, 2, 3
+OP_SPMM, OP_SDDMM, OP_FUSEDMM = 0, 1, 2
+ALGO_NAMES = {0: "auto", 1: "row", 2: "row_nat", 3: "tile", -1: "none"}
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2311_00368_b200.build` "
+        "(there is no fallback implementation)")
+
+lib = ctypes.CDLL(LIB_PATH)
+
+_i, _ll, _vp, _sz = ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_size_t
+
+lib.b2sp_version.restype = _i
+lib.b2sp_status_string.restype = ctypes.c_char_p
+lib.b2sp_status_string.argtypes = [_i]
+lib.b2sp_workspace_bytes.restype = _sz
+lib.b2sp_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _ll]
+lib.b2sp_spmm.restype = _i
+lib.b2sp_spmm.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp, _sz, _i, _vp]
+lib.b2sp_sddmm.restype = _i
+lib.b2sp_sddmm.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp, _vp, _sz, _i, _vp]
+lib.b2sp_fusedmm.restype = _i
+lib.b2sp_fusedmm.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp, _ll, _vp, _ll,
+                             _vp, _sz, _i, _vp]
+lib.b2sp_spmm_host.restype = _i
+lib.b2sp_spmm_host.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.b2sp_sddmm_host.restype = _i
+lib.b2sp_sddmm_host.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.b2sp_fusedmm_host.restype = _i
+lib.b2sp_fusedmm_host.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.b2sp_validate_csr.restype = _i
+lib.b2sp_validate_csr.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
+lib.b2sp_device_status.restype = _i
+lib.b2sp_device_status.argtypes = [_vp, _vp]
+lib.b2sp_last_algo.restype = _i
+lib.b2sp_last_algo.argtypes = [_i]
+lib.b2sp_last_launches.restype = _i
+lib.b2sp_last_launches.argtypes = [_i]
+
+
+class B2spError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {lib.b2sp_status_string(status).decode()} (status {status})")
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise B2spError(status, where)
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ld(t):
+    assert t.dim() == 2 and (t.shape[1] <= 1 or t.stride(1) == 1), "dense operands are row-major"
+    return t.stride(0) if t.shape[0] > 1 else max(t.shape[1], t.stride(0))
+
+
+def _want(t, dtype, name, cuda=True):
+    if t is None:
+        return
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}")
+    if cuda and not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor")
+
+
+def version() -> int:
+    return int(lib.b2sp_version())
+
+
+def workspace_bytes(op: int, M: int, K: int, Kd: int, N: int, nnz: int) -> int:
+    return int(lib.b2sp_workspace_bytes(op, M, K, Kd, N, nnz))
+
+
+_ws_cache = {}
+
+
+def _workspace(op, M, K, Kd, N, nnz, device, workspace):
+    need = workspace_bytes(op, M, K, Kd, N, nnz)
+    if workspace is None:
+        key = (device.index, torch.cuda.current_stream(device).cuda_stream)
+        workspace = _ws_cache.get(key)
+        if workspace is None or workspace.numel() < need:
+            workspace = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=device)
+            _ws_cache[key] = workspace
+    return workspace, workspace.numel()
+
+
+def last_algo(op: int) -> int:
+    return int(lib.b2sp_last_algo(op))
+
+
+def last_launches(op: int) -> int:
+    return int(lib.b2sp_last_launches(op))
+
+
+def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALGO_AUTO):
+    """b2sp_spmm: O = S @ D.  CSR tensors int32/fp32 on the GPU; D [K, N] fp32 row-major."""
+    _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
+    _want(values, torch.float32, "values"); _want(D, torch.float32, "D")
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K = D.shape[0] if K is None else K
+    N = D.shape[1]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=D.device)
+    ws, wsb = _workspace(OP_SPMM, M, K, 0, N, nnz, D.device, workspace)
+    _check(lib.b2sp_spmm(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D), _ld(D),
+                         _ptr(out), _ld(out), _ptr(ws), wsb, algo, _stream()), "b2sp_spmm")
+    return out
+
+
+def sddmm(row_ptr, col_idx, s_values, A, B, out=None, workspace=None, algo=ALGO_AUTO):
+    """b2sp_sddmm: out[p] = s_p * <A[i], B[j]> on S's pattern; s_values=None means all ones."""
+    _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
+    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K, Kd = B.shape
+    if A.shape != (M, Kd):
+        raise ValueError("A must be [M, Kd]")
+    if out is None:
+        out = torch.empty(nnz, dtype=torch.float32, device=A.device)
+    ws, wsb = _workspace(OP_SDDMM, M, K, Kd, 0, nnz, A.device, workspace)
+    _check(lib.b2sp_sddmm(M, K, Kd, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A), _ld(A),
+                          _ptr(B), _ld(B), _ptr(out), _ptr(ws), wsb, algo, _stream()), "b2sp_sddmm")
+    return out
+
+
+def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO):
+    """b2sp_fusedmm: O = (S .* (A @ B.T)) @ D in one pass; the sampled values never reach HBM."""
+    _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
+    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
+    _want(D, torch.float32, "D")
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K, Kd = B.shape
+    N = D.shape[1]
+    if A.shape != (M, Kd) or D.shape[0] != K:
+        raise ValueError("A must be [M, Kd] and D [K, N]")
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=D.device)
+    ws, wsb = _workspace(OP_FUSEDMM, M, K, Kd, N, nnz, D.device, workspace)
+    _check(lib.b2sp_fusedmm(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
+                            _ld(A), _ptr(B), _ld(B), _ptr(D), _ld(D), _ptr(out), _ld(out), _ptr(ws), wsb,
+                            algo, _stream()), "b2sp_fusedmm")
+    return out
+
+
+def _host(t, dtype, name):
+    if t is None:
+        return None
+    if t.is_cuda or t.dtype != dtype or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous CPU tensor of {dtype}")
+    return t
+
+
+def spmm_host(row_ptr, col_idx, values, D, out):
+    """b2sp_spmm_host: host tensors in, host tensor out (copies happen inside the library)."""
+    for t, dt, n in ((row_ptr, torch.int32, "row_ptr"), (col_idx, torch.int32, "col_idx"),
+                     (values, torch.float32, "values"), (D, torch.float32, "D"), (out, torch.float32, "out")):
+        _host(t, dt, n)
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K, N = D.shape
+    _check(lib.b2sp_spmm_host(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D),
+                              _ptr(out), _stream()), "b2sp_spmm_host")
+    return out
+
+
+def sddmm_host(row_ptr, col_idx, s_values, A, B, out):
+    for t, dt, n in ((row_ptr, torch.int32, "row_ptr"), (col_idx, torch.int32, "col_idx"),
+                     (s_values, torch.float32, "s_values"), (A, torch.float32, "A"),
+                     (B, torch.float32, "B"), (out, torch.float32, "out")):
+        _host(t, dt, n)
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K, Kd = B.shape
+    _check(lib.b2sp_sddmm_host(M, K, Kd, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
+                               _ptr(B), _ptr(out), _stream()), "b2sp_sddmm_host")
+    return out
+
+
+def fusedmm_host(row_ptr, col_idx, s_values, A, B, D, out):
+    for t, dt, n in ((row_ptr, torch.int32, "row_ptr"), (col_idx, torch.int32, "col_idx"),
+                     (s_values, torch.float32, "s_values"), (A, torch.float32, "A"),
+                     (B, torch.float32, "B"), (D, torch.float32, "D"), (out, torch.float32, "out")):
+        _host(t, dt, n)
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K, Kd = B.shape
+    N = D.shape[1]
+    _check(lib.b2sp_fusedmm_host(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values),
+                                 _ptr(A), _ptr(B), _ptr(D), _ptr(out), _stream()), "b2sp_fusedmm_host")
+    return out
+
+
+def validate_csr(row_ptr, col_idx, K) -> bool:
+    """b2sp_validate_csr: True if the CSR arrays are well formed (synchronises)."""
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    ws = torch.empty(256, dtype=torch.uint8, device=row_ptr.device)
+    st = lib.b2sp_validate_csr(M, K, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(ws), 256, _stream())
+    if st == 3:
+        return False
+    _check(st, "b2sp_validate_csr")
+    return True
+
+
+def device_status(workspace) -> int:
+    return int(lib.b2sp_device_status(_ptr(workspace), _stream()))

@@ -1,0 +1,492 @@
+// C-ABI entry points of libb2sp: argument checks, workspace carving, kernel dispatch.
+// See include/b2sp.h for the contract of every function.
+#include "../../include/b2sp.h"
+
+#include <climits>
+#include <cstdint>
+
+#include "row_kernels.cuh"
+
+namespace b2sp {
+
+// ---- workspace layout ---------------------------------------------------------------------
+// [0, 128)    int count[32]      row-length histogram            (zeroed per call)
+// [128, 256)  int cursor[32]     scatter cursors                 (zeroed per call)
+// [256, 512)  int status[64]     status[0] = device status word, status[1] = validate flag
+// [512, ...)  int row_order[M]   rows, longest bucket first
+constexpr size_t kHeaderBytes = 512;
+
+inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+
+struct Workspace {
+    int *count, *cursor, *status, *row_order;
+};
+
+inline Workspace carve(void *ws)
+{
+    char *b = static_cast<char *>(ws);
+    Workspace w;
+    w.count = reinterpret_cast<int *>(b);
+    w.cursor = reinterpret_cast<int *>(b + 128);
+    w.status = reinterpret_cast<int *>(b + 256);
+    w.row_order = reinterpret_cast<int *>(b + kHeaderBytes);
+    return w;
+}
+
+thread_local int g_last_algo[3] = {-1, -1, -1};
+thread_local int g_last_launches[3] = {0, 0, 0};
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+inline b2sp_status check_launch()
+{
+    return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
+}
+
+b2sp_status check_workspace(void *ws, size_t have, size_t need)
+{
+    if (!ws || (reinterpret_cast<uintptr_t>(ws) & 255) != 0 || have < need) return B2SP_ERR_WORKSPACE;
+    return B2SP_OK;
+}
+
+// Enqueue the binning pass; returns the row order pointer (NULL for natural order).
+b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t st, int *launches)
+{
+    if (cudaMemsetAsync(w.count, 0, 512, st) != cudaSuccess) return B2SP_ERR_CUDA;
+    int blocks = (M + 255) / 256;
+    bin_count_kernel<<<blocks, 256, 0, st>>>(M, row_ptr, w.count);
+    bin_scatter_kernel<<<blocks, 256, 0, st>>>(M, row_ptr, w.count, w.cursor, w.row_order);
+    *launches += 2;
+    return check_launch();
+}
+
+template <int U, int SPLIT>
+void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
+                 const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
+                 const int *order)
+{
+    spmm_row_kernel<U, SPLIT><<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
+                                                           ldo, order);
+}
+
+// Column geometry for a width N on the float4 path: U float4 per lane, SPLIT sub-warps.
+struct Geom { int U, SPLIT, slab; };
+inline Geom pick_geom(int N)
+{
+    if (N <= 32) return {1, 4, 32};
+    if (N <= 64) return {1, 2, 64};
+    if (N <= 128) return {1, 1, 128};
+    if (N <= 256) return {2, 1, 256};
+    return {4, 1, 512};
+}
+
+inline int pick_ku(int Kd) { return Kd <= 64 ? 2 : Kd <= 128 ? 4 : Kd <= 256 ? 8 : 0; }
+
+template <int KU>
+void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const int *col_idx,
+                  const float *sv, const float *A, int64_t lda, const float *B, int64_t ldb,
+                  float *out, const int *order)
+{
+    size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
+    sddmm_row_kernel<KU><<<grid, kRowThreads, smem, st>>>(Kd, row_ptr, col_idx, sv, A, lda, B, ldb,
+                                                         out, order);
+}
+
+template <int KU, int U, int SPLIT>
+b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
+                         const int *col_idx, const float *sv, const float *A, int64_t lda,
+                         const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
+                         int64_t ldo, const int *order)
+{
+    size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
+                  (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
+    auto kern = fusedmm_row_kernel<KU, U, SPLIT>;
+    if (smem > 48 * 1024) {
+        if (smem > 200 * 1024) return B2SP_ERR_UNSUPPORTED;
+        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+            cudaSuccess)
+            return B2SP_ERR_CUDA;
+    }
+    kern<<<grid, kRowThreads, smem, st>>>(Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
+                                          order);
+    return B2SP_OK;
+}
+
+template <int KU>
+b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int Kd, int N,
+                                const int *row_ptr, const int *col_idx, const float *sv,
+                                const float *A, int64_t lda, const float *B, int64_t ldb,
+                                const float *D, int64_t ldd, float *O, int64_t ldo,
+                                const int *order)
+{
+#define B2SP_F(U_, S_) \
+    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order)
+    if (g.SPLIT == 4) B2SP_F(1, 4);
+    if (g.SPLIT == 2) B2SP_F(1, 2);
+    if (g.U == 1) B2SP_F(1, 1);
+    if (g.U == 2) B2SP_F(2, 1);
+    B2SP_F(4, 1);
+#undef B2SP_F
+}
+
+b2sp_status zero_rows(float *O, int64_t ldo, int M, int N, cudaStream_t st)
+{
+    if (M == 0 || N == 0) return B2SP_OK;
+    return cudaMemset2DAsync(O, sizeof(float) * (size_t)ldo, 0, sizeof(float) * (size_t)N, (size_t)M,
+                             st) == cudaSuccess
+               ? B2SP_OK
+               : B2SP_ERR_CUDA;
+}
+
+bool bad_csr_args(int M, int K, long long nnz, const int *row_ptr, const int *col_idx)
+{
+    if (M < 0 || K < 0 || nnz < 0 || nnz > (long long)INT_MAX) return true;
+    if (M > 0 && !row_ptr) return true;
+    if (nnz > 0 && (!col_idx || K == 0 || M == 0)) return true;
+    return false;
+}
+
+int resolve_algo(int algo)
+{
+    // The dense-tile family is not built into this translation unit yet.
+    if (algo == B2SP_ALGO_AUTO) return B2SP_ALGO_ROW;
+    return algo;
+}
+
+}  // namespace b2sp
+
+using namespace b2sp;
+
+extern "C" {
+
+int b2sp_version(void) { return 100; }
+
+const char *b2sp_status_string(b2sp_status s)
+{
+    switch (s) {
+    case B2SP_OK: return "ok";
+    case B2SP_ERR_INVALID_ARG: return "invalid argument";
+    case B2SP_ERR_UNSUPPORTED: return "unsupported for these arguments";
+    case B2SP_ERR_BAD_CSR: return "malformed CSR";
+    case B2SP_ERR_CUDA: return "CUDA error";
+    case B2SP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case B2SP_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
+{
+    if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
+    return align256(kHeaderBytes + sizeof(int) * (size_t)M);
+}
+
+int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
+int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
+
+b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
+                      const float *values, const float *D, long long ldd, float *O, long long ldo,
+                      void *workspace, size_t workspace_bytes, int algo, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || N < 0) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && N > 0 && (!values || !D || ldd < N)) return B2SP_ERR_INVALID_ARG;
+    b2sp_status rc = check_workspace(workspace, workspace_bytes,
+                                     b2sp_workspace_bytes(B2SP_OP_SPMM, M, K, 0, N, nnz));
+    if (rc != B2SP_OK) return rc;
+    int use = resolve_algo(algo);
+    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    g_last_algo[B2SP_OP_SPMM] = use;
+    int launches = 0;
+    g_last_launches[B2SP_OP_SPMM] = 0;
+    if (M == 0 || N == 0) return B2SP_OK;
+    if (nnz == 0) return zero_rows(O, ldo, M, N, st);
+
+    Workspace w = carve(workspace);
+    const int *order = nullptr;
+    if (use == B2SP_ALGO_ROW) {
+        rc = bin_rows(M, row_ptr, w, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        order = w.row_order;
+    }
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
+    if (vec) {
+        Geom g = pick_geom(N);
+        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
+        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
+        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
+        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
+        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
+        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
+    } else {
+        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
+                                                            ldo, order);
+    }
+    g_last_launches[B2SP_OP_SPMM] = launches + 1;
+    return check_launch();
+}
+
+b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
+                       const float *s_values, const float *A, long long lda, const float *B,
+                       long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
+                       int algo, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && !out_values) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
+    b2sp_status rc = check_workspace(workspace, workspace_bytes,
+                                     b2sp_workspace_bytes(B2SP_OP_SDDMM, M, K, Kd, 0, nnz));
+    if (rc != B2SP_OK) return rc;
+    int use = resolve_algo(algo);
+    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    g_last_algo[B2SP_OP_SDDMM] = use;
+    int launches = 0;
+    g_last_launches[B2SP_OP_SDDMM] = 0;
+    if (M == 0 || nnz == 0) return B2SP_OK;
+    if (Kd == 0)
+        return cudaMemsetAsync(out_values, 0, sizeof(float) * (size_t)nnz, st) == cudaSuccess
+                   ? B2SP_OK
+                   : B2SP_ERR_CUDA;
+
+    Workspace w = carve(workspace);
+    const int *order = nullptr;
+    if (use == B2SP_ALGO_ROW) {
+        rc = bin_rows(M, row_ptr, w, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        order = w.row_order;
+    }
+    dim3 grid((unsigned)M);
+    bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+               Kd <= 40960;
+    if (vec) {
+        switch (pick_ku(Kd)) {
+        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
+        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
+        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
+        default: {
+            size_t smem = sizeof(float) * (size_t)Kd;
+            if (smem > 48 * 1024 &&
+                cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem) != cudaSuccess)
+                return B2SP_ERR_CUDA;
+            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order);
+        }
+        }
+    } else {
+        sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
+                                                             B, ldb, out_values, order);
+    }
+    g_last_launches[B2SP_OP_SDDMM] = launches + 1;
+    return check_launch();
+}
+
+b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+                         const int *col_idx, const float *s_values, const float *A, long long lda,
+                         const float *B, long long ldb, const float *D, long long ldd, float *O,
+                         long long ldo, void *workspace, size_t workspace_bytes, int algo,
+                         void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0 || N < 0) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && N > 0 && (!D || ldd < N)) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && N > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
+    b2sp_status rc = check_workspace(workspace, workspace_bytes,
+                                     b2sp_workspace_bytes(B2SP_OP_FUSEDMM, M, K, Kd, N, nnz));
+    if (rc != B2SP_OK) return rc;
+    int use = resolve_algo(algo);
+    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    g_last_algo[B2SP_OP_FUSEDMM] = use;
+    int launches = 0;
+    g_last_launches[B2SP_OP_FUSEDMM] = 0;
+    if (M == 0 || N == 0) return B2SP_OK;
+    if (nnz == 0 || Kd == 0) return zero_rows(O, ldo, M, N, st);  // empty dot products are 0
+
+    Workspace w = carve(workspace);
+    const int *order = nullptr;
+    if (use == B2SP_ALGO_ROW) {
+        rc = bin_rows(M, row_ptr, w, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        order = w.row_order;
+    }
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
+               Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+               Kd <= 40960;
+    if (vec) {
+        Geom g = pick_geom(N);
+        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
+        switch (pick_ku(Kd)) {
+        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
+        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
+        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
+        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
+        }
+        if (rc != B2SP_OK) return rc;
+    } else {
+        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
+                                                               lda, B, ldb, D, ldd, O, ldo, order);
+    }
+    g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
+    return check_launch();
+}
+
+b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                              void *workspace, size_t workspace_bytes, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (M < 0 || K < 0 || nnz < 0 || nnz > (long long)INT_MAX || !row_ptr || (nnz > 0 && !col_idx))
+        return B2SP_ERR_INVALID_ARG;
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, 256);
+    if (rc != B2SP_OK) return rc;
+    int *flag = static_cast<int *>(workspace);
+    if (cudaMemsetAsync(flag, 0, sizeof(int), st) != cudaSuccess) return B2SP_ERR_CUDA;
+    long long work = nnz > M ? nnz : M;
+    int blocks = (int)((work + 255) / 256);
+    if (blocks < 1) blocks = 1;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    validate_csr_kernel<<<blocks, 256, 0, st>>>(M, K, nnz, row_ptr, col_idx, flag);
+    if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+    int h = 0;
+    if (cudaMemcpyAsync(&h, flag, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return B2SP_ERR_CUDA;
+    return h ? B2SP_ERR_BAD_CSR : B2SP_OK;
+}
+
+b2sp_status b2sp_device_status(const void *workspace, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!workspace) return B2SP_ERR_WORKSPACE;
+    int h = 0;
+    const int *status = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + 256);
+    if (cudaMemcpyAsync(&h, status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return B2SP_ERR_CUDA;
+    return h == 0 ? B2SP_OK : B2SP_ERR_TIMEOUT;
+}
+
+}  // extern "C"
+
+// ---- host-buffer forms ------------------------------------------------------------------------
+namespace {
+
+struct DevArena {
+    cudaStream_t st;
+    void *ptrs[16];
+    int n = 0;
+    bool ok = true;
+    explicit DevArena(cudaStream_t s) : st(s) {}
+    void *alloc(size_t bytes)
+    {
+        void *p = nullptr;
+        if (bytes == 0) bytes = 16;
+        if (!ok || cudaMallocAsync(&p, bytes, st) != cudaSuccess) { ok = false; return nullptr; }
+        ptrs[n++] = p;
+        return p;
+    }
+    template <typename T> T *upload(const T *host, size_t count)
+    {
+        T *d = static_cast<T *>(alloc(sizeof(T) * count));
+        if (d && host && count &&
+            cudaMemcpyAsync(d, host, sizeof(T) * count, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            ok = false;
+        return d;
+    }
+    b2sp_status finish(b2sp_status rc)
+    {
+        for (int i = 0; i < n; ++i) cudaFreeAsync(ptrs[i], st);
+        if (cudaStreamSynchronize(st) != cudaSuccess && rc == B2SP_OK) rc = B2SP_ERR_CUDA;
+        if (!ok && rc == B2SP_OK) rc = B2SP_ERR_CUDA;
+        return rc;
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_ptr,
+                           const int *col_idx, const float *values, const float *D, float *O,
+                           void *stream)
+{
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || N < 0) return B2SP_ERR_INVALID_ARG;
+    if ((M > 0 && N > 0 && !O) || (nnz > 0 && N > 0 && (!values || !D))) return B2SP_ERR_INVALID_ARG;
+    DevArena a(static_cast<cudaStream_t>(stream));
+    int *d_rp = a.upload(row_ptr, (size_t)M + 1);
+    int *d_ci = a.upload(col_idx, (size_t)nnz);
+    float *d_v = a.upload(values, (size_t)nnz);
+    float *d_D = a.upload(D, (size_t)K * N);
+    float *d_O = static_cast<float *>(a.alloc(sizeof(float) * (size_t)M * N));
+    size_t wsb = b2sp_workspace_bytes(B2SP_OP_SPMM, M, K, 0, N, nnz);
+    void *ws = a.alloc(wsb);
+    b2sp_status rc = B2SP_ERR_CUDA;
+    if (a.ok) {
+        rc = b2sp_spmm(M, K, N, nnz, d_rp, d_ci, d_v, d_D, N, d_O, N, ws, wsb, B2SP_ALGO_AUTO, stream);
+        if (rc == B2SP_OK && (size_t)M * N > 0 &&
+            cudaMemcpyAsync(O, d_O, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
+            rc = B2SP_ERR_CUDA;
+    }
+    return a.finish(rc);
+}
+
+b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_ptr,
+                            const int *col_idx, const float *s_values, const float *A,
+                            const float *B, float *out_values, void *stream)
+{
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0) return B2SP_ERR_INVALID_ARG;
+    if (nnz > 0 && (!out_values || (Kd > 0 && (!A || !B)))) return B2SP_ERR_INVALID_ARG;
+    DevArena a(static_cast<cudaStream_t>(stream));
+    int *d_rp = a.upload(row_ptr, (size_t)M + 1);
+    int *d_ci = a.upload(col_idx, (size_t)nnz);
+    float *d_v = s_values ? a.upload(s_values, (size_t)nnz) : nullptr;
+    float *d_A = a.upload(A, (size_t)M * Kd);
+    float *d_B = a.upload(B, (size_t)K * Kd);
+    float *d_C = static_cast<float *>(a.alloc(sizeof(float) * (size_t)nnz));
+    size_t wsb = b2sp_workspace_bytes(B2SP_OP_SDDMM, M, K, Kd, 0, nnz);
+    void *ws = a.alloc(wsb);
+    b2sp_status rc = B2SP_ERR_CUDA;
+    if (a.ok) {
+        rc = b2sp_sddmm(M, K, Kd, nnz, d_rp, d_ci, d_v, d_A, Kd, d_B, Kd, d_C, ws, wsb, B2SP_ALGO_AUTO, stream);
+        if (rc == B2SP_OK && nnz > 0 &&
+            cudaMemcpyAsync(out_values, d_C, sizeof(float) * (size_t)nnz, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
+            rc = B2SP_ERR_CUDA;
+    }
+    return a.finish(rc);
+}
+
+b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+                              const int *col_idx, const float *s_values, const float *A,
+                              const float *B, const float *D, float *O, void *stream)
+{
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0 || N < 0) return B2SP_ERR_INVALID_ARG;
+    if ((M > 0 && N > 0 && !O) || (nnz > 0 && N > 0 && (!D || (Kd > 0 && (!A || !B)))))
+        return B2SP_ERR_INVALID_ARG;
+    DevArena a(static_cast<cudaStream_t>(stream));
+    int *d_rp = a.upload(row_ptr, (size_t)M + 1);
+    int *d_ci = a.upload(col_idx, (size_t)nnz);
+    float *d_v = s_values ? a.upload(s_values, (size_t)nnz) : nullptr;
+    float *d_A = a.upload(A, (size_t)M * Kd);
+    float *d_B = a.upload(B, (size_t)K * Kd);
+    float *d_D = a.upload(D, (size_t)K * N);
+    float *d_O = static_cast<float *>(a.alloc(sizeof(float) * (size_t)M * N));
+    size_t wsb = b2sp_workspace_bytes(B2SP_OP_FUSEDMM, M, K, Kd, N, nnz);
+    void *ws = a.alloc(wsb);
+    b2sp_status rc = B2SP_ERR_CUDA;
+    if (a.ok) {
+        rc = b2sp_fusedmm(M, K, Kd, N, nnz, d_rp, d_ci, d_v, d_A, Kd, d_B, Kd, d_D, N, d_O, N, ws, wsb,
+                          B2SP_ALGO_AUTO, stream);
+        if (rc == B2SP_OK && (size_t)M * N > 0 &&
+            cudaMemcpyAsync(O, d_O, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
+            rc = B2SP_ERR_CUDA;
+    }
+    return a.finish(rc);
+}
+
+}  // extern "C"

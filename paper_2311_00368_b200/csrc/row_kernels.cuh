@@ -1,0 +1,473 @@
+// CUDA-core "row" kernels for SPMM / SDDMM / FusedMM over CSR (sm_100a).
+//
+// One CTA of kRowWarps warps owns one sparse row (and one slab of output columns).  The row's
+// (col_idx, values) segment is consumed in chunks of 32 entries -- the paper's VLC = 32 -- one
+// entry per lane, loaded coalesced and handed round by warp shuffles.  The warps of the CTA
+// take alternate chunks (the paper's "NT threads share a row's nonzeros") and, for SPMM and
+// FusedMM, their partial output rows are combined through shared memory in a fixed order, so
+// results are deterministic.  Rows are visited in the order given by `row_order` (longest
+// first, produced by the binning kernels below) or in natural order when it is NULL.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace b2sp {
+
+constexpr int kRowWarps = 4;
+constexpr int kRowThreads = kRowWarps * 32;
+constexpr int kBuckets = 32;
+constexpr unsigned kFull = 0xffffffffu;
+
+// ------------------------------------------------------------------------------------------
+// Row binning (work assignment): counting sort of the rows by length bucket
+// bucket(len) = number of significant bits of len, longest bucket first.
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int bucket_of(int len) { return len <= 0 ? 0 : 32 - __clz(len); }
+
+__global__ void bin_count_kernel(int M, const int *__restrict__ row_ptr, int *__restrict__ count)
+{
+    __shared__ int h[kBuckets];
+    if (threadIdx.x < kBuckets) h[threadIdx.x] = 0;
+    __syncthreads();
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < M) atomicAdd(&h[bucket_of(row_ptr[i + 1] - row_ptr[i])], 1);
+    __syncthreads();
+    if (threadIdx.x < kBuckets && h[threadIdx.x]) atomicAdd(&count[threadIdx.x], h[threadIdx.x]);
+}
+
+__global__ void bin_scatter_kernel(int M, const int *__restrict__ row_ptr,
+                                   const int *__restrict__ count, int *__restrict__ cursor,
+                                   int *__restrict__ row_order)
+{
+    __shared__ int h[kBuckets];
+    __shared__ int base[kBuckets];
+    if (threadIdx.x < kBuckets) h[threadIdx.x] = 0;
+    __syncthreads();
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    int b = 0, r = 0;
+    if (i < M) {
+        b = bucket_of(row_ptr[i + 1] - row_ptr[i]);
+        r = atomicAdd(&h[b], 1);
+    }
+    __syncthreads();
+    if (threadIdx.x < kBuckets) {
+        int mine = threadIdx.x, start = 0;
+        for (int j = kBuckets - 1; j > mine; --j) start += count[j];
+        base[mine] = h[mine] ? start + atomicAdd(&cursor[mine], h[mine]) : 0;
+    }
+    __syncthreads();
+    if (i < M) row_order[base[b] + r] = i;
+}
+
+// ------------------------------------------------------------------------------------------
+// helpers
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ float4 ldg4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+
+__device__ __forceinline__ void fma4(float4 &acc, float s, const float4 &v)
+{
+    acc.x = fmaf(s, v.x, acc.x);
+    acc.y = fmaf(s, v.y, acc.y);
+    acc.z = fmaf(s, v.z, acc.z);
+    acc.w = fmaf(s, v.w, acc.w);
+}
+
+__device__ __forceinline__ float dot4(const float4 &a, const float4 &b, float acc)
+{
+    acc = fmaf(a.x, b.x, acc);
+    acc = fmaf(a.y, b.y, acc);
+    acc = fmaf(a.z, b.z, acc);
+    acc = fmaf(a.w, b.w, acc);
+    return acc;
+}
+
+// Geometry of the SPMM sweep.  SPLIT sub-warps of LPN = 32/SPLIT lanes each take alternate
+// entries of a chunk; a lane owns U float4 column groups: columns col0 + (sl + LPN*u)*4.
+template <int U, int SPLIT>
+struct SweepGeom {
+    static constexpr int LPN = 32 / SPLIT;
+    static constexpr int SLAB = LPN * 4 * U;
+};
+
+// One chunk (up to 32 entries, lane l holds entry l: column k, scalar s) of the Alg. 2 SAXPY
+// sweep.  SRC(j) gives the lane that holds entry j's scalar.
+template <int U, int SPLIT, bool PERMUTED>
+__device__ __forceinline__ void saxpy_chunk(float4 (&acc)[U], int k, float s, int cnt,
+                                            const float *__restrict__ Dcol, int64_t ldd,
+                                            bool (&live)[U], int sub)
+{
+    constexpr int LPN = 32 / SPLIT;
+    constexpr int STEPS = 32 / SPLIT;
+    if (cnt == 32) {
+#pragma unroll 8
+        for (int jj = 0; jj < STEPS; ++jj) {
+            int j = jj * SPLIT + sub;
+            int src = PERMUTED ? ((j & 3) * 8 + (j >> 2)) : j;
+            int kk = __shfl_sync(kFull, k, j);
+            float ss = __shfl_sync(kFull, s, src);
+            const float *d = Dcol + (int64_t)kk * ldd;
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+                if (live[u]) fma4(acc[u], ss, ldg4(d + u * LPN * 4));
+        }
+    } else {
+        for (int jj = 0; jj < STEPS; ++jj) {
+            int j = jj * SPLIT + sub;
+            int src = PERMUTED ? ((j & 3) * 8 + (j >> 2)) : j;
+            int kk = __shfl_sync(kFull, k, j);
+            float ss = __shfl_sync(kFull, s, src);
+            if (j < cnt) {
+                const float *d = Dcol + (int64_t)kk * ldd;
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+                    if (live[u]) fma4(acc[u], ss, ldg4(d + u * LPN * 4));
+            }
+        }
+    }
+}
+
+// Combine the sub-warps of a warp, then the warps of the CTA (fixed order), and store the row.
+template <int U, int SPLIT>
+__device__ __forceinline__ void reduce_and_store_row(float4 (&acc)[U], float4 *red, int warp,
+                                                     int lane, float *__restrict__ Orow,
+                                                     bool (&live)[U])
+{
+    constexpr int LPN = 32 / SPLIT;
+#pragma unroll
+    for (int off = 16; off >= LPN; off >>= 1) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            acc[u].x += __shfl_xor_sync(kFull, acc[u].x, off);
+            acc[u].y += __shfl_xor_sync(kFull, acc[u].y, off);
+            acc[u].z += __shfl_xor_sync(kFull, acc[u].z, off);
+            acc[u].w += __shfl_xor_sync(kFull, acc[u].w, off);
+        }
+    }
+    if (lane < LPN) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) red[(warp * U + u) * LPN + lane] = acc[u];
+    }
+    __syncthreads();
+    if (warp == 0 && lane < LPN) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (!live[u]) continue;
+            float4 r = red[u * LPN + lane];
+#pragma unroll
+            for (int w = 1; w < kRowWarps; ++w) {
+                float4 t = red[(w * U + u) * LPN + lane];
+                r.x += t.x; r.y += t.y; r.z += t.z; r.w += t.w;
+            }
+            *reinterpret_cast<float4 *>(Orow + u * LPN * 4) = r;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// SPMM  (Alg. 2; float4 path: N, ldd, ldo multiples of 4, D and O 16-byte aligned)
+// ------------------------------------------------------------------------------------------
+template <int U, int SPLIT>
+__global__ void __launch_bounds__(kRowThreads)
+spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
+                const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
+                float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order)
+{
+    using G = SweepGeom<U, SPLIT>;
+    __shared__ float4 red[kRowWarps * U * G::LPN];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / G::LPN, sl = lane % G::LPN;
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int col0 = blockIdx.y * G::SLAB + sl * 4;
+    bool live[U];
+    float4 acc[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        live[u] = col0 + u * G::LPN * 4 < N;
+        acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    const float *Dcol = D + col0;
+    // the next chunk's indices and values are fetched before the current chunk is consumed
+    // (the role of the paper's prefetch of the next ja/avalues block)
+    int k = 0;
+    float s = 0.f;
+    {
+        int p = beg + warp * 32 + lane;
+        if (p < end) {
+            k = __ldg(col_idx + p);
+            s = __ldg(values + p);
+        }
+    }
+    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+        int pn = c + kRowWarps * 32 + lane;
+        int kn = 0;
+        float sn = 0.f;
+        if (pn < end) {
+            kn = __ldg(col_idx + pn);
+            sn = __ldg(values + pn);
+        }
+        saxpy_chunk<U, SPLIT, false>(acc, k, s, min(32, end - c), Dcol, ldd, live, sub);
+        k = kn;
+        s = sn;
+    }
+    reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
+}
+
+// Scalar path for any N / ld / alignment: a lane owns columns col0 + lane + 32u (u < 4).
+__global__ void __launch_bounds__(kRowThreads)
+spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
+                       const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
+                       float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order)
+{
+    __shared__ float red[kRowWarps][128];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int col0 = blockIdx.y * 128 + lane;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+        int p = c + lane;
+        int k = 0;
+        float s = 0.f;
+        if (p < end) {
+            k = __ldg(col_idx + p);
+            s = __ldg(values + p);
+        }
+        int cnt = min(32, end - c);
+        for (int j = 0; j < cnt; ++j) {
+            int kk = __shfl_sync(kFull, k, j);
+            float ss = __shfl_sync(kFull, s, j);
+            const float *d = D + (int64_t)kk * ldd + col0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (col0 + 32 * u >= N) continue;
+            float r = red[0][lane + 32 * u];
+            for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
+            O[(int64_t)row * ldo + col0 + 32 * u] = r;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// SDDMM  (Alg. 1; float4 path: Kd, lda, ldb multiples of 4, A and B 16-byte aligned)
+//
+// A group of 8 lanes computes one sampled dot product: lane t of the group owns elements
+// (t + 8u)*4 .. +3 of the Kd-vector.  KU > 0: A_i is held in KU float4 registers per lane
+// (Kd <= 32*KU).  KU == 0: any Kd, A_i staged in shared memory.  In a chunk of 32 entries,
+// group g takes entries 4r + g (r = 0..7); after the 3-step butterfly every lane of the
+// group has the sum and lane t keeps round t's, so lane 8g + t ends up holding entry 4t + g.
+// ------------------------------------------------------------------------------------------
+template <int KU>
+__device__ __forceinline__ float sddmm_chunk(const float4 (&areg)[KU > 0 ? KU : 1],
+                                             const float *__restrict__ a_smem, int Kd, int k,
+                                             const float *__restrict__ B, int64_t ldb, int lane)
+{
+    const int g = lane >> 3, t = lane & 7;
+    float mine = 0.f;
+#pragma unroll 4
+    for (int r = 0; r < 8; ++r) {
+        int kq = __shfl_sync(kFull, k, 4 * r + g);
+        const float *b = B + (int64_t)kq * ldb + t * 4;
+        float part = 0.f;
+        if (KU > 0) {
+#pragma unroll
+            for (int u = 0; u < KU; ++u)
+                if ((t + 8 * u) * 4 < Kd) part = dot4(areg[u], ldg4(b + u * 32), part);
+        } else {
+            for (int e = t * 4; e < Kd; e += 32)
+                part = dot4(*reinterpret_cast<const float4 *>(a_smem + e), ldg4(b + e - t * 4), part);
+        }
+        part += __shfl_xor_sync(kFull, part, 1);
+        part += __shfl_xor_sync(kFull, part, 2);
+        part += __shfl_xor_sync(kFull, part, 4);
+        if (r == t) mine = part;
+    }
+    return mine;  // lane 8g+t: dot product of entry 4t+g
+}
+
+template <int KU>
+__device__ __forceinline__ void load_a_row(float4 (&areg)[KU > 0 ? KU : 1], float *a_smem,
+                                           const float *__restrict__ Arow, int Kd, int lane)
+{
+    if (KU > 0) {
+        const int t = lane & 7;
+#pragma unroll
+        for (int u = 0; u < (KU > 0 ? KU : 1); ++u)
+            areg[u] = (t + 8 * u) * 4 < Kd ? ldg4(Arow + (t + 8 * u) * 4) : make_float4(0.f, 0.f, 0.f, 0.f);
+    } else {
+        for (int e = threadIdx.x * 4; e < Kd; e += kRowThreads * 4)
+            *reinterpret_cast<float4 *>(a_smem + e) = ldg4(Arow + e);
+        __syncthreads();
+    }
+}
+
+template <int KU>
+__global__ void __launch_bounds__(kRowThreads)
+sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
+                 const float *s_values, const float *__restrict__ A, int64_t lda,
+                 const float *__restrict__ B, int64_t ldb, float *out_values,
+                 const int *__restrict__ row_order)
+{
+    extern __shared__ float4 dyn_smem[];
+    float *a_smem = reinterpret_cast<float *>(dyn_smem);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    float4 areg[KU > 0 ? KU : 1];
+    load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+    const int slot = (lane & 7) * 4 + (lane >> 3);  // entry of the chunk this lane ends up holding
+    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+        int p = c + lane;
+        int k = p < end ? __ldg(col_idx + p) : 0;
+        float dp = sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
+        int q = c + slot;
+        if (q < end) out_values[q] = s_values ? s_values[q] * dp : dp;
+    }
+}
+
+// Scalar path for any Kd / ld / alignment: one lane per entry, serial dot product.
+__global__ void __launch_bounds__(kRowThreads)
+sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
+                        const float *s_values, const float *__restrict__ A, int64_t lda,
+                        const float *__restrict__ B, int64_t ldb, float *out_values,
+                        const int *__restrict__ row_order)
+{
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    const float *a = A + (int64_t)row * lda;
+    for (int p = beg + threadIdx.x; p < end; p += kRowThreads) {
+        const float *b = B + (int64_t)__ldg(col_idx + p) * ldb;
+        float dp = 0.f;
+        for (int l = 0; l < Kd; ++l) dp = fmaf(__ldg(a + l), __ldg(b + l), dp);
+        out_values[p] = s_values ? s_values[p] * dp : dp;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// FusedMM  (Alg. 3): per chunk, the SDDMM values stay in registers (one per lane) and are the
+// scalars of the SAXPY sweep over the same staged column indices; C never reaches memory.
+// ------------------------------------------------------------------------------------------
+template <int KU, int U, int SPLIT>
+__global__ void __launch_bounds__(kRowThreads)
+fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
+                   const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
+                   const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
+                   int64_t ldd, float *__restrict__ O, int64_t ldo,
+                   const int *__restrict__ row_order)
+{
+    using G = SweepGeom<U, SPLIT>;
+    extern __shared__ float4 dyn_smem[];
+    float4 *red = dyn_smem;                                                   // kRowWarps*U*LPN
+    float *a_smem = reinterpret_cast<float *>(dyn_smem + kRowWarps * U * G::LPN);  // Kd (KU == 0)
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane / G::LPN, sl = lane % G::LPN;
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int col0 = blockIdx.y * G::SLAB + sl * 4;
+    bool live[U];
+    float4 acc[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        live[u] = col0 + u * G::LPN * 4 < N;
+        acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    float4 areg[KU > 0 ? KU : 1];
+    load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+    const int slot = (lane & 7) * 4 + (lane >> 3);
+    const float *Dcol = D + col0;
+    int k = 0;
+    float sv = 1.f;
+    {
+        int p = beg + warp * 32 + lane, q = beg + warp * 32 + slot;
+        if (p < end) k = __ldg(col_idx + p);
+        if (s_values && q < end) sv = __ldg(s_values + q);
+    }
+    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+        int pn = c + kRowWarps * 32 + lane, qn = c + kRowWarps * 32 + slot;
+        int kn = pn < end ? __ldg(col_idx + pn) : 0;
+        float svn = (s_values && qn < end) ? __ldg(s_values + qn) : 1.f;
+        float cv = sv * sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
+        saxpy_chunk<U, SPLIT, true>(acc, k, cv, min(32, end - c), Dcol, ldd, live, sub);
+        k = kn;
+        sv = svn;
+    }
+    reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
+}
+
+// Scalar path for any widths / alignment: lane-per-entry dot products, then a scalar sweep.
+__global__ void __launch_bounds__(kRowThreads)
+fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
+                          const int *__restrict__ col_idx, const float *__restrict__ s_values,
+                          const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
+                          int64_t ldb, const float *__restrict__ D, int64_t ldd,
+                          float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order)
+{
+    __shared__ float red[kRowWarps][128];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
+    const int col0 = blockIdx.y * 128 + lane;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    const float *a = A + (int64_t)row * lda;
+    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+        int p = c + lane;
+        int k = 0;
+        float cv = 0.f;
+        if (p < end) {
+            k = __ldg(col_idx + p);
+            const float *b = B + (int64_t)k * ldb;
+            for (int l = 0; l < Kd; ++l) cv = fmaf(__ldg(a + l), __ldg(b + l), cv);
+            if (s_values) cv *= __ldg(s_values + p);
+        }
+        int cnt = min(32, end - c);
+        for (int j = 0; j < cnt; ++j) {
+            int kk = __shfl_sync(kFull, k, j);
+            float ss = __shfl_sync(kFull, cv, j);
+            const float *d = D + (int64_t)kk * ldd + col0;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+                if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (col0 + 32 * u >= N) continue;
+            float r = red[0][lane + 32 * u];
+            for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
+            O[(int64_t)row * ldo + col0 + 32 * u] = r;
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// CSR validation (debug helper)
+// ------------------------------------------------------------------------------------------
+__global__ void validate_csr_kernel(int M, int K, long long nnz, const int *__restrict__ row_ptr,
+                                    const int *__restrict__ col_idx, int *__restrict__ flag)
+{
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    long long stride = (long long)gridDim.x * blockDim.x;
+    bool bad = false;
+    if (i == 0) bad |= row_ptr[0] != 0 || (long long)row_ptr[M] != nnz;
+    for (long long r = i; r < M; r += stride) bad |= row_ptr[r + 1] < row_ptr[r];
+    for (long long p = i; p < nnz; p += stride) {
+        int c = col_idx[p];
+        bad |= c < 0 || c >= K;
+    }
+    if (bad) atomicExch(flag, 1);
+}
+
+}  // namespace b2sp

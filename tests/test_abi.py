@@ -1,0 +1,64 @@
+"""The C-ABI library builds, loads without a GPU and exports every function include/b2sp.h declares.
+No compute call is made here."""
+import ctypes
+import os
+import re
+
+from paper_2311_00368_b200 import build as b2sp_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "b2sp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(b2sp_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_header_declares_the_three_ops():
+    names = declared_functions()
+    for n in ("b2sp_spmm", "b2sp_sddmm", "b2sp_fusedmm", "b2sp_workspace_bytes", "b2sp_spmm_host",
+              "b2sp_sddmm_host", "b2sp_fusedmm_host"):
+        assert n in names
+
+
+def test_library_exports_every_declared_symbol():
+    lib = ctypes.CDLL(b2sp_build.build())
+    for name in declared_functions():
+        assert hasattr(lib, name), f"{name} is declared in b2sp.h but not exported"
+    lib.b2sp_version.restype = ctypes.c_int
+    assert lib.b2sp_version() >= 100
+    lib.b2sp_status_string.restype = ctypes.c_char_p
+    assert lib.b2sp_status_string(0) == b"ok"
+    lib.b2sp_workspace_bytes.restype = ctypes.c_size_t
+    lib.b2sp_workspace_bytes.argtypes = [ctypes.c_int] * 5 + [ctypes.c_longlong]
+    n = lib.b2sp_workspace_bytes(2, 8192, 8192, 128, 512, 20_000_000)
+    assert n >= 4 * 8192 and n % 256 == 0
+    assert lib.b2sp_workspace_bytes(7, 1, 1, 1, 1, 1) == 0
+
+
+def test_argument_errors_need_no_gpu():
+    """Argument checks run before any CUDA call."""
+    lib = ctypes.CDLL(b2sp_build.build())
+    i, ll, vp, sz = ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_size_t
+    lib.b2sp_spmm.restype = i
+    lib.b2sp_spmm.argtypes = [i, i, i, ll, vp, vp, vp, vp, ll, vp, ll, vp, sz, i, vp]
+    assert lib.b2sp_spmm(-1, 4, 4, 0, None, None, None, None, 4, None, 4, None, 0, 0, None) == 1
+    assert lib.b2sp_spmm(4, 4, 4, 2 ** 31, None, None, None, None, 4, None, 4, None, 0, 0, None) == 1
+    assert lib.b2sp_spmm(4, 4, 4, 3, None, None, None, None, 4, None, 4, None, 0, 0, None) == 1
+
+
+def test_binding_refuses_to_run_without_the_library(tmp_path, monkeypatch):
+    """There is no fallback: without libb2sp.so the binding cannot even be imported."""
+    import importlib.util
+    src = os.path.join(ROOT, "paper_2311_00368_b200", "binding.py")
+    dst = tmp_path / "binding_copy.py"
+    dst.write_text(open(src).read())
+    spec = importlib.util.spec_from_file_location("binding_copy", dst)
+    mod = importlib.util.module_from_spec(spec)
+    try:
+        spec.loader.exec_module(mod)
+        raised = False
+    except ImportError:
+        raised = True
+    assert raised
