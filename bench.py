@@ -19,7 +19,6 @@ from __future__ import annotations
 import argparse
 import json
 import os
-import subprocess
 import sys
 import threading
 import time
@@ -39,7 +38,10 @@ L2_FLUSH_BYTES = 256 << 20
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of the dominant kernel,
 # from the ncu captures summarised under profiles/; None where no capture exists yet.
-MEASURED_TRAFFIC_BYTES = {}
+MEASURED_TRAFFIC_BYTES = {
+    # (workload, kernel family of the FusedMM op) -> bytes; see profiles/fusedmm_row_sweep_d30_n128.md
+    ("sweep_d30_n128", "row"): 179_792_128,
+}
 
 
 def make_workload(name: str, rank: int = 0) -> W.Problem:
@@ -72,56 +74,70 @@ def peaks():
 
 
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    """Samples SM clock, power and throttle reasons (read-only NVML queries) from a thread while the
+    timed region runs."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
-
-    def __init__(self, uuid):
-        self.rows, self.proc, self.uuid = [], None, uuid
+    def __init__(self, device_index: int, period_s: float = 0.004):
+        self.idx, self.period, self.rows = device_index, period_s, []
+        self._stop = threading.Event()
+        self.t = None
+        self.err = None
 
     def start(self):
         try:
-            cmd = ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100"]
-            if self.uuid:
-                cmd += ["-i", self.uuid]
-            self.proc = subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            import torch
+            uuid = "GPU-" + str(torch.cuda.get_device_properties(self.idx).uuid)
+            try:
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode())
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(self.idx)
+            self.nv = pynvml
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # noqa: BLE001
+            self.err = f"NVML unavailable: {e}"
+            return
+        self.t = threading.Thread(target=self._loop, daemon=True)
+        self.t.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+    def _loop(self):
+        nv = self.nv
+        while not self._stop.is_set():
+            try:
+                mhz = float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:
+                    reasons = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                try:
+                    power = nv.nvmlDeviceGetPowerUsage(self.h) / 1e3
+                except Exception:
+                    power = float("nan")
+                self.rows.append((mhz, reasons, power))
+            except Exception as e:  # noqa: BLE001
+                self.err = str(e)
+                return
+            time.sleep(self.period)
 
     def stop(self):
-        if not self.proc:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
+        if self.t is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.err or "not sampled"]}
+        self._stop.set()
         self.t.join(timeout=2)
-        sm, mx, reasons, power = [], [], set(), []
-        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
-        for r in self.rows:
-            if len(r) < 7:
-                continue
-            try:
-                sm.append(float(r[0])); mx.append(float(r[1])); power.append(float(r[2]))
-            except ValueError:
-                continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        nv = self.nv
+        bits = {"hw_slowdown": 0x8, "hw_thermal_slowdown": 0x40, "sw_thermal_slowdown": 0x20,
+                "sw_power_cap": 0x4, "hw_power_brake_slowdown": 0x80}
+        seen = set()
+        for _, r, _ in self.rows:
+            for name, bit in bits.items():
+                if r & bit:
+                    seen.add(name)
+        sm = [r[0] for r in self.rows]
+        pw = [r[2] for r in self.rows if r[2] == r[2]]
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": self.max_mhz, "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(seen)}
 
 
 def oracle_sample(p: W.Problem, budget_s: float):
@@ -192,7 +208,7 @@ def workload_config(p, name):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="sweep_d30_n128")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -253,7 +269,7 @@ def main():
     launches = {op: b.last_launches(i) for i, op in enumerate(OPS)}
     algos = {op: b.ALGO_NAMES[b.last_algo(i)] for i, op in enumerate(OPS)}
 
-    sampler = ClockSampler(str(torch.cuda.get_device_properties(device).uuid) if rank == 0 else None)
+    sampler = ClockSampler(local_rank)
     replicas.barrier()
     torch.cuda.synchronize()
     if rank == 0:
@@ -307,7 +323,7 @@ def main():
                 "peak_source": f"hbm_gbs of {peak_src}"}
     roof["frac"] = roof["achieved"] / roof["peak"]
     roof["kernel"] = dom
-    roof["traffic"] = MEASURED_TRAFFIC_BYTES.get(args.workload)
+    roof["traffic"] = MEASURED_TRAFFIC_BYTES.get((args.workload, algos[dom]))
     roof["algorithmic_bytes"] = by[dom]
     roof["algorithmic_flops"] = fl[dom]
 
