@@ -53,7 +53,8 @@ typedef enum {
     B2SP_ERR_BAD_CSR = 3,     /* b2sp_validate_csr: row_ptr not monotone / col_idx out of range */
     B2SP_ERR_CUDA = 4,        /* a CUDA runtime call or a kernel launch failed */
     B2SP_ERR_WORKSPACE = 5,   /* workspace NULL, misaligned or too small */
-    B2SP_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (reported by b2sp_device_status) */
+    B2SP_ERR_TIMEOUT = 6,     /* a bounded device-side wait expired (reported by b2sp_device_status) */
+    B2SP_ERR_TOO_LARGE = 7    /* the problem does not fit the library's built-in scratch array */
 } b2sp_status;
 
 enum { B2SP_ALGO_AUTO = 0, B2SP_ALGO_ROW = 1, B2SP_ALGO_ROW_NAT = 2, B2SP_ALGO_TILE = 3 };
@@ -131,6 +132,41 @@ b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz,
                               const int *row_ptr, const int *col_idx, const float *s_values,
                               const float *A, const float *B, const float *D, float *O,
                               void *stream);
+
+/*
+ * SPMM without any allocation, for callers that cannot obtain device memory of their own.
+ * (The paper has no counterpart; this is a deployment convenience, not part of its method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is not an option -- a plug-in inside a serving
+ * process that gave all device memory to its own arena at start-up, or a latency-critical loop
+ * that must not trigger the device-wide synchronisation an allocation can cause.  Such a caller
+ * owns inputs and outputs but has no workspace to offer, so this entry point keeps the row-binning
+ * workspace in a fixed array inside the library's device image instead.
+ *
+ * Same result and same argument meaning as b2sp_spmm with B2SP_ALGO_ROW (all data pointers are
+ * device pointers; O is fully overwritten), minus the workspace and algo arguments.
+ *
+ * Limits and rules:
+ *   - M <= B2SP_STATIC_SCRATCH_MAX_ROWS, otherwise B2SP_ERR_TOO_LARGE and nothing is enqueued.
+ *     K, N and nnz are unrestricted.
+ *   - The array (512 bytes + 4 bytes per row of the limit, about 257 KiB) occupies device memory on
+ *     every GPU that loads the library, until the process exits, used or not.
+ *   - The first call on each device looks up the array's device address (a host-side runtime
+ *     query, no allocation).  Make that first call with the device current and before starting any
+ *     stream capture on it.
+ *   - All calls on a device share the one array, and it keeps whatever the previous call left.  The
+ *     part that must start from zero is cleared at the start of each call, so back-to-back calls on
+ *     one stream are fine; two calls that can overlap on the GPU (different streams, or different
+ *     host threads with different streams) race on it and give wrong results.  Use b2sp_spmm with
+ *     separate workspaces for concurrent work.
+ *   - The entry point itself calls no cudaMalloc / cudaFree / pool allocator and launches only a
+ *     small memset and kernels on `stream`; it does not synchronise.
+ */
+#define B2SP_STATIC_SCRATCH_MAX_ROWS 65536
+b2sp_status b2sp_spmm_static_scratch(int M, int K, int N, long long nnz,
+                                     const int *row_ptr, const int *col_idx, const float *values,
+                                     const float *D, long long ldd, float *O, long long ldo,
+                                     void *stream);
 
 /*
  * Debug helper: checks on the device that row_ptr[0] = 0, row_ptr is non-decreasing,

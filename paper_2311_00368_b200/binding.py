@@ -49,6 +49,8 @@ lib.b2sp_sddmm_host.restype = _i
 lib.b2sp_sddmm_host.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.b2sp_fusedmm_host.restype = _i
 lib.b2sp_fusedmm_host.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
+lib.b2sp_spmm_static_scratch.restype = _i
+lib.b2sp_spmm_static_scratch.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp]
 lib.b2sp_validate_csr.restype = _i
 lib.b2sp_validate_csr.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_device_status.restype = _i
@@ -134,6 +136,27 @@ def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALG
     ws, wsb = _workspace(OP_SPMM, M, K, 0, N, nnz, D.device, workspace)
     _check(lib.b2sp_spmm(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D), _ld(D),
                          _ptr(out), _ld(out), _ptr(ws), wsb, algo, _stream()), "b2sp_spmm")
+    return out
+
+
+STATIC_SCRATCH_MAX_ROWS = 65536
+
+
+def spmm_static_scratch(row_ptr, col_idx, values, D, K=None, out=None):
+    """b2sp_spmm_static_scratch: SPMM for callers that may not allocate device memory.  The
+    library's built-in scratch array replaces the workspace; M is limited to
+    STATIC_SCRATCH_MAX_ROWS, and calls that could overlap on the GPU must not share a device.
+    (`out` should be passed by such callers; it is only created here for convenience.)"""
+    _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
+    _want(values, torch.float32, "values"); _want(D, torch.float32, "D")
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    K = D.shape[0] if K is None else K
+    N = D.shape[1]
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=D.device)
+    _check(lib.b2sp_spmm_static_scratch(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values),
+                                        _ptr(D), _ld(D), _ptr(out), _ld(out), _stream()),
+           "b2sp_spmm_static_scratch")
     return out
 
 

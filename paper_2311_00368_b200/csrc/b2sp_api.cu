@@ -171,6 +171,7 @@ const char *b2sp_status_string(b2sp_status s)
     case B2SP_ERR_CUDA: return "CUDA error";
     case B2SP_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
     case B2SP_ERR_TIMEOUT: return "device-side wait timed out";
+    case B2SP_ERR_TOO_LARGE: return "problem exceeds the library's built-in scratch array";
     }
     return "unknown status";
 }
