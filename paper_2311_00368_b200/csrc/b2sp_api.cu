@@ -6,6 +6,7 @@
 #include <cstdint>
 
 #include "row_kernels.cuh"
+#include "tile_dispatch.h"
 
 namespace b2sp {
 
@@ -17,6 +18,7 @@ namespace b2sp {
 constexpr size_t kHeaderBytes = 512;
 
 inline size_t align256(size_t x) { return (x + 255) & ~size_t(255); }
+inline size_t row_workspace_bytes(int M) { return align256(kHeaderBytes + sizeof(int) * (size_t)M); }
 
 struct Workspace {
     int *count, *cursor, *status, *row_order;
@@ -63,10 +65,10 @@ b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t
 template <int U, int SPLIT>
 void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
                  const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
-                 const int *order)
+                 const int *order, const int *gate)
 {
     spmm_row_kernel<U, SPLIT><<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                           ldo, order);
+                                                           ldo, order, gate);
 }
 
 // Column geometry for a width N on the float4 path: U float4 per lane, SPLIT sub-warps.
@@ -85,18 +87,18 @@ inline int pick_ku(int Kd) { return Kd <= 64 ? 2 : Kd <= 128 ? 4 : Kd <= 256 ? 8
 template <int KU>
 void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const int *col_idx,
                   const float *sv, const float *A, int64_t lda, const float *B, int64_t ldb,
-                  float *out, const int *order)
+                  float *out, const int *order, const int *gate)
 {
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     sddmm_row_kernel<KU><<<grid, kRowThreads, smem, st>>>(Kd, row_ptr, col_idx, sv, A, lda, B, ldb,
-                                                         out, order);
+                                                         out, order, gate);
 }
 
 template <int KU, int U, int SPLIT>
 b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
                          const int *col_idx, const float *sv, const float *A, int64_t lda,
                          const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
-                         int64_t ldo, const int *order)
+                         int64_t ldo, const int *order, const int *gate)
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
@@ -108,7 +110,7 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
             return B2SP_ERR_CUDA;
     }
     kern<<<grid, kRowThreads, smem, st>>>(Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
-                                          order);
+                                          order, gate);
     return B2SP_OK;
 }
 
@@ -117,10 +119,10 @@ b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int K
                                 const int *row_ptr, const int *col_idx, const float *sv,
                                 const float *A, int64_t lda, const float *B, int64_t ldb,
                                 const float *D, int64_t ldd, float *O, int64_t ldo,
-                                const int *order)
+                                const int *order, const int *gate)
 {
 #define B2SP_F(U_, S_) \
-    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order)
+    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate)
     if (g.SPLIT == 4) B2SP_F(1, 4);
     if (g.SPLIT == 2) B2SP_F(1, 2);
     if (g.U == 1) B2SP_F(1, 1);
@@ -148,7 +150,7 @@ bool bad_csr_args(int M, int K, long long nnz, const int *row_ptr, const int *co
 
 int resolve_algo(int algo)
 {
-    // The dense-tile family is not built into this translation unit yet.
+    // SDDMM and FusedMM: row family only for now.
     if (algo == B2SP_ALGO_AUTO) return B2SP_ALGO_ROW;
     return algo;
 }
@@ -179,11 +181,38 @@ const char *b2sp_status_string(b2sp_status s)
 size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 {
     if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
-    return align256(kHeaderBytes + sizeof(int) * (size_t)M);
+    size_t need = row_workspace_bytes(M);
+    if (op == B2SP_OP_SPMM && tile_profitable(M, K, N, nnz)) {
+        TilePlan p = plan_spmm_tile(M, K, N, nnz, need);
+        if (p.feasible && p.bytes > need) need = p.bytes;
+    }
+    return need;
 }
 
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
+
+// Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
+static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
+                             const float *D, long long ldd, float *O, long long ldo, const int *order,
+                             const int *gate, cudaStream_t st)
+{
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
+    if (vec) {
+        Geom g = pick_geom(N);
+        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
+        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+    } else {
+        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
+                                                            ldo, order, gate);
+    }
+    return check_launch();
+}
 
 b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
                       const float *values, const float *D, long long ldd, float *O, long long ldo,
@@ -194,11 +223,15 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
     if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && (!values || !D || ldd < N)) return B2SP_ERR_INVALID_ARG;
-    b2sp_status rc = check_workspace(workspace, workspace_bytes,
-                                     b2sp_workspace_bytes(B2SP_OP_SPMM, M, K, 0, N, nnz));
+    const size_t row_bytes = row_workspace_bytes(M);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
-    int use = resolve_algo(algo);
-    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    TilePlan plan;
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, N, nnz)))
+        plan = plan_spmm_tile(M, K, N, nnz, row_bytes);
+    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
+    else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_SPMM] = use;
     int launches = 0;
     g_last_launches[B2SP_OP_SPMM] = 0;
@@ -206,28 +239,24 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     if (nnz == 0) return zero_rows(O, ldo, M, N, st);
 
     Workspace w = carve(workspace);
+    if (use == B2SP_ALGO_TILE) {
+        rc = spmm_tile(plan, M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
+        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, st);
+        g_last_launches[B2SP_OP_SPMM] = launches + 1;
+        return rc;
+    }
     const int *order = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
     }
-    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
-    if (vec) {
-        Geom g = pick_geom(N);
-        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
-        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
-        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
-        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
-        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
-        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order);
-    } else {
-        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
-        spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                            ldo, order);
-    }
+    rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, nullptr, st);
     g_last_launches[B2SP_OP_SPMM] = launches + 1;
-    return check_launch();
+    return rc;
 }
 
 b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
@@ -266,21 +295,21 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
                Kd <= 40960;
     if (vec) {
         switch (pick_ku(Kd)) {
-        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
-        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
-        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order); break;
+        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
+        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
+        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
         default: {
             size_t smem = sizeof(float) * (size_t)Kd;
             if (smem > 48 * 1024 &&
                 cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)smem) != cudaSuccess)
                 return B2SP_ERR_CUDA;
-            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order);
+            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr);
         }
         }
     } else {
         sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
-                                                             B, ldb, out_values, order);
+                                                             B, ldb, out_values, order, nullptr);
     }
     g_last_launches[B2SP_OP_SDDMM] = launches + 1;
     return check_launch();
@@ -323,16 +352,16 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
         Geom g = pick_geom(N);
         dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
         switch (pick_ku(Kd)) {
-        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
-        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
-        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
-        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order); break;
+        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
+        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
+        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
+        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
         }
         if (rc != B2SP_OK) return rc;
     } else {
         dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
         fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
-                                                               lda, B, ldb, D, ldd, O, ldo, order);
+                                                               lda, B, ldb, D, ldd, O, ldo, order, nullptr);
     }
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
     return check_launch();

@@ -1,0 +1,177 @@
+// Host side of the dense-tile family: planning (tile shape, K split, workspace carving), TMA
+// tensor maps, launches.
+#include "tile_dispatch.h"
+
+#include <cuda.h>
+
+#include <mutex>
+
+#include "tile_kernels.cuh"
+
+namespace b2sp {
+
+namespace {
+
+constexpr int kSMs = 148;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point query (no link against libcuda).
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+// Packed fp32 tensor [groups][rows][32] (column-blocked dense operand); box = [gbox][rbox][32].
+// `mn_major` selects the 128-byte swizzle in 32-byte units that MN-major tf32 MMA operands need;
+// otherwise the ordinary 128-byte swizzle (K-major operands).
+bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, int rbox, int gbox,
+                      bool mn_major)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {32, (cuuint64_t)rows, (cuuint64_t)groups};
+    cuuint64_t strides[2] = {128, (cuuint64_t)rows * 128};
+    cuuint32_t box[3] = {32, (cuuint32_t)rbox, (cuuint32_t)gbox};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE,
+               mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pick_split(int base_tiles, int Wk)
+{
+    int best = 1;
+    double best_eff = 0.0;
+    for (int ks = 1; ks <= 16 && ks <= Wk && Wk / ks >= 4; ++ks) {
+        long long items = (long long)base_tiles * ks;
+        double eff = (double)items / (double)((items + kSMs - 1) / kSMs * kSMs);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
+        if (eff >= 0.90) return ks;
+    }
+    return best;
+}
+
+template <int TN>
+b2sp_status launch_spmm_tile(const CUtensorMap &hi, const CUtensorMap &lo, const SpmmTileArgs &a, int items,
+                             cudaStream_t st)
+{
+    using Cfg = SpmmTileCfg<TN>;
+    auto kern = spmm_tile_kernel<TN>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+        return B2SP_ERR_CUDA;
+    kern<<<items, kTileThreads, Cfg::SMEM_BYTES, st>>>(hi, lo, a);
+    return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
+}
+
+}  // namespace
+
+bool tile_profitable(int M, int K, int width, long long nnz)
+{
+    if (M < 128 || K < 128 || width < 16 || nnz <= 0) return false;
+    double density = (double)nnz / ((double)M * (double)K);
+    return density >= 0.04;
+}
+
+TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
+{
+    TilePlan p;
+    if (M <= 0 || K <= 0 || N <= 0 || nnz <= 0) return p;
+    p.Wk = (K + kTileKC - 1) / kTileKC;
+    p.Kp = p.Wk * kTileKC;
+    int n32 = (N + 31) / 32 * 32;
+    p.TN = n32 >= 256 ? 256 : n32 >= 128 ? 128 : n32 >= 64 ? 64 : 32;
+    p.Nt = (n32 + p.TN - 1) / p.TN;
+    p.Np = p.Nt * p.TN;
+    p.Mt = (M + kTileM - 1) / kTileM;
+    size_t win_bytes = sizeof(int) * (size_t)M * (size_t)(p.Wk + 1);
+    if (win_bytes > (size_t)2 << 30) return p;  // pattern far too sparse / wide for dense tiles
+    p.KS = pick_split(p.Mt * p.Nt, p.Wk);
+    double per_window = (double)nnz / ((double)M * (double)p.Wk);
+    p.lanes = per_window <= 5.0 ? 8 : per_window <= 11.0 ? 16 : 32;
+    size_t off = align_up(base_off, 1024);
+    p.off_win = off;
+    off = align_up(off + win_bytes, 1024);
+    size_t dbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Np;
+    p.off_dhi = off;
+    off = align_up(off + dbytes, 1024);
+    p.off_dlo = off;
+    off = align_up(off + dbytes, 1024);
+    p.off_part = off;
+    if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * kTileM * (size_t)p.Np;
+    p.bytes = align_up(off, 256);
+    p.feasible = true;
+    return p;
+}
+
+b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, const int *row_ptr,
+                      const int *col_idx, const float *values, const float *D, long long ldd, float *O,
+                      long long ldo, void *workspace, cudaStream_t st, int *launches)
+{
+    (void)nnz;
+    char *ws = static_cast<char *>(workspace);
+    int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
+    int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
+    int *win = reinterpret_cast<int *>(ws + p.off_win);
+    float *dhi = reinterpret_cast<float *>(ws + p.off_dhi);
+    float *dlo = reinterpret_cast<float *>(ws + p.off_dlo);
+    float *part = reinterpret_cast<float *>(ws + p.off_part);
+
+    CUtensorMap tm_hi, tm_lo;
+    if (!make_blocked_map(&tm_hi, dhi, p.Kp, p.Np / 32, kTileKC, p.TN / 32, true) ||
+        !make_blocked_map(&tm_lo, dlo, p.Kp, p.Np / 32, kTileKC, p.TN / 32, true))
+        return B2SP_ERR_CUDA;
+
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
+    tile_windows_kernel<<<(M + 7) / 8, 256, 0, st>>>(M, K, p.Wk, row_ptr, col_idx, win, flags);
+    {
+        long long groups = (long long)p.Kp * (p.Np / 4);
+        int blocks = (int)((groups + 255) / 256 < (long long)kSMs * 8 ? (groups + 255) / 256 : (long long)kSMs * 8);
+        split_dense_kernel<<<blocks, 256, 0, st>>>(D, ldd, K, N, dhi, dlo, p.Kp, p.Np);
+    }
+    *launches += 2;
+    if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+
+    SpmmTileArgs a;
+    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.lanes_per_row = p.lanes;
+    a.col_idx = col_idx; a.values = values; a.win = win;
+    a.flags = flags; a.status = status;
+    if (p.KS == 1) { a.out = O; a.ld_out = ldo; a.slab = 0; }
+    else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kTileM * p.Np; }
+    int items = p.Mt * p.Nt * p.KS;
+    b2sp_status rc;
+    switch (p.TN) {
+    case 256: rc = launch_spmm_tile<256>(tm_hi, tm_lo, a, items, st); break;
+    case 128: rc = launch_spmm_tile<128>(tm_hi, tm_lo, a, items, st); break;
+    case 64: rc = launch_spmm_tile<64>(tm_hi, tm_lo, a, items, st); break;
+    default: rc = launch_spmm_tile<32>(tm_hi, tm_lo, a, items, st); break;
+    }
+    *launches += 1;
+    if (rc != B2SP_OK) return rc;
+    if (p.KS > 1) {
+        long long total = (long long)M * N;
+        int blocks = (int)((total + 255) / 256 < (long long)kSMs * 8 ? (total + 255) / 256 : (long long)kSMs * 8);
+        reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, O, ldo, flags);
+        *launches += 1;
+        if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+    }
+    return B2SP_OK;
+}
+
+}  // namespace b2sp

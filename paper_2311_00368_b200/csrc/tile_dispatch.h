@@ -1,0 +1,34 @@
+// Internal interface between the C-ABI entry points and the dense-tile (tensor-core) family.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+
+#include "../../include/b2sp.h"
+
+namespace b2sp {
+
+// Byte offsets inside the workspace header that both families agree on.
+constexpr size_t kWsStatusOffset = 256;      // int: device status word (0 = ok)
+constexpr size_t kWsTileFlagsOffset = 320;   // int[..]: flags written by the tile pre-pass
+constexpr size_t kWsHeaderBytes = 512;
+
+struct TilePlan {
+    bool feasible = false;
+    int TN = 0, Nt = 0, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0, lanes = 32;
+    size_t off_win = 0, off_dhi = 0, off_dlo = 0, off_part = 0;  // from the workspace base
+    size_t bytes = 0;                                           // total workspace bytes needed
+};
+
+// Plan for SPMM on the dense-tile family; `base_off` = first byte after the row family's region.
+TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off);
+
+// True when the dense-tile family is expected to beat the row family for these sizes.
+bool tile_profitable(int M, int K, int width, long long nnz);
+
+// Enqueues pre-pass + tile kernel (+ reduction).  The kernels leave immediately if the pre-pass
+// finds a row whose columns are not strictly increasing (flag at kWsTileFlagsOffset).
+b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, const int *row_ptr,
+                      const int *col_idx, const float *values, const float *D, long long ldd, float *O,
+                      long long ldo, void *workspace, cudaStream_t st, int *launches);
+
+}  // namespace b2sp

@@ -1,0 +1,308 @@
+// Dense-tile tensor-core kernels (tcgen05 / TMEM / TMA) for SPMM over CSR with 10-30% density.
+//
+// Idea: at these densities a 128 x 32 window of S is a dense tile with 70-90% zeros, and the
+// 5th-generation tensor cores multiply it by a dense D tile an order of magnitude faster than the
+// FP32 pipes can walk its nonzeros.  fp32 accuracy is kept by splitting every operand into two
+// tf32 numbers (x = hi + lo) and issuing three MMAs per product: hi*hi + lo*hi + hi*lo.
+//
+// Pieces:
+//   tile_windows_kernel   per row, the CSR position where each 32-column window starts (needs
+//                         strictly increasing columns in a row; sets a flag otherwise)
+//   split_dense_kernel    dense fp32 operand -> zero-padded (hi, lo) tf32 copies
+//   spmm_tile_kernel      one CTA per (128-row tile, TN-column tile, K split): a TMA warp streams D
+//                         tiles, four builder warps scatter the S window into swizzled shared memory,
+//                         one thread issues tcgen05.mma into a TMEM accumulator, the builders then
+//                         read the accumulator back and store it
+//   reduce_partials_kernel sums the K splits in fixed order
+//
+// Every mbarrier wait is bounded; a wait that gives up records B2SP_ERR_TIMEOUT's flag in the
+// workspace status word and the CTA leaves through the normal teardown (TMEM freed).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "ptx_sm100.cuh"
+
+namespace b2sp {
+
+constexpr int kTileM = 128;       // rows of S per CTA (UMMA M)
+constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-byte swizzle row of tf32)
+constexpr int kTileThreads = 192; // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: builders / epilogue
+constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
+
+// ---- window table -------------------------------------------------------------------------------
+// win[r*(Wk+1) + w] = first position p of row r with col_idx[p] >= 32*w  (w = 0..Wk; Wk = ceil(K/32)).
+__global__ void tile_windows_kernel(int M, int K, int Wk, const int *__restrict__ row_ptr,
+                                    const int *__restrict__ col_idx, int *__restrict__ win,
+                                    int *__restrict__ flags)
+{
+    const int lane = threadIdx.x & 31;
+    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= M) return;
+    const int beg = row_ptr[row], end = row_ptr[row + 1];
+    int *wp = win + (size_t)row * (Wk + 1);
+    if (end <= beg) {
+        for (int w = lane; w <= Wk; w += 32) wp[w] = beg;
+        return;
+    }
+    bool bad = false;
+    for (int p = beg + lane; p < end; p += 32) {
+        int c = col_idx[p];
+        int cprev = p > beg ? col_idx[p - 1] : -1;
+        bad |= c <= cprev || c >= K;
+        int w = min(max(c, 0) >> 5, Wk - 1);
+        int wprev = cprev < 0 ? -1 : min(cprev >> 5, Wk - 1);
+        for (int x = wprev + 1; x <= w; ++x) wp[x] = p;
+        if (p == end - 1)
+            for (int x = w + 1; x <= Wk; ++x) wp[x] = end;
+    }
+    if (bad) atomicExch(&flags[kFlagUnsorted], 1);
+}
+
+// ---- dense operand split ----------------------------------------------------------------------------
+// X [rows x cols] (ld) -> hi, lo in a column-blocked layout: element (r, c) lives at
+// ((c/32)*rows_p + r)*32 + c%32, i.e. [cols_p/32][rows_p][32] floats, zero in the padding
+// (rows_p >= rows, cols_p >= cols, cols_p % 32 == 0).  One 32-float group of a row is one
+// 128-byte swizzle row for TMA, and the whole thing is a plain packed 3-D tensor.
+__global__ void split_dense_kernel(const float *__restrict__ X, long long ld, int rows, int cols,
+                                   float *__restrict__ hi, float *__restrict__ lo, int rows_p, int cols_p)
+{
+    const long long groups = (long long)rows_p * (cols_p >> 2);  // float4 groups
+    for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
+         g += (long long)gridDim.x * blockDim.x) {
+        const int q = (int)(g & 7);                 // float4 inside the 32-float group
+        const long long rg = g >> 3;                // (column group, row) pair
+        const int r = (int)(rg % rows_p);
+        const int c = (int)(rg / rows_p) * 32 + q * 4;
+        uint32_t h[4] = {0, 0, 0, 0}, l[4] = {0, 0, 0, 0};
+        if (r < rows) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (c + i < cols) ptx::split_tf32(__ldg(X + (long long)r * ld + c + i), h[i], l[i]);
+        }
+        reinterpret_cast<uint4 *>(hi)[g] = make_uint4(h[0], h[1], h[2], h[3]);
+        reinterpret_cast<uint4 *>(lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+}
+
+// ---- K-split reduction ------------------------------------------------------------------------------
+__global__ void reduce_partials_kernel(const float *__restrict__ part, int KS, long long slab, int ldp,
+                                       int M, int N, float *__restrict__ O, long long ldo,
+                                       const int *__restrict__ flags)
+{
+    if (flags[kFlagUnsorted] != 0) return;
+    const long long total = (long long)M * N;
+    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
+         e += (long long)gridDim.x * blockDim.x) {
+        int i = (int)(e / N), n = (int)(e % N);
+        const float *p = part + (long long)i * ldp + n;
+        float acc = p[0];
+        for (int s = 1; s < KS; ++s) acc += p[(long long)s * slab];
+        O[(long long)i * ldo + n] = acc;
+    }
+}
+
+// ---- SPMM tile kernel ---------------------------------------------------------------------------------
+template <int TN>
+struct SpmmTileCfg {
+    static constexpr int S_BYTES = kTileM * kTileKC * 4;      // one S window tile (hi or lo): 16 KB
+    static constexpr int D_BYTES = kTileKC * TN * 4;          // one D tile (hi or lo)
+    static constexpr int STAGE_BYTES = 2 * S_BYTES + 2 * D_BYTES;
+    static constexpr int STAGES = (200 * 1024 / STAGE_BYTES) < 4 ? (200 * 1024 / STAGE_BYTES) : 4;
+    static constexpr int TMEM_COLS = TN < 32 ? 32 : TN;       // power of two >= 32
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct SpmmTileArgs {
+    int M, N, Wk, KS, Nt, lanes_per_row;
+    const int *col_idx;
+    const float *values;
+    const int *win;       // [M][Wk+1]
+    float *out;           // O (KS == 1) or the partial slabs
+    long long ld_out;     // leading dimension of `out`
+    long long slab;       // elements between K-split slabs (0 when KS == 1)
+    const int *flags;     // flags[kFlagUnsorted]
+    int *status;          // device status word (set to 1 on a wait that gave up)
+};
+
+template <int TN>
+__global__ void __launch_bounds__(kTileThreads, 1)
+spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
+                 const SpmmTileArgs a)
+{
+    using Cfg = SpmmTileCfg<TN>;
+    constexpr int STAGES = Cfg::STAGES;
+    if (a.flags[kFlagUnsorted] != 0) return;  // whole grid leaves; the row kernels take over
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t bar_base = smem_base + STAGES * Cfg::STAGE_BYTES;
+    auto full_d = [&](int s) { return bar_base + 8u * s; };
+    auto full_s = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto empty = [&](int s) { return bar_base + 8u * (2 * STAGES + s); };
+    const uint32_t acc_full = bar_base + 8u * (3 * STAGES);
+    volatile uint32_t *tmem_slot =
+        reinterpret_cast<volatile uint32_t *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 8 * (3 * STAGES + 1));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // work item
+    const int ks = blockIdx.x % a.KS;
+    const int tile = blockIdx.x / a.KS;
+    const int nt = tile % a.Nt, mt = tile / a.Nt;
+    const int w0 = (int)((long long)a.Wk * ks / a.KS), w1 = (int)((long long)a.Wk * (ks + 1) / a.KS);
+    const int nchunks = w1 - w0;
+    const int m0 = mt * kTileM, n0 = nt * TN;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(full_d(s), 1);
+            ptx::mbar_init(full_s(s), 4);
+            ptx::mbar_init(empty(s), 1);
+        }
+        ptx::mbar_init(acc_full, 1);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), Cfg::TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_acc = *tmem_slot;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ---------------- TMA producer: D_hi / D_lo tiles ----------------
+        if (lane == 0) {
+            ptx::tma_prefetch_desc(&tm_dhi);
+            ptx::tma_prefetch_desc(&tm_dlo);
+            int issued = 0;
+            for (int it = 0; it < nchunks; ++it) {
+                const int s = it % STAGES;
+                if (it >= STAGES && !ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1)) { failed = true; break; }
+                const uint32_t dst = smem_base + s * Cfg::STAGE_BYTES + 2 * Cfg::S_BYTES;
+                ptx::mbar_arrive_expect_tx(full_d(s), 2 * Cfg::D_BYTES);
+                ptx::tma_load_3d(dst, &tm_dhi, full_d(s), 0, (w0 + it) * kTileKC, nt * (TN / 32));
+                ptx::tma_load_3d(dst + Cfg::D_BYTES, &tm_dlo, full_d(s), 0, (w0 + it) * kTileKC, nt * (TN / 32));
+                issued = it + 1;
+            }
+            if (failed) {  // let the copies already in flight land before the CTA goes away
+                for (int it = issued > STAGES ? issued - STAGES : 0; it < issued; ++it)
+                    ptx::mbar_wait(full_d(it % STAGES), (it / STAGES) & 1);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_tf32(kTileM, TN, /*b_mn_major=*/true);
+            for (int it = 0; it < nchunks; ++it) {
+                const int s = it % STAGES;
+                const uint32_t par = (it / STAGES) & 1;
+                if (!ptx::mbar_wait(full_s(s), par) || !ptx::mbar_wait(full_d(s), par)) { failed = true; break; }
+                ptx::tc_fence_after_sync();
+                const uint32_t s_hi = smem_base + s * Cfg::STAGE_BYTES, s_lo = s_hi + Cfg::S_BYTES;
+                const uint32_t d_hi = s_lo + Cfg::S_BYTES, d_lo = d_hi + Cfg::D_BYTES;
+#pragma unroll
+                for (int k8 = 0; k8 < kTileKC / 8; ++k8) {
+                    // A: K-major, 128-byte swizzle rows, 8-row groups 1024 B apart; +32 B per K step of 8
+                    const uint64_t a_hi = ptx::smem_desc_sw128(s_hi + k8 * 32, 16, 1024);
+                    const uint64_t a_lo = ptx::smem_desc_sw128(s_lo + k8 * 32, 16, 1024);
+                    // B: MN-major tf32 (128-byte swizzle in 32-byte units): 32-float column groups
+                    // kTileKC*128 B apart, 4-row K groups 512 B apart; +1024 B per K step of 8 rows
+                    const uint64_t b_hi = ptx::smem_desc(d_hi + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
+                    const uint64_t b_lo = ptx::smem_desc(d_lo + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
+                    ptx::mma_tf32_ss(tmem_acc, a_hi, b_hi, idesc, (it | k8) != 0);
+                    ptx::mma_tf32_ss(tmem_acc, a_lo, b_hi, idesc, 1);
+                    ptx::mma_tf32_ss(tmem_acc, a_hi, b_lo, idesc, 1);
+                }
+                ptx::mma_commit(empty(s));
+            }
+            if (!failed) ptx::mma_commit(acc_full);
+        }
+    } else {
+        // ---------------- builders: scatter the S window into swizzled K-major tiles ----------------
+        const int b = warp - 2;  // rows 32b .. 32b+31 of the tile
+        const int L = a.lanes_per_row;
+        const int sub = lane / L, j = lane % L, rows_per_pass = 32 / L;
+        for (int it = 0; it < nchunks; ++it) {
+            const int s = it % STAGES;
+            bool ok = it < STAGES || ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1);
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }  // warp-uniform decision
+            uint8_t *s_hi = smem_gen + s * Cfg::STAGE_BYTES, *s_lo = s_hi + Cfg::S_BYTES;
+            {   // zero this warp's 32 rows (4 KB) of both tiles
+                uint4 z = make_uint4(0, 0, 0, 0);
+                uint4 *zh = reinterpret_cast<uint4 *>(s_hi + b * 4096) + lane;
+                uint4 *zl = reinterpret_cast<uint4 *>(s_lo + b * 4096) + lane;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { zh[i * 32] = z; zl[i * 32] = z; }
+            }
+            __syncwarp();
+            const int w = w0 + it;
+            for (int r0 = 0; r0 < 32; r0 += rows_per_pass) {
+                const int rt = b * 32 + r0 + sub;  // row inside the tile
+                const int grow = m0 + rt;
+                int beg = 0, end = 0;
+                if (grow < a.M) {
+                    const int *wp = a.win + (size_t)grow * (a.Wk + 1) + w;
+                    beg = __ldg(wp);
+                    end = __ldg(wp + 1);
+                }
+                for (int q = beg + j; q < end; q += L) {
+                    const int kk = __ldg(a.col_idx + q) - w * kTileKC;
+                    uint32_t hi, lo;
+                    ptx::split_tf32(__ldg(a.values + q), hi, lo);
+                    const uint32_t off = rt * 128 + ((((uint32_t)kk >> 2) ^ (rt & 7)) << 4) + ((kk & 3) << 2);
+                    *reinterpret_cast<uint32_t *>(s_hi + off) = hi;
+                    *reinterpret_cast<uint32_t *>(s_lo + off) = lo;
+                }
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(full_s(s));
+        }
+        // ---------------- epilogue: accumulator -> global ----------------
+        {
+            bool ok = !failed && ptx::mbar_wait(acc_full, 0);
+            failed = !__all_sync(0xffffffffu, ok);
+        }
+        if (!failed) {
+            ptx::tc_fence_after_sync();
+            const int q = warp & 3;                 // TMEM lane quarter this warp may access
+            const int grow = m0 + q * 32 + lane;
+            float *orow = a.out + (long long)ks * a.slab + (long long)grow * a.ld_out;
+            const bool vec = (a.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;
+#pragma unroll 1
+            for (int c = 0; c < TN / 32; ++c) {
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
+                ptx::tmem_ld_wait();
+                if (grow < a.M) {
+                    const int n = n0 + c * 32;
+                    if (vec && n + 32 <= a.N) {
+#pragma unroll
+                        for (int i = 0; i < 32; i += 4)
+                            *reinterpret_cast<uint4 *>(orow + n + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 32; ++i)
+                            if (n + i < a.N) orow[n + i] = __uint_as_float(r[i]);
+                    }
+                }
+            }
+        }
+    }
+    if (failed) atomicExch(a.status, 1);
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tmem_dealloc(tmem_acc, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace b2sp

@@ -1,0 +1,117 @@
+"""Parity of the dense-tile (tensor-core, 3xTF32) family against the CPU oracle, through the C ABI.
+Same gate as the row family: |gpu - ref| <= 1e-5 * T + 1e-6 elementwise."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2311_00368_b200 import workloads as W
+from tests.test_gpu_parity import DevProblem, _custom_rows, gate
+
+pytestmark = pytest.mark.gpu
+
+TILE = 3
+
+
+@pytest.fixture(scope="module")
+def b():
+    assert torch.cuda.is_available()
+    from paper_2311_00368_b200 import binding
+    return binding
+
+
+def _ws(b, op, p):
+    n = b.workspace_bytes(op, p.M, p.K, p.Kd, p.N, p.nnz)
+    big = max(n, 64 << 20)
+    return torch.empty(big, dtype=torch.uint8, device="cuda")
+
+
+def spmm_tile_check(b, p, expect_algo=TILE):
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_SPMM, p)
+    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+    out = torch.full((p.M, p.N), float("nan"), device="cuda")
+    b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=out, workspace=ws, algo=TILE)
+    assert b.last_algo(b.OP_SPMM) == expect_algo
+    assert b.device_status(ws) == 0, "a bounded wait inside the tile kernel gave up"
+    r = gate(out, ref, T, f"spmm tile {p.name} M={p.M} K={p.K} N={p.N}")
+    assert d.pattern_untouched()
+    return r
+
+
+@pytest.mark.parametrize("M,K,density,N,kind", [
+    (256, 256, 0.10, 64, "uniform"),     # tiny-config shape
+    (128, 128, 0.30, 32, "uniform"),     # one tile, one column group
+    (257, 333, 0.30, 128, "uniform"),    # ragged M and K (K not a multiple of 32)
+    (300, 512, 0.20, 100, "uniform"),    # N padded to 128 inside the scratch copy
+    (130, 1024, 0.25, 644, "uniform"),   # TN = 256, three column tiles, ragged last one
+    (512, 2048, 0.10, 256, "uniform"),   # several K splits
+    (384, 1024, 0.20, 256, "powerlaw"),  # skewed rows incl. full rows
+    (256, 512, 0.20, 128, "band"),
+    (200, 640, 0.05, 36, "uniform"),     # sparse windows (8 lanes per row), N = 36
+])
+def test_spmm_tile_shapes(b, M, K, density, N, kind):
+    p = W.small_random(2000 + M + N, M, K, density, 0, N, kind=kind)
+    spmm_tile_check(b, p)
+
+
+def test_spmm_tile_row_edges(b):
+    lens = [0, 1, 31, 32, 33, 0, 127, 128, 129, 255, 256, 257, 2048, 0, 2, 64] * 9  # 144 rows
+    p = _custom_rows(lens, 2048, 15, Kd=0, N=128)
+    spmm_tile_check(b, p)
+
+
+def test_spmm_tile_exact_on_small_integers(b):
+    """Integers are exact in tf32 hi parts, so the tensor-core result must equal the exact one."""
+    rng = np.random.default_rng(5)
+    p = W.small_random(77, 256, 256, 0.3, 0, 64)
+    p.values[:] = rng.integers(-4, 5, p.nnz).astype(np.float32)
+    p.D[:] = rng.integers(-8, 9, p.D.shape).astype(np.float32)
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_SPMM, p)
+    out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=TILE)
+    ref, _ = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), ref)
+
+
+def test_spmm_tile_falls_back_on_unsorted_rows(b):
+    """Rows that are not strictly increasing are detected by the pre-pass on the device; the row
+    kernels then produce the result within the same call."""
+    p = W.small_random(91, 256, 300, 0.3, 0, 128)
+    rng = np.random.default_rng(3)
+    ci, v = p.col_idx.copy(), p.values.copy()
+    a, e = p.row_ptr[5], p.row_ptr[6]
+    perm = a + rng.permutation(e - a)
+    ci[a:e], v[a:e] = ci[perm], v[perm]
+    ci[p.row_ptr[9] + 1] = ci[p.row_ptr[9]]  # a duplicate in another row
+    q = W.Problem("unsorted", p.M, p.K, p.row_ptr, ci, v, 0, p.N, None, None, p.D)
+    spmm_tile_check(b, q)
+
+
+def test_spmm_tile_hard_values(b):
+    """Wide dynamic range: the hi/lo split must hold for tiny and large magnitudes alike."""
+    p = W.small_random(123, 256, 512, 0.2, 0, 128)
+    rng = np.random.default_rng(9)
+    p.values[:] = (p.values * np.float32(10.0) ** rng.integers(-6, 7, p.nnz)).astype(np.float32)
+    p.D[:] = (p.D * np.float32(10.0) ** rng.integers(-6, 7, p.D.shape)).astype(np.float32)
+    spmm_tile_check(b, p)
+
+
+def test_spmm_tile_config_and_auto(b):
+    p = W.spmm_case()
+    r = spmm_tile_check(b, p)
+    assert r < 0.5  # 3xTF32 leaves a wide margin under the gate
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_SPMM, p)
+    out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=0)
+    assert b.last_algo(b.OP_SPMM) == TILE  # 20% density: the planner picks the dense-tile family
+    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+    gate(out, ref, T, "spmm auto")
+    # a workspace that only fits the row family makes AUTO use the row family
+    small = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
+    out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=small, algo=0)
+    assert b.last_algo(b.OP_SPMM) == 1
+    gate(out, ref, T, "spmm auto, small workspace")
+    with pytest.raises(b.B2spError) as e:
+        b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=small, algo=TILE)
+    assert e.value.status == 5
