@@ -193,11 +193,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr, uint32_t lbo_
 {
     return smem_desc(addr, lbo_bytes, sbo_bytes, kLayoutSw128);
 }
-// Instruction descriptor: tf32 x tf32 -> fp32, M x N tile, A K-major, B K-major or MN-major.
-__host__ __device__ constexpr uint32_t idesc_tf32(int M, int N, bool b_mn_major)
+// Instruction descriptor: tf32 x tf32 -> fp32, M x N tile; each operand K-major or MN-major.
+__host__ __device__ constexpr uint32_t idesc_tf32(int M, int N, bool a_mn_major, bool b_mn_major)
 {
-    return (1u << 4) | (2u << 7) | (2u << 10) | (0u << 15) | ((b_mn_major ? 1u : 0u) << 16) |
-           ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+    return (1u << 4) | (2u << 7) | (2u << 10) | ((a_mn_major ? 1u : 0u) << 15) |
+           ((b_mn_major ? 1u : 0u) << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 
 // ---- fp32 -> tf32 hi + tf32 lo ------------------------------------------------------------------------

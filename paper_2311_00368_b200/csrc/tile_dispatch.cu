@@ -68,15 +68,15 @@ int pick_split(int base_tiles, int Wk)
     return best;
 }
 
-template <int TN>
+template <int TR>
 b2sp_status launch_spmm_tile(const CUtensorMap &hi, const CUtensorMap &lo, const SpmmTileArgs &a, int items,
                              cudaStream_t st)
 {
-    using Cfg = SpmmTileCfg<TN>;
-    auto kern = spmm_tile_kernel<TN>;
+    using Cfg = SpmmTileCfg<TR>;
+    auto kern = spmm_tile_kernel<TR>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
-    kern<<<items, kTileThreads, Cfg::SMEM_BYTES, st>>>(hi, lo, a);
+    kern<<<items, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(hi, lo, a);
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 
@@ -95,16 +95,13 @@ TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
     if (M <= 0 || K <= 0 || N <= 0 || nnz <= 0) return p;
     p.Wk = (K + kTileKC - 1) / kTileKC;
     p.Kp = p.Wk * kTileKC;
-    int n32 = (N + 31) / 32 * 32;
-    p.TN = n32 >= 256 ? 256 : n32 >= 128 ? 128 : n32 >= 64 ? 64 : 32;
-    p.Nt = (n32 + p.TN - 1) / p.TN;
-    p.Np = p.Nt * p.TN;
-    p.Mt = (M + kTileM - 1) / kTileM;
+    p.Nt = (N + kTileN - 1) / kTileN;
+    p.Np = p.Nt * kTileN;
+    p.TR = M > 128 ? 256 : 128;   // rows of S per CTA (UMMA N)
+    p.Mt = (M + p.TR - 1) / p.TR;
     size_t win_bytes = sizeof(int) * (size_t)M * (size_t)(p.Wk + 1);
     if (win_bytes > (size_t)2 << 30) return p;  // pattern far too sparse / wide for dense tiles
     p.KS = pick_split(p.Mt * p.Nt, p.Wk);
-    double per_window = (double)nnz / ((double)M * (double)p.Wk);
-    p.lanes = per_window <= 5.0 ? 8 : per_window <= 11.0 ? 16 : 32;
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
     off = align_up(off + win_bytes, 1024);
@@ -114,7 +111,7 @@ TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
     p.off_dlo = off;
     off = align_up(off + dbytes, 1024);
     p.off_part = off;
-    if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * kTileM * (size_t)p.Np;
+    if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * p.TR * (size_t)p.Np;
     p.bytes = align_up(off, 256);
     p.feasible = true;
     return p;
@@ -124,7 +121,6 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
                       const int *col_idx, const float *values, const float *D, long long ldd, float *O,
                       long long ldo, void *workspace, cudaStream_t st, int *launches)
 {
-    (void)nnz;
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
@@ -134,12 +130,19 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
     float *part = reinterpret_cast<float *>(ws + p.off_part);
 
     CUtensorMap tm_hi, tm_lo;
-    if (!make_blocked_map(&tm_hi, dhi, p.Kp, p.Np / 32, kTileKC, p.TN / 32, true) ||
-        !make_blocked_map(&tm_lo, dlo, p.Kp, p.Np / 32, kTileKC, p.TN / 32, true))
+    if (!make_blocked_map(&tm_hi, dhi, p.Kp, p.Np / 32, kTileKC, kTileN / 32, true) ||
+        !make_blocked_map(&tm_lo, dlo, p.Kp, p.Np / 32, kTileKC, kTileN / 32, true))
         return B2SP_ERR_CUDA;
 
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
-    tile_windows_kernel<<<(M + 7) / 8, 256, 0, st>>>(M, K, p.Wk, row_ptr, col_idx, win, flags);
+    {
+        // threads per row from the mean row length (32..256)
+        long long avg = nnz / (M > 0 ? M : 1);
+        int G = avg >= 2048 ? 256 : avg >= 512 ? 128 : avg >= 128 ? 64 : 32;
+        long long threads = (long long)M * G;
+        tile_windows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, G, row_ptr, col_idx,
+                                                                                win, flags);
+    }
     {
         long long groups = (long long)p.Kp * (p.Np / 4);
         int blocks = (int)((groups + 255) / 256 < (long long)kSMs * 8 ? (groups + 255) / 256 : (long long)kSMs * 8);
@@ -149,19 +152,15 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
 
     SpmmTileArgs a;
-    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.lanes_per_row = p.lanes;
+    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
     a.col_idx = col_idx; a.values = values; a.win = win;
     a.flags = flags; a.status = status;
     if (p.KS == 1) { a.out = O; a.ld_out = ldo; a.slab = 0; }
-    else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kTileM * p.Np; }
+    else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * p.TR * p.Np; }
     int items = p.Mt * p.Nt * p.KS;
     b2sp_status rc;
-    switch (p.TN) {
-    case 256: rc = launch_spmm_tile<256>(tm_hi, tm_lo, a, items, st); break;
-    case 128: rc = launch_spmm_tile<128>(tm_hi, tm_lo, a, items, st); break;
-    case 64: rc = launch_spmm_tile<64>(tm_hi, tm_lo, a, items, st); break;
-    default: rc = launch_spmm_tile<32>(tm_hi, tm_lo, a, items, st); break;
-    }
+    if (p.TR == 256) rc = launch_spmm_tile<256>(tm_hi, tm_lo, a, items, st);
+    else rc = launch_spmm_tile<128>(tm_hi, tm_lo, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
     if (p.KS > 1) {

@@ -14,7 +14,7 @@ constexpr size_t kWsHeaderBytes = 512;
 
 struct TilePlan {
     bool feasible = false;
-    int TN = 0, Nt = 0, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0, lanes = 32;
+    int TR = 0, Nt = 0, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
     size_t off_win = 0, off_dhi = 0, off_dlo = 0, off_part = 0;  // from the workspace base
     size_t bytes = 0;                                           // total workspace bytes needed
 };

@@ -9,10 +9,10 @@
 //   tile_windows_kernel   per row, the CSR position where each 32-column window starts (needs
 //                         strictly increasing columns in a row; sets a flag otherwise)
 //   split_dense_kernel    dense fp32 operand -> zero-padded (hi, lo) tf32 copies
-//   spmm_tile_kernel      one CTA per (128-row tile, TN-column tile, K split): a TMA warp streams D
-//                         tiles, four builder warps scatter the S window into swizzled shared memory,
-//                         one thread issues tcgen05.mma into a TMEM accumulator, the builders then
-//                         read the accumulator back and store it
+//   spmm_tile_kernel      one CTA per (TR-row tile of S, 128-column tile of D/O, K split): a TMA warp
+//                         streams D tiles, builder warps scatter S windows into swizzled shared
+//                         memory, one thread issues tcgen05.mma into a TMEM accumulator, four warps
+//                         then read the accumulator back and store it
 //   reduce_partials_kernel sums the K splits in fixed order
 //
 // Every mbarrier wait is bounded; a wait that gives up records B2SP_ERR_TIMEOUT's flag in the
@@ -26,33 +26,32 @@
 
 namespace b2sp {
 
-constexpr int kTileM = 128;       // rows of S per CTA (UMMA M)
 constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-byte swizzle row of tf32)
-constexpr int kTileThreads = 192; // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: builders / epilogue
 constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
 
 // ---- window table -------------------------------------------------------------------------------
 // win[r*(Wk+1) + w] = first position p of row r with col_idx[p] >= 32*w  (w = 0..Wk; Wk = ceil(K/32)).
-__global__ void tile_windows_kernel(int M, int K, int Wk, const int *__restrict__ row_ptr,
+__global__ void tile_windows_kernel(int M, int K, int Wk, int G, const int *__restrict__ row_ptr,
                                     const int *__restrict__ col_idx, int *__restrict__ win,
                                     int *__restrict__ flags)
 {
-    const int lane = threadIdx.x & 31;
-    const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // G threads (a power of two, 32..256, dividing blockDim.x) share a row
+    const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const int row = (int)(gt / G), j = (int)(gt % G);
     if (row >= M) return;
     const int beg = row_ptr[row], end = row_ptr[row + 1];
     int *wp = win + (size_t)row * (Wk + 1);
     if (end <= beg) {
-        for (int w = lane; w <= Wk; w += 32) wp[w] = beg;
+        for (int w = j; w <= Wk; w += G) wp[w] = beg;
         return;
     }
     bool bad = false;
-    for (int p = beg + lane; p < end; p += 32) {
-        int c = col_idx[p];
-        int cprev = p > beg ? col_idx[p - 1] : -1;
+    for (int p = beg + j; p < end; p += G) {
+        const int c = __ldg(col_idx + p);
+        const int cprev = p > beg ? __ldg(col_idx + p - 1) : -1;
         bad |= c <= cprev || c >= K;
-        int w = min(max(c, 0) >> 5, Wk - 1);
-        int wprev = cprev < 0 ? -1 : min(cprev >> 5, Wk - 1);
+        const int w = min(max(c, 0) >> 5, Wk - 1);
+        const int wprev = cprev < 0 ? -1 : min(cprev >> 5, Wk - 1);
         for (int x = wprev + 1; x <= w; ++x) wp[x] = p;
         if (p == end - 1)
             for (int x = w + 1; x <= Wk; ++x) wp[x] = end;
@@ -104,18 +103,32 @@ __global__ void reduce_partials_kernel(const float *__restrict__ part, int KS, l
 }
 
 // ---- SPMM tile kernel ---------------------------------------------------------------------------------
-template <int TN>
+// Computes O^T tiles: UMMA M = 128 columns of D/O, UMMA N = TR rows of S, K = 32 columns of S per
+// stage.  A operand = D tile (MN-major tf32, streamed by TMA from the blocked hi/lo copies),
+// B operand = S window tile (K-major, built here from CSR).  The streamed operand is the narrow one,
+// so the L2 -> SM traffic per flop is half of what a 128-row S tile would need.
+//
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, then STAGES builder groups of
+// TR/32 warps; group g owns pipeline slot g.  Stages are independent thanks to the window table, so
+// the groups build different stages concurrently, and each warp prefetches its next window bounds
+// while it works on the current stage.  Group 0's first four warps run the epilogue.
+constexpr int kTileN = 128;  // columns of D / O per CTA (UMMA M)
+
+template <int TR>
 struct SpmmTileCfg {
-    static constexpr int S_BYTES = kTileM * kTileKC * 4;      // one S window tile (hi or lo): 16 KB
-    static constexpr int D_BYTES = kTileKC * TN * 4;          // one D tile (hi or lo)
+    static constexpr int S_BYTES = TR * kTileKC * 4;          // one S window tile (hi or lo)
+    static constexpr int D_BYTES = kTileKC * kTileN * 4;      // one D tile (hi or lo): 16 KB
     static constexpr int STAGE_BYTES = 2 * S_BYTES + 2 * D_BYTES;
-    static constexpr int STAGES = (200 * 1024 / STAGE_BYTES) < 4 ? (200 * 1024 / STAGE_BYTES) : 4;
-    static constexpr int TMEM_COLS = TN < 32 ? 32 : TN;       // power of two >= 32
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int STAGES = TR == 256 ? 2 : 3;
+    static constexpr int GROUP_WARPS = TR / 32;
+    static constexpr int THREADS = (2 + STAGES * GROUP_WARPS) * 32;
+    static constexpr int TMEM_COLS = TR;                      // power of two >= 32
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
+                                      STAGES * GROUP_WARPS * 128 /*pass tables*/;
 };
 
 struct SpmmTileArgs {
-    int M, N, Wk, KS, Nt, lanes_per_row;
+    int M, N, Wk, KS, Nt;
     const int *col_idx;
     const float *values;
     const int *win;       // [M][Wk+1]
@@ -126,12 +139,12 @@ struct SpmmTileArgs {
     int *status;          // device status word (set to 1 on a wait that gave up)
 };
 
-template <int TN>
-__global__ void __launch_bounds__(kTileThreads, 1)
+template <int TR>
+__global__ void __launch_bounds__(SpmmTileCfg<TR>::THREADS, 1)
 spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
                  const SpmmTileArgs a)
 {
-    using Cfg = SpmmTileCfg<TN>;
+    using Cfg = SpmmTileCfg<TR>;
     constexpr int STAGES = Cfg::STAGES;
     if (a.flags[kFlagUnsorted] != 0) return;  // whole grid leaves; the row kernels take over
 
@@ -154,12 +167,12 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
     const int nt = tile % a.Nt, mt = tile / a.Nt;
     const int w0 = (int)((long long)a.Wk * ks / a.KS), w1 = (int)((long long)a.Wk * (ks + 1) / a.KS);
     const int nchunks = w1 - w0;
-    const int m0 = mt * kTileM, n0 = nt * TN;
+    const int m0 = mt * TR, n0 = nt * kTileN;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(full_d(s), 1);
-            ptx::mbar_init(full_s(s), 4);
+            ptx::mbar_init(full_s(s), Cfg::GROUP_WARPS);
             ptx::mbar_init(empty(s), 1);
         }
         ptx::mbar_init(acc_full, 1);
@@ -187,8 +200,8 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
                 if (it >= STAGES && !ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1)) { failed = true; break; }
                 const uint32_t dst = smem_base + s * Cfg::STAGE_BYTES + 2 * Cfg::S_BYTES;
                 ptx::mbar_arrive_expect_tx(full_d(s), 2 * Cfg::D_BYTES);
-                ptx::tma_load_3d(dst, &tm_dhi, full_d(s), 0, (w0 + it) * kTileKC, nt * (TN / 32));
-                ptx::tma_load_3d(dst + Cfg::D_BYTES, &tm_dlo, full_d(s), 0, (w0 + it) * kTileKC, nt * (TN / 32));
+                ptx::tma_load_3d(dst, &tm_dhi, full_d(s), 0, (w0 + it) * kTileKC, nt * (kTileN / 32));
+                ptx::tma_load_3d(dst + Cfg::D_BYTES, &tm_dlo, full_d(s), 0, (w0 + it) * kTileKC, nt * (kTileN / 32));
                 issued = it + 1;
             }
             if (failed) {  // let the copies already in flight land before the CTA goes away
@@ -199,7 +212,8 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_tf32(kTileM, TN, /*b_mn_major=*/true);
+            // A = D tile: MN-major; B = S tile: K-major
+            constexpr uint32_t idesc = ptx::idesc_tf32(kTileN, TR, /*a_mn_major=*/true, /*b_mn_major=*/false);
             for (int it = 0; it < nchunks; ++it) {
                 const int s = it % STAGES;
                 const uint32_t par = (it / STAGES) & 1;
@@ -209,88 +223,136 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
                 const uint32_t d_hi = s_lo + Cfg::S_BYTES, d_lo = d_hi + Cfg::D_BYTES;
 #pragma unroll
                 for (int k8 = 0; k8 < kTileKC / 8; ++k8) {
-                    // A: K-major, 128-byte swizzle rows, 8-row groups 1024 B apart; +32 B per K step of 8
-                    const uint64_t a_hi = ptx::smem_desc_sw128(s_hi + k8 * 32, 16, 1024);
-                    const uint64_t a_lo = ptx::smem_desc_sw128(s_lo + k8 * 32, 16, 1024);
-                    // B: MN-major tf32 (128-byte swizzle in 32-byte units): 32-float column groups
+                    // S: K-major, 128-byte swizzle rows, 8-row groups 1024 B apart; +32 B per K step of 8
+                    const uint64_t b_hi = ptx::smem_desc(s_hi + k8 * 32, 16, 1024, ptx::kLayoutSw128);
+                    const uint64_t b_lo = ptx::smem_desc(s_lo + k8 * 32, 16, 1024, ptx::kLayoutSw128);
+                    // D: MN-major tf32 (128-byte swizzle in 32-byte units): 32-float column groups
                     // kTileKC*128 B apart, 4-row K groups 512 B apart; +1024 B per K step of 8 rows
-                    const uint64_t b_hi = ptx::smem_desc(d_hi + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
-                    const uint64_t b_lo = ptx::smem_desc(d_lo + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
+                    const uint64_t a_hi = ptx::smem_desc(d_hi + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
+                    const uint64_t a_lo = ptx::smem_desc(d_lo + k8 * 1024, kTileKC * 128, 512, ptx::kLayoutSw128Base32);
                     ptx::mma_tf32_ss(tmem_acc, a_hi, b_hi, idesc, (it | k8) != 0);
-                    ptx::mma_tf32_ss(tmem_acc, a_lo, b_hi, idesc, 1);
                     ptx::mma_tf32_ss(tmem_acc, a_hi, b_lo, idesc, 1);
+                    ptx::mma_tf32_ss(tmem_acc, a_lo, b_hi, idesc, 1);
                 }
                 ptx::mma_commit(empty(s));
             }
             if (!failed) ptx::mma_commit(acc_full);
         }
     } else {
-        // ---------------- builders: scatter the S window into swizzled K-major tiles ----------------
-        const int b = warp - 2;  // rows 32b .. 32b+31 of the tile
-        const int L = a.lanes_per_row;
-        const int sub = lane / L, j = lane % L, rows_per_pass = 32 / L;
-        for (int it = 0; it < nchunks; ++it) {
-            const int s = it % STAGES;
-            bool ok = it < STAGES || ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1);
-            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }  // warp-uniform decision
-            uint8_t *s_hi = smem_gen + s * Cfg::STAGE_BYTES, *s_lo = s_hi + Cfg::S_BYTES;
-            {   // zero this warp's 32 rows (4 KB) of both tiles
-                uint4 z = make_uint4(0, 0, 0, 0);
-                uint4 *zh = reinterpret_cast<uint4 *>(s_hi + b * 4096) + lane;
-                uint4 *zl = reinterpret_cast<uint4 *>(s_lo + b * 4096) + lane;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) { zh[i * 32] = z; zl[i * 32] = z; }
+        // ---------------- builders: scatter S windows into swizzled K-major tiles ----------------
+        // Per stage a warp owns 32 rows.  Lane l first holds the window bounds of row l; rows are then
+        // sorted into "long" (more than 16 entries in the window: one pass of 32 lanes) and "short"
+        // (1..16 entries: two rows per pass), empty rows are skipped.  The pass list goes through a
+        // 32-entry shared-memory table per warp; all global loads of up to kPassRound passes are
+        // issued before the first one is consumed.
+        constexpr int kPassRound = 24;
+        const int g = (warp - 2) / Cfg::GROUP_WARPS;   // builder group = pipeline slot
+        const int bw = (warp - 2) % Cfg::GROUP_WARPS;  // rows 32*bw .. 32*bw+31 of the tile
+        uint8_t *s_hi = smem_gen + g * Cfg::STAGE_BYTES, *s_lo = s_hi + Cfg::S_BYTES;
+        volatile int *order = reinterpret_cast<volatile int *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 256) +
+                              (warp - 2) * 32;
+        const int my_row = m0 + bw * 32 + lane;        // the row whose window bounds this lane fetches
+        const int *my_win = a.win + (size_t)(my_row < a.M ? my_row : 0) * (a.Wk + 1) + w0;
+        const unsigned lt_mask = (1u << lane) - 1u;
+        int nb = 0, ne = 0;
+        if (my_row < a.M && g < nchunks) { nb = __ldg(my_win + g); ne = __ldg(my_win + g + 1); }
+        for (int it = g; it < nchunks; it += STAGES) {
+            const int cb = nb, ce = ne;
+            nb = ne = 0;
+            if (my_row < a.M && it + STAGES < nchunks) {   // bounds of this warp's next stage
+                nb = __ldg(my_win + it + STAGES);
+                ne = __ldg(my_win + it + STAGES + 1);
             }
+            const int cnt = ce - cb;
+            const unsigned long_m = __ballot_sync(0xffffffffu, cnt > 16);
+            const unsigned short_m = __ballot_sync(0xffffffffu, cnt > 0 && cnt <= 16);
+            const int nlong = __popc(long_m), nshort = __popc(short_m);
             __syncwarp();
-            const int w = w0 + it;
-            for (int r0 = 0; r0 < 32; r0 += rows_per_pass) {
-                const int rt = b * 32 + r0 + sub;  // row inside the tile
-                const int grow = m0 + rt;
-                int beg = 0, end = 0;
-                if (grow < a.M) {
-                    const int *wp = a.win + (size_t)grow * (a.Wk + 1) + w;
-                    beg = __ldg(wp);
-                    end = __ldg(wp + 1);
+            if (cnt > 16) order[__popc(long_m & lt_mask)] = lane;
+            else if (cnt > 0) order[nlong + __popc(short_m & lt_mask)] = lane;
+            __syncwarp();
+            const int npass = nlong + ((nshort + 1) >> 1);
+            const int kbase = (w0 + it) * kTileKC;
+            bool slot_ready = false;
+            for (int base = 0; base < npass || !slot_ready; base += kPassRound) {
+                int col[kPassRound];
+                float val[kPassRound];
+#pragma unroll
+                for (int p = 0; p < kPassRound; ++p) {
+                    const int pp = base + p;
+                    col[p] = -1;
+                    val[p] = 0.f;
+                    if (pp < npass) {   // warp-uniform
+                        int idx, jj;
+                        if (pp < nlong) { idx = pp; jj = lane; }
+                        else { idx = nlong + 2 * (pp - nlong) + (lane >> 4); jj = lane & 15; }
+                        const bool have = idx < nlong + nshort;
+                        const int r = have ? order[idx] : 0;
+                        const int q = __shfl_sync(0xffffffffu, cb, r) + jj;   // all lanes take part
+                        const int e0 = __shfl_sync(0xffffffffu, ce, r);
+                        const int e = have ? e0 : 0;
+                        if (q < e) {
+                            col[p] = __ldg(a.col_idx + q);
+                            val[p] = __ldg(a.values + q);
+                        }
+                    }
                 }
-                for (int q = beg + j; q < end; q += L) {
-                    const int kk = __ldg(a.col_idx + q) - w * kTileKC;
-                    uint32_t hi, lo;
-                    ptx::split_tf32(__ldg(a.values + q), hi, lo);
-                    const uint32_t off = rt * 128 + ((((uint32_t)kk >> 2) ^ (rt & 7)) << 4) + ((kk & 3) << 2);
-                    *reinterpret_cast<uint32_t *>(s_hi + off) = hi;
-                    *reinterpret_cast<uint32_t *>(s_lo + off) = lo;
+                if (!slot_ready) {
+                    // the slot must have been drained by the MMAs of its previous use
+                    const int use = it / STAGES;
+                    bool ok = use == 0 || ptx::mbar_wait(empty(g), (use - 1) & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                    // zero this warp's 32 rows (4 KB) of both tiles
+                    uint4 z = make_uint4(0, 0, 0, 0);
+                    uint4 *zh = reinterpret_cast<uint4 *>(s_hi + bw * 4096) + lane;
+                    uint4 *zl = reinterpret_cast<uint4 *>(s_lo + bw * 4096) + lane;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) { zh[i * 32] = z; zl[i * 32] = z; }
+                    __syncwarp();
+                    slot_ready = true;
+                }
+#pragma unroll
+                for (int p = 0; p < kPassRound; ++p) {
+                    const int pp = base + p;
+                    if (pp < npass && col[p] >= 0) {
+                        const int idx = pp < nlong ? pp : nlong + 2 * (pp - nlong) + (lane >> 4);
+                        const int rt = bw * 32 + order[idx];
+                        const uint32_t kk = (uint32_t)(col[p] - kbase);
+                        uint32_t hi, lo;
+                        ptx::split_tf32(val[p], hi, lo);
+                        const uint32_t off = rt * 128 + (((kk >> 2) ^ (rt & 7)) << 4) + ((kk & 3) << 2);
+                        *reinterpret_cast<uint32_t *>(s_hi + off) = hi;
+                        *reinterpret_cast<uint32_t *>(s_lo + off) = lo;
+                    }
                 }
             }
+            if (failed) break;
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(full_s(s));
+            if (lane == 0) ptx::mbar_arrive(full_s(g));
         }
-        // ---------------- epilogue: accumulator -> global ----------------
-        {
-            bool ok = !failed && ptx::mbar_wait(acc_full, 0);
-            failed = !__all_sync(0xffffffffu, ok);
-        }
-        if (!failed) {
-            ptx::tc_fence_after_sync();
-            const int q = warp & 3;                 // TMEM lane quarter this warp may access
-            const int grow = m0 + q * 32 + lane;
-            float *orow = a.out + (long long)ks * a.slab + (long long)grow * a.ld_out;
-            const bool vec = (a.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;
+        // ---------------- epilogue (first four builder warps): accumulator -> global ----------------
+        if (warp < 6) {
+            {
+                bool ok = !failed && ptx::mbar_wait(acc_full, 0);
+                failed = !__all_sync(0xffffffffu, ok);
+            }
+            if (!failed) {
+                ptx::tc_fence_after_sync();
+                const int q = warp & 3;                 // TMEM lane quarter this warp may access
+                const int n = n0 + q * 32 + lane;       // O column held by this lane
+                float *obase = a.out + (long long)ks * a.slab + n;
 #pragma unroll 1
-            for (int c = 0; c < TN / 32; ++c) {
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
-                ptx::tmem_ld_wait();
-                if (grow < a.M) {
-                    const int n = n0 + c * 32;
-                    if (vec && n + 32 <= a.N) {
+                for (int c = 0; c < TR / 32; ++c) {
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(tmem_acc + ((uint32_t)(q * 32) << 16) + c * 32, r);
+                    ptx::tmem_ld_wait();
+                    if (n < a.N) {
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            *reinterpret_cast<uint4 *>(orow + n + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-                    } else {
-#pragma unroll
-                        for (int i = 0; i < 32; ++i)
-                            if (n + i < a.N) orow[n + i] = __uint_as_float(r[i]);
+                        for (int i = 0; i < 32; ++i) {
+                            const int row = m0 + c * 32 + i;
+                            if (row < a.M) obase[(long long)row * a.ld_out] = __uint_as_float(r[i]);
+                        }
                     }
                 }
             }
