@@ -16,7 +16,7 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libb2sp.so")
+LIB_PATH = os.environ.get("B2SP_LIB") or os.path.join(_HERE, "libb2sp.so")  # B2SP_LIB: alternate build
 
 ALGO_AUTO, ALGO_ROW, ALGO_ROW_NAT, ALGO_TILE = 0, 1, 2, 3
 OP_SPMM, OP_SDDMM, OP_FUSEDMM = 0, 1, 2

@@ -99,7 +99,7 @@ TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
     p.Np = p.Nt * kTileN;
     p.TR = M > 128 ? 256 : 128;   // rows of S per CTA (UMMA N)
     p.Mt = (M + p.TR - 1) / p.TR;
-    size_t win_bytes = sizeof(int) * (size_t)M * (size_t)(p.Wk + 1);
+    size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30) return p;  // pattern far too sparse / wide for dense tiles
     p.KS = pick_split(p.Mt * p.Nt, p.Wk);
     size_t off = align_up(base_off, 1024);
@@ -124,7 +124,7 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
-    int *win = reinterpret_cast<int *>(ws + p.off_win);
+    int2 *win = reinterpret_cast<int2 *>(ws + p.off_win);
     float *dhi = reinterpret_cast<float *>(ws + p.off_dhi);
     float *dlo = reinterpret_cast<float *>(ws + p.off_dlo);
     float *part = reinterpret_cast<float *>(ws + p.off_part);
@@ -135,13 +135,14 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
         return B2SP_ERR_CUDA;
 
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
+    if (cudaMemsetAsync(win, 0, sizeof(int2) * (size_t)M * (size_t)p.Wk, st) != cudaSuccess) return B2SP_ERR_CUDA;
     {
         // threads per row from the mean row length (32..256)
         long long avg = nnz / (M > 0 ? M : 1);
         int G = avg >= 2048 ? 256 : avg >= 512 ? 128 : avg >= 128 ? 64 : 32;
         long long threads = (long long)M * G;
-        tile_windows_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, G, row_ptr, col_idx,
-                                                                                win, flags);
+        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, G, row_ptr, col_idx, win,
+                                                                              flags);
     }
     {
         long long groups = (long long)p.Kp * (p.Np / 4);
@@ -152,9 +153,10 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
 
     SpmmTileArgs a;
-    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
+    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.nnz = (int)nnz;
     a.col_idx = col_idx; a.values = values; a.win = win;
     a.flags = flags; a.status = status;
+    a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (p.KS == 1) { a.out = O; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * p.TR * p.Np; }
     int items = p.Mt * p.Nt * p.KS;

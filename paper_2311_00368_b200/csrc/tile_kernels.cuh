@@ -6,8 +6,8 @@
 // tf32 numbers (x = hi + lo) and issuing three MMAs per product: hi*hi + lo*hi + hi*lo.
 //
 // Pieces:
-//   tile_windows_kernel   per row, the CSR position where each 32-column window starts (needs
-//                         strictly increasing columns in a row; sets a flag otherwise)
+//   tile_masks_kernel     per row and 32-column window: first CSR position + occupancy bit mask
+//                         (needs strictly increasing columns in a row; sets a flag otherwise)
 //   split_dense_kernel    dense fp32 operand -> zero-padded (hi, lo) tf32 copies
 //   spmm_tile_kernel      one CTA per (TR-row tile of S, 128-column tile of D/O, K split): a TMA warp
 //                         streams D tiles, builder warps scatter S windows into swizzled shared
@@ -24,37 +24,57 @@
 
 #include "ptx_sm100.cuh"
 
+// Optional in-kernel timing of the pipeline roles (build with -DB2SP_TILE_PROFILE): per-CTA cycle
+// totals are added into args.prof[0..15].
+#ifdef B2SP_TILE_PROFILE
+#define B2SP_PROF_DECL long long prof_t0 = 0, prof_acc[4] = {0, 0, 0, 0};
+#define B2SP_PROF_START prof_t0 = clock64();
+#define B2SP_PROF_STOP(i) { long long t_ = clock64(); prof_acc[i] += t_ - prof_t0; prof_t0 = t_; }
+#define B2SP_PROF_FLUSH(base) { if (lane == 0 && a.prof) { for (int i_ = 0; i_ < 4; ++i_) atomicAdd(a.prof + (base) + i_, (unsigned long long)prof_acc[i_]); } }
+#else
+#define B2SP_PROF_DECL
+#define B2SP_PROF_START
+#define B2SP_PROF_STOP(i) {}
+#define B2SP_PROF_FLUSH(base) {}
+#endif
+
 namespace b2sp {
 
 constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-byte swizzle row of tf32)
 constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
 
 // ---- window table -------------------------------------------------------------------------------
-// win[r*(Wk+1) + w] = first position p of row r with col_idx[p] >= 32*w  (w = 0..Wk; Wk = ceil(K/32)).
-__global__ void tile_windows_kernel(int M, int K, int Wk, int G, const int *__restrict__ row_ptr,
-                                    const int *__restrict__ col_idx, int *__restrict__ win,
-                                    int *__restrict__ flags)
+// T[r*Wk + w] = (first CSR position of row r inside column window [32w, 32w+32), occupancy bit mask of
+// that window: bit b set <=> column 32w+b is stored).  The table must be zeroed before the kernel
+// runs; windows without entries keep mask 0.  Needs strictly increasing columns inside a row (then a
+// window's entries are contiguous and at most 32); anything else sets flags[kFlagUnsorted].
+__global__ void tile_masks_kernel(int M, int K, int Wk, int G, const int *__restrict__ row_ptr,
+                                  const int *__restrict__ col_idx, int2 *__restrict__ T,
+                                  int *__restrict__ flags)
 {
-    // G threads (a power of two, 32..256, dividing blockDim.x) share a row
+    // G threads (a power of two, 32..256, dividing blockDim.x) share a row; a warp never spans rows
     const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const int row = (int)(gt / G), j = (int)(gt % G);
     if (row >= M) return;
     const int beg = row_ptr[row], end = row_ptr[row + 1];
-    int *wp = win + (size_t)row * (Wk + 1);
-    if (end <= beg) {
-        for (int w = j; w <= Wk; w += G) wp[w] = beg;
-        return;
-    }
+    int2 *tr = T + (size_t)row * Wk;
     bool bad = false;
-    for (int p = beg + j; p < end; p += G) {
-        const int c = __ldg(col_idx + p);
-        const int cprev = p > beg ? __ldg(col_idx + p - 1) : -1;
-        bad |= c <= cprev || c >= K;
-        const int w = min(max(c, 0) >> 5, Wk - 1);
-        const int wprev = cprev < 0 ? -1 : min(cprev >> 5, Wk - 1);
-        for (int x = wprev + 1; x <= w; ++x) wp[x] = p;
-        if (p == end - 1)
-            for (int x = w + 1; x <= Wk; ++x) wp[x] = end;
+    for (int p0 = beg + (j & ~31); p0 < end; p0 += G) {   // warp-uniform trip count
+        const int p = p0 + (j & 31);
+        const bool live = p < end;
+        int c = 0, cprev = -1;
+        if (live) {
+            c = __ldg(col_idx + p);
+            if (p > beg) cprev = __ldg(col_idx + p - 1);
+            bad |= c <= cprev || c >= K || c < 0;
+        }
+        const int w = live ? min(max(c, 0) >> 5, Wk - 1) : -1 - (j & 31);   // dead lanes match nobody
+        const unsigned peers = __match_any_sync(0xffffffffu, w);
+        const unsigned bits = __reduce_or_sync(peers, live ? 1u << (c & 31) : 0u);
+        if (live) {
+            if ((unsigned)(j & 31) == (unsigned)(__ffs(peers) - 1)) atomicOr(reinterpret_cast<unsigned *>(&tr[w].y), bits);
+            if (cprev < 0 || (cprev >> 5) != w) tr[w].x = p;   // first entry of its window
+        }
     }
     if (bad) atomicExch(&flags[kFlagUnsorted], 1);
 }
@@ -124,19 +144,21 @@ struct SpmmTileCfg {
     static constexpr int THREADS = (2 + STAGES * GROUP_WARPS) * 32;
     static constexpr int TMEM_COLS = TR;                      // power of two >= 32
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                      STAGES * GROUP_WARPS * 128 /*pass tables*/;
+                                      STAGES * GROUP_WARPS * 256 /*pass tables*/;
 };
 
 struct SpmmTileArgs {
     int M, N, Wk, KS, Nt;
+    int nnz;
     const int *col_idx;
     const float *values;
-    const int *win;       // [M][Wk+1]
+    const int2 *win;      // [M][Wk]: (first position, occupancy mask) per row and window
     float *out;           // O (KS == 1) or the partial slabs
     long long ld_out;     // leading dimension of `out`
     long long slab;       // elements between K-split slabs (0 when KS == 1)
     const int *flags;     // flags[kFlagUnsorted]
     int *status;          // device status word (set to 1 on a wait that gave up)
+    unsigned long long *prof;  // optional role timers (only read when built with B2SP_TILE_PROFILE)
 };
 
 template <int TR>
@@ -195,15 +217,20 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
             ptx::tma_prefetch_desc(&tm_dhi);
             ptx::tma_prefetch_desc(&tm_dlo);
             int issued = 0;
+            B2SP_PROF_DECL
+            B2SP_PROF_START
             for (int it = 0; it < nchunks; ++it) {
                 const int s = it % STAGES;
                 if (it >= STAGES && !ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1)) { failed = true; break; }
+                B2SP_PROF_STOP(0)
                 const uint32_t dst = smem_base + s * Cfg::STAGE_BYTES + 2 * Cfg::S_BYTES;
                 ptx::mbar_arrive_expect_tx(full_d(s), 2 * Cfg::D_BYTES);
                 ptx::tma_load_3d(dst, &tm_dhi, full_d(s), 0, (w0 + it) * kTileKC, nt * (kTileN / 32));
                 ptx::tma_load_3d(dst + Cfg::D_BYTES, &tm_dlo, full_d(s), 0, (w0 + it) * kTileKC, nt * (kTileN / 32));
                 issued = it + 1;
+                B2SP_PROF_STOP(1)
             }
+            B2SP_PROF_FLUSH(0)
             if (failed) {  // let the copies already in flight land before the CTA goes away
                 for (int it = issued > STAGES ? issued - STAGES : 0; it < issued; ++it)
                     ptx::mbar_wait(full_d(it % STAGES), (it / STAGES) & 1);
@@ -214,10 +241,15 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
         if (lane == 0) {
             // A = D tile: MN-major; B = S tile: K-major
             constexpr uint32_t idesc = ptx::idesc_tf32(kTileN, TR, /*a_mn_major=*/true, /*b_mn_major=*/false);
+            B2SP_PROF_DECL
+            B2SP_PROF_START
             for (int it = 0; it < nchunks; ++it) {
                 const int s = it % STAGES;
                 const uint32_t par = (it / STAGES) & 1;
-                if (!ptx::mbar_wait(full_s(s), par) || !ptx::mbar_wait(full_d(s), par)) { failed = true; break; }
+                if (!ptx::mbar_wait(full_s(s), par)) { failed = true; break; }
+                B2SP_PROF_STOP(0)
+                if (!ptx::mbar_wait(full_d(s), par)) { failed = true; break; }
+                B2SP_PROF_STOP(1)
                 ptx::tc_fence_after_sync();
                 const uint32_t s_hi = smem_base + s * Cfg::STAGE_BYTES, s_lo = s_hi + Cfg::S_BYTES;
                 const uint32_t d_hi = s_lo + Cfg::S_BYTES, d_lo = d_hi + Cfg::D_BYTES;
@@ -235,102 +267,69 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
                     ptx::mma_tf32_ss(tmem_acc, a_lo, b_hi, idesc, 1);
                 }
                 ptx::mma_commit(empty(s));
+                B2SP_PROF_STOP(2)
             }
+            B2SP_PROF_FLUSH(4)
             if (!failed) ptx::mma_commit(acc_full);
         }
     } else {
-        // ---------------- builders: scatter S windows into swizzled K-major tiles ----------------
-        // Per stage a warp owns 32 rows.  Lane l first holds the window bounds of row l; rows are then
-        // sorted into "long" (more than 16 entries in the window: one pass of 32 lanes) and "short"
-        // (1..16 entries: two rows per pass), empty rows are skipped.  The pass list goes through a
-        // 32-entry shared-memory table per warp; all global loads of up to kPassRound passes are
-        // issued before the first one is consumed.
-        constexpr int kPassRound = 24;
+        // ---------------- builders: expand S windows into swizzled K-major tiles ----------------
+        // Per stage a warp owns 32 rows of the tile and a lane owns one column of the 32-column window.
+        // Lane l first fetches (position, mask) of row l (one stage ahead) and parks it in a small
+        // shared table; then, row by row, lane c reads the row's entry through the warp-uniform mask:
+        // present iff bit c is set, stored at position + popc(mask below c).  Every lane writes its
+        // element (value or 0) of every row, so the tile needs no separate clearing and col_idx is
+        // never read here.  hi = value rounded to tf32, lo = value - hi (exact; the tensor core keeps
+        // its leading tf32 bits).
         const int g = (warp - 2) / Cfg::GROUP_WARPS;   // builder group = pipeline slot
         const int bw = (warp - 2) % Cfg::GROUP_WARPS;  // rows 32*bw .. 32*bw+31 of the tile
-        uint8_t *s_hi = smem_gen + g * Cfg::STAGE_BYTES, *s_lo = s_hi + Cfg::S_BYTES;
-        volatile int *order = reinterpret_cast<volatile int *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 256) +
-                              (warp - 2) * 32;
-        const int my_row = m0 + bw * 32 + lane;        // the row whose window bounds this lane fetches
-        const int *my_win = a.win + (size_t)(my_row < a.M ? my_row : 0) * (a.Wk + 1) + w0;
-        const unsigned lt_mask = (1u << lane) - 1u;
-        int nb = 0, ne = 0;
-        if (my_row < a.M && g < nchunks) { nb = __ldg(my_win + g); ne = __ldg(my_win + g + 1); }
+        uint8_t *w_hi = smem_gen + g * Cfg::STAGE_BYTES + bw * 4096;   // this warp's rows, hi tile
+        int2 *tab = reinterpret_cast<int2 *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 256) + (warp - 2) * 32;
+        const int my_row = m0 + bw * 32 + lane;        // the row whose window record this lane fetches
+        const int2 *my_win = a.win + (size_t)(my_row < a.M ? my_row : 0) * a.Wk + w0;
+        const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
+        uint32_t offs[8];                              // swizzled byte offset of column `lane` in row r: r & 7
+#pragma unroll
+        for (int i = 0; i < 8; ++i) offs[i] = (uint32_t)((lane << 2) ^ (i << 4));
+        int2 nxt = make_int2(0, 0);
+        if (my_row < a.M && g < nchunks) nxt = __ldg(my_win + g);
+        B2SP_PROF_DECL
+        B2SP_PROF_START
         for (int it = g; it < nchunks; it += STAGES) {
-            const int cb = nb, ce = ne;
-            nb = ne = 0;
-            if (my_row < a.M && it + STAGES < nchunks) {   // bounds of this warp's next stage
-                nb = __ldg(my_win + it + STAGES);
-                ne = __ldg(my_win + it + STAGES + 1);
-            }
-            const int cnt = ce - cb;
-            const unsigned long_m = __ballot_sync(0xffffffffu, cnt > 16);
-            const unsigned short_m = __ballot_sync(0xffffffffu, cnt > 0 && cnt <= 16);
-            const int nlong = __popc(long_m), nshort = __popc(short_m);
+            __syncwarp();   // everyone is done with the previous stage's table
+            tab[lane] = nxt;
+            nxt = make_int2(0, 0);
+            if (my_row < a.M && it + STAGES < nchunks) nxt = __ldg(my_win + it + STAGES);
             __syncwarp();
-            if (cnt > 16) order[__popc(long_m & lt_mask)] = lane;
-            else if (cnt > 0) order[nlong + __popc(short_m & lt_mask)] = lane;
-            __syncwarp();
-            const int npass = nlong + ((nshort + 1) >> 1);
-            const int kbase = (w0 + it) * kTileKC;
-            bool slot_ready = false;
-            for (int base = 0; base < npass || !slot_ready; base += kPassRound) {
-                int col[kPassRound];
-                float val[kPassRound];
+            float x[32];
 #pragma unroll
-                for (int p = 0; p < kPassRound; ++p) {
-                    const int pp = base + p;
-                    col[p] = -1;
-                    val[p] = 0.f;
-                    if (pp < npass) {   // warp-uniform
-                        int idx, jj;
-                        if (pp < nlong) { idx = pp; jj = lane; }
-                        else { idx = nlong + 2 * (pp - nlong) + (lane >> 4); jj = lane & 15; }
-                        const bool have = idx < nlong + nshort;
-                        const int r = have ? order[idx] : 0;
-                        const int q = __shfl_sync(0xffffffffu, cb, r) + jj;   // all lanes take part
-                        const int e0 = __shfl_sync(0xffffffffu, ce, r);
-                        const int e = have ? e0 : 0;
-                        if (q < e) {
-                            col[p] = __ldg(a.col_idx + q);
-                            val[p] = __ldg(a.values + q);
-                        }
-                    }
-                }
-                if (!slot_ready) {
-                    // the slot must have been drained by the MMAs of its previous use
-                    const int use = it / STAGES;
-                    bool ok = use == 0 || ptx::mbar_wait(empty(g), (use - 1) & 1);
-                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                    // zero this warp's 32 rows (4 KB) of both tiles
-                    uint4 z = make_uint4(0, 0, 0, 0);
-                    uint4 *zh = reinterpret_cast<uint4 *>(s_hi + bw * 4096) + lane;
-                    uint4 *zl = reinterpret_cast<uint4 *>(s_lo + bw * 4096) + lane;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) { zh[i * 32] = z; zl[i * 32] = z; }
-                    __syncwarp();
-                    slot_ready = true;
-                }
-#pragma unroll
-                for (int p = 0; p < kPassRound; ++p) {
-                    const int pp = base + p;
-                    if (pp < npass && col[p] >= 0) {
-                        const int idx = pp < nlong ? pp : nlong + 2 * (pp - nlong) + (lane >> 4);
-                        const int rt = bw * 32 + order[idx];
-                        const uint32_t kk = (uint32_t)(col[p] - kbase);
-                        uint32_t hi, lo;
-                        ptx::split_tf32(val[p], hi, lo);
-                        const uint32_t off = rt * 128 + (((kk >> 2) ^ (rt & 7)) << 4) + ((kk & 3) << 2);
-                        *reinterpret_cast<uint32_t *>(s_hi + off) = hi;
-                        *reinterpret_cast<uint32_t *>(s_lo + off) = lo;
-                    }
-                }
+            for (int r = 0; r < 32; ++r) {
+                const int2 t = tab[r];
+                x[r] = 0.f;
+                if ((unsigned)t.y & lane_bit) x[r] = __ldg(a.values + t.x + __popc((unsigned)t.y & lt_mask));
             }
-            if (failed) break;
+            B2SP_PROF_STOP(0)
+            {   // the slot must have been drained by the MMAs of its previous use
+                const int use = it / STAGES;
+                bool ok = use == 0 || ptx::mbar_wait(empty(g), (use - 1) & 1);
+                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            }
+            B2SP_PROF_STOP(1)
+#pragma unroll
+            for (int r = 0; r < 32; ++r) {
+                const uint32_t hi = (__float_as_uint(x[r]) + 0x1000u) & 0xffffe000u;
+                const float lo = x[r] - __uint_as_float(hi);
+                uint8_t *dst = w_hi + r * 128 + offs[r & 7];
+                *reinterpret_cast<uint32_t *>(dst) = hi;
+                *reinterpret_cast<float *>(dst + Cfg::S_BYTES) = lo;
+            }
+            B2SP_PROF_STOP(2)
             ptx::fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(full_s(g));
+            B2SP_PROF_STOP(3)
         }
+        if (bw == 0) { B2SP_PROF_FLUSH(8) }
         // ---------------- epilogue (first four builder warps): accumulator -> global ----------------
         if (warp < 6) {
             {
