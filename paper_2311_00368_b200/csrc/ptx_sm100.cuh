@@ -2,20 +2,55 @@
 // TMA tensor loads (never multicast), tensor memory (TMEM) management, tcgen05.mma / commit /
 // ld, proxy fences, and the fp32 -> (tf32 hi, tf32 lo) split.
 //
-// Every wait is bounded: mbar_wait() gives up after kWaitPolls polls and returns false, so a
-// kernel can record the failure and leave instead of spinning forever.
+// Every wait is bounded: mbar_wait() gives up after kWaitLimitNs (and at most kWaitPolls tries) and
+// returns false, so a kernel can record the failure and leave instead of waiting forever.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 namespace b2sp {
 namespace ptx {
 
-constexpr uint32_t kWaitPolls = 1u << 20;  // with the back-off below: a few hundred ms at most
+constexpr uint32_t kWaitPolls = 1u << 22;      // hard cap on tries
+constexpr uint32_t kWaitHintNs = 20000;        // per-try suspend hint
+constexpr uint64_t kWaitLimitNs = 300000000ull; // give up after 0.3 s
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+// ---- explicit shared-state-space accesses (32-bit shared addresses, immediate offsets) -----------------
+__device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ void sts32_off(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.b32 [%0 + %2], %1;" ::"r"(addr), "r"(v), "n"(OFF) : "memory");
+}
+__device__ __forceinline__ void sts64(uint32_t addr, uint32_t v0, uint32_t v1)
+{
+    asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(v0), "r"(v1) : "memory");
+}
+template <int OFF>
+__device__ __forceinline__ void lds64_off(uint32_t addr, uint32_t &v0, uint32_t &v1)
+{
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2 + %3];" : "=r"(v0), "=r"(v1) : "r"(addr), "n"(OFF) : "memory");
+}
+
+// Compile-time row loop: calls f(std::integral_constant<int, r>) for r = 0..N-1, so that row offsets
+// become instruction immediates.
+template <int N, int R = 0, class F>
+__device__ __forceinline__ void for_each_row(F &&f)
+{
+    if constexpr (R < N) {
+        f(std::integral_constant<int, R>{});
+        for_each_row<N, R + 1>(f);
+    }
 }
 
 // ---- mbarrier -----------------------------------------------------------------------------------
@@ -35,24 +70,34 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+// One try: the hardware may park the thread for up to `hint_ns` while the phase is incomplete, so a
+// waiter does not burn issue slots that the working warps of the CTA need.
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t hint_ns)
 {
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(hint_ns)
         : "memory");
     return ok != 0;
 }
-// Bounded wait for the phase with the given parity to complete.  false = gave up.
+__device__ __forceinline__ uint64_t global_timer_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for the phase with the given parity to complete.  false = gave up after kWaitLimitNs.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
 {
+    if (mbar_try_wait(bar, parity, 0)) return true;
+    const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0; i < kWaitPolls; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (i > 64) __nanosleep(i > 4096 ? 256 : 32);
+        if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
+        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
     }
     return false;
 }
@@ -90,6 +135,11 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const void *tmap, uint
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
         : "memory");
+}
+
+__device__ __forceinline__ void prefetch_l2(const void *p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
 }
 
 // ---- tensor memory ----------------------------------------------------------------------------------

@@ -135,13 +135,10 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
         return B2SP_ERR_CUDA;
 
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
-    if (cudaMemsetAsync(win, 0, sizeof(int2) * (size_t)M * (size_t)p.Wk, st) != cudaSuccess) return B2SP_ERR_CUDA;
     {
-        // threads per row from the mean row length (32..256)
-        long long avg = nnz / (M > 0 ? M : 1);
-        int G = avg >= 2048 ? 256 : avg >= 512 ? 128 : avg >= 128 ? 64 : 32;
-        long long threads = (long long)M * G;
-        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, G, row_ptr, col_idx, win,
+        const int GR = (p.Wk + 31) / 32;               // warps per row
+        const long long threads = (long long)M * GR * 32;
+        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, GR, row_ptr, col_idx, win,
                                                                               flags);
     }
     {

@@ -44,37 +44,52 @@ constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-by
 constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
 
 // ---- window table -------------------------------------------------------------------------------
-// T[r*Wk + w] = (first CSR position of row r inside column window [32w, 32w+32), occupancy bit mask of
-// that window: bit b set <=> column 32w+b is stored).  The table must be zeroed before the kernel
-// runs; windows without entries keep mask 0.  Needs strictly increasing columns inside a row (then a
-// window's entries are contiguous and at most 32); anything else sets flags[kFlagUnsorted].
-__global__ void tile_masks_kernel(int M, int K, int Wk, int G, const int *__restrict__ row_ptr,
+// T[r*Wk + w] = (first CSR position of row r whose column is >= 32w, occupancy bit mask of the column
+// window [32w, 32w+32): bit b set <=> column 32w+b is stored).  One lane per window, one warp per 32
+// consecutive windows of a row: a per-lane binary search finds where the window starts, a short loop
+// ORs the bits of its (at most 32) entries, and the warp stores 32 records with one coalesced write.
+// Every window of every row is written, so the table needs no clearing and no atomics.
+// The table is only meaningful when the columns of each row are strictly increasing and in range;
+// each warp also checks that for its share of the row's entries and sets flags[kFlagUnsorted] if not.
+__global__ void tile_masks_kernel(int M, int K, int Wk, int GR, const int *__restrict__ row_ptr,
                                   const int *__restrict__ col_idx, int2 *__restrict__ T,
                                   int *__restrict__ flags)
 {
-    // G threads (a power of two, 32..256, dividing blockDim.x) share a row; a warp never spans rows
-    const long long gt = (long long)blockIdx.x * blockDim.x + threadIdx.x;
-    const int row = (int)(gt / G), j = (int)(gt % G);
+    const int lane = threadIdx.x & 31;
+    const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;   // global warp
+    const int row = (int)(gw / GR), g = (int)(gw % GR);
     if (row >= M) return;
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    int2 *tr = T + (size_t)row * Wk;
+    const int beg = __ldg(row_ptr + row), end = __ldg(row_ptr + row + 1);
+    const int len = end - beg;
+    const int w = g * 32 + lane;
+
+    // lower bound of 32*w among the row's columns (same trip count for the whole warp)
+    int lo = beg, hi = end;
+    const int steps = len > 0 ? 32 - __clz(len) : 0;
+    const int key = w << 5;
+    for (int s = 0; s < steps; ++s) {
+        if (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (__ldg(col_idx + mid) < key) lo = mid + 1; else hi = mid;
+        }
+    }
+    // bits of the window's entries
+    unsigned mask = 0;
+    if (w < Wk) {
+        const int wend = key + 32;
+        for (int p = lo; p < end; ++p) {
+            const int c = __ldg(col_idx + p);
+            if (c >= wend) break;
+            mask |= 1u << (c & 31);
+        }
+        T[(size_t)row * Wk + w] = make_int2(lo, (int)mask);
+    }
+    // order / range check on this warp's share of the row
+    const int v0 = beg + (int)((long long)len * g / GR), v1 = beg + (int)((long long)len * (g + 1) / GR);
     bool bad = false;
-    for (int p0 = beg + (j & ~31); p0 < end; p0 += G) {   // warp-uniform trip count
-        const int p = p0 + (j & 31);
-        const bool live = p < end;
-        int c = 0, cprev = -1;
-        if (live) {
-            c = __ldg(col_idx + p);
-            if (p > beg) cprev = __ldg(col_idx + p - 1);
-            bad |= c <= cprev || c >= K || c < 0;
-        }
-        const int w = live ? min(max(c, 0) >> 5, Wk - 1) : -1 - (j & 31);   // dead lanes match nobody
-        const unsigned peers = __match_any_sync(0xffffffffu, w);
-        const unsigned bits = __reduce_or_sync(peers, live ? 1u << (c & 31) : 0u);
-        if (live) {
-            if ((unsigned)(j & 31) == (unsigned)(__ffs(peers) - 1)) atomicOr(reinterpret_cast<unsigned *>(&tr[w].y), bits);
-            if (cprev < 0 || (cprev >> 5) != w) tr[w].x = p;   // first entry of its window
-        }
+    for (int p = v0 + lane; p < v1; p += 32) {
+        const int c = __ldg(col_idx + p);
+        bad |= c < 0 || c >= K || (p > beg && c <= __ldg(col_idx + p - 1));
     }
     if (bad) atomicExch(&flags[kFlagUnsorted], 1);
 }
@@ -128,10 +143,9 @@ __global__ void reduce_partials_kernel(const float *__restrict__ part, int KS, l
 // B operand = S window tile (K-major, built here from CSR).  The streamed operand is the narrow one,
 // so the L2 -> SM traffic per flop is half of what a 128-row S tile would need.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, then STAGES builder groups of
-// TR/32 warps; group g owns pipeline slot g.  Stages are independent thanks to the window table, so
-// the groups build different stages concurrently, and each warp prefetches its next window bounds
-// while it works on the current stage.  Group 0's first four warps run the epilogue.
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer + TMEM owner, warps 2..31 = builders.  Stages
+// are independent thanks to the window table, so the builders work on (stage, 16-row chunk) items
+// round-robin and prefetch the records of their next item.  Builder warps 2..5 also run the epilogue.
 constexpr int kTileN = 128;  // columns of D / O per CTA (UMMA M)
 
 template <int TR>
@@ -140,11 +154,13 @@ struct SpmmTileCfg {
     static constexpr int D_BYTES = kTileKC * kTileN * 4;      // one D tile (hi or lo): 16 KB
     static constexpr int STAGE_BYTES = 2 * S_BYTES + 2 * D_BYTES;
     static constexpr int STAGES = TR == 256 ? 2 : 3;
-    static constexpr int GROUP_WARPS = TR / 32;
-    static constexpr int THREADS = (2 + STAGES * GROUP_WARPS) * 32;
+    static constexpr int CHUNK_ROWS = 16;                     // rows a builder warp expands per work item
+    static constexpr int CHUNKS = TR / CHUNK_ROWS;            // work items per stage
+    static constexpr int THREADS = 1024;                      // warp 0 TMA, warp 1 MMA, 30 builder warps
+    static constexpr int BUILDERS = THREADS / 32 - 2;
     static constexpr int TMEM_COLS = TR;                      // power of two >= 32
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ +
-                                      STAGES * GROUP_WARPS * 256 /*pass tables*/;
+                                      BUILDERS * CHUNK_ROWS * 8 /*per-warp record tables*/;
 };
 
 struct SpmmTileArgs {
@@ -194,7 +210,7 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             ptx::mbar_init(full_d(s), 1);
-            ptx::mbar_init(full_s(s), Cfg::GROUP_WARPS);
+            ptx::mbar_init(full_s(s), Cfg::CHUNKS);
             ptx::mbar_init(empty(s), 1);
         }
         ptx::mbar_init(acc_full, 1);
@@ -246,10 +262,17 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
             for (int it = 0; it < nchunks; ++it) {
                 const int s = it % STAGES;
                 const uint32_t par = (it / STAGES) & 1;
+#ifdef B2SP_PROF_DFIRST
+                if (!ptx::mbar_wait(full_d(s), par)) { failed = true; break; }
+                B2SP_PROF_STOP(1)
+                if (!ptx::mbar_wait(full_s(s), par)) { failed = true; break; }
+                B2SP_PROF_STOP(0)
+#else
                 if (!ptx::mbar_wait(full_s(s), par)) { failed = true; break; }
                 B2SP_PROF_STOP(0)
                 if (!ptx::mbar_wait(full_d(s), par)) { failed = true; break; }
                 B2SP_PROF_STOP(1)
+#endif
                 ptx::tc_fence_after_sync();
                 const uint32_t s_hi = smem_base + s * Cfg::STAGE_BYTES, s_lo = s_hi + Cfg::S_BYTES;
                 const uint32_t d_hi = s_lo + Cfg::S_BYTES, d_lo = d_hi + Cfg::D_BYTES;
@@ -274,62 +297,77 @@ spmm_tile_kernel(const __grid_constant__ CUtensorMap tm_dhi, const __grid_consta
         }
     } else {
         // ---------------- builders: expand S windows into swizzled K-major tiles ----------------
-        // Per stage a warp owns 32 rows of the tile and a lane owns one column of the 32-column window.
-        // Lane l first fetches (position, mask) of row l (one stage ahead) and parks it in a small
-        // shared table; then, row by row, lane c reads the row's entry through the warp-uniform mask:
-        // present iff bit c is set, stored at position + popc(mask below c).  Every lane writes its
-        // element (value or 0) of every row, so the tile needs no separate clearing and col_idx is
-        // never read here.  hi = value rounded to tf32, lo = value - hi (exact; the tensor core keeps
-        // its leading tf32 bits).
-        const int g = (warp - 2) / Cfg::GROUP_WARPS;   // builder group = pipeline slot
-        const int bw = (warp - 2) % Cfg::GROUP_WARPS;  // rows 32*bw .. 32*bw+31 of the tile
-        uint8_t *w_hi = smem_gen + g * Cfg::STAGE_BYTES + bw * 4096;   // this warp's rows, hi tile
-        int2 *tab = reinterpret_cast<int2 *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 256) + (warp - 2) * 32;
-        const int my_row = m0 + bw * 32 + lane;        // the row whose window record this lane fetches
-        const int2 *my_win = a.win + (size_t)(my_row < a.M ? my_row : 0) * a.Wk + w0;
+        // Work item = (stage, chunk of 16 rows); the builder warps take items round-robin, so the 16
+        // chunks of a stage are expanded by 16 different warps at once and later stages are already
+        // in progress.  Inside an item a lane owns one column of the 32-column window: lanes 0..15
+        // first fetch (position, mask) of the chunk's rows (one item ahead) and park them in a small
+        // shared table; then, row by row, lane c reads the row's entry through the warp-uniform
+        // mask: present iff bit c is set, stored at position + popc(mask below c).  Every lane writes
+        // its element (value or 0) of every row, so the tile needs no separate clearing and col_idx
+        // is never read here.  hi = value rounded to tf32, lo = value - hi (exact; the tensor core
+        // keeps its leading tf32 bits).
+        constexpr int CR = Cfg::CHUNK_ROWS, CH = Cfg::CHUNKS, NB = Cfg::BUILDERS;
+        const int b = warp - 2;
+        const uint32_t tab = smem_base + STAGES * Cfg::STAGE_BYTES + 256 + b * (CR * 8);   // shared address
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
-        uint32_t offs[8];                              // swizzled byte offset of column `lane` in row r: r & 7
-#pragma unroll
-        for (int i = 0; i < 8; ++i) offs[i] = (uint32_t)((lane << 2) ^ (i << 4));
-        int2 nxt = make_int2(0, 0);
-        if (my_row < a.M && g < nchunks) nxt = __ldg(my_win + g);
+        const int nitems = nchunks * CH;
+        auto record = [&](int id) {                    // lanes 0..15: window record of one row of item `id`
+            int2 rec = make_int2(0, 0);
+            const int row = m0 + (id % CH) * CR + lane;
+            if (id < nitems && lane < CR && row < a.M) rec = __ldg(a.win + (size_t)row * a.Wk + w0 + id / CH);
+            return rec;
+        };
+        int2 nxt = record(b);
         B2SP_PROF_DECL
         B2SP_PROF_START
-        for (int it = g; it < nchunks; it += STAGES) {
-            __syncwarp();   // everyone is done with the previous stage's table
-            tab[lane] = nxt;
-            nxt = make_int2(0, 0);
-            if (my_row < a.M && it + STAGES < nchunks) nxt = __ldg(my_win + it + STAGES);
+        for (int id = b; id < nitems; id += NB) {
+            const int it = id / CH, chunk = id % CH, slot = it % STAGES, use = it / STAGES;
+            __syncwarp();   // everyone is done with the previous item's table
+            if (lane < CR) ptx::sts64(tab + lane * 8, (uint32_t)nxt.x, (uint32_t)nxt.y);
+            nxt = record(id + NB);
             __syncwarp();
-            float x[32];
-#pragma unroll
-            for (int r = 0; r < 32; ++r) {
-                const int2 t = tab[r];
+            float x[CR];
+            ptx::for_each_row<CR>([&](auto rc) {
+                constexpr int r = decltype(rc)::value;
+                uint32_t pos, mask;
+                ptx::lds64_off<r * 8>(tab, pos, mask);
                 x[r] = 0.f;
-                if ((unsigned)t.y & lane_bit) x[r] = __ldg(a.values + t.x + __popc((unsigned)t.y & lt_mask));
-            }
+#ifdef B2SP_ABL_NOLOAD
+                if (mask & lane_bit) x[r] = __uint_as_float(pos + __popc(mask & lt_mask));
+#else
+                if (mask & lane_bit) x[r] = __ldg(a.values + (pos + __popc(mask & lt_mask)));
+#endif
+            });
             B2SP_PROF_STOP(0)
             {   // the slot must have been drained by the MMAs of its previous use
-                const int use = it / STAGES;
-                bool ok = use == 0 || ptx::mbar_wait(empty(g), (use - 1) & 1);
+                bool ok = use == 0 || ptx::mbar_wait(empty(slot), (use - 1) & 1);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
             }
             B2SP_PROF_STOP(1)
+            // shared address of this lane's column in row r of the chunk: wb[r & 7] + r * 128
+            const uint32_t w_hi = smem_base + slot * Cfg::STAGE_BYTES + chunk * (CR * 128);
+            uint32_t wb[8];
 #pragma unroll
-            for (int r = 0; r < 32; ++r) {
+            for (int i = 0; i < 8; ++i) wb[i] = w_hi + (uint32_t)((lane << 2) ^ (i << 4));
+            ptx::for_each_row<CR>([&](auto rc) {
+                constexpr int r = decltype(rc)::value;
                 const uint32_t hi = (__float_as_uint(x[r]) + 0x1000u) & 0xffffe000u;
                 const float lo = x[r] - __uint_as_float(hi);
-                uint8_t *dst = w_hi + r * 128 + offs[r & 7];
-                *reinterpret_cast<uint32_t *>(dst) = hi;
-                *reinterpret_cast<float *>(dst + Cfg::S_BYTES) = lo;
-            }
+#ifdef B2SP_ABL_NOSTORE
+                if (hi == 0x12345678u)
+#endif
+                {
+                    ptx::sts32_off<r * 128>(wb[r & 7], hi);
+                    ptx::sts32_off<r * 128 + Cfg::S_BYTES>(wb[r & 7], __float_as_uint(lo));
+                }
+            });
             B2SP_PROF_STOP(2)
             ptx::fence_proxy_async_smem();
             __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(full_s(g));
+            if (lane == 0) ptx::mbar_arrive(full_s(slot));
             B2SP_PROF_STOP(3)
         }
-        if (bw == 0) { B2SP_PROF_FLUSH(8) }
+        if (b < 2) { B2SP_PROF_FLUSH(8) }
         // ---------------- epilogue (first four builder warps): accumulator -> global ----------------
         if (warp < 6) {
             {
