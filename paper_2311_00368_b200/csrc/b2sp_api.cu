@@ -148,13 +148,6 @@ bool bad_csr_args(int M, int K, long long nnz, const int *row_ptr, const int *co
     return false;
 }
 
-int resolve_algo(int algo)
-{
-    // SDDMM and FusedMM: row family only for now.
-    if (algo == B2SP_ALGO_AUTO) return B2SP_ALGO_ROW;
-    return algo;
-}
-
 }  // namespace b2sp
 
 using namespace b2sp;
@@ -184,6 +177,14 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
     size_t need = row_workspace_bytes(M);
     if (op == B2SP_OP_SPMM && tile_profitable(M, K, N, nnz)) {
         TilePlan p = plan_spmm_tile(M, K, N, nnz, need);
+        if (p.feasible && p.bytes > need) need = p.bytes;
+    }
+    if (op == B2SP_OP_SDDMM && tile_profitable(M, K, Kd, nnz)) {
+        FusedPlan p = plan_fused_tile(M, K, Kd, 0, nnz, need, false);
+        if (p.feasible && p.bytes > need) need = p.bytes;
+    }
+    if (op == B2SP_OP_FUSEDMM && tile_profitable(M, K, Kd < N ? Kd : N, nnz)) {
+        FusedPlan p = plan_fused_tile(M, K, Kd, N, nnz, need, true);
         if (p.feasible && p.bytes > need) need = p.bytes;
     }
     return need;
@@ -259,6 +260,35 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     return rc;
 }
 
+// Enqueues the row-family SDDMM.  `gate` != NULL makes it a device-side fallback.
+static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_idx, const float *s_values,
+                              const float *A, long long lda, const float *B, long long ldb,
+                              float *out_values, const int *order, const int *gate, cudaStream_t st)
+{
+    dim3 grid((unsigned)M);
+    bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+               Kd <= 40960;
+    if (vec) {
+        switch (pick_ku(Kd)) {
+        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
+        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
+        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
+        default: {
+            size_t smem = sizeof(float) * (size_t)Kd;
+            if (smem > 48 * 1024 &&
+                cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)smem) != cudaSuccess)
+                return B2SP_ERR_CUDA;
+            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate);
+        }
+        }
+    } else {
+        sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
+                                                             B, ldb, out_values, order, gate);
+    }
+    return check_launch();
+}
+
 b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
                        const float *s_values, const float *A, long long lda, const float *B,
                        long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
@@ -269,11 +299,15 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
     if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && !out_values) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
-    b2sp_status rc = check_workspace(workspace, workspace_bytes,
-                                     b2sp_workspace_bytes(B2SP_OP_SDDMM, M, K, Kd, 0, nnz));
+    const size_t row_bytes = row_workspace_bytes(M);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
-    int use = resolve_algo(algo);
-    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    FusedPlan plan;
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, Kd, nnz)))
+        plan = plan_fused_tile(M, K, Kd, 0, nnz, row_bytes, false);
+    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
+    else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_SDDMM] = use;
     int launches = 0;
     g_last_launches[B2SP_OP_SDDMM] = 0;
@@ -284,34 +318,51 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
                    : B2SP_ERR_CUDA;
 
     Workspace w = carve(workspace);
+    if (use == B2SP_ALGO_TILE) {
+        rc = fused_tile(plan, false, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
+                        out_values, 0, workspace, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, nullptr, gate, st);
+        g_last_launches[B2SP_OP_SDDMM] = launches + 1;
+        return rc;
+    }
     const int *order = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
     }
-    dim3 grid((unsigned)M);
-    bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+    rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr, st);
+    g_last_launches[B2SP_OP_SDDMM] = launches + 1;
+    return rc;
+}
+
+// Enqueues the row-family FusedMM.  `gate` != NULL makes it a device-side fallback.
+static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const int *col_idx,
+                              const float *s_values, const float *A, long long lda, const float *B,
+                              long long ldb, const float *D, long long ldd, float *O, long long ldo,
+                              const int *order, const int *gate, cudaStream_t st)
+{
+    b2sp_status rc = B2SP_OK;
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
+               Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
                Kd <= 40960;
     if (vec) {
+        Geom g = pick_geom(N);
+        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
         switch (pick_ku(Kd)) {
-        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
-        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
-        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr); break;
-        default: {
-            size_t smem = sizeof(float) * (size_t)Kd;
-            if (smem > 48 * 1024 &&
-                cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)smem) != cudaSuccess)
-                return B2SP_ERR_CUDA;
-            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr);
+        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
+        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
+        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
+        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
         }
-        }
+        if (rc != B2SP_OK) return rc;
     } else {
-        sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
-                                                             B, ldb, out_values, order, nullptr);
+        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
+                                                               lda, B, ldb, D, ldd, O, ldo, order, gate);
     }
-    g_last_launches[B2SP_OP_SDDMM] = launches + 1;
     return check_launch();
 }
 
@@ -327,11 +378,15 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && (!D || ldd < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
-    b2sp_status rc = check_workspace(workspace, workspace_bytes,
-                                     b2sp_workspace_bytes(B2SP_OP_FUSEDMM, M, K, Kd, N, nnz));
+    const size_t row_bytes = row_workspace_bytes(M);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
-    int use = resolve_algo(algo);
-    if (use == B2SP_ALGO_TILE) return B2SP_ERR_UNSUPPORTED;
+    FusedPlan plan;
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, Kd < N ? Kd : N, nnz)))
+        plan = plan_fused_tile(M, K, Kd, N, nnz, row_bytes, true);
+    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
+    else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_FUSEDMM] = use;
     int launches = 0;
     g_last_launches[B2SP_OP_FUSEDMM] = 0;
@@ -339,32 +394,24 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     if (nnz == 0 || Kd == 0) return zero_rows(O, ldo, M, N, st);  // empty dot products are 0
 
     Workspace w = carve(workspace);
+    if (use == B2SP_ALGO_TILE) {
+        rc = fused_tile(plan, true, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
+                        workspace, st, &launches);
+        if (rc != B2SP_OK) return rc;
+        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, st);
+        g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
+        return rc;
+    }
     const int *order = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
     }
-    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
-               Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
-               Kd <= 40960;
-    if (vec) {
-        Geom g = pick_geom(N);
-        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
-        switch (pick_ku(Kd)) {
-        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
-        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
-        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
-        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr); break;
-        }
-        if (rc != B2SP_OK) return rc;
-    } else {
-        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
-        fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
-                                                               lda, B, ldb, D, ldd, O, ldo, order, nullptr);
-    }
+    rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
-    return check_launch();
+    return rc;
 }
 
 b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,

@@ -7,6 +7,7 @@
 #include <mutex>
 
 #include "tile_kernels.cuh"
+#include "tile_fused.cuh"
 
 namespace b2sp {
 
@@ -166,6 +167,138 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
         long long total = (long long)M * N;
         int blocks = (int)((total + 255) / 256 < (long long)kSMs * 8 ? (total + 255) / 256 : (long long)kSMs * 8);
         reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, O, ldo, flags);
+        *launches += 1;
+        if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+    }
+    return B2SP_OK;
+}
+
+FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)
+{
+    FusedPlan p;
+    if (M <= 0 || K <= 0 || Kd <= 0 || Kd > 128 || nnz <= 0 || (fused && N <= 0)) return p;
+    p.Wk = (K + kFusedW - 1) / kFusedW;
+    p.Kp = p.Wk * kFusedW;
+    p.Kdp = Kd <= 32 ? 32 : Kd <= 64 ? 64 : 128;
+    p.Mt = (M + kFusedRows - 1) / kFusedRows;
+    p.Nt = fused ? (N + kFusedNT - 1) / kFusedNT : 1;
+    p.Np = fused ? p.Nt * kFusedNT : 0;
+    size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
+    if (win_bytes > (size_t)2 << 30) return p;
+    p.KS = pick_split(p.Mt * p.Nt, p.Wk);
+    size_t off = align_up(base_off, 1024);
+    p.off_win = off;
+    off = align_up(off + win_bytes, 1024);
+    size_t bbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Kdp;
+    p.off_bhi = off;
+    off = align_up(off + bbytes, 1024);
+    p.off_blo = off;
+    off = align_up(off + bbytes, 1024);
+    if (fused) {
+        size_t dbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Np;
+        p.off_dhi = off;
+        off = align_up(off + dbytes, 1024);
+        p.off_dlo = off;
+        off = align_up(off + dbytes, 1024);
+        p.off_part = off;
+        if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * kFusedRows * (size_t)p.Np;
+    }
+    p.bytes = align_up(off, 256);
+    p.feasible = true;
+    return p;
+}
+
+namespace {
+
+template <int KDP, bool FUSED>
+b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
+                              const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
+{
+    using Cfg = FusedCfg<KDP>;
+    auto kern = fused_tile_kernel<KDP, FUSED>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
+        return B2SP_ERR_CUDA;
+    kern<<<items, kFusedThreads, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, a);
+    return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
+}
+
+template <bool FUSED>
+b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
+                             const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
+{
+    if (kdp == 32) return launch_fused_tile<32, FUSED>(bh, bl, dh, dl, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, FUSED>(bh, bl, dh, dl, a, items, st);
+    return launch_fused_tile<128, FUSED>(bh, bl, dh, dl, a, items, st);
+}
+
+void launch_split(const float *X, long long ld, int rows, int cols, float *hi, float *lo, int rows_p, int cols_p,
+                  cudaStream_t st)
+{
+    long long groups = (long long)rows_p * (cols_p / 4);
+    long long want = (groups + 255) / 256, cap = (long long)kSMs * 8;
+    split_dense_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(X, ld, rows, cols, hi, lo, rows_p, cols_p);
+}
+
+}  // namespace
+
+b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int N, long long nnz,
+                       const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
+                       long long lda, const float *B, long long ldb, const float *D, long long ldd,
+                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches)
+{
+    (void)nnz;
+    char *ws = static_cast<char *>(workspace);
+    int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
+    int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
+    int2 *win = reinterpret_cast<int2 *>(ws + p.off_win);
+    float *bhi = reinterpret_cast<float *>(ws + p.off_bhi), *blo = reinterpret_cast<float *>(ws + p.off_blo);
+    float *dhi = reinterpret_cast<float *>(ws + p.off_dhi), *dlo = reinterpret_cast<float *>(ws + p.off_dlo);
+    float *part = reinterpret_cast<float *>(ws + p.off_part);
+
+    CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
+    if (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedW, p.Kdp / 32, false) ||
+        !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedW, p.Kdp / 32, false))
+        return B2SP_ERR_CUDA;
+    if (fused) {
+        if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true) ||
+            !make_blocked_map(&tm_dl, dlo, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true))
+            return B2SP_ERR_CUDA;
+    } else {
+        tm_dh = tm_bh;   // unused by the SDDMM kernel
+        tm_dl = tm_bl;
+    }
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
+    {
+        const int GR = (p.Wk + 31) / 32;
+        const long long threads = (long long)M * GR * 32;
+        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, GR, row_ptr, col_idx, win,
+                                                                              flags);
+    }
+    launch_split(B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, st);
+    *launches += 2;
+    if (fused) {
+        launch_split(D, ldd, K, N, dhi, dlo, p.Kp, p.Np, st);
+        *launches += 1;
+    }
+    if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+
+    FusedTileArgs a;
+    a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
+    a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
+    a.flags = flags; a.status = status;
+    if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
+    else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
+    else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
+    const int items = p.Mt * p.Nt * p.KS;
+    b2sp_status rc = fused ? launch_fused_kdp<true>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
+                           : launch_fused_kdp<false>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
+    *launches += 1;
+    if (rc != B2SP_OK) return rc;
+    if (fused && p.KS > 1) {
+        long long total = (long long)M * N;
+        long long want = (total + 255) / 256, cap = (long long)kSMs * 8;
+        reduce_partials_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, out,
+                                                                                    ldo, flags);
         *launches += 1;
         if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
     }

@@ -22,6 +22,21 @@ struct TilePlan {
 // Plan for SPMM on the dense-tile family; `base_off` = first byte after the row family's region.
 TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off);
 
+// Plans for FusedMM (fused = true) and SDDMM (fused = false) on the dense-tile family.  They need
+// Kd <= 128.  TR is unused; Np is the padded width of D (FusedMM only).
+struct FusedPlan {
+    bool feasible = false;
+    int Kdp = 0, Nt = 1, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
+    size_t off_win = 0, off_bhi = 0, off_blo = 0, off_dhi = 0, off_dlo = 0, off_part = 0;
+    size_t bytes = 0;
+};
+FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused);
+
+b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int N, long long nnz,
+                       const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
+                       long long lda, const float *B, long long ldb, const float *D, long long ldd,
+                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches);
+
 // True when the dense-tile family is expected to beat the row family for these sizes.
 bool tile_profitable(int M, int K, int width, long long nnz);
 

@@ -115,3 +115,116 @@ def test_spmm_tile_config_and_auto(b):
     with pytest.raises(b.B2spError) as e:
         b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=small, algo=TILE)
     assert e.value.status == 5
+
+
+# ---- SDDMM and FusedMM on the dense-tile family -------------------------------------------------
+
+def fused_tile_check(b, p, null_values=False, ops=("sddmm", "fusedmm")):
+    d = DevProblem(p)
+    sv_np = None if null_values else p.values
+    sv = None if null_values else d.values
+    worst = 0.0
+    if "sddmm" in ops:
+        ws = _ws(b, b.OP_SDDMM, p)
+        ref, T = oracle.sddmm(p.row_ptr, p.col_idx, sv_np, p.A, p.B)
+        out = torch.full((p.nnz,), float("nan"), device="cuda")
+        b.sddmm(d.row_ptr, d.col_idx, sv, d.A, d.B, out=out, workspace=ws, algo=TILE)
+        assert b.last_algo(b.OP_SDDMM) == TILE
+        assert b.device_status(ws) == 0, "a bounded wait inside the SDDMM tile kernel gave up"
+        worst = max(worst, gate(out, ref, T, f"sddmm tile {p.name} M={p.M} K={p.K} Kd={p.Kd}"))
+    if "fusedmm" in ops:
+        ws = _ws(b, b.OP_FUSEDMM, p)
+        ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, sv_np, p.A, p.B, p.D)
+        out = torch.full((p.M, p.N), float("nan"), device="cuda")
+        b.fusedmm(d.row_ptr, d.col_idx, sv, d.A, d.B, d.D, out=out, workspace=ws, algo=TILE)
+        assert b.last_algo(b.OP_FUSEDMM) == TILE
+        assert b.device_status(ws) == 0, "a bounded wait inside the FusedMM tile kernel gave up"
+        worst = max(worst, gate(out, ref, T, f"fusedmm tile {p.name} M={p.M} K={p.K} Kd={p.Kd} N={p.N}"))
+    assert d.pattern_untouched()
+    return worst
+
+
+@pytest.mark.parametrize("M,K,density,Kd,N,kind", [
+    (128, 128, 0.30, 32, 32, "uniform"),      # one tile, one window group, smallest Kd
+    (256, 256, 0.10, 64, 64, "uniform"),      # tiny-config shape
+    (257, 333, 0.30, 128, 128, "uniform"),    # ragged M and K
+    (300, 512, 0.20, 100, 100, "uniform"),    # Kd and N padded inside the scratch copies
+    (130, 1024, 0.25, 20, 300, "uniform"),    # three O column tiles, small Kd
+    (512, 2048, 0.10, 128, 256, "uniform"),   # several K splits, two column tiles
+    (384, 1024, 0.20, 64, 128, "powerlaw"),   # skewed rows incl. full rows
+    (256, 512, 0.20, 64, 64, "band"),
+    (200, 640, 0.05, 36, 36, "uniform"),
+])
+def test_fused_and_sddmm_tile_shapes(b, M, K, density, Kd, N, kind):
+    p = W.small_random(3000 + M + N, M, K, density, Kd, N, kind=kind)
+    fused_tile_check(b, p)
+    fused_tile_check(b, p, null_values=True)
+
+
+def test_fused_tile_exact_on_small_integers(b):
+    rng = np.random.default_rng(6)
+    p = W.small_random(78, 256, 256, 0.3, 32, 64)
+    p.values[:] = rng.integers(-2, 3, p.nnz).astype(np.float32)
+    p.A[:] = rng.integers(-3, 4, p.A.shape).astype(np.float32)
+    p.B[:] = rng.integers(-3, 4, p.B.shape).astype(np.float32)
+    p.D[:] = rng.integers(-4, 5, p.D.shape).astype(np.float32)
+    d = DevProblem(p)
+    C = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=_ws(b, b.OP_SDDMM, p), algo=TILE)
+    ref, _ = oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B)
+    assert np.array_equal(C.cpu().numpy().astype(np.float64), ref)
+    O = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=_ws(b, b.OP_FUSEDMM, p), algo=TILE)
+    ref, _ = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)
+    assert np.array_equal(O.cpu().numpy().astype(np.float64), ref)
+
+
+def test_fused_tile_row_edges_and_inplace_sddmm(b):
+    lens = [0, 1, 31, 32, 33, 0, 127, 128, 129, 255, 256, 257, 2048, 0, 2, 64] * 9
+    p = _custom_rows(lens, 2048, 16, Kd=64, N=128)
+    fused_tile_check(b, p)
+    d = DevProblem(p)
+    ref, T = oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B)
+    vals = d.values.clone()
+    b.sddmm(d.row_ptr, d.col_idx, vals, d.A, d.B, out=vals, workspace=_ws(b, b.OP_SDDMM, p), algo=TILE)
+    gate(vals, ref, T, "sddmm tile in place")
+
+
+def test_fused_tile_falls_back_on_unsorted_rows_and_large_kd(b):
+    p = W.small_random(92, 256, 300, 0.3, 64, 128)
+    rng = np.random.default_rng(4)
+    ci, v = p.col_idx.copy(), p.values.copy()
+    a, e = p.row_ptr[7], p.row_ptr[8]
+    perm = a + rng.permutation(e - a)
+    ci[a:e], v[a:e] = ci[perm], v[perm]
+    q = W.Problem("unsorted", p.M, p.K, p.row_ptr, ci, v, p.Kd, p.N, p.A, p.B, p.D)
+    fused_tile_check(b, q)
+    # Kd > 128 is outside the tile family: an explicit request is refused, AUTO uses the row kernels
+    big = W.small_random(93, 256, 256, 0.2, 160, 64)
+    d = DevProblem(big)
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    with pytest.raises(b.B2spError) as e:
+        b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=TILE)
+    assert e.value.status == 2
+    out = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=0)
+    assert b.last_algo(b.OP_FUSEDMM) == 1
+    ref, T = oracle.fusedmm(big.row_ptr, big.col_idx, big.values, big.A, big.B, big.D)
+    gate(out, ref, T, "fusedmm auto, Kd=160")
+
+
+def test_fused_tile_configs(b):
+    p = W.sddmm_case()
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_SDDMM, p)
+    ref, T = oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B)
+    out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=0)
+    assert b.last_algo(b.OP_SDDMM) == TILE and b.device_status(ws) == 0
+    assert gate(out, ref, T, "sddmm config, auto") < 0.5
+    p = W.attention_case(3)
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_FUSEDMM, p)
+    out = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=0)
+    assert b.last_algo(b.OP_FUSEDMM) == TILE and b.device_status(ws) == 0
+    rows = (0, 37, 2048, 4095)
+    for r in rows:
+        ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D, rows=(r, r + 1))
+        ok, ratio = oracle.within_tolerance(out[r:r + 1].cpu().numpy(), ref, T)
+        assert ok, f"attention row {r}: {ratio:.3g}"
