@@ -39,7 +39,8 @@ __device__ __forceinline__ void sts64(uint32_t addr, uint32_t v0, uint32_t v1)
 template <int OFF>
 __device__ __forceinline__ void lds64_off(uint32_t addr, uint32_t &v0, uint32_t &v1)
 {
-    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2 + %3];" : "=r"(v0), "=r"(v1) : "r"(addr), "n"(OFF) : "memory");
+    // no memory clobber: callers order these reads against shared-memory writes with __syncwarp()
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2 + %3];" : "=r"(v0), "=r"(v1) : "r"(addr), "n"(OFF));
 }
 
 // Compile-time row loop: calls f(std::integral_constant<int, r>) for r = 0..N-1, so that row offsets

@@ -286,6 +286,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     a.flags = flags; a.status = status;
+    a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }

@@ -21,6 +21,18 @@
 
 #include "ptx_sm100.cuh"
 
+#ifdef B2SP_TILE_PROFILE
+#define B2SP_FPROF_DECL long long fp_t0 = 0, fp_acc[6] = {0, 0, 0, 0, 0, 0};
+#define B2SP_FPROF_START fp_t0 = clock64();
+#define B2SP_FPROF_STOP(i) { long long t_ = clock64(); fp_acc[i] += t_ - fp_t0; fp_t0 = t_; }
+#define B2SP_FPROF_FLUSH(base) { if (lane == 0 && a.prof) { for (int i_ = 0; i_ < 6; ++i_) atomicAdd(a.prof + (base) + i_, (unsigned long long)fp_acc[i_]); } }
+#else
+#define B2SP_FPROF_DECL
+#define B2SP_FPROF_START
+#define B2SP_FPROF_STOP(i) {}
+#define B2SP_FPROF_FLUSH(base) {}
+#endif
+
 namespace b2sp {
 
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
@@ -40,6 +52,7 @@ struct FusedTileArgs {
     long long ld_out, slab;
     const int *flags;
     int *status;
+    unsigned long long *prof;  // optional role timers (profiling builds only)
 };
 
 template <int KDP>
@@ -48,7 +61,7 @@ struct FusedCfg {
     static constexpr int D_BYTES = kFusedW * kFusedNT * 4;     // D window tile (hi or lo): 16 KB
     static constexpr int STAGE_BYTES = 2 * B_BYTES + 2 * D_BYTES;
     static constexpr int STAGE_BYTES_SDDMM = 2 * B_BYTES;
-    static constexpr int AUX_BYTES = 256 /*barriers*/ + 4 * 256 /*record tables*/ + 4 * 4096 /*value staging*/;
+    static constexpr int AUX_BYTES = 256 /*barriers*/ + 4 * 512 /*record tables*/ + 4 * 4096 /*value staging*/;
     static constexpr int SMEM_BYTES = kFusedStages * STAGE_BYTES + 1024 + AUX_BYTES;
 };
 
@@ -171,10 +184,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedW, false, false);
             constexpr uint32_t idesc2 = ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
+            B2SP_FPROF_DECL
+            B2SP_FPROF_START
             auto gemm1 = [&](int it) -> bool {   // P[it & 1] = A_tile * B_window^T
                 const int s = it % STAGES, pb = it & 1;
                 if (!ptx::mbar_wait(full(s), (it / STAGES) & 1)) return false;
+                B2SP_FPROF_STOP(0)
                 if (it >= 2 && !ptx::mbar_wait(p_free(pb), ((it >> 1) - 1) & 1)) return false;
+                B2SP_FPROF_STOP(1)
                 ptx::tc_fence_after_sync();
                 const uint32_t b_hi = smem_base + s * STAGE_BYTES, b_lo = b_hi + Cfg::B_BYTES;
                 const uint32_t pacc = tmem + kColP + pb * kFusedW;
@@ -190,6 +207,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 ptx::mma_commit(p_full(pb));
                 if (!FUSED) ptx::mma_commit(empty(s));   // SDDMM: the stage only held B
+                B2SP_FPROF_STOP(2)
                 return true;
             };
             if (nwin > 0 && !gemm1(0)) failed = true;
@@ -198,6 +216,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (FUSED) {
                     const int s = it % STAGES;
                     if (!ptx::mbar_wait(pp_full, it & 1)) { failed = true; break; }
+                    B2SP_FPROF_STOP(3)
                     ptx::tc_fence_after_sync();
                     const uint32_t d_hi = smem_base + s * STAGE_BYTES + 2 * Cfg::B_BYTES, d_lo = d_hi + Cfg::D_BYTES;
 #pragma unroll
@@ -212,64 +231,90 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     }
                     ptx::mma_commit(pp_free);
                     ptx::mma_commit(empty(s));
+                    B2SP_FPROF_STOP(4)
                 }
             }
+            B2SP_FPROF_FLUSH(0)
             if (FUSED && !failed) ptx::mma_commit(o_full);
         }
     } else {
         // ---------------- element-wise warps (thread = row) ----------------
+        // Software pipeline over windows: while window t is processed, the stored values of window
+        // t+1 are already in flight (loaded cooperatively with lane = column, then transposed through
+        // shared memory so that each thread gets its own row), and the record of window t+2 is loading.
         const int ew = warp - 2;
-        const uint32_t rec_tab = aux + 256 + ew * 256;              // 32 records of this warp's rows
-        const uint32_t stage_v = aux + 256 + 4 * 256 + ew * 4096;   // 32 x 32 floats, swizzled chunks
+        const uint32_t rec_tab = aux + 256 + ew * 512;              // 2 x 32 records of this warp's rows
+        const uint32_t stage_v = aux + 256 + 4 * 512 + ew * 4096;   // 32 x 32 floats, swizzled chunks
         const int grow = m0 + row;
         const int2 *my_win = a.win + (size_t)(grow < a.M ? grow : 0) * a.Wk + w0;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
         const bool has_values = a.s_values != nullptr;
-        int2 nxt = make_int2(0, 0);
-        if (grow < a.M && nwin > 0) nxt = __ldg(my_win);
+        const bool use_tab = has_values || !FUSED;
+        auto load_rec = [&](int t) {
+            int2 r = make_int2(0, 0);
+            if (grow < a.M && t < nwin) r = __ldg(my_win + t);
+            return r;
+        };
+        // column-owner loads of one window's stored values (lane = column, register r = row r of the warp)
+        auto issue_values = [&](uint32_t tab, float (&vn)[32]) {
+            ptx::for_each_row<32>([&](auto rc) {
+                constexpr int r = decltype(rc)::value;
+                uint32_t pos, m;
+                ptx::lds64_off<r * 8>(tab, pos, m);
+                vn[r] = 0.f;
+                if (m & lane_bit) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
+            });
+        };
+        // transpose through shared memory: afterwards sv[c] = value of (this thread's row, column c)
+        auto transpose_values = [&](const float (&vn)[32], float (&sv)[32]) {
+            __syncwarp();
+            ptx::for_each_row<32>([&](auto rc) {
+                constexpr int r = decltype(rc)::value;
+                ptx::sts32_off<r * 128>(stage_v + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
+            });
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t x0, x1, x2, x3;
+                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                             : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+                             : "r"(stage_v + lane * 128 + (uint32_t)((j ^ (lane & 7)) << 4)));
+                sv[4 * j] = __uint_as_float(x0); sv[4 * j + 1] = __uint_as_float(x1);
+                sv[4 * j + 2] = __uint_as_float(x2); sv[4 * j + 3] = __uint_as_float(x3);
+            }
+        };
+        float sv[32], vn[32];
+        int2 cur = load_rec(0), nxt = load_rec(1);
+        if (use_tab) {
+            ptx::sts64(rec_tab + lane * 8, (uint32_t)cur.x, (uint32_t)cur.y);
+            __syncwarp();
+        }
+        if (has_values) {
+            issue_values(rec_tab, vn);
+            transpose_values(vn, sv);
+        }
+        B2SP_FPROF_DECL
+        B2SP_FPROF_START
         for (int it = 0; it < nwin; ++it) {
             const int pb = it & 1;
-            const int2 rec = nxt;
-            nxt = make_int2(0, 0);
-            if (grow < a.M && it + 1 < nwin) nxt = __ldg(my_win + it + 1);
-            const unsigned mask = (unsigned)rec.y;
-
-            // Stored values of the window, densified per row (0 where nothing is stored).  Expansion is
-            // cooperative: for each row of the warp, lane = column.
-            float sv[32];
-            if (has_values || !FUSED) {
-                __syncwarp();
-                ptx::sts64(rec_tab + lane * 8, (uint32_t)rec.x, mask);
+            const uint32_t tab_cur = rec_tab + (it & 1) * 256, tab_nxt = rec_tab + ((it + 1) & 1) * 256;
+            const unsigned mask = (unsigned)cur.y;
+            if (use_tab) {   // records of window it+1 for the whole warp; its values start loading now
+                ptx::sts64(tab_nxt + lane * 8, (uint32_t)nxt.x, (uint32_t)nxt.y);
                 __syncwarp();
             }
-            if (has_values) {
-                ptx::for_each_row<32>([&](auto rc) {
-                    constexpr int r = decltype(rc)::value;
-                    uint32_t pos, m;
-                    ptx::lds64_off<r * 8>(rec_tab, pos, m);
-                    float v = 0.f;
-                    if (m & lane_bit) v = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
-                    ptx::sts32_off<r * 128>(stage_v + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(v));
-                });
-                __syncwarp();
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t x0, x1, x2, x3;
-                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                                 : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
-                                 : "r"(stage_v + lane * 128 + (uint32_t)((j ^ (lane & 7)) << 4)));
-                    sv[4 * j] = __uint_as_float(x0); sv[4 * j + 1] = __uint_as_float(x1);
-                    sv[4 * j + 2] = __uint_as_float(x2); sv[4 * j + 3] = __uint_as_float(x3);
-                }
-            } else {
+            if (has_values && it + 1 < nwin) issue_values(tab_nxt, vn);
+            const int2 nxt2 = load_rec(it + 2);
+            if (!has_values) {
 #pragma unroll
                 for (int c = 0; c < 32; ++c) sv[c] = (mask >> c) & 1u ? 1.f : 0.f;
             }
-
+            B2SP_FPROF_STOP(0)
             {   // P is ready?
                 bool ok = ptx::mbar_wait(p_full(pb), (it >> 1) & 1);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
             }
+            B2SP_FPROF_STOP(1)
             ptx::tc_fence_after_sync();
             uint32_t p0[16], p1[16];
             ptx::tmem_ld_32x16(tmem + lane_addr + kColP + pb * kFusedW, p0);
@@ -278,6 +323,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(p_free(pb));
+            B2SP_FPROF_STOP(2)
 
             if (FUSED) {
                 uint32_t hi[16], lo[16];
@@ -286,6 +332,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
                 }
+                B2SP_FPROF_STOP(3)
 #pragma unroll
                 for (int c = 0; c < 16; ++c) ptx::split_tf32_fast(__uint_as_float(p0[c]) * sv[c], hi[c], lo[c]);
                 ptx::tmem_st_32x16(tmem + lane_addr + kColPPhi, hi);
@@ -298,6 +345,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(pp_full);
+                B2SP_FPROF_STOP(4)
             } else {
                 // SDDMM: stage the masked, scaled row (dense, 32 columns) and write the stored entries
                 // row by row with lane = column, so each row's outputs are one contiguous store.
@@ -317,12 +365,17 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::for_each_row<32>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     uint32_t pos, m, v;
-                    ptx::lds64_off<r * 8>(rec_tab, pos, m);
+                    ptx::lds64_off<r * 8>(tab_cur, pos, m);
                     asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(stage_v + (uint32_t)((lane << 2) ^ ((r & 7) << 4))), "n"(r * 128));
                     if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = __uint_as_float(v);
                 });
             }
+            // the values of window it+1 have had the whole step to arrive: give each thread its row
+            if (has_values && it + 1 < nwin) transpose_values(vn, sv);
+            cur = nxt;
+            nxt = nxt2;
         }
+        if (ew == 0) { B2SP_FPROF_FLUSH(8) }
         // ---------------- epilogue: O accumulator -> global ----------------
         if (FUSED) {
             {
