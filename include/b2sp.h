@@ -31,9 +31,15 @@
  *   B2SP_ALGO_AUTO     the library chooses (fastest family whose preconditions hold);
  *   B2SP_ALGO_ROW      CUDA-core row kernels, rows taken longest-first (binned by length);
  *   B2SP_ALGO_ROW_NAT  the same kernels, rows in natural order (no binning pass);
- *   B2SP_ALGO_TILE     dense-tile tensor-core kernels (tcgen05, 3xTF32 split).  They need
- *                      column indices sorted within each row; if an explicit request cannot be
- *                      met the call returns B2SP_ERR_UNSUPPORTED.
+ *   B2SP_ALGO_TILE     dense-tile tensor-core kernels (tcgen05 + tensor memory, every operand
+ *                      split into two tf32 numbers so that fp32 accuracy is kept).  A pre-pass
+ *                      over col_idx builds a table of 32-column windows; it also detects rows
+ *                      whose columns are not strictly increasing, in which case the row kernels
+ *                      produce the result instead (decided on the device, inside the same call).
+ *                      B2SP_ERR_UNSUPPORTED if the sizes are outside the family (SDDMM/FusedMM:
+ *                      Kd > 128), B2SP_ERR_WORKSPACE if the workspace is too small for it.
+ *   B2SP_ALGO_TILE_PREPARED  as TILE, but the window table is taken from the workspace, where an
+ *                      earlier b2sp_prepare_pattern call for the same S left it (see there).
  * Floating-point results of the families differ in summation order only; all stay within
  * |x - exact| <= 1e-5 * sum|terms| + 1e-6.
  */
@@ -57,7 +63,8 @@ typedef enum {
     B2SP_ERR_TOO_LARGE = 7    /* the problem does not fit the library's built-in scratch array */
 } b2sp_status;
 
-enum { B2SP_ALGO_AUTO = 0, B2SP_ALGO_ROW = 1, B2SP_ALGO_ROW_NAT = 2, B2SP_ALGO_TILE = 3 };
+enum { B2SP_ALGO_AUTO = 0, B2SP_ALGO_ROW = 1, B2SP_ALGO_ROW_NAT = 2, B2SP_ALGO_TILE = 3,
+       B2SP_ALGO_TILE_PREPARED = 4 };
 enum { B2SP_OP_SPMM = 0, B2SP_OP_SDDMM = 1, B2SP_OP_FUSEDMM = 2 };
 
 /* Library version (major*10000 + minor*100 + patch). */
@@ -72,6 +79,22 @@ const char *b2sp_status_string(b2sp_status s);
  * (Kd for SPMM, N for SDDMM) may be 0.  Returns 0 on invalid arguments.
  */
 size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz);
+
+/*
+ * Pattern analysis shared by the dense-tile kernels of all three ops (work assignment and index
+ * staging: where the paper's kernels cut each row's ja array into blocks of VLC = 32 entries on the
+ * fly, this library cuts each row into windows of 32 columns once).  Builds, in `workspace`, the
+ * table of (first position, occupancy mask) per row and window from row_ptr / col_idx and records
+ * which arrays it was built from.  Any later b2sp_spmm / b2sp_sddmm / b2sp_fusedmm call with
+ * algo = B2SP_ALGO_TILE_PREPARED, the same workspace and the same M, K, nnz, row_ptr, col_idx
+ * skips its own pre-pass.  The caller promises that the contents of row_ptr and col_idx did not
+ * change in between; a workspace that does not hold a matching table (never prepared, prepared for
+ * another S, or used by a B2SP_ALGO_ROW call since) is detected on the device and the row kernels
+ * produce the result instead.  `workspace` must be at least as large as b2sp_workspace_bytes says
+ * for the ops that will use it.  Asynchronous on `stream`.
+ */
+b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                                 void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * SPMM, Eq. 2 / Alg. 2 (SPMM-ROW):  O[i, :] = sum over stored entries (s, k) of row i of

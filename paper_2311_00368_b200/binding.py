@@ -18,9 +18,9 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.environ.get("B2SP_LIB") or os.path.join(_HERE, "libb2sp.so")  # B2SP_LIB: alternate build
 
-ALGO_AUTO, ALGO_ROW, ALGO_ROW_NAT, ALGO_TILE = 0, 1, 2, 3
+ALGO_AUTO, ALGO_ROW, ALGO_ROW_NAT, ALGO_TILE, ALGO_TILE_PREPARED = 0, 1, 2, 3, 4
 OP_SPMM, OP_SDDMM, OP_FUSEDMM = 0, 1, 2
-ALGO_NAMES = {0: "auto", 1: "row", 2: "row_nat", 3: "tile", -1: "none"}
+ALGO_NAMES = {0: "auto", 1: "row", 2: "row_nat", 3: "tile", 4: "tile_prepared", -1: "none"}
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -51,6 +51,8 @@ lib.b2sp_fusedmm_host.restype = _i
 lib.b2sp_fusedmm_host.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.b2sp_spmm_static_scratch.restype = _i
 lib.b2sp_spmm_static_scratch.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp]
+lib.b2sp_prepare_pattern.restype = _i
+lib.b2sp_prepare_pattern.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_validate_csr.restype = _i
 lib.b2sp_validate_csr.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_device_status.restype = _i
@@ -238,6 +240,14 @@ def fusedmm_host(row_ptr, col_idx, s_values, A, B, D, out):
     _check(lib.b2sp_fusedmm_host(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values),
                                  _ptr(A), _ptr(B), _ptr(D), _ptr(out), _stream()), "b2sp_fusedmm_host")
     return out
+
+
+def prepare_pattern(row_ptr, col_idx, K, workspace):
+    """b2sp_prepare_pattern: build S's window table in `workspace` once; later calls that pass the same
+    workspace and algo=ALGO_TILE_PREPARED reuse it."""
+    M, nnz = row_ptr.numel() - 1, col_idx.numel()
+    _check(lib.b2sp_prepare_pattern(M, K, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(workspace),
+                                    workspace.numel(), _stream()), "b2sp_prepare_pattern")
 
 
 def validate_csr(row_ptr, col_idx, K) -> bool:

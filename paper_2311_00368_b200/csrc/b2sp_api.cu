@@ -221,7 +221,9 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || N < 0) return B2SP_ERR_INVALID_ARG;
-    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return B2SP_ERR_INVALID_ARG;
+    const bool prepared = algo == B2SP_ALGO_TILE_PREPARED;
+    if (prepared) algo = B2SP_ALGO_TILE;
     if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && (!values || !D || ldd < N)) return B2SP_ERR_INVALID_ARG;
     const size_t row_bytes = row_workspace_bytes(M);
@@ -241,7 +243,7 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
-        rc = spmm_tile(plan, M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, st, &launches);
+        rc = spmm_tile(plan, prepared, M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
@@ -296,7 +298,9 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0) return B2SP_ERR_INVALID_ARG;
-    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return B2SP_ERR_INVALID_ARG;
+    const bool prepared = algo == B2SP_ALGO_TILE_PREPARED;
+    if (prepared) algo = B2SP_ALGO_TILE;
     if (nnz > 0 && !out_values) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
     const size_t row_bytes = row_workspace_bytes(M);
@@ -319,7 +323,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
-        rc = fused_tile(plan, false, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
+        rc = fused_tile(plan, prepared, false, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
                         out_values, 0, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
@@ -374,7 +378,9 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0 || N < 0) return B2SP_ERR_INVALID_ARG;
-    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE) return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return B2SP_ERR_INVALID_ARG;
+    const bool prepared = algo == B2SP_ALGO_TILE_PREPARED;
+    if (prepared) algo = B2SP_ALGO_TILE;
     if (M > 0 && N > 0 && (!O || ldo < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && (!D || ldd < N)) return B2SP_ERR_INVALID_ARG;
     if (nnz > 0 && N > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
@@ -395,7 +401,7 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
-        rc = fused_tile(plan, true, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
+        rc = fused_tile(plan, prepared, true, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
                         workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
@@ -412,6 +418,18 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
     return rc;
+}
+
+b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                                 void *workspace, size_t workspace_bytes, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || M == 0 || K == 0 || nnz == 0) return B2SP_ERR_INVALID_ARG;
+    const size_t need = pattern_table_offset(M) + pattern_table_bytes(M, K);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, need);
+    if (rc != B2SP_OK) return rc;
+    int launches = 0;
+    return pattern_pass(false, M, K, nnz, row_ptr, col_idx, workspace, st, &launches);
 }
 
 b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,

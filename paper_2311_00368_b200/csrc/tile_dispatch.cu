@@ -83,11 +83,51 @@ b2sp_status launch_spmm_tile(const CUtensorMap &hi, const CUtensorMap &lo, const
 
 }  // namespace
 
+size_t pattern_table_offset(int M)
+{
+    return align_up(align_up(kWsHeaderBytes + sizeof(int) * (size_t)M, 256), 1024);
+}
+size_t pattern_table_bytes(int M, int K)
+{
+    return sizeof(int2) * (size_t)M * (size_t)((K + kTileKC - 1) / kTileKC);
+}
+
+b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                         void *workspace, cudaStream_t st, int *launches)
+{
+    char *ws = static_cast<char *>(workspace);
+    int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
+    PatternSignature *sig_dev = reinterpret_cast<PatternSignature *>(ws + kWsSignatureOffset);
+    const int Wk = (K + kTileKC - 1) / kTileKC;
+    PatternSignature sig{kPatternMagic, M, K, Wk, nnz, row_ptr, col_idx};
+    if (prepared) {
+        // keep the table, its flag and its signature; clear only the status / profiling words
+        if (cudaMemsetAsync(ws + kWsStatusOffset, 0, kWsTileFlagsOffset - kWsStatusOffset, st) != cudaSuccess ||
+            cudaMemsetAsync(ws + kWsStatusOffset + 128, 0, kWsSignatureOffset - kWsStatusOffset - 128, st) != cudaSuccess)
+            return B2SP_ERR_CUDA;
+        check_signature_kernel<<<1, 1, 0, st>>>(sig, sig_dev, flags);
+        *launches += 1;
+        return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
+    }
+    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
+    int2 *win = reinterpret_cast<int2 *>(ws + pattern_table_offset(M));
+    const int GR = (Wk + 31) / 32;               // warps per row
+    const long long threads = (long long)M * GR * 32;
+    tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, Wk, GR, row_ptr, col_idx, win, flags);
+    write_signature_kernel<<<1, 1, 0, st>>>(sig, sig_dev);
+    *launches += 2;
+    return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
+}
+
 bool tile_profitable(int M, int K, int width, long long nnz)
 {
-    if (M < 128 || K < 128 || width < 16 || nnz <= 0) return false;
-    double density = (double)nnz / ((double)M * (double)K);
-    return density >= 0.04;
+    // Measured on B200: the dense-tile family pays a pattern pre-pass and does
+    // 3 / density times the useful flops on the tensor cores; it overtakes the row family from
+    // about 15% density, earlier on large matrices where the pre-pass amortises.
+    if (M < 256 || K < 256 || width < 16 || nnz <= 0) return false;
+    const double cells = (double)M * (double)K;
+    const double density = (double)nnz / cells;
+    return density >= 0.15 || (density >= 0.08 && cells >= 48.0e6);
 }
 
 TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
@@ -118,7 +158,7 @@ TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
     return p;
 }
 
-b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, const int *row_ptr,
+b2sp_status spmm_tile(const TilePlan &p, bool prepared, int M, int K, int N, long long nnz, const int *row_ptr,
                       const int *col_idx, const float *values, const float *D, long long ldd, float *O,
                       long long ldo, void *workspace, cudaStream_t st, int *launches)
 {
@@ -135,19 +175,16 @@ b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, con
         !make_blocked_map(&tm_lo, dlo, p.Kp, p.Np / 32, kTileKC, kTileN / 32, true))
         return B2SP_ERR_CUDA;
 
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
     {
-        const int GR = (p.Wk + 31) / 32;               // warps per row
-        const long long threads = (long long)M * GR * 32;
-        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, GR, row_ptr, col_idx, win,
-                                                                              flags);
+        b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
+        if (prc != B2SP_OK) return prc;
     }
     {
         long long groups = (long long)p.Kp * (p.Np / 4);
         int blocks = (int)((groups + 255) / 256 < (long long)kSMs * 8 ? (groups + 255) / 256 : (long long)kSMs * 8);
         split_dense_kernel<<<blocks, 256, 0, st>>>(D, ldd, K, N, dhi, dlo, p.Kp, p.Np);
     }
-    *launches += 2;
+    *launches += 1;
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
 
     SpmmTileArgs a;
@@ -241,12 +278,11 @@ void launch_split(const float *X, long long ld, int rows, int cols, float *hi, f
 
 }  // namespace
 
-b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int N, long long nnz,
+b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches)
 {
-    (void)nnz;
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
@@ -267,15 +303,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int
         tm_dh = tm_bh;   // unused by the SDDMM kernel
         tm_dl = tm_bl;
     }
-    if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
     {
-        const int GR = (p.Wk + 31) / 32;
-        const long long threads = (long long)M * GR * 32;
-        tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, p.Wk, GR, row_ptr, col_idx, win,
-                                                                              flags);
+        b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
+        if (prc != B2SP_OK) return prc;
     }
     launch_split(B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, st);
-    *launches += 2;
+    *launches += 1;
     if (fused) {
         launch_split(D, ldd, K, N, dhi, dlo, p.Kp, p.Np, st);
         *launches += 1;

@@ -10,6 +10,7 @@ namespace b2sp {
 // Byte offsets inside the workspace header that both families agree on.
 constexpr size_t kWsStatusOffset = 256;      // int: device status word (0 = ok)
 constexpr size_t kWsTileFlagsOffset = 320;   // int[..]: flags written by the tile pre-pass
+constexpr size_t kWsSignatureOffset = 448;   // int[16]: which CSR arrays the window table was built from
 constexpr size_t kWsHeaderBytes = 512;
 
 struct TilePlan {
@@ -32,7 +33,7 @@ struct FusedPlan {
 };
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused);
 
-b2sp_status fused_tile(const FusedPlan &p, bool fused, int M, int K, int Kd, int N, long long nnz,
+b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches);
@@ -42,8 +43,17 @@ bool tile_profitable(int M, int K, int width, long long nnz);
 
 // Enqueues pre-pass + tile kernel (+ reduction).  The kernels leave immediately if the pre-pass
 // finds a row whose columns are not strictly increasing (flag at kWsTileFlagsOffset).
-b2sp_status spmm_tile(const TilePlan &p, int M, int K, int N, long long nnz, const int *row_ptr,
+b2sp_status spmm_tile(const TilePlan &p, bool prepared, int M, int K, int N, long long nnz, const int *row_ptr,
                       const int *col_idx, const float *values, const float *D, long long ldd, float *O,
                       long long ldo, void *workspace, cudaStream_t st, int *launches);
+
+// Offset of the window table inside the workspace (the same for every op) and its size.
+size_t pattern_table_offset(int M);
+size_t pattern_table_bytes(int M, int K);
+
+// Builds the window table (`prepared` = false) or checks that the workspace holds one for these
+// arrays (`prepared` = true; a mismatch raises the device flag that sends the work to the row kernels).
+b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+                         void *workspace, cudaStream_t st, int *launches);
 
 }  // namespace b2sp

@@ -94,6 +94,25 @@ __global__ void tile_masks_kernel(int M, int K, int Wk, int GR, const int *__res
     if (bad) atomicExch(&flags[kFlagUnsorted], 1);
 }
 
+// ---- table signature ------------------------------------------------------------------------------------
+struct PatternSignature {
+    int magic, M, K, Wk;
+    long long nnz;
+    const int *row_ptr, *col_idx;
+};
+constexpr int kPatternMagic = 0x62327370;
+
+__global__ void write_signature_kernel(PatternSignature sig, PatternSignature *dst) { *dst = sig; }
+
+// Raises flags[kFlagUnsorted] when the workspace does not hold a table built from these arrays.
+__global__ void check_signature_kernel(PatternSignature want, const PatternSignature *have, int *flags)
+{
+    const PatternSignature h = *have;
+    if (h.magic != want.magic || h.M != want.M || h.K != want.K || h.Wk != want.Wk || h.nnz != want.nnz ||
+        h.row_ptr != want.row_ptr || h.col_idx != want.col_idx)
+        atomicExch(&flags[kFlagUnsorted], 1);
+}
+
 // ---- dense operand split ----------------------------------------------------------------------------
 // X [rows x cols] (ld) -> hi, lo in a column-blocked layout: element (r, c) lives at
 // ((c/32)*rows_p + r)*32 + c%32, i.e. [cols_p/32][rows_p][32] floats, zero in the padding

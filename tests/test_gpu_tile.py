@@ -215,9 +215,12 @@ def test_fused_tile_configs(b):
     d = DevProblem(p)
     ws = _ws(b, b.OP_SDDMM, p)
     ref, T = oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B)
-    out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=0)
+    out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=TILE)
     assert b.last_algo(b.OP_SDDMM) == TILE and b.device_status(ws) == 0
-    assert gate(out, ref, T, "sddmm config, auto") < 0.5
+    assert gate(out, ref, T, "sddmm config, tile") < 0.5
+    out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=0)
+    assert b.last_algo(b.OP_SDDMM) == 1   # 10% density at 4096^2: the planner keeps the row kernels
+    gate(out, ref, T, "sddmm config, auto")
     p = W.attention_case(3)
     d = DevProblem(p)
     ws = _ws(b, b.OP_FUSEDMM, p)
@@ -228,3 +231,41 @@ def test_fused_tile_configs(b):
         ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D, rows=(r, r + 1))
         ok, ratio = oracle.within_tolerance(out[r:r + 1].cpu().numpy(), ref, T)
         assert ok, f"attention row {r}: {ratio:.3g}"
+
+
+# ---- prepared pattern ------------------------------------------------------------------------------
+
+def test_prepared_pattern_is_shared_by_all_ops_and_stale_tables_are_detected(b):
+    PREP = 4
+    p = W.small_random(501, 300, 700, 0.25, 64, 128)
+    d = DevProblem(p)
+    n = max(b.workspace_bytes(op, p.M, p.K, p.Kd, p.N, p.nnz) for op in range(3))
+    ws = torch.empty(max(n, 1 << 20), dtype=torch.uint8, device="cuda")
+    b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
+    refs = {"spmm": oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D),
+            "sddmm": oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B),
+            "fusedmm": oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)}
+
+    def run_all(tag):
+        for _ in range(2):   # the table survives repeated use by all three ops
+            out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=PREP)
+            gate(out, *refs["spmm"], f"spmm prepared {tag}")
+            out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=PREP)
+            gate(out, *refs["sddmm"], f"sddmm prepared {tag}")
+            out = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=PREP)
+            gate(out, *refs["fusedmm"], f"fusedmm prepared {tag}")
+            assert b.device_status(ws) == 0
+
+    run_all("fresh")
+    # a workspace prepared for another matrix must not be trusted: the result stays correct
+    q = W.small_random(502, 300, 700, 0.25, 64, 128)
+    dq = DevProblem(q)
+    b.prepare_pattern(dq.row_ptr, dq.col_idx, q.K, ws)
+    run_all("stale table")
+    # neither must a workspace that was never prepared (garbage header)
+    ws.fill_(0x5a)
+    run_all("garbage workspace")
+    # nor one whose header a row-family call has rewritten
+    b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
+    b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=1)
+    run_all("after a row-family call")
