@@ -215,14 +215,14 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     FusedPlan p;
     if (M <= 0 || K <= 0 || Kd <= 0 || Kd > 128 || nnz <= 0 || (fused && N <= 0)) return p;
     p.Wk = (K + kFusedW - 1) / kFusedW;
-    p.Kp = p.Wk * kFusedW;
+    p.Kp = (K + kFusedBlk - 1) / kFusedBlk * kFusedBlk;   // operand copies padded to whole 128-column blocks
     p.Kdp = Kd <= 32 ? 32 : Kd <= 64 ? 64 : 128;
     p.Mt = (M + kFusedRows - 1) / kFusedRows;
     p.Nt = fused ? (N + kFusedNT - 1) / kFusedNT : 1;
     p.Np = fused ? p.Nt * kFusedNT : 0;
     size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30) return p;
-    p.KS = pick_split(p.Mt * p.Nt, p.Wk);
+    p.KS = pick_split(p.Mt * p.Nt, p.Kp / kFusedBlk);
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
     off = align_up(off + win_bytes, 1024);
@@ -251,7 +251,7 @@ template <int KDP, bool FUSED>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                               const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
 {
-    using Cfg = FusedCfg<KDP>;
+    using Cfg = FusedCfg<KDP, FUSED>;
     auto kern = fused_tile_kernel<KDP, FUSED>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
@@ -292,8 +292,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int
     float *part = reinterpret_cast<float *>(ws + p.off_part);
 
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
-    if (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedW, p.Kdp / 32, false) ||
-        !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedW, p.Kdp / 32, false))
+    if (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
+        !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false))
         return B2SP_ERR_CUDA;
     if (fused) {
         if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true) ||

@@ -1,19 +1,21 @@
 // Dense-tile FusedMM and SDDMM (tcgen05 / TMEM / TMA, 3xTF32) over the window table of S.
 //
-// One CTA owns 128 rows of S (= rows of A and O) and a range of 32-column windows of S.
-//   * A_tile (128 x Kd) is split into tf32 hi/lo once and kept in tensor memory for the CTA's life.
-//   * Per window: GEMM1  P = A_tile * B_window^T  (128 x 32, A from TMEM, B rows by TMA), into one of
-//     two P accumulators in TMEM.
-//   * Four warps (thread = row) read P, apply the window's occupancy mask and the stored values
-//     (the sampled C of the paper exists only in these registers), split the result into hi/lo and
-//     write it back to TMEM as P'.
-//   * FusedMM: GEMM2  O += P' * D_window  (A = P' from TMEM, B = D rows by TMA, MN-major), O in TMEM.
-//     SDDMM: the masked values are written to out_values instead (coalesced through shared memory).
-// The MMA thread issues GEMM1 of window t+1 before GEMM2 of window t, so the tensor pipe works while
-// the element-wise stage of window t runs.
+// One CTA owns 128 rows of S (= rows of A and O) and a range of 128-column blocks of S (4 windows).
+//   * A_tile (128 x Kd) is split into tf32 hi/lo once: A_hi lives in tensor memory for the CTA's
+//     life; A_lo lives in tensor memory too (SDDMM) or in shared memory (FusedMM, where TMEM is
+//     needed for O and P').
+//   * Per block: GEMM1  P = A_tile * B_block^T  (128 x 128).  The B rows of the block arrive by TMA
+//     in chunks of 32 k (hi + lo, 32 KB); N = 128 MMAs run the tensor pipe at full rate (a 128xNx8
+//     tf32 MMA costs max(N/2, 45.6) cycles, so 32-column GEMMs would waste two thirds of it).
+//   * Four warps (thread = row) read P window by window (32 columns), apply the window's occupancy
+//     mask and stored values (the sampled C of the paper exists only in these registers), and
+//       - FusedMM: split the result into hi/lo and write it back to TMEM as P' (two buffers); GEMM2
+//         O += P'_window * D_window (A = P' from TMEM, B = D rows by TMA, MN-major) accumulates O in TMEM;
+//       - SDDMM: write the stored entries to out_values (coalesced through shared memory).
 //
-// TMEM columns (512 allocated): O [0,128)  P0 [128,160)  P1 [160,192)  P'hi [192,224)  P'lo [224,256)
-//                               A_hi [256, 256+Kdp)      A_lo [384, 384+Kdp)          (Kdp <= 128)
+// TMEM columns (512 allocated)
+//   FusedMM: O [0,128)  P [128,256)  P'0 hi/lo [256,288)/[288,320)  P'1 hi/lo [320,352)/[352,384)  A_hi [384,384+Kdp)
+//   SDDMM:   P0 [0,128) P1 [128,256) A_hi [256,256+Kdp)  A_lo [384,384+Kdp)
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -36,11 +38,11 @@
 namespace b2sp {
 
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
-constexpr int kFusedW = 32;         // S columns per stage (one window)
-constexpr int kFusedStages = 3;
+constexpr int kFusedW = 32;         // S columns per window
+constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 constexpr int kFusedThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: element-wise / epilogue
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
-constexpr uint32_t kColO = 0, kColP = 128, kColPPhi = 192, kColPPlo = 224, kColAhi = 256, kColAlo = 384;
+constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
@@ -55,14 +57,17 @@ struct FusedTileArgs {
     unsigned long long *prof;  // optional role timers (profiling builds only)
 };
 
-template <int KDP>
+template <int KDP, bool FUSED>
 struct FusedCfg {
-    static constexpr int B_BYTES = kFusedW * KDP * 4;          // B window tile (hi or lo)
-    static constexpr int D_BYTES = kFusedW * kFusedNT * 4;     // D window tile (hi or lo): 16 KB
-    static constexpr int STAGE_BYTES = 2 * B_BYTES + 2 * D_BYTES;
-    static constexpr int STAGE_BYTES_SDDMM = 2 * B_BYTES;
+    static constexpr int NCH_B = KDP / 32;                     // B chunks per block
+    static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
+    static constexpr int ALO_BYTES = FUSED ? kFusedRows * KDP * 4 : 0;
+    static constexpr int RING = FUSED ? 4 : 6;
     static constexpr int AUX_BYTES = 256 /*barriers*/ + 4 * 512 /*record tables*/ + 4 * 4096 /*value staging*/;
-    static constexpr int SMEM_BYTES = kFusedStages * STAGE_BYTES + 1024 + AUX_BYTES;
+    static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
+    // tensor-memory columns
+    static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
+    static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
 
 // FUSED = true: FusedMM (GEMM2 + O epilogue).  FUSED = false: SDDMM (write the sampled values).
@@ -72,36 +77,43 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
                   const FusedTileArgs a)
 {
-    using Cfg = FusedCfg<KDP>;
-    constexpr int STAGES = kFusedStages;
-    constexpr int STAGE_BYTES = FUSED ? Cfg::STAGE_BYTES : Cfg::STAGE_BYTES_SDDMM;
+    using Cfg = FusedCfg<KDP, FUSED>;
+    constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B, NCH_D = Cfg::NCH_D;
+    constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
     if (a.flags[0] != 0) return;  // pattern not usable for tiles: the row kernels take over
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t aux = smem_base + STAGES * STAGE_BYTES;
+    const uint32_t ring = smem_base;                               // RING chunks of 32 KB
+    const uint32_t alo_smem = smem_base + RING * kFusedChunk;      // FusedMM: A_lo, K-major, 16 KB per 32 k
+    const uint32_t aux = alo_smem + Cfg::ALO_BYTES;
     auto full = [&](int s) { return aux + 8u * s; };
-    auto empty = [&](int s) { return aux + 8u * (STAGES + s); };
-    auto p_full = [&](int b) { return aux + 8u * (2 * STAGES + b); };
-    auto p_free = [&](int b) { return aux + 8u * (2 * STAGES + 2 + b); };
-    const uint32_t pp_full = aux + 8u * (2 * STAGES + 4), pp_free = aux + 8u * (2 * STAGES + 5);
-    const uint32_t o_full = aux + 8u * (2 * STAGES + 6);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + STAGES * STAGE_BYTES + 8 * (2 * STAGES + 7));
+    auto empty = [&](int s) { return aux + 8u * (RING + s); };
+    auto p_full = [&](int b) { return aux + 8u * (2 * RING + b); };
+    auto p_free = [&](int b) { return aux + 8u * (2 * RING + 2 + b); };
+    auto pp_full = [&](int b) { return aux + 8u * (2 * RING + 4 + b); };
+    auto pp_free = [&](int b) { return aux + 8u * (2 * RING + 6 + b); };
+    const uint32_t o_full = aux + 8u * (2 * RING + 8);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 9));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ks = blockIdx.x % a.KS;
     const int tile = blockIdx.x / a.KS;
     const int nt = tile % a.Nt, mt = tile / a.Nt;
-    const int w0 = (int)((long long)a.Wk * ks / a.KS), w1 = (int)((long long)a.Wk * (ks + 1) / a.KS);
-    const int nwin = w1 - w0;
+    const int nblk_all = (a.Wk + WPB - 1) / WPB;
+    const int b0 = (int)((long long)nblk_all * ks / a.KS), b1 = (int)((long long)nblk_all * (ks + 1) / a.KS);
+    const int nblk = b1 - b0;
     const int m0 = mt * kFusedRows, n0 = nt * kFusedNT;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
-        for (int b = 0; b < 2; ++b) { ptx::mbar_init(p_full(b), 1); ptx::mbar_init(p_free(b), 4); }
-        ptx::mbar_init(pp_full, 4);
-        ptx::mbar_init(pp_free, 1);
+        for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(p_full(b), 1);
+            ptx::mbar_init(p_free(b), 4);
+            ptx::mbar_init(pp_full(b), 4);
+            ptx::mbar_init(pp_free(b), 1);
+        }
         ptx::mbar_init(o_full, 1);
         ptx::fence_mbar_init();
     }
@@ -116,7 +128,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const uint32_t tmem = *tmem_slot;
     bool failed = false;
 
-    // ---- A tile -> TMEM (hi / lo), done by the element-wise warps; thread = row ----
+    // ---- A tile -> TMEM (hi, and lo for SDDMM) / shared memory (lo for FusedMM); thread = row ----
     const int q = warp & 3;                 // TMEM lane quarter of warps 2..5
     const int row = q * 32 + lane;          // row inside the tile (warps >= 2)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
@@ -145,93 +157,118 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
 #pragma unroll
             for (int i = 0; i < 16; ++i) ptx::split_tf32_fast(v[i], hi[i], lo[i]);
-            ptx::tmem_st_32x16(tmem + lane_addr + kColAhi + c, hi);
-            ptx::tmem_st_32x16(tmem + lane_addr + kColAlo + c, lo);
+            ptx::tmem_st_32x16(tmem + lane_addr + Cfg::COL_AHI + c, hi);
+            if (FUSED) {
+                // K-major, 128-byte swizzle: 16 KB sub-tile per 32 k, row = 128 B, 16-byte chunk j at j ^ (row & 7)
+                const uint32_t base = alo_smem + (c >> 5) * (kFusedRows * 128) + row * 128;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t chunk = (uint32_t)(((c & 31) >> 2) + j);
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(base + ((chunk ^ (row & 7)) << 4)),
+                                 "r"(lo[4 * j]), "r"(lo[4 * j + 1]), "r"(lo[4 * j + 2]), "r"(lo[4 * j + 3]) : "memory");
+                }
+            } else {
+                ptx::tmem_st_32x16(tmem + lane_addr + Cfg::COL_ALO + c, lo);
+            }
         }
         ptx::tmem_st_wait();
+        if (FUSED) ptx::fence_proxy_async_smem();
     }
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
 
     if (warp == 0) {
-        // ---------------- TMA producer ----------------
+        // ---------------- TMA producer: per block NCH_B chunks of B rows, then NCH_D chunks of D rows ----------------
         if (lane == 0) {
             ptx::tma_prefetch_desc(&tm_bhi);
             ptx::tma_prefetch_desc(&tm_blo);
             if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); ptx::tma_prefetch_desc(&tm_dlo); }
-            int issued = 0;
-            for (int it = 0; it < nwin; ++it) {
-                const int s = it % STAGES;
-                if (it >= STAGES && !ptx::mbar_wait(empty(s), ((it / STAGES) - 1) & 1)) { failed = true; break; }
-                const uint32_t dst = smem_base + s * STAGE_BYTES;
-                ptx::mbar_arrive_expect_tx(full(s), STAGE_BYTES);
-                const int krow = (w0 + it) * kFusedW;
-                ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, krow, 0);
-                ptx::tma_load_3d(dst + Cfg::B_BYTES, &tm_blo, full(s), 0, krow, 0);
-                if (FUSED) {
-                    ptx::tma_load_3d(dst + 2 * Cfg::B_BYTES, &tm_dhi, full(s), 0, krow, nt * (kFusedNT / 32));
-                    ptx::tma_load_3d(dst + 2 * Cfg::B_BYTES + Cfg::D_BYTES, &tm_dlo, full(s), 0, krow, nt * (kFusedNT / 32));
+            int c = 0;
+            for (int b = 0; b < nblk && !failed; ++b) {
+                const int col0 = (b0 + b) * kFusedBlk;
+                for (int i = 0; i < NCH_B + NCH_D; ++i, ++c) {
+                    const int s = c % RING;
+                    if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) { failed = true; break; }
+                    const uint32_t dst = ring + s * kFusedChunk;
+                    ptx::mbar_arrive_expect_tx(full(s), kFusedChunk);
+                    if (i < NCH_B) {   // B rows col0..col0+127, k group i
+                        ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
+                        ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
+                    } else {           // D rows of window i - NCH_B
+                        const int krow = col0 + (i - NCH_B) * kFusedW;
+                        ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (kFusedNT / 32));
+                        ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (kFusedNT / 32));
+                    }
                 }
-                issued = it + 1;
             }
             if (failed)
-                for (int it = issued > STAGES ? issued - STAGES : 0; it < issued; ++it)
-                    ptx::mbar_wait(full(it % STAGES), (it / STAGES) & 1);
+                for (int j = c > RING ? c - RING : 0; j < c; ++j) ptx::mbar_wait(full(j % RING), (j / RING) & 1);
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
-            constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedW, false, false);
+            constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedBlk, false, false);
             constexpr uint32_t idesc2 = ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
             B2SP_FPROF_DECL
             B2SP_FPROF_START
-            auto gemm1 = [&](int it) -> bool {   // P[it & 1] = A_tile * B_window^T
-                const int s = it % STAGES, pb = it & 1;
-                if (!ptx::mbar_wait(full(s), (it / STAGES) & 1)) return false;
+            int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
+            for (int b = 0; b < nblk && !failed; ++b) {
+                const int pb = FUSED ? 0 : (b & 1);
+                // P buffer drained by the element-wise warps?
+                const int puse = FUSED ? b : (b >> 1);
+                if (puse > 0 && !ptx::mbar_wait(p_free(pb), (puse - 1) & 1)) { failed = true; break; }
                 B2SP_FPROF_STOP(0)
-                if (it >= 2 && !ptx::mbar_wait(p_free(pb), ((it >> 1) - 1) & 1)) return false;
-                B2SP_FPROF_STOP(1)
-                ptx::tc_fence_after_sync();
-                const uint32_t b_hi = smem_base + s * STAGE_BYTES, b_lo = b_hi + Cfg::B_BYTES;
-                const uint32_t pacc = tmem + kColP + pb * kFusedW;
-#pragma unroll
-                for (int kk = 0; kk < KDP / 8; ++kk) {
-                    // B window: K-major, one 4 KB sub-tile (32 rows x 128 B, 128-byte swizzle) per 32 k
-                    const uint32_t off = (kk >> 2) * (kFusedW * 128) + (kk & 3) * 32;
-                    const uint64_t dbh = ptx::smem_desc(b_hi + off, 16, 1024, ptx::kLayoutSw128);
-                    const uint64_t dbl = ptx::smem_desc(b_lo + off, 16, 1024, ptx::kLayoutSw128);
-                    ptx::mma_tf32_ts(pacc, tmem + kColAhi + kk * 8, dbh, idesc1, kk != 0);
-                    ptx::mma_tf32_ts(pacc, tmem + kColAlo + kk * 8, dbh, idesc1, 1);
-                    ptx::mma_tf32_ts(pacc, tmem + kColAhi + kk * 8, dbl, idesc1, 1);
-                }
-                ptx::mma_commit(p_full(pb));
-                if (!FUSED) ptx::mma_commit(empty(s));   // SDDMM: the stage only held B
-                B2SP_FPROF_STOP(2)
-                return true;
-            };
-            if (nwin > 0 && !gemm1(0)) failed = true;
-            for (int it = 0; it < nwin && !failed; ++it) {
-                if (it + 1 < nwin && !gemm1(it + 1)) { failed = true; break; }
-                if (FUSED) {
-                    const int s = it % STAGES;
-                    if (!ptx::mbar_wait(pp_full, it & 1)) { failed = true; break; }
-                    B2SP_FPROF_STOP(3)
+                const uint32_t pacc = tmem + Cfg::COL_P + pb * kFusedBlk;
+                for (int i = 0; i < NCH_B; ++i, ++c) {
+                    const int s = c % RING;
+                    if (!ptx::mbar_wait(full(s), (c / RING) & 1)) { failed = true; break; }
+                    B2SP_FPROF_STOP(1)
                     ptx::tc_fence_after_sync();
-                    const uint32_t d_hi = smem_base + s * STAGE_BYTES + 2 * Cfg::B_BYTES, d_lo = d_hi + Cfg::D_BYTES;
+                    const uint32_t b_hi = ring + s * kFusedChunk, b_lo = b_hi + kFusedChunk / 2;
 #pragma unroll
-                    for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
-                        // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
-                        // groups 512 B apart, +1 KB per K step of 8 rows
-                        const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                        const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                        ptx::mma_tf32_ts(tmem + kColO, tmem + kColPPhi + k8 * 8, ddh, idesc2, (it | k8) != 0);
-                        ptx::mma_tf32_ts(tmem + kColO, tmem + kColPPlo + k8 * 8, ddh, idesc2, 1);
-                        ptx::mma_tf32_ts(tmem + kColO, tmem + kColPPhi + k8 * 8, ddl, idesc2, 1);
+                    for (int k8 = 0; k8 < 4; ++k8) {
+                        const uint64_t dbh = ptx::smem_desc(b_hi + k8 * 32, 16, 1024, ptx::kLayoutSw128);
+                        const uint64_t dbl = ptx::smem_desc(b_lo + k8 * 32, 16, 1024, ptx::kLayoutSw128);
+                        const uint32_t acol = i * 32 + k8 * 8;
+                        ptx::mma_tf32_ts(pacc, tmem + Cfg::COL_AHI + acol, dbh, idesc1, (i | k8) != 0);
+                        ptx::mma_tf32_ts(pacc, tmem + Cfg::COL_AHI + acol, dbl, idesc1, 1);
+                        if (FUSED) {
+                            const uint64_t dal = ptx::smem_desc(alo_smem + i * (kFusedRows * 128) + k8 * 32, 16, 1024, ptx::kLayoutSw128);
+                            ptx::mma_tf32_ss(pacc, dal, dbh, idesc1, 1);
+                        } else {
+                            ptx::mma_tf32_ts(pacc, tmem + Cfg::COL_ALO + acol, dbh, idesc1, 1);
+                        }
                     }
-                    ptx::mma_commit(pp_free);
                     ptx::mma_commit(empty(s));
-                    B2SP_FPROF_STOP(4)
+                    B2SP_FPROF_STOP(2)
+                }
+                if (failed) break;
+                ptx::mma_commit(p_full(pb));
+                if (FUSED) {
+                    for (int w = 0; w < WPB; ++w, ++c, ++ppu) {
+                        const int s = c % RING, ppb = ppu & 1;
+                        if (!ptx::mbar_wait(pp_full(ppb), (ppu >> 1) & 1)) { failed = true; break; }
+                        B2SP_FPROF_STOP(3)
+                        if (!ptx::mbar_wait(full(s), (c / RING) & 1)) { failed = true; break; }
+                        B2SP_FPROF_STOP(1)
+                        ptx::tc_fence_after_sync();
+                        const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
+                        const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
+#pragma unroll
+                        for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
+                            // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
+                            // groups 512 B apart, +1 KB per K step of 8 rows
+                            const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                            const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, (b | w | k8) != 0);
+                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, ppl + k8 * 8, ddh, idesc2, 1);
+                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddl, idesc2, 1);
+                        }
+                        ptx::mma_commit(pp_free(ppb));
+                        ptx::mma_commit(empty(s));
+                        B2SP_FPROF_STOP(4)
+                    }
                 }
             }
             B2SP_FPROF_FLUSH(0)
@@ -246,16 +283,16 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         const uint32_t rec_tab = aux + 256 + ew * 512;              // 2 x 32 records of this warp's rows
         const uint32_t stage_v = aux + 256 + 4 * 512 + ew * 4096;   // 32 x 32 floats, swizzled chunks
         const int grow = m0 + row;
-        const int2 *my_win = a.win + (size_t)(grow < a.M ? grow : 0) * a.Wk + w0;
+        const int wbase = b0 * WPB, nwin = nblk * WPB;              // windows of this CTA (the tail may pass Wk)
+        const int2 *my_win = a.win + (size_t)(grow < a.M ? grow : 0) * a.Wk;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
         const bool has_values = a.s_values != nullptr;
         const bool use_tab = has_values || !FUSED;
         auto load_rec = [&](int t) {
             int2 r = make_int2(0, 0);
-            if (grow < a.M && t < nwin) r = __ldg(my_win + t);
+            if (grow < a.M && t < nwin && wbase + t < a.Wk) r = __ldg(my_win + wbase + t);
             return r;
         };
-        // column-owner loads of one window's stored values (lane = column, register r = row r of the warp)
         auto issue_values = [&](uint32_t tab, float (&vn)[32]) {
             ptx::for_each_row<32>([&](auto rc) {
                 constexpr int r = decltype(rc)::value;
@@ -265,7 +302,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (m & lane_bit) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
             });
         };
-        // transpose through shared memory: afterwards sv[c] = value of (this thread's row, column c)
         auto transpose_values = [&](const float (&vn)[32], float (&sv)[32]) {
             __syncwarp();
             ptx::for_each_row<32>([&](auto rc) {
@@ -296,7 +332,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         B2SP_FPROF_DECL
         B2SP_FPROF_START
         for (int it = 0; it < nwin; ++it) {
-            const int pb = it & 1;
+            const int blk = it / WPB, w = it % WPB;
+            const int pb = FUSED ? 0 : (blk & 1);
             const uint32_t tab_cur = rec_tab + (it & 1) * 256, tab_nxt = rec_tab + ((it + 1) & 1) * 256;
             const unsigned mask = (unsigned)cur.y;
             if (use_tab) {   // records of window it+1 for the whole warp; its values start loading now
@@ -310,41 +347,47 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 for (int c = 0; c < 32; ++c) sv[c] = (mask >> c) & 1u ? 1.f : 0.f;
             }
             B2SP_FPROF_STOP(0)
-            {   // P is ready?
-                bool ok = ptx::mbar_wait(p_full(pb), (it >> 1) & 1);
+            if (w == 0) {   // P of this block ready?
+                const int puse = FUSED ? blk : (blk >> 1);
+                bool ok = ptx::mbar_wait(p_full(pb), puse & 1);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                ptx::tc_fence_after_sync();
             }
             B2SP_FPROF_STOP(1)
-            ptx::tc_fence_after_sync();
             uint32_t p0[16], p1[16];
-            ptx::tmem_ld_32x16(tmem + lane_addr + kColP + pb * kFusedW, p0);
-            ptx::tmem_ld_32x16(tmem + lane_addr + kColP + pb * kFusedW + 16, p1);
+            const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + pb * kFusedBlk + w * kFusedW;
+            ptx::tmem_ld_32x16(pcol, p0);
+            ptx::tmem_ld_32x16(pcol + 16, p1);
             ptx::tmem_ld_wait();
-            ptx::tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) ptx::mbar_arrive(p_free(pb));
+            if (w == WPB - 1) {   // the whole block has been read: GEMM1 may overwrite this P buffer
+                ptx::tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(p_free(pb));
+            }
             B2SP_FPROF_STOP(2)
 
             if (FUSED) {
                 uint32_t hi[16], lo[16];
-                if (it > 0) {
-                    bool ok = ptx::mbar_wait(pp_free, (it - 1) & 1);
+                const int ppb = it & 1, ppuse = it >> 1;
+                if (ppuse > 0) {
+                    bool ok = ptx::mbar_wait(pp_free(ppb), (ppuse - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
                 }
                 B2SP_FPROF_STOP(3)
+                const uint32_t pph = tmem + lane_addr + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) ptx::split_tf32_fast(__uint_as_float(p0[c]) * sv[c], hi[c], lo[c]);
-                ptx::tmem_st_32x16(tmem + lane_addr + kColPPhi, hi);
-                ptx::tmem_st_32x16(tmem + lane_addr + kColPPlo, lo);
+                ptx::tmem_st_32x16(pph, hi);
+                ptx::tmem_st_32x16(ppl, lo);
 #pragma unroll
                 for (int c = 0; c < 16; ++c) ptx::split_tf32_fast(__uint_as_float(p1[c]) * sv[16 + c], hi[c], lo[c]);
-                ptx::tmem_st_32x16(tmem + lane_addr + kColPPhi + 16, hi);
-                ptx::tmem_st_32x16(tmem + lane_addr + kColPPlo + 16, lo);
+                ptx::tmem_st_32x16(pph + 16, hi);
+                ptx::tmem_st_32x16(ppl + 16, lo);
                 ptx::tmem_st_wait();
                 ptx::tc_fence_before_sync();
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(pp_full);
+                if (lane == 0) ptx::mbar_arrive(pp_full(ppb));
                 B2SP_FPROF_STOP(4)
             } else {
                 // SDDMM: stage the masked, scaled row (dense, 32 columns) and write the stored entries
@@ -389,7 +432,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 #pragma unroll 1
                 for (int c = 0; c < kFusedNT / 32; ++c) {
                     uint32_t r[32];
-                    ptx::tmem_ld_32x32(tmem + lane_addr + kColO + c * 32, r);
+                    ptx::tmem_ld_32x32(tmem + lane_addr + Cfg::COL_O + c * 32, r);
                     ptx::tmem_ld_wait();
                     if (grow < a.M) {
                         const int n = n0 + c * 32;
