@@ -7,7 +7,8 @@
 //   * Per block: GEMM1  P = A_tile * B_block^T  (128 x 128).  The B rows of the block arrive by TMA
 //     in chunks of 32 k (hi + lo, 32 KB); N = 128 MMAs run the tensor pipe at full rate (a 128xNx8
 //     tf32 MMA costs max(N/2, 45.6) cycles, so 32-column GEMMs would waste two thirds of it).
-//   * Four warps (thread = row) read P window by window (32 columns), apply the window's occupancy
+//   * Two sets of four warps (thread = row; set s takes the windows of parity s and owns P' buffer s)
+//     read P window by window (32 columns), apply the window's occupancy
 //     mask and stored values (the sampled C of the paper exists only in these registers), and
 //       - FusedMM: split the result into hi/lo and write it back to TMEM as P' (two buffers); GEMM2
 //         O += P'_window * D_window (A = P' from TMEM, B = D rows by TMA, MN-major) accumulates O in TMEM;
@@ -40,7 +41,7 @@ namespace b2sp {
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
-constexpr int kFusedThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: element-wise / epilogue
+constexpr int kFusedThreads = 320;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-9: element-wise (two sets of four)
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
@@ -62,8 +63,8 @@ struct FusedCfg {
     static constexpr int NCH_B = KDP / 32;                     // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = FUSED ? kFusedRows * KDP * 4 : 0;
-    static constexpr int RING = FUSED ? 4 : 6;
-    static constexpr int AUX_BYTES = 256 /*barriers*/ + 4 * 512 /*record tables*/ + 4 * 4096 /*value staging*/;
+    static constexpr int RING = FUSED ? 3 : 5;
+    static constexpr int AUX_BYTES = 256 /*barriers*/ + 8 * 512 /*record tables*/ + 8 * 4096 /*value staging*/;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
@@ -110,7 +111,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(p_full(b), 1);
-            ptx::mbar_init(p_free(b), 4);
+            ptx::mbar_init(p_free(b), 8);
             ptx::mbar_init(pp_full(b), 4);
             ptx::mbar_init(pp_free(b), 1);
         }
@@ -132,7 +133,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int q = warp & 3;                 // TMEM lane quarter of warps 2..5
     const int row = q * 32 + lane;          // row inside the tile (warps >= 2)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    if (warp >= 2) {
+    if (warp >= 2 && warp < 6) {
         const int grow = m0 + row;
         const float *arow = a.A + (long long)(grow < a.M ? grow : 0) * a.lda;
         const bool vec = (a.lda & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
@@ -280,8 +281,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // t+1 are already in flight (loaded cooperatively with lane = column, then transposed through
         // shared memory so that each thread gets its own row), and the record of window t+2 is loading.
         const int ew = warp - 2;
+        const int set = ew >> 2;                                    // windows of parity `set`, P' buffer `set`
         const uint32_t rec_tab = aux + 256 + ew * 512;              // 2 x 32 records of this warp's rows
-        const uint32_t stage_v = aux + 256 + 4 * 512 + ew * 4096;   // 32 x 32 floats, swizzled chunks
+        const uint32_t stage_v = aux + 256 + 8 * 512 + ew * 4096;   // 32 x 32 floats, swizzled chunks
         const int grow = m0 + row;
         const int wbase = b0 * WPB, nwin = nblk * WPB;              // windows of this CTA (the tail may pass Wk)
         const int2 *my_win = a.win + (size_t)(grow < a.M ? grow : 0) * a.Wk;
@@ -320,7 +322,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
         };
         float sv[32], vn[32];
-        int2 cur = load_rec(0), nxt = load_rec(1);
+        int2 cur = load_rec(set), nxt = load_rec(set + 2);
         if (use_tab) {
             ptx::sts64(rec_tab + lane * 8, (uint32_t)cur.x, (uint32_t)cur.y);
             __syncwarp();
@@ -331,23 +333,24 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         }
         B2SP_FPROF_DECL
         B2SP_FPROF_START
-        for (int it = 0; it < nwin; ++it) {
+        for (int it = set; it < nwin; it += 2) {
             const int blk = it / WPB, w = it % WPB;
             const int pb = FUSED ? 0 : (blk & 1);
-            const uint32_t tab_cur = rec_tab + (it & 1) * 256, tab_nxt = rec_tab + ((it + 1) & 1) * 256;
+            const int step = it >> 1;   // this set's own window counter
+            const uint32_t tab_cur = rec_tab + (step & 1) * 256, tab_nxt = rec_tab + ((step + 1) & 1) * 256;
             const unsigned mask = (unsigned)cur.y;
             if (use_tab) {   // records of window it+1 for the whole warp; its values start loading now
                 ptx::sts64(tab_nxt + lane * 8, (uint32_t)nxt.x, (uint32_t)nxt.y);
                 __syncwarp();
             }
-            if (has_values && it + 1 < nwin) issue_values(tab_nxt, vn);
-            const int2 nxt2 = load_rec(it + 2);
+            if (has_values && it + 2 < nwin) issue_values(tab_nxt, vn);
+            const int2 nxt2 = load_rec(it + 4);
             if (!has_values) {
 #pragma unroll
                 for (int c = 0; c < 32; ++c) sv[c] = (mask >> c) & 1u ? 1.f : 0.f;
             }
             B2SP_FPROF_STOP(0)
-            if (w == 0) {   // P of this block ready?
+            if (w < 2) {   // first window of this set in the block: P of this block ready?
                 const int puse = FUSED ? blk : (blk >> 1);
                 bool ok = ptx::mbar_wait(p_full(pb), puse & 1);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -359,7 +362,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::tmem_ld_32x16(pcol, p0);
             ptx::tmem_ld_32x16(pcol + 16, p1);
             ptx::tmem_ld_wait();
-            if (w == WPB - 1) {   // the whole block has been read: GEMM1 may overwrite this P buffer
+            if (w >= WPB - 2) {   // this set has read its share of the block (both sets arrive: count 8)
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(p_free(pb));
@@ -368,7 +371,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 
             if (FUSED) {
                 uint32_t hi[16], lo[16];
-                const int ppb = it & 1, ppuse = it >> 1;
+                const int ppb = set, ppuse = step;
                 if (ppuse > 0) {
                     bool ok = ptx::mbar_wait(pp_free(ppb), (ppuse - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -414,13 +417,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 });
             }
             // the values of window it+1 have had the whole step to arrive: give each thread its row
-            if (has_values && it + 1 < nwin) transpose_values(vn, sv);
+            if (has_values && it + 2 < nwin) transpose_values(vn, sv);
             cur = nxt;
             nxt = nxt2;
         }
         if (ew == 0) { B2SP_FPROF_FLUSH(8) }
-        // ---------------- epilogue: O accumulator -> global ----------------
-        if (FUSED) {
+        // ---------------- epilogue (first set): O accumulator -> global ----------------
+        if (FUSED && set == 0) {
             {
                 bool ok = !failed && ptx::mbar_wait(o_full, 0);
                 failed = !__all_sync(0xffffffffu, ok);
