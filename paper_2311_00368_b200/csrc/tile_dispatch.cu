@@ -4,6 +4,7 @@
 
 #include <cuda.h>
 
+#include <cstdlib>
 #include <mutex>
 
 #include "tile_kernels.cuh"
@@ -58,15 +59,18 @@ bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, 
 
 int pick_split(int base_tiles, int Wk)
 {
-    int best = 1;
-    double best_eff = 0.0;
-    for (int ks = 1; ks <= 16 && ks <= Wk && Wk / ks >= 4; ++ks) {
-        long long items = (long long)base_tiles * ks;
-        double eff = (double)items / (double)((items + kSMs - 1) / kSMs * kSMs);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
-        if (eff >= 0.90) return ks;
+    if (const char *e = getenv("B2SP_FORCE_KS")) {   // tuning aid
+        int ks = atoi(e);
+        if (ks >= 1 && ks <= Wk) return ks;
     }
-    return best;
+    // One wave of long-lived CTAs beats several waves of short ones (each CTA pays a prologue, an
+    // epilogue and a partial-output slab): take the largest split that still fits one wave, as long
+    // as every split keeps a few pipeline steps.
+    if (base_tiles >= kSMs) return 1;
+    int ks = kSMs / base_tiles;
+    if (ks > Wk / 4) ks = Wk / 4;
+    if (ks > 32) ks = 32;
+    return ks < 1 ? 1 : ks;
 }
 
 template <int TR>

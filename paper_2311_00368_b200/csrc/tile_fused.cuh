@@ -79,7 +79,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                   const FusedTileArgs a)
 {
     using Cfg = FusedCfg<KDP, FUSED>;
-    constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B, NCH_D = Cfg::NCH_D;
+    constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
     if (a.flags[0] != 0) return;  // pattern not usable for tiles: the row kernels take over
 
@@ -185,23 +185,31 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::tma_prefetch_desc(&tm_bhi);
             ptx::tma_prefetch_desc(&tm_blo);
             if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); ptx::tma_prefetch_desc(&tm_dlo); }
+            // Chunk order = the order the MMA thread consumes them: B(0); then per block b:
+            // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only).
             int c = 0;
-            for (int b = 0; b < nblk && !failed; ++b) {
-                const int col0 = (b0 + b) * kFusedBlk;
-                for (int i = 0; i < NCH_B + NCH_D; ++i, ++c) {
-                    const int s = c % RING;
-                    if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) { failed = true; break; }
-                    const uint32_t dst = ring + s * kFusedChunk;
-                    ptx::mbar_arrive_expect_tx(full(s), kFusedChunk);
-                    if (i < NCH_B) {   // B rows col0..col0+127, k group i
-                        ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
-                        ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
-                    } else {           // D rows of window i - NCH_B
-                        const int krow = col0 + (i - NCH_B) * kFusedW;
-                        ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (kFusedNT / 32));
-                        ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (kFusedNT / 32));
-                    }
+            auto put = [&](bool is_b, int blk, int i) -> bool {
+                const int s = c % RING;
+                if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
+                const uint32_t dst = ring + s * kFusedChunk;
+                const int col0 = (b0 + blk) * kFusedBlk;
+                ptx::mbar_arrive_expect_tx(full(s), kFusedChunk);
+                if (is_b) {   // B rows col0..col0+127, k group i
+                    ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
+                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
+                } else {      // D rows of window i of the block
+                    const int krow = col0 + i * kFusedW;
+                    ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (kFusedNT / 32));
+                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (kFusedNT / 32));
                 }
+                ++c;
+                return true;
+            };
+            for (int i = 0; i < NCH_B && nblk > 0 && !failed; ++i) failed = !put(true, 0, i);
+            for (int b = 0; b < nblk && !failed; ++b) {
+                if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !put(false, b, w);
+                if (b + 1 < nblk) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
+                if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !put(false, b, w);
             }
             if (failed)
                 for (int j = c > RING ? c - RING : 0; j < c; ++j) ptx::mbar_wait(full(j % RING), (j / RING) & 1);
@@ -214,16 +222,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             B2SP_FPROF_DECL
             B2SP_FPROF_START
             int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
-            for (int b = 0; b < nblk && !failed; ++b) {
+            auto gemm1 = [&](int b) -> bool {   // P = A_tile * B_block^T over NCH_B chunks
                 const int pb = FUSED ? 0 : (b & 1);
-                // P buffer drained by the element-wise warps?
                 const int puse = FUSED ? b : (b >> 1);
-                if (puse > 0 && !ptx::mbar_wait(p_free(pb), (puse - 1) & 1)) { failed = true; break; }
+                if (puse > 0 && !ptx::mbar_wait(p_free(pb), (puse - 1) & 1)) return false;   // P drained?
                 B2SP_FPROF_STOP(0)
                 const uint32_t pacc = tmem + Cfg::COL_P + pb * kFusedBlk;
                 for (int i = 0; i < NCH_B; ++i, ++c) {
                     const int s = c % RING;
-                    if (!ptx::mbar_wait(full(s), (c / RING) & 1)) { failed = true; break; }
+                    if (!ptx::mbar_wait(full(s), (c / RING) & 1)) return false;
                     B2SP_FPROF_STOP(1)
                     ptx::tc_fence_after_sync();
                     const uint32_t b_hi = ring + s * kFusedChunk, b_lo = b_hi + kFusedChunk / 2;
@@ -244,33 +251,43 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     ptx::mma_commit(empty(s));
                     B2SP_FPROF_STOP(2)
                 }
-                if (failed) break;
                 ptx::mma_commit(p_full(pb));
-                if (FUSED) {
-                    for (int w = 0; w < WPB; ++w, ++c, ++ppu) {
-                        const int s = c % RING, ppb = ppu & 1;
-                        if (!ptx::mbar_wait(pp_full(ppb), (ppu >> 1) & 1)) { failed = true; break; }
-                        B2SP_FPROF_STOP(3)
-                        if (!ptx::mbar_wait(full(s), (c / RING) & 1)) { failed = true; break; }
-                        B2SP_FPROF_STOP(1)
-                        ptx::tc_fence_after_sync();
-                        const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
-                        const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
+                return true;
+            };
+            auto gemm2 = [&](int b, int w) -> bool {   // O += P'_window * D_window
+                const int s = c % RING, ppb = ppu & 1;
+                if (!ptx::mbar_wait(pp_full(ppb), (ppu >> 1) & 1)) return false;
+                B2SP_FPROF_STOP(3)
+                if (!ptx::mbar_wait(full(s), (c / RING) & 1)) return false;
+                B2SP_FPROF_STOP(1)
+                ptx::tc_fence_after_sync();
+                const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
+                const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
 #pragma unroll
-                        for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
-                            // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
-                            // groups 512 B apart, +1 KB per K step of 8 rows
-                            const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                            const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, (b | w | k8) != 0);
-                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, ppl + k8 * 8, ddh, idesc2, 1);
-                            ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddl, idesc2, 1);
-                        }
-                        ptx::mma_commit(pp_free(ppb));
-                        ptx::mma_commit(empty(s));
-                        B2SP_FPROF_STOP(4)
-                    }
+                for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
+                    // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
+                    // groups 512 B apart, +1 KB per K step of 8 rows
+                    const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                    const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, (b | w | k8) != 0);
+                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, ppl + k8 * 8, ddh, idesc2, 1);
+                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddl, idesc2, 1);
                 }
+                ptx::mma_commit(pp_free(ppb));
+                ptx::mma_commit(empty(s));
+                ++c;
+                ++ppu;
+                B2SP_FPROF_STOP(4)
+                return true;
+            };
+            // GEMM1 of block b+1 is issued between the second and third GEMM2 of block b: by then the
+            // element-wise warps have read all of P(b), and the tensor pipe has work while they
+            // process the last two windows of block b.
+            if (nblk > 0 && !gemm1(0)) failed = true;
+            for (int b = 0; b < nblk && !failed; ++b) {
+                if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !gemm2(b, w);
+                if (b + 1 < nblk && !failed) failed = !gemm1(b + 1);
+                if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !gemm2(b, w);
             }
             B2SP_FPROF_FLUSH(0)
             if (FUSED && !failed) ptx::mma_commit(o_full);
