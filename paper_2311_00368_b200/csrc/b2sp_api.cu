@@ -3,6 +3,7 @@
 #include "../../include/b2sp.h"
 
 #include <climits>
+#include <cstdlib>
 #include <cstdint>
 
 #include "row_kernels.cuh"
@@ -193,6 +194,14 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
 
+static bool spmm_via_fused_pipeline()
+{
+    // Default: SPMM runs through the FusedMM tile pipeline (P' = the stored values).  The older kernel
+    // that builds S tiles in shared memory (spmm_tile_kernel) stays selectable for comparison.
+    const char *e = getenv("B2SP_SPMM_IMPL");   // tuning aid: "builder" selects the shared-memory builder
+    return !(e && e[0] == 'b');
+}
+
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
                              const float *D, long long ldd, float *O, long long ldo, const int *order,
@@ -242,6 +251,18 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     if (nnz == 0) return zero_rows(O, ldo, M, N, st);
 
     Workspace w = carve(workspace);
+    if (use == B2SP_ALGO_TILE && spmm_via_fused_pipeline()) {
+        FusedPlan fp = plan_fused_tile(M, K, 0, N, nnz, row_bytes, true);
+        if (fp.feasible && workspace_bytes >= fp.bytes) {
+            rc = fused_tile(fp, prepared, 2, M, K, 0, N, nnz, row_ptr, col_idx, values, nullptr, 0, nullptr, 0, D, ldd,
+                            O, ldo, workspace, st, &launches);
+            if (rc != B2SP_OK) return rc;
+            const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+            rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, st);
+            g_last_launches[B2SP_OP_SPMM] = launches + 1;
+            return rc;
+        }
+    }
     if (use == B2SP_ALGO_TILE) {
         rc = spmm_tile(plan, prepared, M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
@@ -323,7 +344,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
-        rc = fused_tile(plan, prepared, false, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
+        rc = fused_tile(plan, prepared, 0, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
                         out_values, 0, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
@@ -401,7 +422,7 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
-        rc = fused_tile(plan, prepared, true, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
+        rc = fused_tile(plan, prepared, 1, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
                         workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
@@ -477,7 +498,21 @@ struct DevArena {
     void *ptrs[16];
     int n = 0;
     bool ok = true;
-    explicit DevArena(cudaStream_t s) : st(s) {}
+    explicit DevArena(cudaStream_t s) : st(s)
+    {
+        // keep freed blocks in the stream-ordered pool across calls (the default returns them to the
+        // driver at every synchronisation, which makes each call pay for fresh allocations)
+        static thread_local int tuned_device = -1;
+        int dev = -1;
+        if (cudaGetDevice(&dev) == cudaSuccess && dev != tuned_device) {
+            cudaMemPool_t pool;
+            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+                unsigned long long keep = ~0ull;
+                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+            }
+            tuned_device = dev;
+        }
+    }
     void *alloc(size_t bytes)
     {
         void *p = nullptr;

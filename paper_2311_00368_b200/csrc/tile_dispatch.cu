@@ -217,10 +217,10 @@ b2sp_status spmm_tile(const TilePlan &p, bool prepared, int M, int K, int N, lon
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)
 {
     FusedPlan p;
-    if (M <= 0 || K <= 0 || Kd <= 0 || Kd > 128 || nnz <= 0 || (fused && N <= 0)) return p;
+    if (M <= 0 || K <= 0 || Kd < 0 || Kd > 128 || nnz <= 0 || (fused && N <= 0) || (!fused && Kd == 0)) return p;
     p.Wk = (K + kFusedW - 1) / kFusedW;
     p.Kp = (K + kFusedBlk - 1) / kFusedBlk * kFusedBlk;   // operand copies padded to whole 128-column blocks
-    p.Kdp = Kd <= 32 ? 32 : Kd <= 64 ? 64 : 128;
+    p.Kdp = Kd == 0 ? 0 : Kd <= 32 ? 32 : Kd <= 64 ? 64 : 128;   // Kd == 0: SPMM through the fused pipeline
     p.Mt = (M + kFusedRows - 1) / kFusedRows;
     p.Nt = fused ? (N + kFusedNT - 1) / kFusedNT : 1;
     p.Np = fused ? p.Nt * kFusedNT : 0;
@@ -251,25 +251,25 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
 
 namespace {
 
-template <int KDP, bool FUSED>
+template <int KDP, int MODE>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                               const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
 {
-    using Cfg = FusedCfg<KDP, FUSED>;
-    auto kern = fused_tile_kernel<KDP, FUSED>;
+    using Cfg = FusedCfg<KDP, MODE>;
+    auto kern = fused_tile_kernel<KDP, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
     kern<<<items, kFusedThreads, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, a);
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 
-template <bool FUSED>
+template <int MODE>
 b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                              const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
 {
-    if (kdp == 32) return launch_fused_tile<32, FUSED>(bh, bl, dh, dl, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, FUSED>(bh, bl, dh, dl, a, items, st);
-    return launch_fused_tile<128, FUSED>(bh, bl, dh, dl, a, items, st);
+    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE>(bh, bl, dh, dl, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, MODE>(bh, bl, dh, dl, a, items, st);
+    return launch_fused_tile<128, MODE>(bh, bl, dh, dl, a, items, st);
 }
 
 void launch_split(const float *X, long long ld, int rows, int cols, float *hi, float *lo, int rows_p, int cols_p,
@@ -282,7 +282,7 @@ void launch_split(const float *X, long long ld, int rows, int cols, float *hi, f
 
 }  // namespace
 
-b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int K, int Kd, int N, long long nnz,
+b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches)
@@ -295,9 +295,10 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int
     float *dhi = reinterpret_cast<float *>(ws + p.off_dhi), *dlo = reinterpret_cast<float *>(ws + p.off_dlo);
     float *part = reinterpret_cast<float *>(ws + p.off_part);
 
+    const bool fused = mode != kModeSddmm, spmm = mode == kModeSpmm;
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
-    if (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
-        !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false))
+    if (!spmm && (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
+                  !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
         return B2SP_ERR_CUDA;
     if (fused) {
         if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true) ||
@@ -307,12 +308,15 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int
         tm_dh = tm_bh;   // unused by the SDDMM kernel
         tm_dl = tm_bl;
     }
+    if (spmm) { tm_bh = tm_dh; tm_bl = tm_dl; }   // unused by the SPMM mode
     {
         b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
         if (prc != B2SP_OK) return prc;
     }
-    launch_split(B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, st);
-    *launches += 1;
+    if (!spmm) {
+        launch_split(B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, st);
+        *launches += 1;
+    }
     if (fused) {
         launch_split(D, ldd, K, N, dhi, dlo, p.Kp, p.Np, st);
         *launches += 1;
@@ -328,8 +332,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
     const int items = p.Mt * p.Nt * p.KS;
-    b2sp_status rc = fused ? launch_fused_kdp<true>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
-                           : launch_fused_kdp<false>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
+    b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
+                     : fused ? launch_fused_kdp<kModeFused>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
+                             : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
     if (fused && p.KS > 1) {

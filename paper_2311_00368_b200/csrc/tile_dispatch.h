@@ -33,7 +33,8 @@ struct FusedPlan {
 };
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused);
 
-b2sp_status fused_tile(const FusedPlan &p, bool prepared, bool fused, int M, int K, int Kd, int N, long long nnz,
+// mode: 0 = SDDMM, 1 = FusedMM, 2 = SPMM through the FusedMM pipeline (P' = the stored values)
+b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches);

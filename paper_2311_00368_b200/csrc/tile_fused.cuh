@@ -58,12 +58,18 @@ struct FusedTileArgs {
     unsigned long long *prof;  // optional role timers (profiling builds only)
 };
 
-template <int KDP, bool FUSED>
+// MODE: which op the kernel runs.  SPMM reuses the FusedMM pipeline with P' = the stored values
+// themselves (no A, no GEMM1).
+constexpr int kModeSddmm = 0, kModeFused = 1, kModeSpmm = 2;
+
+template <int KDP, int MODE>
 struct FusedCfg {
-    static constexpr int NCH_B = KDP / 32;                     // B chunks per block
+    static constexpr bool FUSED = MODE != kModeSddmm;          // has GEMM2 / O
+    static constexpr bool SPMM = MODE == kModeSpmm;
+    static constexpr int NCH_B = SPMM ? 0 : KDP / 32;          // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
-    static constexpr int ALO_BYTES = FUSED ? kFusedRows * KDP * 4 : 0;
-    static constexpr int RING = FUSED ? 3 : 5;
+    static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
+    static constexpr int RING = SPMM ? 5 : FUSED ? 3 : 5;
     static constexpr int AUX_BYTES = 256 /*barriers*/ + 8 * 512 /*record tables*/ + 8 * 4096 /*value staging*/;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
@@ -71,14 +77,14 @@ struct FusedCfg {
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
 
-// FUSED = true: FusedMM (GEMM2 + O epilogue).  FUSED = false: SDDMM (write the sampled values).
-template <int KDP, bool FUSED>
+template <int KDP, int MODE>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
                   const FusedTileArgs a)
 {
-    using Cfg = FusedCfg<KDP, FUSED>;
+    using Cfg = FusedCfg<KDP, MODE>;
+    constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
     constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
     if (a.flags[0] != 0) return;  // pattern not usable for tiles: the row kernels take over
@@ -133,7 +139,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int q = warp & 3;                 // TMEM lane quarter of warps 2..5
     const int row = q * 32 + lane;          // row inside the tile (warps >= 2)
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    if (warp >= 2 && warp < 6) {
+    if (!SPMM && warp >= 2 && warp < 6) {
         const int grow = m0 + row;
         const float *arow = a.A + (long long)(grow < a.M ? grow : 0) * a.lda;
         const bool vec = (a.lda & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
@@ -182,8 +188,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     if (warp == 0) {
         // ---------------- TMA producer: per block NCH_B chunks of B rows, then NCH_D chunks of D rows ----------------
         if (lane == 0) {
-            ptx::tma_prefetch_desc(&tm_bhi);
-            ptx::tma_prefetch_desc(&tm_blo);
+            if (!SPMM) { ptx::tma_prefetch_desc(&tm_bhi); ptx::tma_prefetch_desc(&tm_blo); }
             if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); ptx::tma_prefetch_desc(&tm_dlo); }
             // Chunk order = the order the MMA thread consumes them: B(0); then per block b:
             // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only).
@@ -208,7 +213,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             for (int i = 0; i < NCH_B && nblk > 0 && !failed; ++i) failed = !put(true, 0, i);
             for (int b = 0; b < nblk && !failed; ++b) {
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !put(false, b, w);
-                if (b + 1 < nblk) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
+                if (!SPMM && b + 1 < nblk) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !put(false, b, w);
             }
             if (failed)
@@ -283,10 +288,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             // GEMM1 of block b+1 is issued between the second and third GEMM2 of block b: by then the
             // element-wise warps have read all of P(b), and the tensor pipe has work while they
             // process the last two windows of block b.
-            if (nblk > 0 && !gemm1(0)) failed = true;
+            if (!SPMM && nblk > 0 && !gemm1(0)) failed = true;
             for (int b = 0; b < nblk && !failed; ++b) {
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !gemm2(b, w);
-                if (b + 1 < nblk && !failed) failed = !gemm1(b + 1);
+                if (!SPMM && b + 1 < nblk && !failed) failed = !gemm1(b + 1);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !gemm2(b, w);
             }
             B2SP_FPROF_FLUSH(0)
@@ -367,7 +372,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 for (int c = 0; c < 32; ++c) sv[c] = (mask >> c) & 1u ? 1.f : 0.f;
             }
             B2SP_FPROF_STOP(0)
-            if (w < 2) {   // first window of this set in the block: P of this block ready?
+            if (!SPMM && w < 2) {   // first window of this set in the block: P of this block ready?
                 const int puse = FUSED ? blk : (blk >> 1);
                 bool ok = ptx::mbar_wait(p_full(pb), puse & 1);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
@@ -375,14 +380,19 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
             B2SP_FPROF_STOP(1)
             uint32_t p0[16], p1[16];
-            const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + pb * kFusedBlk + w * kFusedW;
-            ptx::tmem_ld_32x16(pcol, p0);
-            ptx::tmem_ld_32x16(pcol + 16, p1);
-            ptx::tmem_ld_wait();
-            if (w >= WPB - 2) {   // this set has read its share of the block (both sets arrive: count 8)
-                ptx::tc_fence_before_sync();
-                __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(p_free(pb));
+            if (SPMM) {   // P' is S itself
+#pragma unroll
+                for (int c = 0; c < 16; ++c) { p0[c] = 0x3f800000u; p1[c] = 0x3f800000u; }
+            } else {
+                const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + pb * kFusedBlk + w * kFusedW;
+                ptx::tmem_ld_32x16(pcol, p0);
+                ptx::tmem_ld_32x16(pcol + 16, p1);
+                ptx::tmem_ld_wait();
+                if (w >= WPB - 2) {   // this set has read its share of the block (both sets arrive: count 8)
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(p_free(pb));
+                }
             }
             B2SP_FPROF_STOP(2)
 
