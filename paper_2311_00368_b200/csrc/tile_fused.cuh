@@ -7,9 +7,10 @@
 //   * Per block: GEMM1  P = A_tile * B_block^T  (128 x 128).  The B rows of the block arrive by TMA
 //     in chunks of 32 k (hi + lo, 32 KB); N = 128 MMAs run the tensor pipe at full rate (a 128xNx8
 //     tf32 MMA costs max(N/2, 45.6) cycles, so 32-column GEMMs would waste two thirds of it).
-//   * Two sets of four warps (thread = row; set s takes the windows of parity s and owns P' buffer s)
-//     read P window by window (32 columns), apply the window's occupancy
-//     mask and stored values (the sampled C of the paper exists only in these registers), and
+//   * Four processor warps (thread = row) read P window by window (32 columns) and multiply it by the
+//     window's stored values (0 where nothing is stored), which eight helper warps fetch with lane =
+//     column (coalesced), densify and transpose through shared-memory slots.  The sampled C of the
+//     paper exists only in these registers.  Then
 //       - FusedMM: split the result into hi/lo and write it back to TMEM as P' (two buffers); GEMM2
 //         O += P'_window * D_window (A = P' from TMEM, B = D rows by TMA, MN-major) accumulates O in TMEM;
 //       - SDDMM: write the stored entries to out_values (coalesced through shared memory).
@@ -41,7 +42,9 @@ namespace b2sp {
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
-constexpr int kFusedThreads = 320;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-9: element-wise (two sets of four)
+constexpr int kFusedThreads = 576;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: processors, warps 6-17: helpers
+constexpr int kFusedSlots = 12;     // shared-memory slots (4 KB) between helpers and processors: 3 windows deep
+constexpr int kFusedHelpers = 12;
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
@@ -70,7 +73,7 @@ struct FusedCfg {
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
     static constexpr int RING = SPMM ? 5 : FUSED ? 3 : 5;
-    static constexpr int AUX_BYTES = 256 /*barriers*/ + 8 * 512 /*record tables*/ + 8 * 4096 /*value staging*/;
+    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedHelpers * 256 /*record tables*/ + kFusedSlots * 4096;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
@@ -102,7 +105,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     auto pp_full = [&](int b) { return aux + 8u * (2 * RING + 4 + b); };
     auto pp_free = [&](int b) { return aux + 8u * (2 * RING + 6 + b); };
     const uint32_t o_full = aux + 8u * (2 * RING + 8);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 9));
+    constexpr int NSLOT = kFusedSlots, NH = kFusedHelpers;
+    auto sl_full = [&](int s) { return aux + 8u * (2 * RING + 9 + s); };
+    auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 9 + 2 * NSLOT));
+    const uint32_t helper_tabs = aux + 512, slots = aux + 512 + NH * 256;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ks = blockIdx.x % a.KS;
@@ -117,11 +124,12 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(p_full(b), 1);
-            ptx::mbar_init(p_free(b), 8);
+            ptx::mbar_init(p_free(b), 4);
             ptx::mbar_init(pp_full(b), 4);
             ptx::mbar_init(pp_free(b), 1);
         }
         ptx::mbar_init(o_full, 1);
+        for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(sl_full(s), 1); ptx::mbar_init(sl_empty(s), 1); }
         ptx::fence_mbar_init();
     }
     if (warp == 1) {
@@ -297,114 +305,62 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             B2SP_FPROF_FLUSH(0)
             if (FUSED && !failed) ptx::mma_commit(o_full);
         }
-    } else {
-        // ---------------- element-wise warps (thread = row) ----------------
-        // Software pipeline over windows: while window t is processed, the stored values of window
-        // t+1 are already in flight (loaded cooperatively with lane = column, then transposed through
-        // shared memory so that each thread gets its own row), and the record of window t+2 is loading.
-        const int ew = warp - 2;
-        const int set = ew >> 2;                                    // windows of parity `set`, P' buffer `set`
-        const uint32_t rec_tab = aux + 256 + ew * 512;              // 2 x 32 records of this warp's rows
-        const uint32_t stage_v = aux + 256 + 8 * 512 + ew * 4096;   // 32 x 32 floats, swizzled chunks
+    } else if (warp < 6) {
+        // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
+        // FusedMM / SPMM: per window, take the row's stored values (densified and transposed by a
+        // helper warp into a shared-memory slot), multiply them into P (or use them as they are for
+        // SPMM), split to hi/lo and write P' to tensor memory.
+        // SDDMM: per window, copy the row of P into a slot; a helper warp writes the stored entries.
         const int grow = m0 + row;
-        const int wbase = b0 * WPB, nwin = nblk * WPB;              // windows of this CTA (the tail may pass Wk)
-        const int2 *my_win = a.win + (size_t)(grow < a.M ? grow : 0) * a.Wk;
-        const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
-        const bool has_values = a.s_values != nullptr;
-        const bool use_tab = has_values || !FUSED;
-        auto load_rec = [&](int t) {
-            int2 r = make_int2(0, 0);
-            if (grow < a.M && t < nwin && wbase + t < a.Wk) r = __ldg(my_win + wbase + t);
-            return r;
-        };
-        auto issue_values = [&](uint32_t tab, float (&vn)[32]) {
-            ptx::for_each_row<32>([&](auto rc) {
-                constexpr int r = decltype(rc)::value;
-                uint32_t pos, m;
-                ptx::lds64_off<r * 8>(tab, pos, m);
-                vn[r] = 0.f;
-                if (m & lane_bit) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
-            });
-        };
-        auto transpose_values = [&](const float (&vn)[32], float (&sv)[32]) {
-            __syncwarp();
-            ptx::for_each_row<32>([&](auto rc) {
-                constexpr int r = decltype(rc)::value;
-                ptx::sts32_off<r * 128>(stage_v + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
-            });
-            __syncwarp();
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                uint32_t x0, x1, x2, x3;
-                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                             : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
-                             : "r"(stage_v + lane * 128 + (uint32_t)((j ^ (lane & 7)) << 4)));
-                sv[4 * j] = __uint_as_float(x0); sv[4 * j + 1] = __uint_as_float(x1);
-                sv[4 * j + 2] = __uint_as_float(x2); sv[4 * j + 3] = __uint_as_float(x3);
-            }
-        };
-        float sv[32], vn[32];
-        int2 cur = load_rec(set), nxt = load_rec(set + 2);
-        if (use_tab) {
-            ptx::sts64(rec_tab + lane * 8, (uint32_t)cur.x, (uint32_t)cur.y);
-            __syncwarp();
-        }
-        if (has_values) {
-            issue_values(rec_tab, vn);
-            transpose_values(vn, sv);
-        }
-        B2SP_FPROF_DECL
-        B2SP_FPROF_START
-        for (int it = set; it < nwin; it += 2) {
+        const int nwin = nblk * WPB;
+        for (int it = 0; it < nwin; ++it) {
             const int blk = it / WPB, w = it % WPB;
-            const int pb = FUSED ? 0 : (blk & 1);
-            const int step = it >> 1;   // this set's own window counter
-            const uint32_t tab_cur = rec_tab + (step & 1) * 256, tab_nxt = rec_tab + ((step + 1) & 1) * 256;
-            const unsigned mask = (unsigned)cur.y;
-            if (use_tab) {   // records of window it+1 for the whole warp; its values start loading now
-                ptx::sts64(tab_nxt + lane * 8, (uint32_t)nxt.x, (uint32_t)nxt.y);
-                __syncwarp();
-            }
-            if (has_values && it + 2 < nwin) issue_values(tab_nxt, vn);
-            const int2 nxt2 = load_rec(it + 4);
-            if (!has_values) {
-#pragma unroll
-                for (int c = 0; c < 32; ++c) sv[c] = (mask >> c) & 1u ? 1.f : 0.f;
-            }
-            B2SP_FPROF_STOP(0)
-            if (!SPMM && w < 2) {   // first window of this set in the block: P of this block ready?
-                const int puse = FUSED ? blk : (blk >> 1);
-                bool ok = ptx::mbar_wait(p_full(pb), puse & 1);
-                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                ptx::tc_fence_after_sync();
-            }
-            B2SP_FPROF_STOP(1)
-            uint32_t p0[16], p1[16];
-            if (SPMM) {   // P' is S itself
-#pragma unroll
-                for (int c = 0; c < 16; ++c) { p0[c] = 0x3f800000u; p1[c] = 0x3f800000u; }
-            } else {
-                const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + pb * kFusedBlk + w * kFusedW;
-                ptx::tmem_ld_32x16(pcol, p0);
-                ptx::tmem_ld_32x16(pcol + 16, p1);
-                ptx::tmem_ld_wait();
-                if (w >= WPB - 2) {   // this set has read its share of the block (both sets arrive: count 8)
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(p_free(pb));
-                }
-            }
-            B2SP_FPROF_STOP(2)
-
+            const int j = it * 4 + q, s = j % NSLOT, use = j / NSLOT;
+            const uint32_t slot = slots + s * 4096 + lane * 128;
             if (FUSED) {
-                uint32_t hi[16], lo[16];
-                const int ppb = set, ppuse = step;
+                float sv[32];
+                {
+                    bool ok = ptx::mbar_wait(sl_full(s), use & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                }
+#pragma unroll
+                for (int jj = 0; jj < 8; ++jj) {
+                    uint32_t x0, x1, x2, x3;
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                                 : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+                                 : "r"(slot + (uint32_t)((jj ^ (lane & 7)) << 4)) : "memory");
+                    sv[4 * jj] = __uint_as_float(x0); sv[4 * jj + 1] = __uint_as_float(x1);
+                    sv[4 * jj + 2] = __uint_as_float(x2); sv[4 * jj + 3] = __uint_as_float(x3);
+                }
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(sl_empty(s));
+                uint32_t p0[16], p1[16];
+                if (SPMM) {
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) { p0[c] = 0x3f800000u; p1[c] = 0x3f800000u; }
+                } else {
+                    if (w == 0) {
+                        bool ok = ptx::mbar_wait(p_full(0), blk & 1);
+                        if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                        ptx::tc_fence_after_sync();
+                    }
+                    const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + w * kFusedW;
+                    ptx::tmem_ld_32x16(pcol, p0);
+                    ptx::tmem_ld_32x16(pcol + 16, p1);
+                    ptx::tmem_ld_wait();
+                    if (w == WPB - 1) {   // the whole block has been read: GEMM1 may overwrite P
+                        ptx::tc_fence_before_sync();
+                        __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(p_free(0));
+                    }
+                }
+                const int ppb = it & 1, ppuse = it >> 1;
                 if (ppuse > 0) {
                     bool ok = ptx::mbar_wait(pp_free(ppb), (ppuse - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
                 }
-                B2SP_FPROF_STOP(3)
+                uint32_t hi[16], lo[16];
                 const uint32_t pph = tmem + lane_addr + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
 #pragma unroll
                 for (int c = 0; c < 16; ++c) ptx::split_tf32_fast(__uint_as_float(p0[c]) * sv[c], hi[c], lo[c]);
@@ -418,39 +374,39 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(pp_full(ppb));
-                B2SP_FPROF_STOP(4)
             } else {
-                // SDDMM: stage the masked, scaled row (dense, 32 columns) and write the stored entries
-                // row by row with lane = column, so each row's outputs are one contiguous store.
-                __syncwarp();
+                const int pb = blk & 1;
+                if (w == 0) {
+                    bool ok = ptx::mbar_wait(p_full(pb), (blk >> 1) & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                    ptx::tc_fence_after_sync();
+                }
+                uint32_t p0[16], p1[16];
+                const uint32_t pcol = tmem + lane_addr + Cfg::COL_P + pb * kFusedBlk + w * kFusedW;
+                ptx::tmem_ld_32x16(pcol, p0);
+                ptx::tmem_ld_32x16(pcol + 16, p1);
+                ptx::tmem_ld_wait();
+                if (w == WPB - 1) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(p_free(pb));
+                }
+                if (use > 0) {
+                    bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                }
 #pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t x[4];
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int c = 4 * j + i;
-                        x[i] = __float_as_uint(__uint_as_float(c < 16 ? p0[c] : p1[c - 16]) * sv[c]);
-                    }
-                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage_v + lane * 128 + (uint32_t)((j ^ (lane & 7)) << 4)),
-                                 "r"(x[0]), "r"(x[1]), "r"(x[2]), "r"(x[3]) : "memory");
+                for (int jj = 0; jj < 8; ++jj) {
+                    const uint32_t *src = jj < 4 ? &p0[4 * jj] : &p1[4 * (jj - 4)];
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(slot + (uint32_t)((jj ^ (lane & 7)) << 4)),
+                                 "r"(src[0]), "r"(src[1]), "r"(src[2]), "r"(src[3]) : "memory");
                 }
                 __syncwarp();
-                ptx::for_each_row<32>([&](auto rc) {
-                    constexpr int r = decltype(rc)::value;
-                    uint32_t pos, m, v;
-                    ptx::lds64_off<r * 8>(tab_cur, pos, m);
-                    asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(stage_v + (uint32_t)((lane << 2) ^ ((r & 7) << 4))), "n"(r * 128));
-                    if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = __uint_as_float(v);
-                });
+                if (lane == 0) ptx::mbar_arrive(sl_full(s));
             }
-            // the values of window it+1 have had the whole step to arrive: give each thread its row
-            if (has_values && it + 2 < nwin) transpose_values(vn, sv);
-            cur = nxt;
-            nxt = nxt2;
         }
-        if (ew == 0) { B2SP_FPROF_FLUSH(8) }
-        // ---------------- epilogue (first set): O accumulator -> global ----------------
-        if (FUSED && set == 0) {
+        // ---------------- epilogue: O accumulator -> global ----------------
+        if (FUSED) {
             {
                 bool ok = !failed && ptx::mbar_wait(o_full, 0);
                 failed = !__all_sync(0xffffffffu, ok);
@@ -477,6 +433,69 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         }
                     }
                 }
+            }
+        }
+    } else {
+        // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
+        // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
+        // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
+        // values) and write them transposed into a slot, from which the processor thread of each row
+        // reads its row.  SDDMM: prefetch the stored values the same way, then take the P rows the
+        // processors left in the slot and write the stored entries, one coalesced run per row.
+        const int h = warp - 6;
+        const uint32_t tab = helper_tabs + h * 256;   // 32 records (position, mask) of the item's rows
+        const int wbase = b0 * WPB, nitems = nblk * WPB * 4;
+        const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
+        const bool has_values = a.s_values != nullptr;
+        auto load_rec = [&](int jj) {   // lane = row: window record of one row of item jj
+            int2 r = make_int2(0, 0);
+            const int hrow = m0 + (jj & 3) * 32 + lane, wglob = wbase + (jj >> 2);
+            if (jj < nitems && hrow < a.M && wglob < a.Wk) r = __ldg(a.win + (size_t)hrow * a.Wk + wglob);
+            return r;
+        };
+        int2 rec_next = load_rec(h);
+        for (int j = h; j < nitems; j += NH) {
+            const int s = j % NSLOT, use = j / NSLOT;
+            const int2 rec = rec_next;
+            rec_next = load_rec(j + NH);   // the next item's records load while this item is processed
+            __syncwarp();   // everyone is done with the previous item's records
+            ptx::sts64(tab + lane * 8, (uint32_t)rec.x, (uint32_t)rec.y);
+            __syncwarp();
+            float vn[32];
+            ptx::for_each_row<32>([&](auto rc) {
+                constexpr int r = decltype(rc)::value;
+                uint32_t pos, m;
+                ptx::lds64_off<r * 8>(tab, pos, m);
+                const bool present = (m & lane_bit) != 0;
+                vn[r] = (present && (!FUSED || !has_values)) ? 1.f : 0.f;
+                if (present && has_values) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
+            });
+            const uint32_t slot = slots + s * 4096;
+            if (FUSED) {
+                if (use > 0) {
+                    bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                }
+                ptx::for_each_row<32>([&](auto rc) {
+                    constexpr int r = decltype(rc)::value;
+                    ptx::sts32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
+                });
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(sl_full(s));
+            } else {
+                {
+                    bool ok = ptx::mbar_wait(sl_full(s), use & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                }
+                ptx::for_each_row<32>([&](auto rc) {
+                    constexpr int r = decltype(rc)::value;
+                    uint32_t pos, m, v;
+                    ptx::lds64_off<r * 8>(tab, pos, m);
+                    asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4))), "n"(r * 128) : "memory");
+                    if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = vn[r] * __uint_as_float(v);
+                });
+                __syncwarp();
+                if (lane == 0) ptx::mbar_arrive(sl_empty(s));
             }
         }
     }
