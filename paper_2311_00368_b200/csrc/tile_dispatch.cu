@@ -115,9 +115,11 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     }
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
     int2 *win = reinterpret_cast<int2 *>(ws + pattern_table_offset(M));
-    const int GR = (Wk + 31) / 32;               // warps per row
-    const long long threads = (long long)M * GR * 32;
-    tile_masks_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(M, K, Wk, GR, row_ptr, col_idx, win, flags);
+    if (Wk > kMasksMaxWk) return B2SP_ERR_UNSUPPORTED;
+    if (cudaFuncSetAttribute(tile_masks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMasksMaxWk * 4) != cudaSuccess)
+        return B2SP_ERR_CUDA;
+    const int cap = kSMs * 64;
+    tile_masks_kernel<<<M < cap ? M : cap, kMasksWarps * 32, (size_t)Wk * 4, st>>>(M, K, Wk, nnz, row_ptr, col_idx, win, flags);
     write_signature_kernel<<<1, 1, 0, st>>>(sig, sig_dev);
     *launches += 2;
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
@@ -145,7 +147,7 @@ TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
     p.TR = M > 128 ? 256 : 128;   // rows of S per CTA (UMMA N)
     p.Mt = (M + p.TR - 1) / p.TR;
     size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
-    if (win_bytes > (size_t)2 << 30) return p;  // pattern far too sparse / wide for dense tiles
+    if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;  // pattern far too sparse / wide for dense tiles
     p.KS = pick_split(p.Mt * p.Nt, p.Wk);
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
@@ -225,7 +227,7 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     p.Nt = fused ? (N + kFusedNT - 1) / kFusedNT : 1;
     p.Np = fused ? p.Nt * kFusedNT : 0;
     size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
-    if (win_bytes > (size_t)2 << 30) return p;
+    if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(p.Mt * p.Nt, p.Kp / kFusedBlk);
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
@@ -349,3 +351,13 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 }
 
 }  // namespace b2sp
+
+#ifdef B2SP_TILE_PROFILE
+// Profiling builds only: copies the fused tile kernel's role timers to the host and clears them.
+extern "C" int b2sp_prof_fetch(unsigned long long *host32)
+{
+    unsigned long long zero[32] = {};
+    if (cudaMemcpyFromSymbol(host32, b2sp::g_fused_prof, sizeof(zero)) != cudaSuccess) return 1;
+    return cudaMemcpyToSymbol(b2sp::g_fused_prof, zero, sizeof(zero)) != cudaSuccess;
+}
+#endif

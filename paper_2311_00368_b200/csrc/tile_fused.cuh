@@ -29,7 +29,8 @@
 #define B2SP_FPROF_DECL long long fp_t0 = 0, fp_acc[6] = {0, 0, 0, 0, 0, 0};
 #define B2SP_FPROF_START fp_t0 = clock64();
 #define B2SP_FPROF_STOP(i) { long long t_ = clock64(); fp_acc[i] += t_ - fp_t0; fp_t0 = t_; }
-#define B2SP_FPROF_FLUSH(base) { if (lane == 0 && a.prof) { for (int i_ = 0; i_ < 6; ++i_) atomicAdd(a.prof + (base) + i_, (unsigned long long)fp_acc[i_]); } }
+#define B2SP_FPROF_FLUSH(base) { if (lane == 0) { for (int i_ = 0; i_ < 6; ++i_) atomicAdd(b2sp::g_fused_prof + (base) + i_, (unsigned long long)fp_acc[i_]); } }
+namespace b2sp { __device__ unsigned long long g_fused_prof[32]; }
 #else
 #define B2SP_FPROF_DECL
 #define B2SP_FPROF_START
@@ -42,9 +43,12 @@ namespace b2sp {
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
-constexpr int kFusedThreads = 576;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: processors, warps 6-17: helpers
+constexpr int kFusedThreads = 672;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: processors, warps 6-20: helpers (not 9, 13, 17)
 constexpr int kFusedSlots = 12;     // shared-memory slots (4 KB) between helpers and processors: 3 windows deep
-constexpr int kFusedHelpers = 12;
+constexpr int kFusedHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) gets no helper: its issue slots feed the tensor pipe
+// A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one phase
+// away: every slot must always be filled by the same helper and drained by the same processor warp.
+static_assert(kFusedSlots % kFusedHelpers == 0 && kFusedSlots % 4 == 0, "slot ownership must be fixed");
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
@@ -313,6 +317,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // SDDMM: per window, copy the row of P into a slot; a helper warp writes the stored entries.
         const int grow = m0 + row;
         const int nwin = nblk * WPB;
+        B2SP_FPROF_DECL
+        B2SP_FPROF_START
         for (int it = 0; it < nwin; ++it) {
             const int blk = it / WPB, w = it % WPB;
             const int j = it * 4 + q, s = j % NSLOT, use = j / NSLOT;
@@ -323,6 +329,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     bool ok = ptx::mbar_wait(sl_full(s), use & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
+                B2SP_FPROF_STOP(0)
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
                     uint32_t x0, x1, x2, x3;
@@ -334,6 +341,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
+                B2SP_FPROF_STOP(1)
                 uint32_t p0[16], p1[16];
                 if (SPMM) {
 #pragma unroll
@@ -354,12 +362,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         if (lane == 0) ptx::mbar_arrive(p_free(0));
                     }
                 }
+                B2SP_FPROF_STOP(2)
                 const int ppb = it & 1, ppuse = it >> 1;
                 if (ppuse > 0) {
                     bool ok = ptx::mbar_wait(pp_free(ppb), (ppuse - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
                 }
+                B2SP_FPROF_STOP(3)
                 uint32_t hi[16], lo[16];
                 const uint32_t pph = tmem + lane_addr + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
 #pragma unroll
@@ -374,6 +384,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(pp_full(ppb));
+                B2SP_FPROF_STOP(4)
             } else {
                 const int pb = blk & 1;
                 if (w == 0) {
@@ -391,10 +402,12 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(p_free(pb));
                 }
+                B2SP_FPROF_STOP(2)
                 if (use > 0) {
                     bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
+                B2SP_FPROF_STOP(0)
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
                     const uint32_t *src = jj < 4 ? &p0[4 * jj] : &p1[4 * (jj - 4)];
@@ -403,8 +416,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_full(s));
+                B2SP_FPROF_STOP(4)
             }
         }
+        B2SP_FPROF_FLUSH(8)
         // ---------------- epilogue: O accumulator -> global ----------------
         if (FUSED) {
             {
@@ -435,14 +450,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
             }
         }
-    } else {
+    } else if ((warp & 3) != 1) {
         // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
         // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
         // values) and write them transposed into a slot, from which the processor thread of each row
         // reads its row.  SDDMM: prefetch the stored values the same way, then take the P rows the
         // processors left in the slot and write the stored entries, one coalesced run per row.
-        const int h = warp - 6;
+        const int h = (warp - 6) - ((warp - 5) >> 2);   // warps 6,7,8,10,11,12,14,... -> 0,1,2,3,...
         const uint32_t tab = helper_tabs + h * 256;   // 32 records (position, mask) of the item's rows
         const int wbase = b0 * WPB, nitems = nblk * WPB * 4;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
@@ -454,6 +469,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             return r;
         };
         int2 rec_next = load_rec(h);
+        B2SP_FPROF_DECL
+        B2SP_FPROF_START
         for (int j = h; j < nitems; j += NH) {
             const int s = j % NSLOT, use = j / NSLOT;
             const int2 rec = rec_next;
@@ -471,22 +488,26 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (present && has_values) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
             });
             const uint32_t slot = slots + s * 4096;
+            B2SP_FPROF_STOP(0)
             if (FUSED) {
                 if (use > 0) {
                     bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
+                B2SP_FPROF_STOP(1)
                 ptx::for_each_row<32>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     ptx::sts32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
                 });
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_full(s));
+                B2SP_FPROF_STOP(2)
             } else {
                 {
                     bool ok = ptx::mbar_wait(sl_full(s), use & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
+                B2SP_FPROF_STOP(1)
                 ptx::for_each_row<32>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     uint32_t pos, m, v;
@@ -496,8 +517,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 });
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
+                B2SP_FPROF_STOP(2)
             }
         }
+        B2SP_FPROF_FLUSH(16)
     }
     if (failed) atomicExch(a.status, 1);
     ptx::tc_fence_before_sync();

@@ -45,51 +45,101 @@ constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not s
 
 // ---- window table -------------------------------------------------------------------------------
 // T[r*Wk + w] = (first CSR position of row r whose column is >= 32w, occupancy bit mask of the column
-// window [32w, 32w+32): bit b set <=> column 32w+b is stored).  One lane per window, one warp per 32
-// consecutive windows of a row: a per-lane binary search finds where the window starts, a short loop
-// ORs the bits of its (at most 32) entries, and the warp stores 32 records with one coalesced write.
-// Every window of every row is written, so the table needs no clearing and no atomics.
+// window [32w, 32w+32): bit b set <=> column 32w+b is stored).
+// One block of four warps per row (rows differ a lot in length; blocks are scheduled as they finish),
+// one mask word per window of the row in shared memory.  First sweep: the warps read the row's column
+// indices 128 at a time (coalesced, four per lane); a lane merges the bits of its entries that fall
+// into the same window and ORs them into the window's word.  Second sweep: thread = window; the
+// position of a window is the row start plus the entries of all earlier windows (a block prefix sum
+// over the pop counts).  Every window of every row is written, so the table needs no clearing.
 // The table is only meaningful when the columns of each row are strictly increasing and in range;
-// each warp also checks that for its share of the row's entries and sets flags[kFlagUnsorted] if not.
-__global__ void tile_masks_kernel(int M, int K, int Wk, int GR, const int *__restrict__ row_ptr,
-                                  const int *__restrict__ col_idx, int2 *__restrict__ T,
-                                  int *__restrict__ flags)
-{
-    const int lane = threadIdx.x & 31;
-    const long long gw = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;   // global warp
-    const int row = (int)(gw / GR), g = (int)(gw % GR);
-    if (row >= M) return;
-    const int beg = __ldg(row_ptr + row), end = __ldg(row_ptr + row + 1);
-    const int len = end - beg;
-    const int w = g * 32 + lane;
+// the first sweep checks exactly that and sets flags[kFlagUnsorted] if not.
+constexpr int kMasksWarps = 4;
+constexpr int kMasksMaxWk = 24 * 1024;   // the mask row must fit in the shared memory a block may ask for (96 KB)
 
-    // lower bound of 32*w among the row's columns (same trip count for the whole warp)
-    int lo = beg, hi = end;
-    const int steps = len > 0 ? 32 - __clz(len) : 0;
-    const int key = w << 5;
-    for (int s = 0; s < steps; ++s) {
-        if (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            if (__ldg(col_idx + mid) < key) lo = mid + 1; else hi = mid;
-        }
-    }
-    // bits of the window's entries
-    unsigned mask = 0;
-    if (w < Wk) {
-        const int wend = key + 32;
-        for (int p = lo; p < end; ++p) {
-            const int c = __ldg(col_idx + p);
-            if (c >= wend) break;
-            mask |= 1u << (c & 31);
-        }
-        T[(size_t)row * Wk + w] = make_int2(lo, (int)mask);
-    }
-    // order / range check on this warp's share of the row
-    const int v0 = beg + (int)((long long)len * g / GR), v1 = beg + (int)((long long)len * (g + 1) / GR);
+__global__ void __launch_bounds__(kMasksWarps * 32)
+tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ row_ptr,
+                  const int *__restrict__ col_idx, int2 *__restrict__ T, int *__restrict__ flags)
+{
+    extern __shared__ __align__(16) unsigned mask[];     // Wk words
+    __shared__ int warp_total[kMasksWarps];
+    constexpr unsigned kFull = 0xffffffffu;
+    constexpr int NT = kMasksWarps * 32;
+    const bool vec = (reinterpret_cast<uintptr_t>(col_idx) & 15) == 0;
+    const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     bool bad = false;
-    for (int p = v0 + lane; p < v1; p += 32) {
-        const int c = __ldg(col_idx + p);
-        bad |= c < 0 || c >= K || (p > beg && c <= __ldg(col_idx + p - 1));
+    for (int row = blockIdx.x; row < M; row += gridDim.x) {
+        for (int w = threadIdx.x; w < Wk; w += NT) mask[w] = 0u;
+        __syncthreads();
+        const int beg = __ldg(row_ptr + row), end = __ldg(row_ptr + row + 1);
+        // lane l of a warp takes positions p .. p + 3 (one 16-byte load when the array allows it); the
+        // warp's next load is in flight while this one is checked.
+        auto load4 = [&](int p) {
+            int4 c = make_int4(0, 0, 0, 0);
+            if (p >= end) return c;
+            if (vec && p + 3 < nnz) return __ldg(reinterpret_cast<const int4 *>(col_idx + p));
+            c.x = __ldg(col_idx + p);
+            if (p + 1 < end) c.y = __ldg(col_idx + p + 1);
+            if (p + 2 < end) c.z = __ldg(col_idx + p + 2);
+            if (p + 3 < end) c.w = __ldg(col_idx + p + 3);
+            return c;
+        };
+        const int abeg = beg & ~3;
+        int4 c_next = load4(abeg + 128 * wib + 4 * lane);
+        for (int p0 = abeg + 128 * wib; p0 < end; p0 += 128 * kMasksWarps) {
+            const int p = p0 + 4 * lane;
+            const int4 c = c_next;
+            c_next = load4(p + 128 * kMasksWarps);
+            int prev = __shfl_up_sync(kFull, c.w, 1);
+            if (lane == 0 && p > beg) prev = __ldg(col_idx + p - 1);
+            int cur_w = -1;
+            unsigned cur_bits = 0u;
+            auto visit = [&](int q, int col, int before) {
+                if (q >= beg && q < end) {
+                    const bool ok = col >= 0 && col < K;
+                    bad |= !ok || (q > beg && col <= before);
+                    if (ok) {
+                        const int w = col >> 5;
+                        if (w != cur_w) {
+                            if (cur_w >= 0) atomicOr(&mask[cur_w], cur_bits);
+                            cur_w = w;
+                            cur_bits = 0u;
+                        }
+                        cur_bits |= 1u << (col & 31);
+                    }
+                }
+            };
+            visit(p, c.x, prev);
+            visit(p + 1, c.y, c.x);
+            visit(p + 2, c.z, c.y);
+            visit(p + 3, c.w, c.z);
+            if (cur_w >= 0) atomicOr(&mask[cur_w], cur_bits);
+        }
+        __syncthreads();
+        int run = beg;
+        for (int w0 = 0; w0 < Wk; w0 += NT) {
+            const int w = w0 + threadIdx.x;
+            const unsigned m = w < Wk ? mask[w] : 0u;
+            const int cnt = __popc(m);
+            int incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int t = __shfl_up_sync(kFull, incl, d);
+                if (lane >= d) incl += t;
+            }
+            if (lane == 31) warp_total[wib] = incl;
+            __syncthreads();
+            int before = 0, all = 0;
+#pragma unroll
+            for (int i = 0; i < kMasksWarps; ++i) {
+                const int t = warp_total[i];
+                if (i < wib) before += t;
+                all += t;
+            }
+            if (w < Wk) T[(size_t)row * Wk + w] = make_int2(run + before + incl - cnt, (int)m);
+            run += all;
+            __syncthreads();   // warp_total and mask are reused
+        }
     }
     if (bad) atomicExch(&flags[kFlagUnsorted], 1);
 }
