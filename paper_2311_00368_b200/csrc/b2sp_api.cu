@@ -63,13 +63,23 @@ b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t
     return check_launch();
 }
 
+// A gated launch (the row family as the dense-tile family's fallback) almost always finds its gate
+// closed: it gets a small grid whose blocks walk the rows, so that the usual case costs little.
+inline unsigned gated_blocks(unsigned rows, const int *gate)
+{
+    const unsigned cap = 148u * 4u;
+    return gate && rows > cap ? cap : rows;
+}
+
 template <int U, int SPLIT>
 void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
                  const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
                  const int *order, const int *gate)
 {
+    const int nrows = (int)grid.x;
+    grid.x = gated_blocks(grid.x, gate);
     spmm_row_kernel<U, SPLIT><<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                           ldo, order, gate);
+                                                           ldo, order, gate, nrows);
 }
 
 // Column geometry for a width N on the float4 path: U float4 per lane, SPLIT sub-warps.
@@ -91,8 +101,10 @@ void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const 
                   float *out, const int *order, const int *gate)
 {
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
+    const int nrows = (int)grid.x;
+    grid.x = gated_blocks(grid.x, gate);
     sddmm_row_kernel<KU><<<grid, kRowThreads, smem, st>>>(Kd, row_ptr, col_idx, sv, A, lda, B, ldb,
-                                                         out, order, gate);
+                                                         out, order, gate, nrows);
 }
 
 template <int KU, int U, int SPLIT>
@@ -110,8 +122,10 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
             cudaSuccess)
             return B2SP_ERR_CUDA;
     }
+    const int nrows = (int)grid.x;
+    grid.x = gated_blocks(grid.x, gate);
     kern<<<grid, kRowThreads, smem, st>>>(Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
-                                          order, gate);
+                                          order, gate, nrows);
     return B2SP_OK;
 }
 
@@ -217,9 +231,9 @@ static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_id
         else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
         else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
     } else {
-        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
         spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                            ldo, order, gate);
+                                                            ldo, order, gate, M);
     }
     return check_launch();
 }
@@ -306,8 +320,9 @@ static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_
         }
         }
     } else {
+        grid.x = gated_blocks(grid.x, gate);
         sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
-                                                             B, ldb, out_values, order, gate);
+                                                             B, ldb, out_values, order, gate, M);
     }
     return check_launch();
 }
@@ -384,9 +399,9 @@ static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const in
         }
         if (rc != B2SP_OK) return rc;
     } else {
-        dim3 grid((unsigned)M, (unsigned)((N + 127) / 128));
+        dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
         fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
-                                                               lda, B, ldb, D, ldd, O, ldo, order, gate);
+                                                               lda, B, ldb, D, ldd, O, ldo, order, gate, M);
     }
     return check_launch();
 }

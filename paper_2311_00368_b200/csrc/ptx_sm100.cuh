@@ -43,6 +43,14 @@ __device__ __forceinline__ void lds64_off(uint32_t addr, uint32_t &v0, uint32_t 
     asm volatile("ld.shared.v2.b32 {%0, %1}, [%2 + %3];" : "=r"(v0), "=r"(v1) : "r"(addr), "n"(OFF));
 }
 
+template <int OFF>
+__device__ __forceinline__ uint32_t lds32_off(uint32_t addr)
+{
+    uint32_t v;   // no memory clobber, as above
+    asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+
 // Compile-time row loop: calls f(std::integral_constant<int, r>) for r = 0..N-1, so that row offsets
 // become instruction immediates.
 template <int N, int R = 0, class F>

@@ -173,48 +173,51 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                 const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                 float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                const int *__restrict__ gate)
+                const int *__restrict__ gate, int nrows)
 {
     using G = SweepGeom<U, SPLIT>;
     __shared__ float4 red[kRowWarps * U * G::LPN];
     if (gate && *gate == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / G::LPN, sl = lane % G::LPN;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int col0 = blockIdx.y * G::SLAB + sl * 4;
-    bool live[U];
-    float4 acc[U];
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int col0 = blockIdx.y * G::SLAB + sl * 4;
+        bool live[U];
+        float4 acc[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        live[u] = col0 + u * G::LPN * 4 < N;
-        acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    const float *Dcol = D + col0;
-    // the next chunk's indices and values are fetched before the current chunk is consumed
-    // (the role of the paper's prefetch of the next ja/avalues block)
-    int k = 0;
-    float s = 0.f;
-    {
-        int p = beg + warp * 32 + lane;
-        if (p < end) {
-            k = __ldg(col_idx + p);
-            s = __ldg(values + p);
+        for (int u = 0; u < U; ++u) {
+            live[u] = col0 + u * G::LPN * 4 < N;
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
-    }
-    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
-        int pn = c + kRowWarps * 32 + lane;
-        int kn = 0;
-        float sn = 0.f;
-        if (pn < end) {
-            kn = __ldg(col_idx + pn);
-            sn = __ldg(values + pn);
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        const float *Dcol = D + col0;
+        // the next chunk's indices and values are fetched before the current chunk is consumed
+        // (the role of the paper's prefetch of the next ja/avalues block)
+        int k = 0;
+        float s = 0.f;
+        {
+            int p = beg + warp * 32 + lane;
+            if (p < end) {
+                k = __ldg(col_idx + p);
+                s = __ldg(values + p);
+            }
         }
-        saxpy_chunk<U, SPLIT, false>(acc, k, s, min(32, end - c), Dcol, ldd, live, sub);
-        k = kn;
-        s = sn;
+        for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+            int pn = c + kRowWarps * 32 + lane;
+            int kn = 0;
+            float sn = 0.f;
+            if (pn < end) {
+                kn = __ldg(col_idx + pn);
+                sn = __ldg(values + pn);
+            }
+            saxpy_chunk<U, SPLIT, false>(acc, k, s, min(32, end - c), Dcol, ldd, live, sub);
+            k = kn;
+            s = sn;
+        }
+        reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
+        __syncthreads();   // shared memory is reused by the next row
     }
-    reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
 }
 
 // Scalar path for any N / ld / alignment: a lane owns columns col0 + lane + 32u (u < 4).
@@ -222,44 +225,47 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                        const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                        float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                       const int *__restrict__ gate)
+                       const int *__restrict__ gate, int nrows)
 {
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int col0 = blockIdx.y * 128 + lane;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
-        int p = c + lane;
-        int k = 0;
-        float s = 0.f;
-        if (p < end) {
-            k = __ldg(col_idx + p);
-            s = __ldg(values + p);
-        }
-        int cnt = min(32, end - c);
-        for (int j = 0; j < cnt; ++j) {
-            int kk = __shfl_sync(kFull, k, j);
-            float ss = __shfl_sync(kFull, s, j);
-            const float *d = D + (int64_t)kk * ldd + col0;
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int col0 = blockIdx.y * 128 + lane;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+            int p = c + lane;
+            int k = 0;
+            float s = 0.f;
+            if (p < end) {
+                k = __ldg(col_idx + p);
+                s = __ldg(values + p);
+            }
+            int cnt = min(32, end - c);
+            for (int j = 0; j < cnt; ++j) {
+                int kk = __shfl_sync(kFull, k, j);
+                float ss = __shfl_sync(kFull, s, j);
+                const float *d = D + (int64_t)kk * ldd + col0;
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+                for (int u = 0; u < 4; ++u)
+                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+            }
         }
-    }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
-    __syncthreads();
-    if (warp == 0) {
+        for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
+        __syncthreads();
+        if (warp == 0) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (col0 + 32 * u >= N) continue;
-            float r = red[0][lane + 32 * u];
-            for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
-            O[(int64_t)row * ldo + col0 + 32 * u] = r;
+            for (int u = 0; u < 4; ++u) {
+                if (col0 + 32 * u >= N) continue;
+                float r = red[0][lane + 32 * u];
+                for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
+                O[(int64_t)row * ldo + col0 + 32 * u] = r;
+            }
         }
+        __syncthreads();   // shared memory is reused by the next row
     }
 }
 
@@ -321,23 +327,26 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                  const float *s_values, const float *__restrict__ A, int64_t lda,
                  const float *__restrict__ B, int64_t ldb, float *out_values,
-                 const int *__restrict__ row_order, const int *__restrict__ gate)
+                 const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
 {
     extern __shared__ float4 dyn_smem[];
     float *a_smem = reinterpret_cast<float *>(dyn_smem);
     if (gate && *gate == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    float4 areg[KU > 0 ? KU : 1];
-    load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
-    const int slot = (lane & 7) * 4 + (lane >> 3);  // entry of the chunk this lane ends up holding
-    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
-        int p = c + lane;
-        int k = p < end ? __ldg(col_idx + p) : 0;
-        float dp = sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
-        int q = c + slot;
-        if (q < end) out_values[q] = s_values ? s_values[q] * dp : dp;
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        float4 areg[KU > 0 ? KU : 1];
+        load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+        const int slot = (lane & 7) * 4 + (lane >> 3);  // entry of the chunk this lane ends up holding
+        for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+            int p = c + lane;
+            int k = p < end ? __ldg(col_idx + p) : 0;
+            float dp = sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
+            int q = c + slot;
+            if (q < end) out_values[q] = s_values ? s_values[q] * dp : dp;
+        }
+        __syncthreads();   // shared memory is reused by the next row
     }
 }
 
@@ -346,17 +355,20 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                         const float *s_values, const float *__restrict__ A, int64_t lda,
                         const float *__restrict__ B, int64_t ldb, float *out_values,
-                        const int *__restrict__ row_order, const int *__restrict__ gate)
+                        const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
 {
     if (gate && *gate == 0) return;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    const float *a = A + (int64_t)row * lda;
-    for (int p = beg + threadIdx.x; p < end; p += kRowThreads) {
-        const float *b = B + (int64_t)__ldg(col_idx + p) * ldb;
-        float dp = 0.f;
-        for (int l = 0; l < Kd; ++l) dp = fmaf(__ldg(a + l), __ldg(b + l), dp);
-        out_values[p] = s_values ? s_values[p] * dp : dp;
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        const float *a = A + (int64_t)row * lda;
+        for (int p = beg + threadIdx.x; p < end; p += kRowThreads) {
+            const float *b = B + (int64_t)__ldg(col_idx + p) * ldb;
+            float dp = 0.f;
+            for (int l = 0; l < Kd; ++l) dp = fmaf(__ldg(a + l), __ldg(b + l), dp);
+            out_values[p] = s_values ? s_values[p] * dp : dp;
+        }
+        __syncthreads();   // shared memory is reused by the next row
     }
 }
 
@@ -370,7 +382,7 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
                    const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
-                   const int *__restrict__ row_order, const int *__restrict__ gate)
+                   const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
 {
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
@@ -379,37 +391,40 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
     float *a_smem = reinterpret_cast<float *>(dyn_smem + kRowWarps * U * G::LPN);  // Kd (KU == 0)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / G::LPN, sl = lane % G::LPN;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int col0 = blockIdx.y * G::SLAB + sl * 4;
-    bool live[U];
-    float4 acc[U];
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int col0 = blockIdx.y * G::SLAB + sl * 4;
+        bool live[U];
+        float4 acc[U];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-        live[u] = col0 + u * G::LPN * 4 < N;
-        acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int u = 0; u < U; ++u) {
+            live[u] = col0 + u * G::LPN * 4 < N;
+            acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        float4 areg[KU > 0 ? KU : 1];
+        load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+        const int slot = (lane & 7) * 4 + (lane >> 3);
+        const float *Dcol = D + col0;
+        int k = 0;
+        float sv = 1.f;
+        {
+            int p = beg + warp * 32 + lane, q = beg + warp * 32 + slot;
+            if (p < end) k = __ldg(col_idx + p);
+            if (s_values && q < end) sv = __ldg(s_values + q);
+        }
+        for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+            int pn = c + kRowWarps * 32 + lane, qn = c + kRowWarps * 32 + slot;
+            int kn = pn < end ? __ldg(col_idx + pn) : 0;
+            float svn = (s_values && qn < end) ? __ldg(s_values + qn) : 1.f;
+            float cv = sv * sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
+            saxpy_chunk<U, SPLIT, true>(acc, k, cv, min(32, end - c), Dcol, ldd, live, sub);
+            k = kn;
+            sv = svn;
+        }
+        reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
+        __syncthreads();   // shared memory is reused by the next row
     }
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    float4 areg[KU > 0 ? KU : 1];
-    load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
-    const int slot = (lane & 7) * 4 + (lane >> 3);
-    const float *Dcol = D + col0;
-    int k = 0;
-    float sv = 1.f;
-    {
-        int p = beg + warp * 32 + lane, q = beg + warp * 32 + slot;
-        if (p < end) k = __ldg(col_idx + p);
-        if (s_values && q < end) sv = __ldg(s_values + q);
-    }
-    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
-        int pn = c + kRowWarps * 32 + lane, qn = c + kRowWarps * 32 + slot;
-        int kn = pn < end ? __ldg(col_idx + pn) : 0;
-        float svn = (s_values && qn < end) ? __ldg(s_values + qn) : 1.f;
-        float cv = sv * sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
-        saxpy_chunk<U, SPLIT, true>(acc, k, cv, min(32, end - c), Dcol, ldd, live, sub);
-        k = kn;
-        sv = svn;
-    }
-    reduce_and_store_row<U, SPLIT>(acc, red, warp, lane, O + (int64_t)row * ldo + col0, live);
 }
 
 // Scalar path for any widths / alignment: lane-per-entry dot products, then a scalar sweep.
@@ -419,47 +434,50 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
                           const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
                           int64_t ldb, const float *__restrict__ D, int64_t ldd,
                           float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                          const int *__restrict__ gate)
+                          const int *__restrict__ gate, int nrows)
 {
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int row = row_order ? row_order[blockIdx.x] : blockIdx.x;
-    const int col0 = blockIdx.y * 128 + lane;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    const int beg = row_ptr[row], end = row_ptr[row + 1];
-    const float *a = A + (int64_t)row * lda;
-    for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
-        int p = c + lane;
-        int k = 0;
-        float cv = 0.f;
-        if (p < end) {
-            k = __ldg(col_idx + p);
-            const float *b = B + (int64_t)k * ldb;
-            for (int l = 0; l < Kd; ++l) cv = fmaf(__ldg(a + l), __ldg(b + l), cv);
-            if (s_values) cv *= __ldg(s_values + p);
-        }
-        int cnt = min(32, end - c);
-        for (int j = 0; j < cnt; ++j) {
-            int kk = __shfl_sync(kFull, k, j);
-            float ss = __shfl_sync(kFull, cv, j);
-            const float *d = D + (int64_t)kk * ldd + col0;
+    for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
+        const int row = row_order ? row_order[rb] : rb;
+        const int col0 = blockIdx.y * 128 + lane;
+        float acc[4] = {0.f, 0.f, 0.f, 0.f};
+        const int beg = row_ptr[row], end = row_ptr[row + 1];
+        const float *a = A + (int64_t)row * lda;
+        for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
+            int p = c + lane;
+            int k = 0;
+            float cv = 0.f;
+            if (p < end) {
+                k = __ldg(col_idx + p);
+                const float *b = B + (int64_t)k * ldb;
+                for (int l = 0; l < Kd; ++l) cv = fmaf(__ldg(a + l), __ldg(b + l), cv);
+                if (s_values) cv *= __ldg(s_values + p);
+            }
+            int cnt = min(32, end - c);
+            for (int j = 0; j < cnt; ++j) {
+                int kk = __shfl_sync(kFull, k, j);
+                float ss = __shfl_sync(kFull, cv, j);
+                const float *d = D + (int64_t)kk * ldd + col0;
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
-                if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+                for (int u = 0; u < 4; ++u)
+                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+            }
         }
-    }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
-    __syncthreads();
-    if (warp == 0) {
+        for (int u = 0; u < 4; ++u) red[warp][lane + 32 * u] = acc[u];
+        __syncthreads();
+        if (warp == 0) {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (col0 + 32 * u >= N) continue;
-            float r = red[0][lane + 32 * u];
-            for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
-            O[(int64_t)row * ldo + col0 + 32 * u] = r;
+            for (int u = 0; u < 4; ++u) {
+                if (col0 + 32 * u >= N) continue;
+                float r = red[0][lane + 32 * u];
+                for (int w = 1; w < kRowWarps; ++w) r += red[w][lane + 32 * u];
+                O[(int64_t)row * ldo + col0 + 32 * u] = r;
+            }
         }
+        __syncthreads();   // shared memory is reused by the next row
     }
 }
 

@@ -119,9 +119,8 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     if (cudaFuncSetAttribute(tile_masks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMasksMaxWk * 4) != cudaSuccess)
         return B2SP_ERR_CUDA;
     const int cap = kSMs * 64;
-    tile_masks_kernel<<<M < cap ? M : cap, kMasksWarps * 32, (size_t)Wk * 4, st>>>(M, K, Wk, nnz, row_ptr, col_idx, win, flags);
-    write_signature_kernel<<<1, 1, 0, st>>>(sig, sig_dev);
-    *launches += 2;
+    tile_masks_kernel<<<M < cap ? M : cap, kMasksWarps * 32, (size_t)Wk * 4, st>>>(M, K, Wk, nnz, row_ptr, col_idx, win, flags, sig, sig_dev);
+    *launches += 1;
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 

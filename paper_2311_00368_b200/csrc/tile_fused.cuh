@@ -468,13 +468,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             if (jj < nitems && hrow < a.M && wglob < a.Wk) r = __ldg(a.win + (size_t)hrow * a.Wk + wglob);
             return r;
         };
-        int2 rec_next = load_rec(h);
+        // the records of the next two items are in flight while an item is processed
+        int2 rec_next = load_rec(h), rec_next2 = load_rec(h + NH);
         B2SP_FPROF_DECL
         B2SP_FPROF_START
         for (int j = h; j < nitems; j += NH) {
             const int s = j % NSLOT, use = j / NSLOT;
             const int2 rec = rec_next;
-            rec_next = load_rec(j + NH);   // the next item's records load while this item is processed
+            rec_next = rec_next2;
+            rec_next2 = load_rec(j + 2 * NH);
             __syncwarp();   // everyone is done with the previous item's records
             ptx::sts64(tab + lane * 8, (uint32_t)rec.x, (uint32_t)rec.y);
             __syncwarp();
@@ -508,15 +510,19 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
                 B2SP_FPROF_STOP(1)
+                // all reads of the slot first (independent loads), then the stores
                 ptx::for_each_row<32>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
-                    uint32_t pos, m, v;
-                    ptx::lds64_off<r * 8>(tab, pos, m);
-                    asm volatile("ld.shared.b32 %0, [%1 + %2];" : "=r"(v) : "r"(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4))), "n"(r * 128) : "memory");
-                    if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = vn[r] * __uint_as_float(v);
+                    vn[r] *= __uint_as_float(ptx::lds32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4))));
                 });
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
+                ptx::for_each_row<32>([&](auto rc) {
+                    constexpr int r = decltype(rc)::value;
+                    uint32_t pos, m;
+                    ptx::lds64_off<r * 8>(tab, pos, m);
+                    if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = vn[r];
+                });
                 B2SP_FPROF_STOP(2)
             }
         }

@@ -43,13 +43,21 @@ namespace b2sp {
 constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-byte swizzle row of tf32)
 constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
 
+// ---- table signature ------------------------------------------------------------------------------------
+struct PatternSignature {
+    int magic, M, K, Wk;
+    long long nnz;
+    const int *row_ptr, *col_idx;
+};
+constexpr int kPatternMagic = 0x62327370;
+
 // ---- window table -------------------------------------------------------------------------------
 // T[r*Wk + w] = (first CSR position of row r whose column is >= 32w, occupancy bit mask of the column
 // window [32w, 32w+32): bit b set <=> column 32w+b is stored).
 // One block of four warps per row (rows differ a lot in length; blocks are scheduled as they finish),
 // one mask word per window of the row in shared memory.  First sweep: the warps read the row's column
 // indices 128 at a time (coalesced, four per lane); a lane merges the bits of its entries that fall
-// into the same window and ORs them into the window's word.  Second sweep: thread = window; the
+// into the same window and ORs them into the window's word (shared-memory atomics).  Second sweep: thread = window; the
 // position of a window is the row start plus the entries of all earlier windows (a block prefix sum
 // over the pop counts).  Every window of every row is written, so the table needs no clearing.
 // The table is only meaningful when the columns of each row are strictly increasing and in range;
@@ -59,9 +67,11 @@ constexpr int kMasksMaxWk = 24 * 1024;   // the mask row must fit in the shared 
 
 __global__ void __launch_bounds__(kMasksWarps * 32)
 tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ row_ptr,
-                  const int *__restrict__ col_idx, int2 *__restrict__ T, int *__restrict__ flags)
+                  const int *__restrict__ col_idx, int2 *__restrict__ T, int *__restrict__ flags,
+                  PatternSignature sig, PatternSignature *__restrict__ sig_out)
 {
     extern __shared__ __align__(16) unsigned mask[];     // Wk words
+    if (blockIdx.x == 0 && threadIdx.x == 0) *sig_out = sig;   // what the table is built from
     __shared__ int warp_total[kMasksWarps];
     constexpr unsigned kFull = 0xffffffffu;
     constexpr int NT = kMasksWarps * 32;
@@ -92,28 +102,33 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
             c_next = load4(p + 128 * kMasksWarps);
             int prev = __shfl_up_sync(kFull, c.w, 1);
             if (lane == 0 && p > beg) prev = __ldg(col_idx + p - 1);
-            int cur_w = -1;
-            unsigned cur_bits = 0u;
-            auto visit = [&](int q, int col, int before) {
-                if (q >= beg && q < end) {
-                    const bool ok = col >= 0 && col < K;
-                    bad |= !ok || (q > beg && col <= before);
-                    if (ok) {
-                        const int w = col >> 5;
-                        if (w != cur_w) {
-                            if (cur_w >= 0) atomicOr(&mask[cur_w], cur_bits);
-                            cur_w = w;
-                            cur_bits = 0u;
-                        }
-                        cur_bits |= 1u << (col & 31);
-                    }
+            const bool inside = p >= beg && p + 3 < end;
+            const bool in_range = (unsigned)c.x < (unsigned)K && (unsigned)c.y < (unsigned)K &&
+                                  (unsigned)c.z < (unsigned)K && (unsigned)c.w < (unsigned)K;
+            if (inside && in_range) {
+                // common case: four valid entries, almost always in one or two windows
+                bad |= (p > beg && c.x <= prev) || c.y <= c.x || c.z <= c.y || c.w <= c.z;
+                const int wx = c.x >> 5, wy = c.y >> 5, wz = c.z >> 5, ww = c.w >> 5;
+                const unsigned bx = 1u << (c.x & 31), by = 1u << (c.y & 31), bz = 1u << (c.z & 31), bw = 1u << (c.w & 31);
+                atomicOr(&mask[wx], bx | (wy == wx ? by : 0u) | (wz == wx ? bz : 0u) | (ww == wx ? bw : 0u));
+                if (ww != wx) {
+                    atomicOr(&mask[ww], bw | (wz == ww ? bz : 0u) | (wy == ww ? by : 0u));
+                    if (wy != wx && wy != ww) atomicOr(&mask[wy], by);
+                    if (wz != wx && wz != ww) atomicOr(&mask[wz], bz);
                 }
-            };
-            visit(p, c.x, prev);
-            visit(p + 1, c.y, c.x);
-            visit(p + 2, c.z, c.y);
-            visit(p + 3, c.w, c.z);
-            if (cur_w >= 0) atomicOr(&mask[cur_w], cur_bits);
+            } else {
+                auto visit = [&](int q, int col, int before) {
+                    if (q >= beg && q < end) {
+                        const bool ok = (unsigned)col < (unsigned)K;
+                        bad |= !ok || (q > beg && col <= before);
+                        if (ok) atomicOr(&mask[col >> 5], 1u << (col & 31));
+                    }
+                };
+                visit(p, c.x, prev);
+                visit(p + 1, c.y, c.x);
+                visit(p + 2, c.z, c.y);
+                visit(p + 3, c.w, c.z);
+            }
         }
         __syncthreads();
         int run = beg;
@@ -143,16 +158,6 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
     }
     if (bad) atomicExch(&flags[kFlagUnsorted], 1);
 }
-
-// ---- table signature ------------------------------------------------------------------------------------
-struct PatternSignature {
-    int magic, M, K, Wk;
-    long long nnz;
-    const int *row_ptr, *col_idx;
-};
-constexpr int kPatternMagic = 0x62327370;
-
-__global__ void write_signature_kernel(PatternSignature sig, PatternSignature *dst) { *dst = sig; }
 
 // Raises flags[kFlagUnsorted] when the workspace does not hold a table built from these arrays.
 __global__ void check_signature_kernel(PatternSignature want, const PatternSignature *have, int *flags)
