@@ -191,7 +191,7 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
     if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
     size_t need = row_workspace_bytes(M);
     if (op == B2SP_OP_SPMM && tile_profitable(M, K, N, nnz)) {
-        TilePlan p = plan_spmm_tile(M, K, N, nnz, need);
+        FusedPlan p = plan_fused_tile(M, K, 0, N, nnz, need, true);
         if (p.feasible && p.bytes > need) need = p.bytes;
     }
     if (op == B2SP_OP_SDDMM && tile_profitable(M, K, Kd, nnz)) {
@@ -207,14 +207,6 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
-
-static bool spmm_via_fused_pipeline()
-{
-    // Default: SPMM runs through the FusedMM tile pipeline (P' = the stored values).  The older kernel
-    // that builds S tiles in shared memory (spmm_tile_kernel) stays selectable for comparison.
-    const char *e = getenv("B2SP_SPMM_IMPL");   // tuning aid: "builder" selects the shared-memory builder
-    return !(e && e[0] == 'b');
-}
 
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
@@ -252,9 +244,9 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     const size_t row_bytes = row_workspace_bytes(M);
     b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
-    TilePlan plan;
+    FusedPlan plan;   // SPMM runs through the FusedMM tile pipeline with P' = the stored values (Kd = 0)
     if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, N, nnz)))
-        plan = plan_spmm_tile(M, K, N, nnz, row_bytes);
+        plan = plan_fused_tile(M, K, 0, N, nnz, row_bytes, true);
     int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
     if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
     else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
@@ -265,20 +257,9 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     if (nnz == 0) return zero_rows(O, ldo, M, N, st);
 
     Workspace w = carve(workspace);
-    if (use == B2SP_ALGO_TILE && spmm_via_fused_pipeline()) {
-        FusedPlan fp = plan_fused_tile(M, K, 0, N, nnz, row_bytes, true);
-        if (fp.feasible && workspace_bytes >= fp.bytes) {
-            rc = fused_tile(fp, prepared, 2, M, K, 0, N, nnz, row_ptr, col_idx, values, nullptr, 0, nullptr, 0, D, ldd,
-                            O, ldo, workspace, st, &launches);
-            if (rc != B2SP_OK) return rc;
-            const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
-            rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, st);
-            g_last_launches[B2SP_OP_SPMM] = launches + 1;
-            return rc;
-        }
-    }
     if (use == B2SP_ALGO_TILE) {
-        rc = spmm_tile(plan, prepared, M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, st, &launches);
+        rc = fused_tile(plan, prepared, 2, M, K, 0, N, nnz, row_ptr, col_idx, values, nullptr, 0, nullptr, 0, D, ldd,
+                        O, ldo, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);

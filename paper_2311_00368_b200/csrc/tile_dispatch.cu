@@ -73,18 +73,6 @@ int pick_split(int base_tiles, int Wk)
     return ks < 1 ? 1 : ks;
 }
 
-template <int TR>
-b2sp_status launch_spmm_tile(const CUtensorMap &hi, const CUtensorMap &lo, const SpmmTileArgs &a, int items,
-                             cudaStream_t st)
-{
-    using Cfg = SpmmTileCfg<TR>;
-    auto kern = spmm_tile_kernel<TR>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-        return B2SP_ERR_CUDA;
-    kern<<<items, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(hi, lo, a);
-    return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
-}
-
 }  // namespace
 
 size_t pattern_table_offset(int M)
@@ -104,15 +92,9 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     PatternSignature *sig_dev = reinterpret_cast<PatternSignature *>(ws + kWsSignatureOffset);
     const int Wk = (K + kTileKC - 1) / kTileKC;
     PatternSignature sig{kPatternMagic, M, K, Wk, nnz, row_ptr, col_idx};
-    if (prepared) {
-        // keep the table, its flag and its signature; clear only the status / profiling words
-        if (cudaMemsetAsync(ws + kWsStatusOffset, 0, kWsTileFlagsOffset - kWsStatusOffset, st) != cudaSuccess ||
-            cudaMemsetAsync(ws + kWsStatusOffset + 128, 0, kWsSignatureOffset - kWsStatusOffset - 128, st) != cudaSuccess)
-            return B2SP_ERR_CUDA;
-        check_signature_kernel<<<1, 1, 0, st>>>(sig, sig_dev, flags);
-        *launches += 1;
-        return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
-    }
+    // A prepared table is used as it is: the tile kernel itself compares the signature stored beside
+    // the table with these arrays and raises the fallback flag on a mismatch.
+    if (prepared) return B2SP_OK;
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
     int2 *win = reinterpret_cast<int2 *>(ws + pattern_table_offset(M));
     if (Wk > kMasksMaxWk) return B2SP_ERR_UNSUPPORTED;
@@ -133,86 +115,6 @@ bool tile_profitable(int M, int K, int width, long long nnz)
     const double cells = (double)M * (double)K;
     const double density = (double)nnz / cells;
     return density >= 0.15 || (density >= 0.08 && cells >= 48.0e6);
-}
-
-TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off)
-{
-    TilePlan p;
-    if (M <= 0 || K <= 0 || N <= 0 || nnz <= 0) return p;
-    p.Wk = (K + kTileKC - 1) / kTileKC;
-    p.Kp = p.Wk * kTileKC;
-    p.Nt = (N + kTileN - 1) / kTileN;
-    p.Np = p.Nt * kTileN;
-    p.TR = M > 128 ? 256 : 128;   // rows of S per CTA (UMMA N)
-    p.Mt = (M + p.TR - 1) / p.TR;
-    size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
-    if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;  // pattern far too sparse / wide for dense tiles
-    p.KS = pick_split(p.Mt * p.Nt, p.Wk);
-    size_t off = align_up(base_off, 1024);
-    p.off_win = off;
-    off = align_up(off + win_bytes, 1024);
-    size_t dbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Np;
-    p.off_dhi = off;
-    off = align_up(off + dbytes, 1024);
-    p.off_dlo = off;
-    off = align_up(off + dbytes, 1024);
-    p.off_part = off;
-    if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * p.TR * (size_t)p.Np;
-    p.bytes = align_up(off, 256);
-    p.feasible = true;
-    return p;
-}
-
-b2sp_status spmm_tile(const TilePlan &p, bool prepared, int M, int K, int N, long long nnz, const int *row_ptr,
-                      const int *col_idx, const float *values, const float *D, long long ldd, float *O,
-                      long long ldo, void *workspace, cudaStream_t st, int *launches)
-{
-    char *ws = static_cast<char *>(workspace);
-    int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
-    int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
-    int2 *win = reinterpret_cast<int2 *>(ws + p.off_win);
-    float *dhi = reinterpret_cast<float *>(ws + p.off_dhi);
-    float *dlo = reinterpret_cast<float *>(ws + p.off_dlo);
-    float *part = reinterpret_cast<float *>(ws + p.off_part);
-
-    CUtensorMap tm_hi, tm_lo;
-    if (!make_blocked_map(&tm_hi, dhi, p.Kp, p.Np / 32, kTileKC, kTileN / 32, true) ||
-        !make_blocked_map(&tm_lo, dlo, p.Kp, p.Np / 32, kTileKC, kTileN / 32, true))
-        return B2SP_ERR_CUDA;
-
-    {
-        b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
-        if (prc != B2SP_OK) return prc;
-    }
-    {
-        long long groups = (long long)p.Kp * (p.Np / 4);
-        int blocks = (int)((groups + 255) / 256 < (long long)kSMs * 8 ? (groups + 255) / 256 : (long long)kSMs * 8);
-        split_dense_kernel<<<blocks, 256, 0, st>>>(D, ldd, K, N, dhi, dlo, p.Kp, p.Np);
-    }
-    *launches += 1;
-    if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
-
-    SpmmTileArgs a;
-    a.M = M; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.nnz = (int)nnz;
-    a.col_idx = col_idx; a.values = values; a.win = win;
-    a.flags = flags; a.status = status;
-    a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
-    if (p.KS == 1) { a.out = O; a.ld_out = ldo; a.slab = 0; }
-    else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * p.TR * p.Np; }
-    int items = p.Mt * p.Nt * p.KS;
-    b2sp_status rc;
-    if (p.TR == 256) rc = launch_spmm_tile<256>(tm_hi, tm_lo, a, items, st);
-    else rc = launch_spmm_tile<128>(tm_hi, tm_lo, a, items, st);
-    *launches += 1;
-    if (rc != B2SP_OK) return rc;
-    if (p.KS > 1) {
-        long long total = (long long)M * N;
-        int blocks = (int)((total + 255) / 256 < (long long)kSMs * 8 ? (total + 255) / 256 : (long long)kSMs * 8);
-        reduce_partials_kernel<<<blocks, 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, O, ldo, flags);
-        *launches += 1;
-        if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
-    }
-    return B2SP_OK;
 }
 
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)
@@ -273,12 +175,15 @@ b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &
     return launch_fused_tile<128, MODE>(bh, bl, dh, dl, a, items, st);
 }
 
-void launch_split(const float *X, long long ld, int rows, int cols, float *hi, float *lo, int rows_p, int cols_p,
-                  cudaStream_t st)
+// Splits one or two dense operands (job 1 optional) and clears the device status word.
+void launch_split(const SplitJob &j0, const SplitJob *j1, int *status, cudaStream_t st)
 {
-    long long groups = (long long)rows_p * (cols_p / 4);
-    long long want = (groups + 255) / 256, cap = (long long)kSMs * 8;
-    split_dense_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(X, ld, rows, cols, hi, lo, rows_p, cols_p);
+    auto groups = [](const SplitJob &j) { return (long long)j.rows_p * (j.cols_p >> 2); };
+    long long most = groups(j0);
+    if (j1 && groups(*j1) > most) most = groups(*j1);
+    const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
+    dim3 grid((unsigned)(want < cap ? want : cap), j1 ? 2u : 1u);
+    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, status);
 }
 
 }  // namespace
@@ -314,12 +219,11 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
         if (prc != B2SP_OK) return prc;
     }
-    if (!spmm) {
-        launch_split(B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, st);
-        *launches += 1;
-    }
-    if (fused) {
-        launch_split(D, ldd, K, N, dhi, dlo, p.Kp, p.Np, st);
+    {
+        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp}, jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np};
+        if (spmm) launch_split(jd, nullptr, status, st);
+        else if (fused) launch_split(jb, &jd, status, st);
+        else launch_split(jb, nullptr, status, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
@@ -328,6 +232,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     a.flags = flags; a.status = status;
+    a.sig_want = PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx};
+    a.sig_have = reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset);
     a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }

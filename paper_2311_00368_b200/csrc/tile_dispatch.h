@@ -13,18 +13,9 @@ constexpr size_t kWsTileFlagsOffset = 320;   // int[..]: flags written by the ti
 constexpr size_t kWsSignatureOffset = 448;   // int[16]: which CSR arrays the window table was built from
 constexpr size_t kWsHeaderBytes = 512;
 
-struct TilePlan {
-    bool feasible = false;
-    int TR = 0, Nt = 0, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
-    size_t off_win = 0, off_dhi = 0, off_dlo = 0, off_part = 0;  // from the workspace base
-    size_t bytes = 0;                                           // total workspace bytes needed
-};
-
-// Plan for SPMM on the dense-tile family; `base_off` = first byte after the row family's region.
-TilePlan plan_spmm_tile(int M, int K, int N, long long nnz, size_t base_off);
-
-// Plans for FusedMM (fused = true) and SDDMM (fused = false) on the dense-tile family.  They need
-// Kd <= 128.  TR is unused; Np is the padded width of D (FusedMM only).
+// Plans for FusedMM / SPMM (fused = true; SPMM passes Kd = 0) and SDDMM (fused = false) on the dense-tile
+// family; `base_off` = first byte after the row family's region.  They need Kd <= 128.  Np is the padded
+// width of D (fused only).
 struct FusedPlan {
     bool feasible = false;
     int Kdp = 0, Nt = 1, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
@@ -33,6 +24,9 @@ struct FusedPlan {
 };
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused);
 
+// Enqueues pre-pass (or the check of a prepared table), operand splits, tile kernel and K-split reduction.
+// The tile kernel leaves immediately if the pre-pass found a row whose columns are not strictly increasing
+// (flag at kWsTileFlagsOffset).
 // mode: 0 = SDDMM, 1 = FusedMM, 2 = SPMM through the FusedMM pipeline (P' = the stored values)
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
@@ -41,12 +35,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 
 // True when the dense-tile family is expected to beat the row family for these sizes.
 bool tile_profitable(int M, int K, int width, long long nnz);
-
-// Enqueues pre-pass + tile kernel (+ reduction).  The kernels leave immediately if the pre-pass
-// finds a row whose columns are not strictly increasing (flag at kWsTileFlagsOffset).
-b2sp_status spmm_tile(const TilePlan &p, bool prepared, int M, int K, int N, long long nnz, const int *row_ptr,
-                      const int *col_idx, const float *values, const float *D, long long ldd, float *O,
-                      long long ldo, void *workspace, cudaStream_t st, int *launches);
 
 // Offset of the window table inside the workspace (the same for every op) and its size.
 size_t pattern_table_offset(int M);

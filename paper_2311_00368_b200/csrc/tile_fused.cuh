@@ -24,6 +24,7 @@
 #include <stdint.h>
 
 #include "ptx_sm100.cuh"
+#include "tile_kernels.cuh"
 
 #ifdef B2SP_TILE_PROFILE
 #define B2SP_FPROF_DECL long long fp_t0 = 0, fp_acc[6] = {0, 0, 0, 0, 0, 0};
@@ -60,7 +61,9 @@ struct FusedTileArgs {
     long long lda;
     float *out;               // FusedMM: O or partial slabs; SDDMM: out_values
     long long ld_out, slab;
-    const int *flags;
+    int *flags;                // flags[0] != 0: the table cannot be used, the row kernels take over
+    PatternSignature sig_want; // the arrays this call was given ...
+    const PatternSignature *sig_have;   // ... and what the table in the workspace was built from
     int *status;
     unsigned long long *prof;  // optional role timers (profiling builds only)
 };
@@ -95,6 +98,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
     if (a.flags[0] != 0) return;  // pattern not usable for tiles: the row kernels take over
+    if (!signature_matches(a.sig_want, a.sig_have)) {   // stale or foreign table (uniform over the grid)
+        if (threadIdx.x == 0) atomicExch(&a.flags[kFlagUnsorted], 1);
+        return;
+    }
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
