@@ -51,6 +51,13 @@ __device__ __forceinline__ uint32_t lds32_off(uint32_t addr)
     return v;
 }
 
+// Four fp32 additions to global memory in one reduction (no return value); 16-byte aligned address.
+__device__ __forceinline__ void red_add_v4(float *addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(__uint_as_float(x)),
+                 "f"(__uint_as_float(y)), "f"(__uint_as_float(z)), "f"(__uint_as_float(w)) : "memory");
+}
+
 // Compile-time row loop: calls f(std::integral_constant<int, r>) for r = 0..N-1, so that row offsets
 // become instruction immediates.
 template <int N, int R = 0, class F>

@@ -175,15 +175,17 @@ b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &
     return launch_fused_tile<128, MODE>(bh, bl, dh, dl, a, items, st);
 }
 
-// Splits one or two dense operands (job 1 optional) and clears the device status word.
-void launch_split(const SplitJob &j0, const SplitJob *j1, int *status, cudaStream_t st)
+// Splits one or two dense operands (job 1 optional), clears the device status word and optionally
+// zero-fills an output matrix.
+void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int *status, cudaStream_t st)
 {
     auto groups = [](const SplitJob &j) { return (long long)j.rows_p * (j.cols_p >> 2); };
     long long most = groups(j0);
     if (j1 && groups(*j1) > most) most = groups(*j1);
     const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
-    dim3 grid((unsigned)(want < cap ? want : cap), j1 ? 2u : 1u);
-    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, status);
+    const int njobs = j1 ? 2 : 1;
+    dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(njobs + (z.out ? 1 : 0)));
+    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, njobs, z, status);
 }
 
 }  // namespace
@@ -202,6 +204,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     float *part = reinterpret_cast<float *>(ws + p.off_part);
 
     const bool fused = mode != kModeSddmm, spmm = mode == kModeSpmm;
+    const bool accumulate = fused && p.KS == 2;
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
     if (!spmm && (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
                   !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
@@ -221,9 +224,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     }
     {
         const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp}, jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np};
-        if (spmm) launch_split(jd, nullptr, status, st);
-        else if (fused) launch_split(jb, &jd, status, st);
-        else launch_split(jb, nullptr, status, st);
+        // Two K splits add their partial tiles straight into O (x + y does not depend on the order, so
+        // the result is still deterministic); more splits go through partial slabs and a fixed-order sum.
+        const ZeroJob z{accumulate ? out : nullptr, ldo, M, N};
+        if (spmm) launch_split(jd, nullptr, z, status, st);
+        else if (fused) launch_split(jb, &jd, z, status, st);
+        else launch_split(jb, nullptr, z, status, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
@@ -231,12 +237,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     FusedTileArgs a;
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
-    a.flags = flags; a.status = status;
+    a.flags = flags; a.status = status; a.accumulate = accumulate ? 1 : 0;
     a.sig_want = PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx};
     a.sig_have = reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset);
     a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
-    else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
+    else if (p.KS == 1 || accumulate) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
     const int items = p.Mt * p.Nt * p.KS;
     b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
@@ -244,7 +250,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
                              : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
-    if (fused && p.KS > 1) {
+    if (fused && p.KS > 1 && !accumulate) {
         long long total = (long long)M * N;
         long long want = (total + 255) / 256, cap = (long long)kSMs * 8;
         reduce_partials_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, out,

@@ -55,6 +55,7 @@ constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
+    int accumulate;           // FusedMM / SPMM with two K splits: add the tile into `out` (zero-filled before the launch)
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
     const float *A;           // M x Kd
@@ -444,7 +445,16 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     ptx::tmem_ld_wait();
                     if (grow < a.M) {
                         const int n = n0 + c * 32;
-                        if (vec && n + 32 <= a.N) {
+                        if (a.accumulate) {
+                            if (vec && n + 32 <= a.N) {
+#pragma unroll
+                                for (int i = 0; i < 32; i += 4) ptx::red_add_v4(orow + n + i, r[i], r[i + 1], r[i + 2], r[i + 3]);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 32; ++i)
+                                    if (n + i < a.N) atomicAdd(orow + n + i, __uint_as_float(r[i]));
+                            }
+                        } else if (vec && n + 32 <= a.N) {
 #pragma unroll
                             for (int i = 0; i < 32; i += 4)
                                 *reinterpret_cast<uint4 *>(orow + n + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);

@@ -152,7 +152,8 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // (rows_p >= rows, cols_p >= cols, cols_p % 32 == 0).  One 32-float group of a row is one
 // 128-byte swizzle row for TMA, and the whole thing is a plain packed 3-D tensor.
 // One launch splits up to two operands (blockIdx.y picks the job) and, being the first kernel of
-// every tile op, also clears the workspace's device status word.
+// every tile op, also clears the workspace's device status word and, when asked to, zero-fills the
+// output matrix (the last blockIdx.y) for tile kernels that add their K-split partial sums into it.
 struct SplitJob {
     const float *X;
     long long ld;
@@ -161,10 +162,23 @@ struct SplitJob {
     int rows_p, cols_p;
 };
 
-__global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int *__restrict__ status)
+struct ZeroJob {
+    float *out;      // NULL: nothing to clear
+    long long ld;
+    int rows, cols;
+};
+
+__global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status)
 {
-    const SplitJob j = blockIdx.y ? j1 : j0;
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
+    if ((int)blockIdx.y == njobs) {   // zero-fill job
+        const long long total = (long long)z.rows * z.cols;
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
+             i += (long long)gridDim.x * blockDim.x)
+            z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
+        return;
+    }
+    const SplitJob j = blockIdx.y ? j1 : j0;
     const bool vec = (j.ld & 3) == 0 && (reinterpret_cast<uintptr_t>(j.X) & 15) == 0;
     const long long groups = (long long)j.rows_p * (j.cols_p >> 2);  // float4 groups
     for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
