@@ -44,7 +44,12 @@ namespace b2sp {
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
-constexpr int kFusedThreads = 672;  // warp 0: TMA, warp 1: MMA + TMEM, warps 2-5: processors, warps 6-20: helpers (not 9, 13, 17)
+// 20 warps = 5 per scheduler (a sixth would cut the register budget from 96 to 80 per thread).
+// Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors; warp 0 and warps 6-19
+// except 9, 13, 17: helpers.  Warps 13 and 17 idle: the scheduler of warps 1, 5, 9, 13, 17 keeps its
+// issue slots for the MMA warp.
+constexpr int kFusedThreads = 640;
+constexpr int kFusedTmaWarp = 9;
 constexpr int kFusedSlots = 12;     // shared-memory slots (4 KB) between helpers and processors: 3 windows deep
 constexpr int kFusedHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) gets no helper: its issue slots feed the tensor pipe
 // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one phase
@@ -205,7 +210,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     __syncthreads();
     ptx::tc_fence_after_sync();
 
-    if (warp == 0) {
+    if (warp == kFusedTmaWarp) {
         // ---------------- TMA producer: per block NCH_B chunks of B rows, then NCH_D chunks of D rows ----------------
         if (lane == 0) {
             if (!SPMM) { ptx::tma_prefetch_desc(&tm_bhi); ptx::tma_prefetch_desc(&tm_blo); }
@@ -317,7 +322,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             B2SP_FPROF_FLUSH(0)
             if (FUSED && !failed) ptx::mma_commit(o_full);
         }
-    } else if (warp < 6) {
+    } else if (warp >= 2 && warp < 6) {
         // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
         // FusedMM / SPMM: per window, take the row's stored values (densified and transposed by a
         // helper warp into a shared-memory slot), multiply them into P (or use them as they are for
@@ -467,14 +472,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
             }
         }
-    } else if ((warp & 3) != 1) {
+    } else if ((warp & 3) != 1) {   // warp 0 and warps 6.. that do not share the MMA warp's scheduler
         // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
         // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
         // values) and write them transposed into a slot, from which the processor thread of each row
         // reads its row.  SDDMM: prefetch the stored values the same way, then take the P rows the
         // processors left in the slot and write the stored entries, one coalesced run per row.
-        const int h = (warp - 6) - ((warp - 5) >> 2);   // warps 6,7,8,10,11,12,14,... -> 0,1,2,3,...
+        const int h = warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);   // warps 0,6,7,8,10,11,12,14,... -> 0,1,2,3,...
         const uint32_t tab = helper_tabs + h * 256;   // 32 records (position, mask) of the item's rows
         const int wbase = b0 * WPB, nitems = nblk * WPB * 4;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
@@ -498,13 +503,16 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::sts64(tab + lane * 8, (uint32_t)rec.x, (uint32_t)rec.y);
             __syncwarp();
             float vn[32];
+            int idx[FUSED ? 1 : 32];   // SDDMM: CSR position of the lane's entry in each row (-1: nothing stored)
             ptx::for_each_row<32>([&](auto rc) {
                 constexpr int r = decltype(rc)::value;
                 uint32_t pos, m;
                 ptx::lds64_off<r * 8>(tab, pos, m);
                 const bool present = (m & lane_bit) != 0;
+                const int at = (int)pos + __popc(m & lt_mask);
                 vn[r] = (present && (!FUSED || !has_values)) ? 1.f : 0.f;
-                if (present && has_values) vn[r] = __ldg(a.s_values + (pos + __popc(m & lt_mask)));
+                if (present && has_values) vn[r] = __ldg(a.s_values + at);
+                if (!FUSED) idx[r] = present ? at : -1;
             });
             const uint32_t slot = slots + s * 4096;
             B2SP_FPROF_STOP(0)
@@ -536,9 +544,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
                 ptx::for_each_row<32>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
-                    uint32_t pos, m;
-                    ptx::lds64_off<r * 8>(tab, pos, m);
-                    if (m & lane_bit) a.out[pos + __popc(m & lt_mask)] = vn[r];
+                    if (idx[FUSED ? 0 : r] >= 0) a.out[idx[FUSED ? 0 : r]] = vn[r];
                 });
                 B2SP_FPROF_STOP(2)
             }
