@@ -74,11 +74,19 @@ int b2sp_version(void);
 const char *b2sp_status_string(b2sp_status s);
 
 /*
- * Bytes of device workspace an op needs for the given sizes (an upper bound over all algo
- * values; always a multiple of 256, never 0).  `op` is one of B2SP_OP_*.  Unused sizes
+ * Bytes of device workspace an op needs for the given sizes: an upper bound over all algo values
+ * the sizes allow (always a multiple of 256, never 0).  `op` is one of B2SP_OP_*.  Unused sizes
  * (Kd for SPMM, N for SDDMM) may be 0.  Returns 0 on invalid arguments.
  */
 size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz);
+
+/*
+ * The same for one algo value: B2SP_ALGO_AUTO gives what the automatic choice will use (the row
+ * family's few bytes per row when it would not pick the dense-tile family), B2SP_ALGO_ROW /
+ * B2SP_ALGO_ROW_NAT the row family's size, B2SP_ALGO_TILE / B2SP_ALGO_TILE_PREPARED the dense-tile
+ * family's (0 if these sizes are outside that family).  Returns 0 on invalid arguments.
+ */
+size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz);
 
 /*
  * Pattern analysis shared by the dense-tile kernels of all three ops (work assignment and index

@@ -36,6 +36,8 @@ lib.b2sp_status_string.restype = ctypes.c_char_p
 lib.b2sp_status_string.argtypes = [_i]
 lib.b2sp_workspace_bytes.restype = _sz
 lib.b2sp_workspace_bytes.argtypes = [_i, _i, _i, _i, _i, _ll]
+lib.b2sp_workspace_bytes_algo.restype = _sz
+lib.b2sp_workspace_bytes_algo.argtypes = [_i, _i, _i, _i, _i, _i, _ll]
 lib.b2sp_spmm.restype = _i
 lib.b2sp_spmm.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp, _sz, _i, _vp]
 lib.b2sp_sddmm.restype = _i
@@ -100,16 +102,19 @@ def version() -> int:
     return int(lib.b2sp_version())
 
 
-def workspace_bytes(op: int, M: int, K: int, Kd: int, N: int, nnz: int) -> int:
-    return int(lib.b2sp_workspace_bytes(op, M, K, Kd, N, nnz))
+def workspace_bytes(op: int, M: int, K: int, Kd: int, N: int, nnz: int, algo=None) -> int:
+    """b2sp_workspace_bytes (upper bound over all algo values) or, with `algo`, b2sp_workspace_bytes_algo."""
+    if algo is None:
+        return int(lib.b2sp_workspace_bytes(op, M, K, Kd, N, nnz))
+    return int(lib.b2sp_workspace_bytes_algo(op, algo, M, K, Kd, N, nnz))
 
 
 _ws_cache = {}
 
 
-def _workspace(op, M, K, Kd, N, nnz, device, workspace):
-    need = workspace_bytes(op, M, K, Kd, N, nnz)
+def _workspace(op, M, K, Kd, N, nnz, device, workspace, algo=0):
     if workspace is None:
+        need = workspace_bytes(op, M, K, Kd, N, nnz, algo)
         key = (device.index, torch.cuda.current_stream(device).cuda_stream)
         workspace = _ws_cache.get(key)
         if workspace is None or workspace.numel() < need:
@@ -135,7 +140,7 @@ def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALG
     N = D.shape[1]
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=D.device)
-    ws, wsb = _workspace(OP_SPMM, M, K, 0, N, nnz, D.device, workspace)
+    ws, wsb = _workspace(OP_SPMM, M, K, 0, N, nnz, D.device, workspace, algo)
     _check(lib.b2sp_spmm(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D), _ld(D),
                          _ptr(out), _ld(out), _ptr(ws), wsb, algo, _stream()), "b2sp_spmm")
     return out
@@ -172,7 +177,7 @@ def sddmm(row_ptr, col_idx, s_values, A, B, out=None, workspace=None, algo=ALGO_
         raise ValueError("A must be [M, Kd]")
     if out is None:
         out = torch.empty(nnz, dtype=torch.float32, device=A.device)
-    ws, wsb = _workspace(OP_SDDMM, M, K, Kd, 0, nnz, A.device, workspace)
+    ws, wsb = _workspace(OP_SDDMM, M, K, Kd, 0, nnz, A.device, workspace, algo)
     _check(lib.b2sp_sddmm(M, K, Kd, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A), _ld(A),
                           _ptr(B), _ld(B), _ptr(out), _ptr(ws), wsb, algo, _stream()), "b2sp_sddmm")
     return out
@@ -190,7 +195,7 @@ def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=
         raise ValueError("A must be [M, Kd] and D [K, N]")
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=D.device)
-    ws, wsb = _workspace(OP_FUSEDMM, M, K, Kd, N, nnz, D.device, workspace)
+    ws, wsb = _workspace(OP_FUSEDMM, M, K, Kd, N, nnz, D.device, workspace, algo)
     _check(lib.b2sp_fusedmm(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
                             _ld(A), _ptr(B), _ld(B), _ptr(D), _ld(D), _ptr(out), _ld(out), _ptr(ws), wsb,
                             algo, _stream()), "b2sp_fusedmm")

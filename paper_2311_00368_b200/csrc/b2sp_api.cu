@@ -186,23 +186,34 @@ const char *b2sp_status_string(b2sp_status s)
     return "unknown status";
 }
 
+// Workspace of the dense-tile family for an op (0: these sizes are outside the family).
+static size_t tile_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz, size_t row_bytes)
+{
+    FusedPlan p = op == B2SP_OP_SPMM    ? plan_fused_tile(M, K, 0, N, nnz, row_bytes, true)
+                  : op == B2SP_OP_SDDMM ? plan_fused_tile(M, K, Kd, 0, nnz, row_bytes, false)
+                                        : plan_fused_tile(M, K, Kd, N, nnz, row_bytes, true);
+    return p.feasible ? p.bytes : 0;
+}
+
+static int tile_width(int op, int Kd, int N) { return op == B2SP_OP_SPMM ? N : op == B2SP_OP_SDDMM ? Kd : (Kd < N ? Kd : N); }
+
+size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz)
+{
+    if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return 0;
+    const size_t rows = row_workspace_bytes(M);
+    if (algo == B2SP_ALGO_ROW || algo == B2SP_ALGO_ROW_NAT) return rows;
+    const size_t tile = tile_workspace_bytes(op, M, K, Kd, N, nnz, rows);
+    if (algo == B2SP_ALGO_TILE || algo == B2SP_ALGO_TILE_PREPARED) return tile;
+    return tile > rows && tile_profitable(M, K, tile_width(op, Kd, N), nnz) ? tile : rows;
+}
+
 size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 {
     if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
-    size_t need = row_workspace_bytes(M);
-    if (op == B2SP_OP_SPMM && tile_profitable(M, K, N, nnz)) {
-        FusedPlan p = plan_fused_tile(M, K, 0, N, nnz, need, true);
-        if (p.feasible && p.bytes > need) need = p.bytes;
-    }
-    if (op == B2SP_OP_SDDMM && tile_profitable(M, K, Kd, nnz)) {
-        FusedPlan p = plan_fused_tile(M, K, Kd, 0, nnz, need, false);
-        if (p.feasible && p.bytes > need) need = p.bytes;
-    }
-    if (op == B2SP_OP_FUSEDMM && tile_profitable(M, K, Kd < N ? Kd : N, nnz)) {
-        FusedPlan p = plan_fused_tile(M, K, Kd, N, nnz, need, true);
-        if (p.feasible && p.bytes > need) need = p.bytes;
-    }
-    return need;
+    const size_t rows = row_workspace_bytes(M);
+    const size_t tile = tile_workspace_bytes(op, M, K, Kd, N, nnz, rows);
+    return tile > rows ? tile : rows;
 }
 
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
@@ -550,7 +561,7 @@ b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_pt
     float *d_v = a.upload(values, (size_t)nnz);
     float *d_D = a.upload(D, (size_t)K * N);
     float *d_O = static_cast<float *>(a.alloc(sizeof(float) * (size_t)M * N));
-    size_t wsb = b2sp_workspace_bytes(B2SP_OP_SPMM, M, K, 0, N, nnz);
+    size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_SPMM, B2SP_ALGO_AUTO, M, K, 0, N, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
     if (a.ok) {
@@ -575,7 +586,7 @@ b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_
     float *d_A = a.upload(A, (size_t)M * Kd);
     float *d_B = a.upload(B, (size_t)K * Kd);
     float *d_C = static_cast<float *>(a.alloc(sizeof(float) * (size_t)nnz));
-    size_t wsb = b2sp_workspace_bytes(B2SP_OP_SDDMM, M, K, Kd, 0, nnz);
+    size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_SDDMM, B2SP_ALGO_AUTO, M, K, Kd, 0, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
     if (a.ok) {
@@ -602,7 +613,7 @@ b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const 
     float *d_B = a.upload(B, (size_t)K * Kd);
     float *d_D = a.upload(D, (size_t)K * N);
     float *d_O = static_cast<float *>(a.alloc(sizeof(float) * (size_t)M * N));
-    size_t wsb = b2sp_workspace_bytes(B2SP_OP_FUSEDMM, M, K, Kd, N, nnz);
+    size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_FUSEDMM, B2SP_ALGO_AUTO, M, K, Kd, N, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
     if (a.ok) {

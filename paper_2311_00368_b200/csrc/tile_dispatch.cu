@@ -108,13 +108,16 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
 
 bool tile_profitable(int M, int K, int width, long long nnz)
 {
-    // Measured on B200: the dense-tile family pays a pattern pre-pass and does
-    // 3 / density times the useful flops on the tensor cores; it overtakes the row family from
-    // about 15% density, earlier on large matrices where the pre-pass amortises.
+    // Measured on B200: the dense-tile family costs a fixed ~35 us (pattern pre-pass, operand splits,
+    // tile prologue) plus ~1.3 us per million cells of S whatever the density, the row family ~22 us
+    // plus ~31 us per million stored entries (width 128).  The cross-over density is therefore about
+    // 4.5% on large matrices and rises as the matrix shrinks (16% at 2048^2, never at 1024^2); narrow
+    // operands favour the row family a little longer.
     if (M < 256 || K < 256 || width < 16 || nnz <= 0) return false;
     const double cells = (double)M * (double)K;
     const double density = (double)nnz / cells;
-    return density >= 0.15 || (density >= 0.08 && cells >= 48.0e6);
+    const double crossover = 0.045 + 0.5e6 / cells;
+    return density >= (width >= 64 ? crossover : 1.5 * crossover);
 }
 
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)

@@ -35,6 +35,18 @@ def test_library_exports_every_declared_symbol():
     n = lib.b2sp_workspace_bytes(2, 8192, 8192, 128, 512, 20_000_000)
     assert n >= 4 * 8192 and n % 256 == 0
     assert lib.b2sp_workspace_bytes(7, 1, 1, 1, 1, 1) == 0
+    # per-algo sizes: the row family needs a few bytes per row, the dense-tile family the window table
+    # and operand copies; AUTO reports what it would use; the general query bounds them all
+    lib.b2sp_workspace_bytes_algo.restype = ctypes.c_size_t
+    lib.b2sp_workspace_bytes_algo.argtypes = [ctypes.c_int] * 6 + [ctypes.c_longlong]
+    dims = (8192, 8192, 128, 512, 20_000_000)
+    row, tile, auto = (lib.b2sp_workspace_bytes_algo(2, a, *dims) for a in (1, 3, 0))
+    assert 4 * 8192 <= row < 1 << 20 and tile > 8 * 8192 * 256 and auto == tile == n
+    sparse = (8192, 8192, 128, 512, 100_000)     # 0.15% density: AUTO stays with the row family
+    assert lib.b2sp_workspace_bytes_algo(2, 0, *sparse) == lib.b2sp_workspace_bytes_algo(2, 1, *sparse)
+    assert lib.b2sp_workspace_bytes(2, *sparse) >= lib.b2sp_workspace_bytes_algo(2, 3, *sparse) > 0
+    assert lib.b2sp_workspace_bytes_algo(2, 3, 64, 64, 200, 64, 100) == 0   # Kd > 128: outside the tile family
+    assert lib.b2sp_workspace_bytes_algo(2, 9, *dims) == 0
 
 
 def test_argument_errors_need_no_gpu():
