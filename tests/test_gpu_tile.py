@@ -270,3 +270,28 @@ def test_prepared_pattern_is_shared_by_all_ops_and_stale_tables_are_detected(b):
     b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
     b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=1)
     run_all("after a row-family call")
+
+
+@pytest.mark.parametrize("ks", [1, 2, 3])
+def test_k_split_epilogues(b, ks, monkeypatch):
+    """One K split stores O, two splits add their tiles into a zero-filled O, more go through slabs
+    and the fixed-order sum: all three must give the same result, also for a ragged width, an output
+    whose rows are padded, and an output that held NaNs before the call; repeated calls are bit-equal."""
+    monkeypatch.setenv("B2SP_FORCE_KS", str(ks))
+    p = W.small_random(4100 + ks, 300, 1024, 0.2, 48, 100)
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_FUSEDMM, p)
+    ref_f, T_f = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)
+    ref_s, T_s = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+    for name, ref, T, call in (
+            ("fusedmm", ref_f, T_f, lambda o: b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=o, workspace=ws, algo=TILE)),
+            ("spmm", ref_s, T_s, lambda o: b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=o, workspace=ws, algo=TILE))):
+        padded = torch.full((p.M, p.N + 12), float("nan"), device="cuda")
+        out = padded[:, :p.N]                     # ld = N + 12
+        call(out)
+        assert b.device_status(ws) == 0
+        gate(out, ref, T, f"{name} tile, {ks} K split(s), padded rows")
+        assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
+        again = torch.full((p.M, p.N), float("nan"), device="cuda")
+        call(again)
+        assert torch.equal(again, out.contiguous()), f"{name}: two runs differ ({ks} K splits)"
