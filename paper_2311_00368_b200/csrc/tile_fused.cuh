@@ -1,6 +1,8 @@
-// Dense-tile FusedMM and SDDMM (tcgen05 / TMEM / TMA, 3xTF32) over the window table of S.
+// Dense-tile FusedMM, SDDMM and SPMM (tcgen05 / TMEM / TMA, 3xTF32) over the window table of S:
+// one kernel, three modes.
 //
-// One CTA owns 128 rows of S (= rows of A and O) and a range of 128-column blocks of S (4 windows).
+// One CTA owns 128 rows of S (= rows of A and O), a range of 128-column blocks of S (4 windows of 32
+// columns each) and, for FusedMM / SPMM, one 128-column tile of O.
 //   * A_tile (128 x Kd) is split into tf32 hi/lo once: A_hi lives in tensor memory for the CTA's
 //     life; A_lo lives in tensor memory too (SDDMM) or in shared memory (FusedMM, where TMEM is
 //     needed for O and P').
@@ -8,15 +10,18 @@
 //     in chunks of 32 k (hi + lo, 32 KB); N = 128 MMAs run the tensor pipe at full rate (a 128xNx8
 //     tf32 MMA costs max(N/2, 45.6) cycles, so 32-column GEMMs would waste two thirds of it).
 //   * Four processor warps (thread = row) read P window by window (32 columns) and multiply it by the
-//     window's stored values (0 where nothing is stored), which eight helper warps fetch with lane =
+//     window's stored values (0 where nothing is stored), which twelve helper warps fetch with lane =
 //     column (coalesced), densify and transpose through shared-memory slots.  The sampled C of the
-//     paper exists only in these registers.  Then
+//     paper (Alg. 3) exists only in these registers.  Then
 //       - FusedMM: split the result into hi/lo and write it back to TMEM as P' (two buffers); GEMM2
 //         O += P'_window * D_window (A = P' from TMEM, B = D rows by TMA, MN-major) accumulates O in TMEM;
-//       - SDDMM: write the stored entries to out_values (coalesced through shared memory).
+//       - SDDMM (Alg. 1): the processors hand their rows of P to the helpers through the slots; the
+//         helpers multiply by the stored values and write each row's entries as one contiguous run.
+//   * SPMM (Alg. 2) is the FusedMM pipeline with P' = the stored values themselves: no A, no B, no GEMM1.
 //
 // TMEM columns (512 allocated)
 //   FusedMM: O [0,128)  P [128,256)  P'0 hi/lo [256,288)/[288,320)  P'1 hi/lo [320,352)/[352,384)  A_hi [384,384+Kdp)
+//   SPMM:    O [0,128)  P' as for FusedMM
 //   SDDMM:   P0 [0,128) P1 [128,256) A_hi [256,256+Kdp)  A_lo [384,384+Kdp)
 #pragma once
 #include <cuda.h>
