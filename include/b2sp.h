@@ -89,6 +89,16 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz);
 size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz);
 
 /*
+ * Measurement aid with no counterpart in the paper: the FP32 FMA rate the current device sustains
+ * right now (8 independent register-only FMA chains per thread, 2048 threads on every SM, best of 10
+ * launches timed with CUDA events), in GFLOP/s, for the denominator of a roofline fraction.
+ * `iters` = chain length in units of 64 FMAs per thread (4096 takes about a millisecond);
+ * `scratch` = DEVICE pointer to at least one float (never written in practice); `gflops_host` =
+ * HOST pointer for the result.  Synchronises `stream`.  B2SP_ERR_INVALID_ARG / B2SP_ERR_CUDA.
+ */
+b2sp_status b2sp_probe_fp32_peak(int iters, float *scratch, double *gflops_host, void *stream);
+
+/*
  * Pattern analysis shared by the dense-tile kernels of all three ops (work assignment and index
  * staging: where the paper's kernels cut each row's ja array into blocks of VLC = 32 entries on the
  * fly, this library cuts each row into windows of 32 columns once).  Builds, in `workspace`, the

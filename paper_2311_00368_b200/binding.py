@@ -57,6 +57,8 @@ lib.b2sp_prepare_pattern.restype = _i
 lib.b2sp_prepare_pattern.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_validate_csr.restype = _i
 lib.b2sp_validate_csr.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
+lib.b2sp_probe_fp32_peak.restype = _i
+lib.b2sp_probe_fp32_peak.argtypes = [_i, _vp, ctypes.POINTER(ctypes.c_double), _vp]
 lib.b2sp_device_status.restype = _i
 lib.b2sp_device_status.argtypes = [_vp, _vp]
 lib.b2sp_last_algo.restype = _i
@@ -121,6 +123,14 @@ def _workspace(op, M, K, Kd, N, nnz, device, workspace, algo=0):
             workspace = torch.empty(max(need, 1 << 20), dtype=torch.uint8, device=device)
             _ws_cache[key] = workspace
     return workspace, workspace.numel()
+
+
+def probe_fp32_peak(iters: int = 4096, device=None) -> float:
+    """b2sp_probe_fp32_peak: sustained FP32 FMA rate of the current device in GFLOP/s (synchronises)."""
+    scratch = torch.zeros(1, dtype=torch.float32, device=device or "cuda")
+    out = ctypes.c_double(0.0)
+    _check(lib.b2sp_probe_fp32_peak(iters, _ptr(scratch), ctypes.byref(out), _stream()), "b2sp_probe_fp32_peak")
+    return float(out.value)
 
 
 def last_algo(op: int) -> int:
