@@ -64,6 +64,8 @@ def make_workload(name: str, rank: int = 0) -> W.Problem:
         return p
     if name.startswith("attn"):
         return W.attention_case(int(name[4:] or 0) + 8 * rank)
+    if name.startswith("grid_"):
+        return W.paper_grid_case(name, seed=replicas.instance_seed(5, rank))
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -227,6 +229,72 @@ def workload_config(p, name):
             "l2": "flushed between steps (256 MiB write, untimed)"}
 
 
+def run_grid(args):
+    """The paper's evaluation grid on one GPU: per case and op, the minimum of 20 warm calls (the paper's
+    protocol: minimum of 20 runs, operands cache-warm) through the stateless C-ABI entry points with
+    algo = AUTO, the fraction of the roofline, and the parity of the timed outputs against the oracle on a
+    bounded sample of rows (with the oracle's own rate on that sample: the cpu_baseline of the case)."""
+    import torch
+    from paper_2311_00368_b200 import binding as b
+    import oracle
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback")
+    device = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    hbm_gbs, sm_max_mhz, _ = peaks()
+    fp32_peak = SM_COUNT * FP32_LANES_PER_SM * 2 * sm_max_mhz / 1e3   # GFLOP/s
+    stream = torch.cuda.current_stream()
+    for name in W.paper_grid_names():
+        if args.grid_filter and args.grid_filter not in name:
+            continue
+        p = make_workload(name)
+        dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(device)
+        rp, ci, v, A, B, D = map(dev, (p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D))
+        O = torch.empty((p.M, p.N), dtype=torch.float32, device=device)
+        O2 = torch.empty_like(O)
+        C = torch.empty(p.nnz, dtype=torch.float32, device=device)
+        ws = torch.empty(max(b.workspace_bytes(op, p.M, p.K, p.Kd, p.N, p.nnz, 0) for op in range(3)),
+                         dtype=torch.uint8, device=device)
+        calls = {"sddmm": lambda: b.sddmm(rp, ci, v, A, B, out=C, workspace=ws, algo=0),
+                 "spmm": lambda: b.spmm(rp, ci, v, D, K=p.K, out=O2, workspace=ws, algo=0),
+                 "fusedmm": lambda: b.fusedmm(rp, ci, v, A, B, D, out=O, workspace=ws, algo=0)}
+        line = {"workload": name, "M": p.M, "K": p.K, "N": p.N, "nnz": p.nnz, "ops": {}}
+        for i, op in enumerate(("sddmm", "spmm", "fusedmm")):
+            for _ in range(3):
+                calls[op]()
+            ev = []
+            for _ in range(20):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                calls[op]()
+                e1.record(stream)
+                ev.append((e0, e1))
+            torch.cuda.synchronize()
+            ms = [x.elapsed_time(y) for x, y in ev]
+            fl = W.flops(op, p.nnz, p.Kd, p.N)
+            by = W.compulsory_bytes(op, p.M, p.K, p.nnz, p.Kd, p.N)
+            t_roof = max(fl / (fp32_peak * 1e9), by / (hbm_gbs * 1e9))
+            line["ops"][op] = {"ms_min": round(float(np.min(ms)), 4), "ms_median": round(float(np.median(ms)), 4),
+                               "gflops_at_min": round(fl / float(np.min(ms)) / 1e6, 1),
+                               "roofline_frac_at_min": round(t_roof / (float(np.min(ms)) * 1e-3), 4),
+                               "algo": b.ALGO_NAMES[b.last_algo({"spmm": 0, "sddmm": 1, "fusedmm": 2}[op])]}
+        rows = min(p.M, 64)
+        t0 = time.perf_counter()
+        par = parity_on_sample(p, rows, O2, C, O)
+        t = time.perf_counter() - t0
+        nnz_s = int(p.row_ptr[rows])
+        line["parity_ok"] = par["ok"]
+        line["parity_worst"] = max(x["worst_error_over_allowed"] for x in par["ops"].values())
+        line["cpu_baseline"] = {"value": round(sum(W.flops(op, nnz_s, p.Kd, p.N) for op in OPS) / t / 1e9, 2),
+                                "unit": "GFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": f"rows 0..{rows}, spmm+sddmm+fusedmm once"}
+        print(json.dumps(line), flush=True)
+        del rp, ci, v, A, B, D, O, O2, C, ws
+        torch.cuda.empty_cache()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -241,9 +309,14 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--min-warmup", type=int, default=3,
                     help="lower bound on warm-up steps (only profiler captures go below 3)")
+    ap.add_argument("--grid", action="store_true",
+                    help="run the paper's 72-case grid (uniform-random stand-ins), one JSON line per case")
+    ap.add_argument("--grid-filter", default="", help="only grid cases whose name contains this text")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.grid:
+        return run_grid(args)
 
     import torch
     from paper_2311_00368_b200 import binding as b  # raises if libb2sp.so is missing

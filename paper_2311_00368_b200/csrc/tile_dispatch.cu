@@ -57,20 +57,24 @@ bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-int pick_split(int base_tiles, int Wk)
+// K splits of a tile; `blocks` = 128-column blocks of S.
+int pick_split(int base_tiles, int blocks)
 {
     if (const char *e = getenv("B2SP_FORCE_KS")) {   // tuning aid
         int ks = atoi(e);
-        if (ks >= 1 && ks <= Wk) return ks;
+        if (ks >= 1 && ks <= blocks) return ks;
     }
     // One wave of long-lived CTAs beats several waves of short ones (each CTA pays a prologue, an
     // epilogue and a partial-output slab): take the largest split that still fits one wave, as long
     // as every split keeps a few pipeline steps.
-    if (base_tiles >= kSMs) return 1;
-    int ks = kSMs / base_tiles;
-    if (ks > Wk / 4) ks = Wk / 4;
-    if (ks > 32) ks = 32;
-    return ks < 1 ? 1 : ks;
+    int ks = 1;
+    if (base_tiles < kSMs) {
+        ks = kSMs / base_tiles;
+        if (ks > blocks / 4) ks = blocks / 4;
+        if (ks > 32) ks = 32;
+        if (ks < 1) ks = 1;
+    }
+    return ks;
 }
 
 }  // namespace
@@ -149,6 +153,8 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
         off = align_up(off + dbytes, 1024);
         p.off_part = off;
         if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * kFusedRows * (size_t)p.Np;
+        p.off_cnt = off;   // one arrival counter per output tile (more than one K split only)
+        if (p.KS > 1) off = align_up(off + sizeof(int) * (size_t)p.Mt * (size_t)p.Nt, 256);
     }
     p.bytes = align_up(off, 256);
     p.feasible = true;
@@ -207,7 +213,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     float *part = reinterpret_cast<float *>(ws + p.off_part);
 
     const bool fused = mode != kModeSddmm, spmm = mode == kModeSpmm;
-    const bool accumulate = fused && p.KS == 2;
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
     if (!spmm && (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
                   !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
@@ -227,9 +232,10 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     }
     {
         const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp}, jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np};
-        // Two K splits add their partial tiles straight into O (x + y does not depend on the order, so
-        // the result is still deterministic); more splits go through partial slabs and a fixed-order sum.
-        const ZeroJob z{accumulate ? out : nullptr, ldo, M, N};
+        // With several K splits the CTA that finishes an output tile last sums the splits' slabs: the
+        // per-tile arrival counters start at zero.
+        const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), p.Mt * p.Nt, 1, p.Mt * p.Nt}
+                                            : ZeroJob{nullptr, 0, 0, 0};
         if (spmm) launch_split(jd, nullptr, z, status, st);
         else if (fused) launch_split(jb, &jd, z, status, st);
         else launch_split(jb, nullptr, z, status, st);
@@ -240,12 +246,14 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     FusedTileArgs a;
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
-    a.flags = flags; a.status = status; a.accumulate = accumulate ? 1 : 0;
+    a.flags = flags; a.status = status;
+    a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
+    a.O = out; a.ldo = ldo;
     a.sig_want = PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx};
     a.sig_have = reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset);
     a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
-    else if (p.KS == 1 || accumulate) { a.out = out; a.ld_out = ldo; a.slab = 0; }
+    else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
     const int items = p.Mt * p.Nt * p.KS;
     b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
@@ -253,14 +261,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
                              : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
-    if (fused && p.KS > 1 && !accumulate) {
-        long long total = (long long)M * N;
-        long long want = (total + 255) / 256, cap = (long long)kSMs * 8;
-        reduce_partials_kernel<<<(unsigned)(want < cap ? want : cap), 256, 0, st>>>(part, p.KS, a.slab, p.Np, M, N, out,
-                                                                                    ldo, flags);
-        *launches += 1;
-        if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
-    }
     return B2SP_OK;
 }
 

@@ -61,17 +61,25 @@ constexpr int kFusedHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) 
 // away: every slot must always be filled by the same helper and drained by the same processor warp.
 static_assert(kFusedSlots % kFusedHelpers == 0 && kFusedSlots % 4 == 0, "slot ownership must be fixed");
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
+// The tensor core adds every MMA into its fp32 accumulator with truncation: a bias of about -2e-8 of
+// the running sum per MMA, which nothing cancels on same-sign data (measured: -3.0e-5 after the 1536
+// MMAs of 32 blocks, three times the 1e-5 gate).  So O is accumulated in tensor memory over at most
+// kFusedFlushBlocks blocks (192 MMAs, bias <= 4e-6), then added into the output in global memory with
+// round-to-nearest fp32 reductions and restarted from zero.
+constexpr int kFusedFlushBlocks = 4;
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
-    int accumulate;           // FusedMM / SPMM with two K splits: add the tile into `out` (zero-filled before the launch)
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
     const float *A;           // M x Kd
     long long lda;
-    float *out;               // FusedMM: O or partial slabs; SDDMM: out_values
+    float *out;               // FusedMM / SPMM: O (one K split) or the K splits' slabs; SDDMM: out_values
     long long ld_out, slab;
+    float *O;                 // FusedMM / SPMM with several K splits: the output the slabs are summed into ...
+    long long ldo;
+    int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
     int *flags;                // flags[0] != 0: the table cannot be used, the row kernels take over
     PatternSignature sig_want; // the arrays this call was given ...
     const PatternSignature *sig_have;   // ... and what the table in the workspace was built from
@@ -91,7 +99,8 @@ struct FusedCfg {
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
     static constexpr int RING = SPMM ? 5 : FUSED ? 3 : 5;
-    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedHelpers * 256 /*record tables*/ + kFusedSlots * 4096;
+    static constexpr int FLUSH_BYTES = FUSED ? 4 * 2048 : 0;   // 32 rows x 16 columns per processor warp (see the flush)
+    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedHelpers * 256 /*record tables*/ + kFusedSlots * 4096 + FLUSH_BYTES;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
@@ -130,8 +139,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     constexpr int NSLOT = kFusedSlots, NH = kFusedHelpers;
     auto sl_full = [&](int s) { return aux + 8u * (2 * RING + 9 + s); };
     auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 9 + 2 * NSLOT));
+    const uint32_t o_free = aux + 8u * (2 * RING + 9 + 2 * NSLOT);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 10 + 2 * NSLOT));
     const uint32_t helper_tabs = aux + 512, slots = aux + 512 + NH * 256;
+    const uint32_t flush_stage = slots + NSLOT * 4096;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int ks = blockIdx.x % a.KS;
@@ -151,6 +162,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::mbar_init(pp_free(b), 1);
         }
         ptx::mbar_init(o_full, 1);
+        ptx::mbar_init(o_free, 4);
         for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(sl_full(s), 1); ptx::mbar_init(sl_empty(s), 1); }
         ptx::fence_mbar_init();
     }
@@ -304,7 +316,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     // groups 512 B apart, +1 KB per K step of 8 rows
                     const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
                     const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, (b | w | k8) != 0);
+                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
                     ptx::mma_tf32_ts(tmem + Cfg::COL_O, ppl + k8 * 8, ddh, idesc2, 1);
                     ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddl, idesc2, 1);
                 }
@@ -320,12 +332,20 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             // process the last two windows of block b.
             if (!SPMM && nblk > 0 && !gemm1(0)) failed = true;
             for (int b = 0; b < nblk && !failed; ++b) {
+                // O restarts from zero every kFusedFlushBlocks blocks, once the processors have taken the
+                // previous partial sum out of tensor memory
+                if (FUSED && b > 0 && b % kFusedFlushBlocks == 0) {
+                    B2SP_FPROF_STOP(4)
+                    failed = !ptx::mbar_wait(o_free, (b / kFusedFlushBlocks - 1) & 1);
+                    B2SP_FPROF_STOP(5)
+                }
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !gemm2(b, w);
                 if (!SPMM && b + 1 < nblk && !failed) failed = !gemm1(b + 1);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !gemm2(b, w);
+                if (FUSED && !failed && (b % kFusedFlushBlocks == kFusedFlushBlocks - 1 || b == nblk - 1))
+                    ptx::mma_commit(o_full);
             }
             B2SP_FPROF_FLUSH(0)
-            if (FUSED && !failed) ptx::mma_commit(o_full);
         }
     } else if (warp >= 2 && warp < 6) {
         // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
@@ -333,7 +353,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // helper warp into a shared-memory slot), multiply them into P (or use them as they are for
         // SPMM), split to hi/lo and write P' to tensor memory.
         // SDDMM: per window, copy the row of P into a slot; a helper warp writes the stored entries.
-        const int grow = m0 + row;
         const int nwin = nblk * WPB;
         B2SP_FPROF_DECL
         B2SP_FPROF_START
@@ -403,6 +422,71 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(pp_full(ppb));
                 B2SP_FPROF_STOP(4)
+                // ---- flush: after every kFusedFlushBlocks-th block (and after the last block) the partial O
+                // leaves tensor memory: each thread adds its row into the output (or
+                // its K split's slab): the first partial sum is stored, the later ones are added with fp32
+                // reductions (round to nearest).  A given element is only ever touched by the same lane of this
+                // warp, in program order, so the sum is reproducible.
+                // The flush of a chunk of blocks is done one window late (after P' of the next chunk's first
+                // window is ready), so that the tensor core has work again the moment O is free.
+                const bool chunk_ended = w == 0 && blk > 0 && blk % kFusedFlushBlocks == 0;
+                if (chunk_ended || it == nwin - 1) {
+                    const int chunk = chunk_ended ? blk / kFusedFlushBlocks - 1 : blk / kFusedFlushBlocks;
+                    bool ok = ptx::mbar_wait(o_full, chunk & 1);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                    ptx::tc_fence_after_sync();
+                    // 16 columns at a time go through 2 KB of shared memory per warp, so that one reduction
+                    // instruction covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes
+                    // (16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3): conflict-free both ways).
+                    float *obase = a.out + (long long)ks * a.slab + (long long)(m0 + q * 32) * a.ld_out;
+                    const bool vec = (a.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;
+                    const int ncols = a.KS == 1 ? a.N : a.Nt * kFusedNT;   // slabs are padded to whole tiles
+                    const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
+                    const uint32_t stage = flush_stage + (uint32_t)q * 2048;
+#pragma unroll 1
+                    for (int c = 0; c < kFusedNT / 16; ++c) {
+                        uint32_t r[16];
+                        ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + c * 16, r);
+                        ptx::tmem_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
+                                         "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                        __syncwarp();
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int rr = t * 8 + (lane >> 2), pc = lane & 3;
+                            uint32_t x0, x1, x2, x3;
+                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+                                         : "r"(stage + (uint32_t)rr * 64 + (uint32_t)((pc ^ ((rr >> 1) & 3)) << 4)) : "memory");
+                            const int n = n0 + c * 16 + pc * 4;
+                            if (m0 + q * 32 + rr < nrows) {
+                                float *dst = obase + (long long)rr * a.ld_out + n;
+                                if (chunk == 0) {   // the first partial sum initialises the target
+                                    if (vec && n + 4 <= ncols) {
+                                        *reinterpret_cast<uint4 *>(dst) = make_uint4(x0, x1, x2, x3);
+                                    } else {
+                                        if (n < ncols) dst[0] = __uint_as_float(x0);
+                                        if (n + 1 < ncols) dst[1] = __uint_as_float(x1);
+                                        if (n + 2 < ncols) dst[2] = __uint_as_float(x2);
+                                        if (n + 3 < ncols) dst[3] = __uint_as_float(x3);
+                                    }
+                                } else if (vec && n + 4 <= ncols) {
+                                    ptx::red_add_v4(dst, x0, x1, x2, x3);
+                                } else {
+                                    if (n < ncols) atomicAdd(dst, __uint_as_float(x0));
+                                    if (n + 1 < ncols) atomicAdd(dst + 1, __uint_as_float(x1));
+                                    if (n + 2 < ncols) atomicAdd(dst + 2, __uint_as_float(x2));
+                                    if (n + 3 < ncols) atomicAdd(dst + 3, __uint_as_float(x3));
+                                }
+                            }
+                        }
+                        __syncwarp();
+                    }
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(o_free);
+                }
             } else {
                 const int pb = blk & 1;
                 if (w == 0) {
@@ -438,45 +522,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
         }
         B2SP_FPROF_FLUSH(8)
-        // ---------------- epilogue: O accumulator -> global ----------------
-        if (FUSED) {
-            {
-                bool ok = !failed && ptx::mbar_wait(o_full, 0);
-                failed = !__all_sync(0xffffffffu, ok);
-            }
-            if (!failed) {
-                ptx::tc_fence_after_sync();
-                float *orow = a.out + (long long)ks * a.slab + (long long)grow * a.ld_out;
-                const bool vec = (a.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;
-#pragma unroll 1
-                for (int c = 0; c < kFusedNT / 32; ++c) {
-                    uint32_t r[32];
-                    ptx::tmem_ld_32x32(tmem + lane_addr + Cfg::COL_O + c * 32, r);
-                    ptx::tmem_ld_wait();
-                    if (grow < a.M) {
-                        const int n = n0 + c * 32;
-                        if (a.accumulate) {
-                            if (vec && n + 32 <= a.N) {
-#pragma unroll
-                                for (int i = 0; i < 32; i += 4) ptx::red_add_v4(orow + n + i, r[i], r[i + 1], r[i + 2], r[i + 3]);
-                            } else {
-#pragma unroll
-                                for (int i = 0; i < 32; ++i)
-                                    if (n + i < a.N) atomicAdd(orow + n + i, __uint_as_float(r[i]));
-                            }
-                        } else if (vec && n + 32 <= a.N) {
-#pragma unroll
-                            for (int i = 0; i < 32; i += 4)
-                                *reinterpret_cast<uint4 *>(orow + n + i) = make_uint4(r[i], r[i + 1], r[i + 2], r[i + 3]);
-                        } else {
-#pragma unroll
-                            for (int i = 0; i < 32; ++i)
-                                if (n + i < a.N) orow[n + i] = __uint_as_float(r[i]);
-                        }
-                    }
-                }
-            }
-        }
     } else if ((warp & 3) != 1) {   // warp 0 and warps 6.. that do not share the MMA warp's scheduler
         // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
@@ -557,8 +602,39 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         B2SP_FPROF_FLUSH(16)
     }
     if (failed) atomicExch(a.status, 1);
+    if (FUSED && a.KS > 1) __threadfence();   // this CTA's slab is complete before its arrival is counted
     ptx::tc_fence_before_sync();
     __syncthreads();
+    if (FUSED && a.KS > 1) {
+        // The CTA that arrives last at its output tile's counter sums the K splits' slabs, always in
+        // the order of the splits, into O: no CTA waits for another and the result is reproducible.
+        int *last_flag = reinterpret_cast<int *>(smem_gen + (helper_tabs - smem_base));   // the record tables are idle now
+        if (threadIdx.x == 0) *last_flag = atomicAdd(a.tile_arrivals + tile, 1) == a.KS - 1;
+        __syncthreads();
+        if (*last_flag) {
+            __threadfence();
+            for (int e = threadIdx.x; e < kFusedRows * (kFusedNT / 4); e += kFusedThreads) {
+                const int r = e / (kFusedNT / 4), c = (e % (kFusedNT / 4)) * 4;
+                const int grow = m0 + r, n = n0 + c;
+                if (grow >= a.M || n >= a.N) continue;
+                const float *src = a.out + (long long)grow * a.ld_out + n;
+                float4 acc = __ldcg(reinterpret_cast<const float4 *>(src));
+                for (int k = 1; k < a.KS; ++k) {
+                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + (long long)k * a.slab));
+                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+                }
+                float *dst = a.O + (long long)grow * a.ldo + n;
+                if (n + 3 < a.N && (a.ldo & 3) == 0 && (reinterpret_cast<uintptr_t>(a.O) & 15) == 0) {
+                    *reinterpret_cast<float4 *>(dst) = acc;
+                } else {
+                    dst[0] = acc.x;
+                    if (n + 1 < a.N) dst[1] = acc.y;
+                    if (n + 2 < a.N) dst[2] = acc.z;
+                    if (n + 3 < a.N) dst[3] = acc.w;
+                }
+            }
+        }
+    }
     if (warp == 1) {
         __syncwarp();
         ptx::tmem_dealloc(tmem, 512);

@@ -9,7 +9,6 @@
 //   tile_masks_kernel      per row and 32-column window: first CSR position + occupancy bit mask
 //                          (needs strictly increasing columns in a row; sets a flag otherwise)
 //   split_dense_kernel     dense fp32 operands -> zero-padded (hi, lo) tf32 copies
-//   reduce_partials_kernel sums the K splits in fixed order
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -152,8 +151,8 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // (rows_p >= rows, cols_p >= cols, cols_p % 32 == 0).  One 32-float group of a row is one
 // 128-byte swizzle row for TMA, and the whole thing is a plain packed 3-D tensor.
 // One launch splits up to two operands (blockIdx.y picks the job) and, being the first kernel of
-// every tile op, also clears the workspace's device status word and, when asked to, zero-fills the
-// output matrix (the last blockIdx.y) for tile kernels that add their K-split partial sums into it.
+// every tile op, also clears the workspace's device status word and, when asked to, zero-fills an
+// array (the last blockIdx.y): the per-tile arrival counters of a FusedMM / SPMM with several K splits.
 struct SplitJob {
     const float *X;
     long long ld;
@@ -165,7 +164,8 @@ struct SplitJob {
 struct ZeroJob {
     float *out;      // NULL: nothing to clear
     long long ld;
-    int rows, cols;
+    long long rows;
+    int cols;
 };
 
 __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status)
@@ -173,9 +173,13 @@ __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob 
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
     if ((int)blockIdx.y == njobs) {   // zero-fill job
         const long long total = (long long)z.rows * z.cols;
-        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-             i += (long long)gridDim.x * blockDim.x)
-            z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
+        const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
+        if (z.ld == z.cols && (total & 3) == 0 && (reinterpret_cast<uintptr_t>(z.out) & 15) == 0) {
+            for (long long i = t0; i < total / 4; i += step)
+                reinterpret_cast<float4 *>(z.out)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            for (long long i = t0; i < total; i += step) z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
+        }
         return;
     }
     const SplitJob j = blockIdx.y ? j1 : j0;
@@ -204,23 +208,6 @@ __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob 
         }
         reinterpret_cast<uint4 *>(j.hi)[g] = make_uint4(h[0], h[1], h[2], h[3]);
         reinterpret_cast<uint4 *>(j.lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
-    }
-}
-
-// ---- K-split reduction ------------------------------------------------------------------------------
-__global__ void reduce_partials_kernel(const float *__restrict__ part, int KS, long long slab, int ldp,
-                                       int M, int N, float *__restrict__ O, long long ldo,
-                                       const int *__restrict__ flags)
-{
-    if (flags[kFlagUnsorted] != 0) return;
-    const long long total = (long long)M * N;
-    for (long long e = (long long)blockIdx.x * blockDim.x + threadIdx.x; e < total;
-         e += (long long)gridDim.x * blockDim.x) {
-        int i = (int)(e / N), n = (int)(e % N);
-        const float *p = part + (long long)i * ldp + n;
-        float acc = p[0];
-        for (int s = 1; s < KS; ++s) acc += p[(long long)s * slab];
-        O[(long long)i * ldo + n] = acc;
     }
 }
 

@@ -231,6 +231,31 @@ def sweep_case(density: float, N: int, seed: int = 4, M: int = 8192, K: int = 81
     return _finish(f"sweep_d{int(round(density * 100))}_n{N}", rng, M, K, rp, ci, False, Kd, N)
 
 
+# The paper's evaluation grid (the x axis of its benchmark figures): 12 shapes x N in {32, 128} x
+# sparsity in {70, 80, 90}%.  Its matrices (a public collection) are not available here; these are
+# uniform-random stand-ins of the same shape and density.  "1k" is read as 1024.
+PAPER_GRID_SHAPES = [(1, 1), (3, 1), (4, 1), (2, 2), (6, 2), (8, 2), (4, 4), (12, 4), (16, 4), (8, 8), (24, 8), (32, 8)]
+PAPER_GRID_WIDTHS = (32, 128)
+PAPER_GRID_SPARSITIES = (70, 80, 90)
+
+
+def paper_grid_names() -> list:
+    """Names of the 72 grid cases, in the order of the paper's figures (N = 32 first)."""
+    return [f"grid_{m}k_{k}k_{n}_{sp}" for n in PAPER_GRID_WIDTHS for (m, k) in PAPER_GRID_SHAPES
+            for sp in PAPER_GRID_SPARSITIES]
+
+
+def paper_grid_case(name: str, seed: int = 5) -> Problem:
+    """`grid_<M>k_<K>k_<N>_<sparsity%>`: S is M x K uniform-random at density 1 - sparsity with values
+    U(-1,1); A is M x N, B and D are K x N (the paper uses one width N for the dot product and for
+    the output).  The generator is seeded by (seed, M, K, N, sparsity)."""
+    _, m, k, n, sp = name.split("_")
+    M, K, N, sp = int(m[:-1]) * 1024, int(k[:-1]) * 1024, int(n), int(sp)
+    rng = np.random.default_rng([seed, M, K, N, sp])
+    rp, ci = pattern_uniform(rng, M, K, 1.0 - sp / 100.0)
+    return _finish(name, rng, M, K, rp, ci, False, N, N)
+
+
 def small_random(seed: int, M: int, K: int, density: float, Kd: int, N: int,
                  unit_values: bool = False, kind: str = "uniform") -> Problem:
     """Arbitrary small instance for parity and edge-case tests."""

@@ -295,3 +295,18 @@ def test_k_split_epilogues(b, ks, monkeypatch):
         again = torch.full((p.M, p.N), float("nan"), device="cuda")
         call(again)
         assert torch.equal(again, out.contiguous()), f"{name}: two runs differ ({ks} K splits)"
+
+
+def test_tile_accuracy_on_same_sign_data_and_long_rows(b):
+    """The tensor core adds into its fp32 accumulator with truncation, a bias that grows with the
+    number of MMAs per output; on same-sign data nothing cancels it.  The planner caps the columns of
+    S per K split, so the error must stay well inside the gate for K = 32768 as for K = 8192."""
+    for M, K in ((256, 8192), (128, 32768)):
+        p = W.small_random(4200 + K, M, K, 0.3, 64, 128)
+        rng = np.random.default_rng(5)
+        p.values = rng.uniform(0.5, 1.5, p.nnz).astype(np.float32)
+        p.A = rng.uniform(0.5, 1.5, p.A.shape).astype(np.float32)
+        p.B = rng.uniform(0.5, 1.5, p.B.shape).astype(np.float32)
+        p.D = rng.uniform(0.5, 1.5, p.D.shape).astype(np.float32)
+        assert spmm_tile_check(b, p) < 0.6
+        assert fused_tile_check(b, p) < 0.6
