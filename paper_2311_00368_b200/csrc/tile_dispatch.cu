@@ -58,6 +58,21 @@ bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, 
 }
 
 // K splits of a tile; `blocks` = 128-column blocks of S.
+// fp32 matrix [rows][cols] with row stride `ld` elements, as the target of the tile kernel's flush:
+// boxes of 16 columns x 32 rows, 64-byte swizzle.  Needs a 16-byte aligned base and row stride.
+bool make_output_map(CUtensorMap *tm, float *base, long long rows, int cols, long long ld)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {16, 32};
+    cuuint32_t estr[2] = {1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+               CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 int pick_split(int base_tiles, int blocks)
 {
     if (const char *e = getenv("B2SP_FORCE_KS")) {   // tuning aid
@@ -165,23 +180,25 @@ namespace {
 
 template <int KDP, int MODE>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
-                              const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
+                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
+                              cudaStream_t st)
 {
     using Cfg = FusedCfg<KDP, MODE>;
     auto kern = fused_tile_kernel<KDP, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
-    kern<<<items, kFusedThreads, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, a);
+    kern<<<items, kFusedThreads, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, out, a);
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 
 template <int MODE>
 b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
-                             const CUtensorMap &dl, const FusedTileArgs &a, int items, cudaStream_t st)
+                             const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
+                             cudaStream_t st)
 {
-    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE>(bh, bl, dh, dl, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, MODE>(bh, bl, dh, dl, a, items, st);
-    return launch_fused_tile<128, MODE>(bh, bl, dh, dl, a, items, st);
+    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE>(bh, bl, dh, dl, out, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, MODE>(bh, bl, dh, dl, out, a, items, st);
+    return launch_fused_tile<128, MODE>(bh, bl, dh, dl, out, a, items, st);
 }
 
 // Splits one or two dense operands (job 1 optional), clears the device status word and optionally
@@ -255,10 +272,23 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
+    // The flush goes through TMA when the target's rows are 16-byte aligned (slabs always are).
+    CUtensorMap tm_out = tm_dh;
+    a.out_tma = 0;
+    a.slab_rows = p.Mt * kFusedRows;
+    if (fused) {
+        const bool aligned = (reinterpret_cast<uintptr_t>(a.out) & 15) == 0 && (a.ld_out & 3) == 0;
+        if (aligned) {
+            const long long rows = p.KS == 1 ? M : (long long)p.KS * a.slab_rows;
+            const int cols = p.KS == 1 ? N : p.Np;
+            if (!make_output_map(&tm_out, a.out, rows, cols, a.ld_out)) return B2SP_ERR_CUDA;
+            a.out_tma = 1;
+        }
+    }
     const int items = p.Mt * p.Nt * p.KS;
-    b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
-                     : fused ? launch_fused_kdp<kModeFused>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st)
-                             : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, a, items, st);
+    b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
+                     : fused ? launch_fused_kdp<kModeFused>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
+                             : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
     return B2SP_OK;

@@ -21,7 +21,7 @@
 //
 // TMEM columns (512 allocated)
 //   FusedMM: O [0,128)  P [128,256)  P'0 hi/lo [256,288)/[288,320)  P'1 hi/lo [320,352)/[352,384)  A_hi [384,384+Kdp)
-//   SPMM:    O [0,128)  P' as for FusedMM
+//   SPMM:    O0 [0,128)  O1 [128,256)  P' as for FusedMM
 //   SDDMM:   P0 [0,128) P1 [128,256) A_hi [256,256+Kdp)  A_lo [384,384+Kdp)
 #pragma once
 #include <cuda.h>
@@ -55,11 +55,7 @@ constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 // issue slots for the MMA warp.
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
-constexpr int kFusedSlots = 12;     // shared-memory slots (4 KB) between helpers and processors: 3 windows deep
-constexpr int kFusedHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) gets no helper: its issue slots feed the tensor pipe
-// A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one phase
-// away: every slot must always be filled by the same helper and drained by the same processor warp.
-static_assert(kFusedSlots % kFusedHelpers == 0 && kFusedSlots % 4 == 0, "slot ownership must be fixed");
+constexpr int kFusedMaxHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) gets no helper: its issue slots feed the tensor pipe
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 // The tensor core adds every MMA into its fp32 accumulator with truncation: a bias of about -2e-8 of
 // the running sum per MMA, which nothing cancels on same-sign data (measured: -3.0e-5 after the 1536
@@ -77,6 +73,8 @@ struct FusedTileArgs {
     long long lda;
     float *out;               // FusedMM / SPMM: O (one K split) or the K splits' slabs; SDDMM: out_values
     long long ld_out, slab;
+    int out_tma;              // the flush may use TMA on `out` (tm_out covers it; 16-byte aligned rows)
+    int slab_rows;            // rows of one slab (TMA y coordinate of slab ks = ks * slab_rows)
     float *O;                 // FusedMM / SPMM with several K splits: the output the slabs are summed into ...
     long long ldo;
     int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
@@ -98,11 +96,21 @@ struct FusedCfg {
     static constexpr int NCH_B = SPMM ? 0 : KDP / 32;          // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
-    static constexpr int RING = SPMM ? 5 : FUSED ? 3 : 5;
-    static constexpr int FLUSH_BYTES = FUSED ? 4 * 2048 : 0;   // 32 rows x 16 columns per processor warp (see the flush)
-    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedHelpers * 256 /*record tables*/ + kFusedSlots * 4096 + FLUSH_BYTES;
+    static constexpr int RING = SPMM ? 4 : FUSED ? 3 : 5;
+    // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
+    // 4 KB slots (two windows deep).  SPMM and SDDMM are bound by the helpers: twelve, twelve slots.
+    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : kFusedMaxHelpers;
+    static constexpr int SLOTS = HELPERS;
+    // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one
+    // phase away: every slot is always filled by the same helper and drained by the same processor warp.
+    static_assert(SLOTS % HELPERS == 0 && SLOTS % 4 == 0, "slot ownership must be fixed");
+    static constexpr int FLUSH_BYTES = FUSED ? 4 * 4096 : 0;   // per processor warp: two buffers of 32 rows x 16 columns
+    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * 4096 + FLUSH_BYTES;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
+    // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
+    // chunk of blocks while the previous partial sum is flushed.
+    static constexpr int NOB = SPMM ? 2 : 1;
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
@@ -111,7 +119,7 @@ template <int KDP, int MODE>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
-                  const FusedTileArgs a)
+                  const __grid_constant__ CUtensorMap tm_out, const FusedTileArgs a)
 {
     using Cfg = FusedCfg<KDP, MODE>;
     constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
@@ -135,13 +143,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     auto p_free = [&](int b) { return aux + 8u * (2 * RING + 2 + b); };
     auto pp_full = [&](int b) { return aux + 8u * (2 * RING + 4 + b); };
     auto pp_free = [&](int b) { return aux + 8u * (2 * RING + 6 + b); };
-    const uint32_t o_full = aux + 8u * (2 * RING + 8);
-    constexpr int NSLOT = kFusedSlots, NH = kFusedHelpers;
+    constexpr int NSLOT = Cfg::SLOTS, NH = Cfg::HELPERS, NOB = Cfg::NOB;
+    auto o_full = [&](int b) { return aux + 8u * (b == 0 ? 2 * RING + 8 : 2 * RING + 11 + 2 * NSLOT); };
     auto sl_full = [&](int s) { return aux + 8u * (2 * RING + 9 + s); };
     auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
-    const uint32_t o_free = aux + 8u * (2 * RING + 9 + 2 * NSLOT);
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 10 + 2 * NSLOT));
-    const uint32_t helper_tabs = aux + 512, slots = aux + 512 + NH * 256;
+    auto o_free = [&](int b) { return aux + 8u * (2 * RING + 9 + 2 * NSLOT + b); };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 12 + 2 * NSLOT));
+    const uint32_t helper_tabs = aux + 512, slots = aux + 512 + kFusedMaxHelpers * 256;
     const uint32_t flush_stage = slots + NSLOT * 4096;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -161,8 +169,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             ptx::mbar_init(pp_full(b), 4);
             ptx::mbar_init(pp_free(b), 1);
         }
-        ptx::mbar_init(o_full, 1);
-        ptx::mbar_init(o_free, 4);
+        for (int b = 0; b < NOB; ++b) { ptx::mbar_init(o_full(b), 1); ptx::mbar_init(o_free(b), 4); }
         for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(sl_full(s), 1); ptx::mbar_init(sl_empty(s), 1); }
         ptx::fence_mbar_init();
     }
@@ -310,15 +317,16 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::tc_fence_after_sync();
                 const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
                 const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
+                const uint32_t oacc = tmem + Cfg::COL_O + ((b / kFusedFlushBlocks) % NOB) * kFusedNT;
 #pragma unroll
                 for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
                     // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
                     // groups 512 B apart, +1 KB per K step of 8 rows
                     const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
                     const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
-                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, ppl + k8 * 8, ddh, idesc2, 1);
-                    ptx::mma_tf32_ts(tmem + Cfg::COL_O, pph + k8 * 8, ddl, idesc2, 1);
+                    ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
+                    ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
+                    ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
                 }
                 ptx::mma_commit(pp_free(ppb));
                 ptx::mma_commit(empty(s));
@@ -334,16 +342,17 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             for (int b = 0; b < nblk && !failed; ++b) {
                 // O restarts from zero every kFusedFlushBlocks blocks, once the processors have taken the
                 // previous partial sum out of tensor memory
-                if (FUSED && b > 0 && b % kFusedFlushBlocks == 0) {
+                if (FUSED && b % kFusedFlushBlocks == 0 && b / kFusedFlushBlocks >= NOB) {
+                    const int ch = b / kFusedFlushBlocks;   // chunk ch reuses the accumulator of chunk ch - NOB
                     B2SP_FPROF_STOP(4)
-                    failed = !ptx::mbar_wait(o_free, (b / kFusedFlushBlocks - 1) & 1);
+                    failed = !ptx::mbar_wait(o_free(ch % NOB), (ch / NOB - 1) & 1);
                     B2SP_FPROF_STOP(5)
                 }
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !gemm2(b, w);
                 if (!SPMM && b + 1 < nblk && !failed) failed = !gemm1(b + 1);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !gemm2(b, w);
                 if (FUSED && !failed && (b % kFusedFlushBlocks == kFusedFlushBlocks - 1 || b == nblk - 1))
-                    ptx::mma_commit(o_full);
+                    ptx::mma_commit(o_full((b / kFusedFlushBlocks) % NOB));
             }
             B2SP_FPROF_FLUSH(0)
         }
@@ -432,60 +441,85 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 const bool chunk_ended = w == 0 && blk > 0 && blk % kFusedFlushBlocks == 0;
                 if (chunk_ended || it == nwin - 1) {
                     const int chunk = chunk_ended ? blk / kFusedFlushBlocks - 1 : blk / kFusedFlushBlocks;
-                    bool ok = ptx::mbar_wait(o_full, chunk & 1);
+                    const int ob = chunk % NOB;
+                    bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
-                    // 16 columns at a time go through 2 KB of shared memory per warp, so that one reduction
-                    // instruction covers 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes
-                    // (16-byte piece j of row r sits at piece j ^ ((r >> 1) & 3): conflict-free both ways).
-                    float *obase = a.out + (long long)ks * a.slab + (long long)(m0 + q * 32) * a.ld_out;
-                    const bool vec = (a.ld_out & 3) == 0 && (reinterpret_cast<uintptr_t>(a.out) & 15) == 0;
-                    const int ncols = a.KS == 1 ? a.N : a.Nt * kFusedNT;   // slabs are padded to whole tiles
-                    const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
-                    const uint32_t stage = flush_stage + (uint32_t)q * 2048;
-#pragma unroll 1
-                    for (int c = 0; c < kFusedNT / 16; ++c) {
-                        uint32_t r[16];
-                        ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + c * 16, r);
-                        ptx::tmem_ld_wait();
-#pragma unroll
-                        for (int j = 0; j < 4; ++j)
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
-                                         "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                    // 16 columns at a time go through shared memory (per warp two buffers of 32 rows x 16
+                    // columns, 64-byte swizzle: 16-byte piece j of row r at piece j ^ ((r >> 1) & 3)).  From
+                    // there one TMA store (first partial sum) or fp32 add-reduction per buffer moves whole
+                    // 64-byte row pieces; rows and columns outside the output are clipped by TMA.  O is free
+                    // for the tensor core again as soon as its last columns have been read.
+                    const uint32_t stage = flush_stage + (uint32_t)q * 4096;
+                    if (a.out_tma) {
+                        if (lane == 0) ptx::bulk_wait<0>();   // the previous flush's reductions are complete (order of the sums)
                         __syncwarp();
+                        const int y = ks * a.slab_rows + m0 + q * 32;
+#pragma unroll 1
+                        for (int c = 0; c < kFusedNT / 16; ++c) {
+                            const uint32_t buf = stage + (uint32_t)(c & 1) * 2048;
+                            if (c >= 2) {
+                                if (lane == 0) ptx::bulk_wait_read<1>();   // the buffer's previous contents have been read
+                                __syncwarp();
+                            }
+                            uint32_t r[16];
+                            ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                            ptx::tmem_ld_wait();
+                            if (c == kFusedNT / 16 - 1) {
+                                ptx::tc_fence_before_sync();
+                                __syncwarp();
+                                if (lane == 0) ptx::mbar_arrive(o_free(ob));
+                            }
 #pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int rr = t * 8 + (lane >> 2), pc = lane & 3;
-                            uint32_t x0, x1, x2, x3;
-                            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
-                                         : "r"(stage + (uint32_t)rr * 64 + (uint32_t)((pc ^ ((rr >> 1) & 3)) << 4)) : "memory");
-                            const int n = n0 + c * 16 + pc * 4;
-                            if (m0 + q * 32 + rr < nrows) {
-                                float *dst = obase + (long long)rr * a.ld_out + n;
-                                if (chunk == 0) {   // the first partial sum initialises the target
-                                    if (vec && n + 4 <= ncols) {
-                                        *reinterpret_cast<uint4 *>(dst) = make_uint4(x0, x1, x2, x3);
-                                    } else {
-                                        if (n < ncols) dst[0] = __uint_as_float(x0);
-                                        if (n + 1 < ncols) dst[1] = __uint_as_float(x1);
-                                        if (n + 2 < ncols) dst[2] = __uint_as_float(x2);
-                                        if (n + 3 < ncols) dst[3] = __uint_as_float(x3);
-                                    }
-                                } else if (vec && n + 4 <= ncols) {
-                                    ptx::red_add_v4(dst, x0, x1, x2, x3);
-                                } else {
-                                    if (n < ncols) atomicAdd(dst, __uint_as_float(x0));
-                                    if (n + 1 < ncols) atomicAdd(dst + 1, __uint_as_float(x1));
-                                    if (n + 2 < ncols) atomicAdd(dst + 2, __uint_as_float(x2));
-                                    if (n + 3 < ncols) atomicAdd(dst + 3, __uint_as_float(x3));
-                                }
+                            for (int j = 0; j < 4; ++j)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
+                                             "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                if (chunk == 0) ptx::tma_store_2d(&tm_out, buf, n0 + c * 16, y);
+                                else ptx::tma_reduce_add_2d(&tm_out, buf, n0 + c * 16, y);
+                                ptx::bulk_commit();
                             }
                         }
+                    } else {
+                        // output rows that are not 16-byte aligned: the same through plain stores / atomics
+                        float *obase = a.out + (long long)ks * a.slab + (long long)(m0 + q * 32) * a.ld_out;
+                        const int ncols = a.KS == 1 ? a.N : a.Nt * kFusedNT;   // slabs are padded to whole tiles
+                        const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
+#pragma unroll 1
+                        for (int c = 0; c < kFusedNT / 16; ++c) {
+                            uint32_t r[16];
+                            ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                            ptx::tmem_ld_wait();
+#pragma unroll
+                            for (int j = 0; j < 4; ++j)
+                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
+                                             "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                            __syncwarp();
+#pragma unroll
+                            for (int t = 0; t < 4; ++t) {
+                                const int rr = t * 8 + (lane >> 2), pc = lane & 3;
+                                uint32_t x[4];
+                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                                             : "r"(stage + (uint32_t)rr * 64 + (uint32_t)((pc ^ ((rr >> 1) & 3)) << 4)) : "memory");
+                                const int n = n0 + c * 16 + pc * 4;
+                                if (m0 + q * 32 + rr < nrows) {
+                                    float *dst = obase + (long long)rr * a.ld_out + n;
+#pragma unroll
+                                    for (int e = 0; e < 4; ++e) {
+                                        if (n + e >= ncols) continue;
+                                        if (chunk == 0) dst[e] = __uint_as_float(x[e]);   // the first partial sum initialises the target
+                                        else atomicAdd(dst + e, __uint_as_float(x[e]));
+                                    }
+                                }
+                            }
+                            __syncwarp();
+                        }
+                        ptx::tc_fence_before_sync();
                         __syncwarp();
+                        if (lane == 0) ptx::mbar_arrive(o_free(ob));
                     }
-                    ptx::tc_fence_before_sync();
-                    __syncwarp();
-                    if (lane == 0) ptx::mbar_arrive(o_free);
                 }
             } else {
                 const int pb = blk & 1;
@@ -522,7 +556,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
         }
         B2SP_FPROF_FLUSH(8)
-    } else if ((warp & 3) != 1) {   // warp 0 and warps 6.. that do not share the MMA warp's scheduler
+    } else if ((warp & 3) != 1 && (warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2)) < NH) {
+        // warp 0 and warps 6.. that do not share the MMA warp's scheduler, as many as this mode uses
         // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
         // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
@@ -602,6 +637,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         B2SP_FPROF_FLUSH(16)
     }
     if (failed) atomicExch(a.status, 1);
+    if (FUSED && warp >= 2 && warp < 6 && lane == 0) {   // this warp's TMA stores / reductions have been performed
+        ptx::bulk_wait<0>();
+        ptx::fence_proxy_async_all();
+    }
     if (FUSED && a.KS > 1) __threadfence();   // this CTA's slab is complete before its arrival is counted
     ptx::tc_fence_before_sync();
     __syncthreads();

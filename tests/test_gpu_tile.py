@@ -286,12 +286,13 @@ def test_k_split_epilogues(b, ks, monkeypatch):
     for name, ref, T, call in (
             ("fusedmm", ref_f, T_f, lambda o: b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=o, workspace=ws, algo=TILE)),
             ("spmm", ref_s, T_s, lambda o: b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=o, workspace=ws, algo=TILE))):
-        padded = torch.full((p.M, p.N + 12), float("nan"), device="cuda")
-        out = padded[:, :p.N]                     # ld = N + 12
-        call(out)
-        assert b.device_status(ws) == 0
-        gate(out, ref, T, f"{name} tile, {ks} K split(s), padded rows")
-        assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
+        for pad in (12, 13):                          # ld = 112 (rows 16-byte aligned: TMA flush) and 113 (plain stores / atomics)
+            padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
+            out = padded[:, :p.N]
+            call(out)
+            assert b.device_status(ws) == 0
+            gate(out, ref, T, f"{name} tile, {ks} K split(s), rows padded by {pad}")
+            assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
         again = torch.full((p.M, p.N), float("nan"), device="cuda")
         call(again)
         assert torch.equal(again, out.contiguous()), f"{name}: two runs differ ({ks} K splits)"
