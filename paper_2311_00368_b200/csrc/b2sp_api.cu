@@ -205,7 +205,7 @@ size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, 
     if (algo == B2SP_ALGO_ROW || algo == B2SP_ALGO_ROW_NAT) return rows;
     const size_t tile = tile_workspace_bytes(op, M, K, Kd, N, nnz, rows);
     if (algo == B2SP_ALGO_TILE || algo == B2SP_ALGO_TILE_PREPARED) return tile;
-    return tile > rows && tile_profitable(M, K, tile_width(op, Kd, N), nnz) ? tile : rows;
+    return tile > rows && tile_profitable(op, M, K, tile_width(op, Kd, N), nnz) ? tile : rows;
 }
 
 size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
@@ -218,6 +218,10 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
+
+// The row family under AUTO: the binning pass (two small launches, ~10 us) orders the rows longest
+// first, which only pays when the CTAs of the row kernel need several waves on the GPU.
+static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_ALGO_ROW; }
 
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
@@ -256,9 +260,9 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
     FusedPlan plan;   // SPMM runs through the FusedMM tile pipeline with P' = the stored values (Kd = 0)
-    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, N, nnz)))
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(B2SP_OP_SPMM, M, K, N, nnz)))
         plan = plan_fused_tile(M, K, 0, N, nnz, row_bytes, true);
-    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    int use = algo == B2SP_ALGO_AUTO ? auto_row_algo(M) : algo;
     if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
     else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_SPMM] = use;
@@ -335,9 +339,9 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
     b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
     FusedPlan plan;
-    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, Kd, nnz)))
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(B2SP_OP_SDDMM, M, K, Kd, nnz)))
         plan = plan_fused_tile(M, K, Kd, 0, nnz, row_bytes, false);
-    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    int use = algo == B2SP_ALGO_AUTO ? auto_row_algo(M) : algo;
     if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
     else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_SDDMM] = use;
@@ -416,9 +420,9 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
     if (rc != B2SP_OK) return rc;
     FusedPlan plan;
-    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(M, K, Kd < N ? Kd : N, nnz)))
+    if (algo == B2SP_ALGO_TILE || (algo == B2SP_ALGO_AUTO && tile_profitable(B2SP_OP_FUSEDMM, M, K, Kd < N ? Kd : N, nnz)))
         plan = plan_fused_tile(M, K, Kd, N, nnz, row_bytes, true);
-    int use = algo == B2SP_ALGO_AUTO ? B2SP_ALGO_ROW : algo;
+    int use = algo == B2SP_ALGO_AUTO ? auto_row_algo(M) : algo;
     if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
     else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
     g_last_algo[B2SP_OP_FUSEDMM] = use;

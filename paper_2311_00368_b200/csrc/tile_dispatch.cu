@@ -125,18 +125,21 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 
-bool tile_profitable(int M, int K, int width, long long nnz)
+bool tile_profitable(int op, int M, int K, int width, long long nnz)
 {
     // Measured on B200: the dense-tile family costs a fixed ~35 us (pattern pre-pass, operand splits,
     // tile prologue) plus ~1.3 us per million cells of S whatever the density, the row family ~22 us
     // plus ~31 us per million stored entries (width 128).  The cross-over density is therefore about
-    // 4.5% on large matrices and rises as the matrix shrinks (16% at 2048^2, never at 1024^2); narrow
-    // operands favour the row family a little longer.
+    // 4.5% on large matrices and rises as the matrix shrinks (16% at 2048^2, never at 1024^2).
+    // Operands narrower than 64 use a quarter of the 128-wide tiles while the row kernels lose
+    // nothing (sub-warps share a row): measured at width 32 on 1k^2 ... 32k x 8k, the cross-over is
+    // about 5.5x higher for SPMM (tile only at 30% on large matrices), 3x for SDDMM, 2.5x for FusedMM.
     if (M < 256 || K < 256 || width < 16 || nnz <= 0) return false;
     const double cells = (double)M * (double)K;
     const double density = (double)nnz / cells;
     const double crossover = 0.045 + 0.5e6 / cells;
-    return density >= (width >= 64 ? crossover : 1.5 * crossover);
+    const double narrow = op == B2SP_OP_SPMM ? 5.5 : op == B2SP_OP_SDDMM ? 3.0 : 2.5;
+    return density >= (width >= 64 ? crossover : narrow * crossover);
 }
 
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)

@@ -33,8 +33,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches);
 
-// True when the dense-tile family is expected to beat the row family for these sizes.
-bool tile_profitable(int M, int K, int width, long long nnz);
+// True when the dense-tile family is expected to beat the row family for these sizes (op = B2SP_OP_*,
+// width = N for SPMM, Kd for SDDMM, the smaller of the two for FusedMM).
+bool tile_profitable(int op, int M, int K, int width, long long nnz);
 
 // Offset of the window table inside the workspace (the same for every op) and its size.
 size_t pattern_table_offset(int M);

@@ -110,7 +110,7 @@ def test_spmm_tile_config_and_auto(b):
     # a workspace that only fits the row family makes AUTO use the row family
     small = torch.empty(1 << 16, dtype=torch.uint8, device="cuda")
     out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=small, algo=0)
-    assert b.last_algo(b.OP_SPMM) == 1
+    assert b.last_algo(b.OP_SPMM) in (1, 2)   # the row family (natural order for few rows)
     gate(out, ref, T, "spmm auto, small workspace")
     with pytest.raises(b.B2spError) as e:
         b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=small, algo=TILE)
@@ -205,7 +205,7 @@ def test_fused_tile_falls_back_on_unsorted_rows_and_large_kd(b):
         b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=TILE)
     assert e.value.status == 2
     out = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=0)
-    assert b.last_algo(b.OP_FUSEDMM) == 1
+    assert b.last_algo(b.OP_FUSEDMM) in (1, 2)
     ref, T = oracle.fusedmm(big.row_ptr, big.col_idx, big.values, big.A, big.B, big.D)
     gate(out, ref, T, "fusedmm auto, Kd=160")
 
