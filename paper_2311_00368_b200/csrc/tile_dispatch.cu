@@ -280,7 +280,10 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.out_tma = 0;
     a.slab_rows = p.Mt * kFusedRows;
     if (fused) {
-        const bool aligned = (reinterpret_cast<uintptr_t>(a.out) & 15) == 0 && (a.ld_out & 3) == 0;
+        // (TMA clips out-of-range columns in units of 16 bytes: a width that is not a multiple of four
+        // would let it write up to three floats past the end of every row of O)
+        const bool aligned = (reinterpret_cast<uintptr_t>(a.out) & 15) == 0 && (a.ld_out & 3) == 0 &&
+                             (p.KS > 1 || (N & 3) == 0);
         if (aligned) {
             const long long rows = p.KS == 1 ? M : (long long)p.KS * a.slab_rows;
             const int cols = p.KS == 1 ? N : p.Np;

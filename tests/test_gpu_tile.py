@@ -272,13 +272,14 @@ def test_prepared_pattern_is_shared_by_all_ops_and_stale_tables_are_detected(b):
     run_all("after a row-family call")
 
 
+@pytest.mark.parametrize("width", [100, 101])
 @pytest.mark.parametrize("ks", [1, 2, 3])
-def test_k_split_epilogues(b, ks, monkeypatch):
+def test_k_split_epilogues(b, ks, width, monkeypatch):
     """One K split stores O, two splits add their tiles into a zero-filled O, more go through slabs
     and the fixed-order sum: all three must give the same result, also for a ragged width, an output
     whose rows are padded, and an output that held NaNs before the call; repeated calls are bit-equal."""
     monkeypatch.setenv("B2SP_FORCE_KS", str(ks))
-    p = W.small_random(4100 + ks, 300, 1024, 0.2, 48, 100)
+    p = W.small_random(4100 + ks, 300, 1024, 0.2, 48, width)
     d = DevProblem(p)
     ws = _ws(b, b.OP_FUSEDMM, p)
     ref_f, T_f = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)
@@ -286,7 +287,7 @@ def test_k_split_epilogues(b, ks, monkeypatch):
     for name, ref, T, call in (
             ("fusedmm", ref_f, T_f, lambda o: b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=o, workspace=ws, algo=TILE)),
             ("spmm", ref_s, T_s, lambda o: b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=o, workspace=ws, algo=TILE))):
-        for pad in (12, 13):                          # ld = 112 (rows 16-byte aligned: TMA flush) and 113 (plain stores / atomics)
+        for pad in (12, 13, 3):                       # rows 16-byte aligned (TMA flush, unless the width is odd) or not (plain stores / atomics)
             padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
             out = padded[:, :p.N]
             call(out)
