@@ -219,6 +219,14 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
 
+// The workspace's device status word (read by b2sp_device_status) is 0 after a call whose kernels
+// could not fail; the binning pass and the tile family's first kernel reset it themselves.
+static b2sp_status clear_status(void *workspace, cudaStream_t st)
+{
+    return cudaMemsetAsync(static_cast<char *>(workspace) + kWsStatusOffset, 0, 64, st) == cudaSuccess ? B2SP_OK
+                                                                                                       : B2SP_ERR_CUDA;
+}
+
 // The row family under AUTO: the binning pass (two small launches, ~10 us) orders the rows longest
 // first, which only pays when the CTAs of the row kernel need several waves on the GPU.
 static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_ALGO_ROW; }
@@ -287,6 +295,8 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
+    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
+        return B2SP_ERR_CUDA;
     }
     rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, nullptr, st);
     g_last_launches[B2SP_OP_SPMM] = launches + 1;
@@ -368,6 +378,8 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
+    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
+        return B2SP_ERR_CUDA;
     }
     rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr, st);
     g_last_launches[B2SP_OP_SDDMM] = launches + 1;
@@ -446,6 +458,8 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
+    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
+        return B2SP_ERR_CUDA;
     }
     rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;

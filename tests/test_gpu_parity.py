@@ -305,3 +305,22 @@ def test_config_sweep_sampled(b, density, N):
     p = W.sweep_case(density, N)
     assert p.nnz == round(density * 8192 * 8192)
     check_sampled(b, p, (0,), ("spmm", "sddmm", "fusedmm"))
+
+
+def test_device_status_is_reset_by_every_family(b):
+    """b2sp_device_status reports the last call on a workspace: a stale word (here: garbage left in the
+    buffer) must not survive a call of any kernel family."""
+    p = W.small_random(77, 300, 400, 0.2, 32, 64)
+    d = DevProblem(p)
+    n = max(b.workspace_bytes(op, p.M, p.K, p.Kd, p.N, p.nnz) for op in range(3))
+    for algo in (0, 1, 2, 3):
+        ws = torch.full((max(n, 1 << 20),), 0x5a, dtype=torch.uint8, device="cuda")
+        assert b.device_status(ws) != 0
+        b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=algo)
+        assert b.device_status(ws) == 0, f"spmm algo={algo}"
+        ws.fill_(0x5a)
+        b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=algo)
+        assert b.device_status(ws) == 0, f"sddmm algo={algo}"
+        ws.fill_(0x5a)
+        b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=algo)
+        assert b.device_status(ws) == 0, f"fusedmm algo={algo}"
