@@ -19,7 +19,8 @@
  *     them, including the workspace; the library allocates nothing;
  *   - inputs are read-only; outputs are fully overwritten (never accumulated into; an empty
  *     row gives a zero output row, Alg. 2 line 1);
- *   - the call enqueues kernels on `stream` and returns without synchronising;
+ *   - the call enqueues kernels on `stream` and returns without synchronising; it may be captured
+ *     into a CUDA graph (make one ordinary call first: it does the library's one-time driver queries);
  *   - `workspace` is scratch of at least b2sp_workspace_bytes(...) bytes, 256-byte aligned;
  *     its contents are overwritten by every call, so two calls that may overlap in time on
  *     the GPU (different streams) need different workspaces;

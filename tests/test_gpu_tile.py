@@ -312,3 +312,34 @@ def test_tile_accuracy_on_same_sign_data_and_long_rows(b):
         p.D = rng.uniform(0.5, 1.5, p.D.shape).astype(np.float32)
         assert spmm_tile_check(b, p) < 0.6
         assert fused_tile_check(b, p) < 0.6
+
+
+def test_entry_points_can_be_captured_in_a_cuda_graph(b):
+    """The device entry points only enqueue work (no allocation, no synchronisation), so a step of
+    all three ops, row family and dense-tile family alike, can be captured once and replayed."""
+    p = W.small_random(4300, 384, 1024, 0.2, 64, 128)
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_FUSEDMM, p)
+    O1 = torch.empty((p.M, p.N), device="cuda")
+    O2 = torch.empty((p.M, p.N), device="cuda")
+    C = torch.empty(p.nnz, device="cuda")
+    refs = (oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D),
+            oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B),
+            oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D))
+    for algo in (TILE, 1):
+        def step():
+            b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=O1, workspace=ws, algo=algo)
+            b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, out=C, workspace=ws, algo=algo)
+            b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=O2, workspace=ws, algo=algo)
+        step()                                   # first use outside the capture (one-time driver queries)
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            step()
+        for out in (O1, O2, C):
+            out.fill_(float("nan"))
+        g.replay()
+        torch.cuda.synchronize()
+        assert b.device_status(ws) == 0
+        for name, out, (ref, T) in zip(("spmm", "sddmm", "fusedmm"), (O1, C, O2), refs):
+            gate(out, ref, T, f"{name} replayed from a CUDA graph, algo={algo}")
