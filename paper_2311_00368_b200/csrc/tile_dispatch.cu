@@ -179,6 +179,18 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     return p;
 }
 
+TwoPhasePlan plan_two_phase(int M, int K, int Kd, int N, long long nnz, size_t base_off)
+{
+    TwoPhasePlan t;
+    t.sddmm = plan_fused_tile(M, K, Kd, 0, nnz, base_off, false);
+    t.spmm = plan_fused_tile(M, K, 0, N, nnz, base_off, true);
+    if (!t.sddmm.feasible || !t.spmm.feasible) return t;
+    t.off_c = align_up(t.sddmm.bytes > t.spmm.bytes ? t.sddmm.bytes : t.spmm.bytes, 256);
+    t.bytes = align_up(t.off_c + sizeof(float) * (size_t)nnz, 256);
+    t.feasible = true;
+    return t;
+}
+
 namespace {
 
 template <int KDP, int MODE>
@@ -222,7 +234,7 @@ void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int 
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
-                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches)
+                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches, bool keep_status)
 {
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
@@ -256,9 +268,10 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         // per-tile arrival counters start at zero.
         const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), p.Mt * p.Nt, 1, p.Mt * p.Nt}
                                             : ZeroJob{nullptr, 0, 0, 0};
-        if (spmm) launch_split(jd, nullptr, z, status, st);
-        else if (fused) launch_split(jb, &jd, z, status, st);
-        else launch_split(jb, nullptr, z, status, st);
+        int *clear = keep_status ? nullptr : status;
+        if (spmm) launch_split(jd, nullptr, z, clear, st);
+        else if (fused) launch_split(jb, &jd, z, clear, st);
+        else launch_split(jb, nullptr, z, clear, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;

@@ -31,7 +31,17 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
-                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches);
+                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches,
+                       bool keep_status = false);
+
+// FusedMM with an output wider than two 128-column tiles runs as SDDMM into a scratch C followed by SPMM
+// on C (see b2sp_fusedmm): the plans of the two phases and where C sits in the workspace.
+struct TwoPhasePlan {
+    bool feasible = false;
+    FusedPlan sddmm, spmm;
+    size_t off_c = 0, bytes = 0;
+};
+TwoPhasePlan plan_two_phase(int M, int K, int Kd, int N, long long nnz, size_t base_off);
 
 // True when the dense-tile family is expected to beat the row family for these sizes (op = B2SP_OP_*,
 // width = N for SPMM, Kd for SDDMM, the smaller of the two for FusedMM).

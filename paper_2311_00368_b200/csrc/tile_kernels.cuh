@@ -151,7 +151,8 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // (rows_p >= rows, cols_p >= cols, cols_p % 32 == 0).  One 32-float group of a row is one
 // 128-byte swizzle row for TMA, and the whole thing is a plain packed 3-D tensor.
 // One launch splits up to two operands (blockIdx.y picks the job) and, being the first kernel of
-// every tile op, also clears the workspace's device status word and, when asked to, zero-fills an
+// every tile op, also clears the workspace's device status word (unless `status` is NULL: the second
+// kernel of a two-phase op keeps what the first one reported) and, when asked to, zero-fills an
 // array (the last blockIdx.y): the per-tile arrival counters of a FusedMM / SPMM with several K splits.
 struct SplitJob {
     const float *X;
@@ -170,7 +171,7 @@ struct ZeroJob {
 
 __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status)
 {
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
+    if (status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
     if ((int)blockIdx.y == njobs) {   // zero-fill job
         const long long total = (long long)z.rows * z.cols;
         const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
