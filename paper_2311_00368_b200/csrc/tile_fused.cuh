@@ -240,7 +240,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             if (!SPMM) { ptx::tma_prefetch_desc(&tm_bhi); ptx::tma_prefetch_desc(&tm_blo); }
             if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); ptx::tma_prefetch_desc(&tm_dlo); }
             // Chunk order = the order the MMA thread consumes them: B(0); then per block b:
-            // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only).
+            // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only; last block of a chunk: B(b+1) last).
             int c = 0;
             auto put = [&](bool is_b, int blk, int i) -> bool {
                 const int s = c % RING;
@@ -261,9 +261,12 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             };
             for (int i = 0; i < NCH_B && nblk > 0 && !failed; ++i) failed = !put(true, 0, i);
             for (int b = 0; b < nblk && !failed; ++b) {
+                // (FusedMM: at the end of a chunk of blocks GEMM1 of the next block comes last, see the MMA thread)
+                const bool late_b = FUSED && b % kFusedFlushBlocks == kFusedFlushBlocks - 1;
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !put(false, b, w);
-                if (!SPMM && b + 1 < nblk) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
+                if (!SPMM && b + 1 < nblk && !late_b) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !put(false, b, w);
+                if (!SPMM && b + 1 < nblk && late_b) for (int i = 0; i < NCH_B && !failed; ++i) failed = !put(true, b + 1, i);
             }
             if (failed)
                 for (int j = c > RING ? c - RING : 0; j < c; ++j) ptx::mbar_wait(full(j % RING), (j / RING) & 1);
@@ -348,11 +351,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     failed = !ptx::mbar_wait(o_free(ch % NOB), (ch / NOB - 1) & 1);
                     B2SP_FPROF_STOP(5)
                 }
+                // At the end of a chunk GEMM1 of the next block is issued after the chunk's last GEMM2, so that
+                // the tensor core works on it while the processors take O out of tensor memory.
+                const bool late_b = FUSED && b % kFusedFlushBlocks == kFusedFlushBlocks - 1;
                 if (FUSED) for (int w = 0; w < 2 && !failed; ++w) failed = !gemm2(b, w);
-                if (!SPMM && b + 1 < nblk && !failed) failed = !gemm1(b + 1);
+                if (!SPMM && b + 1 < nblk && !late_b && !failed) failed = !gemm1(b + 1);
                 if (FUSED) for (int w = 2; w < WPB && !failed; ++w) failed = !gemm2(b, w);
-                if (FUSED && !failed && (b % kFusedFlushBlocks == kFusedFlushBlocks - 1 || b == nblk - 1))
+                if (FUSED && !failed && (late_b || b == nblk - 1))
                     ptx::mma_commit(o_full((b / kFusedFlushBlocks) % NOB));
+                if (!SPMM && b + 1 < nblk && late_b && !failed) failed = !gemm1(b + 1);
             }
             B2SP_FPROF_FLUSH(0)
         }
@@ -436,11 +443,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 // its K split's slab): the first partial sum is stored, the later ones are added with fp32
                 // reductions (round to nearest).  A given element is only ever touched by the same lane of this
                 // warp, in program order, so the sum is reproducible.
-                // The flush of a chunk of blocks is done one window late (after P' of the next chunk's first
-                // window is ready), so that the tensor core has work again the moment O is free.
-                const bool chunk_ended = w == 0 && blk > 0 && blk % kFusedFlushBlocks == 0;
+                // SPMM: the flush of a chunk of blocks is done one window late (after P' of the next chunk's
+                // first window is ready), so that the tensor core has work again the moment O is free.
+                // FusedMM: right away; the tensor core runs GEMM1 of the next block meanwhile.
+                const bool chunk_ended = SPMM ? (w == 0 && blk > 0 && blk % kFusedFlushBlocks == 0)
+                                              : (w == WPB - 1 && blk % kFusedFlushBlocks == kFusedFlushBlocks - 1);
                 if (chunk_ended || it == nwin - 1) {
-                    const int chunk = chunk_ended ? blk / kFusedFlushBlocks - 1 : blk / kFusedFlushBlocks;
+                    const int chunk = (chunk_ended && SPMM) ? blk / kFusedFlushBlocks - 1 : blk / kFusedFlushBlocks;
                     const int ob = chunk % NOB;
                     bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
