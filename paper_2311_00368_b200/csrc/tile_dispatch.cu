@@ -323,4 +323,9 @@ extern "C" int b2sp_prof_fetch(unsigned long long *host32)
     if (cudaMemcpyFromSymbol(host32, b2sp::g_fused_prof, sizeof(zero)) != cudaSuccess) return 1;
     return cudaMemcpyToSymbol(b2sp::g_fused_prof, zero, sizeof(zero)) != cudaSuccess;
 }
+// Profiling builds only: per CTA the global-timer stamps (start, end of the MMA loop, end) and the SM id.
+extern "C" int b2sp_prof_cta_times(unsigned long long *host4096)
+{
+    return cudaMemcpyFromSymbol(host4096, b2sp::g_fused_cta, 4096 * sizeof(unsigned long long)) != cudaSuccess;
+}
 #endif

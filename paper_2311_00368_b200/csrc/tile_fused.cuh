@@ -36,8 +36,16 @@
 #define B2SP_FPROF_START fp_t0 = clock64();
 #define B2SP_FPROF_STOP(i) { long long t_ = clock64(); fp_acc[i] += t_ - fp_t0; fp_t0 = t_; }
 #define B2SP_FPROF_FLUSH(base) { if (lane == 0) { for (int i_ = 0; i_ < 6; ++i_) atomicAdd(b2sp::g_fused_prof + (base) + i_, (unsigned long long)fp_acc[i_]); } }
-namespace b2sp { __device__ unsigned long long g_fused_prof[32]; }
+#define B2SP_FPROF_STAMP(var) const long long var = clock64();
+#define B2SP_FPROF_ADD(i, v) { atomicAdd(b2sp::g_fused_prof + (i), (unsigned long long)(v)); }
+namespace b2sp { __device__ unsigned long long g_fused_prof[32]; __device__ unsigned long long g_fused_cta[1024 * 4]; }
+__device__ __forceinline__ unsigned long long b2sp_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+__device__ __forceinline__ unsigned b2sp_smid() { unsigned t; asm volatile("mov.u32 %0, %smid;" : "=r"(t)); return t; }
+#define B2SP_FPROF_CTA(i) { if (threadIdx.x == 32 && blockIdx.x < 1024) { b2sp::g_fused_cta[blockIdx.x * 4 + (i)] = b2sp_gtime(); b2sp::g_fused_cta[blockIdx.x * 4 + 3] = b2sp_smid(); } }
 #else
+#define B2SP_FPROF_CTA(i) {}
+#define B2SP_FPROF_STAMP(var)
+#define B2SP_FPROF_ADD(i, v) {}
 #define B2SP_FPROF_DECL
 #define B2SP_FPROF_START
 #define B2SP_FPROF_STOP(i) {}
@@ -153,6 +161,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const uint32_t flush_stage = slots + NSLOT * 4096;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    B2SP_FPROF_STAMP(fp_kernel_start)
+    B2SP_FPROF_CTA(0)
     const int ks = blockIdx.x % a.KS;
     const int tile = blockIdx.x / a.KS;
     const int nt = tile % a.Nt, mt = tile / a.Nt;
@@ -278,6 +288,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             constexpr uint32_t idesc2 = ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
             B2SP_FPROF_DECL
             B2SP_FPROF_START
+            B2SP_FPROF_STAMP(fp_loop_start)
             int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
             auto gemm1 = [&](int b) -> bool {   // P = A_tile * B_block^T over NCH_B chunks
                 const int pb = FUSED ? 0 : (b & 1);
@@ -362,6 +373,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (!SPMM && b + 1 < nblk && late_b && !failed) failed = !gemm1(b + 1);
             }
             B2SP_FPROF_FLUSH(0)
+            B2SP_FPROF_ADD(26, fp_loop_start - fp_kernel_start)
+            B2SP_FPROF_ADD(27, clock64() - fp_loop_start)
+            B2SP_FPROF_CTA(1)
         }
     } else if (warp >= 2 && warp < 6) {
         // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
@@ -687,6 +701,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         __syncwarp();
         ptx::tmem_dealloc(tmem, 512);
     }
+    if (threadIdx.x == 32) B2SP_FPROF_ADD(28, clock64() - fp_kernel_start)
+    B2SP_FPROF_CTA(2)
 }
 
 }  // namespace b2sp
