@@ -59,11 +59,12 @@ constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 // 20 warps = 5 per scheduler (a sixth would cut the register budget from 96 to 80 per thread).
 // Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors; warp 0 and warps 6-19
-// except 9, 13, 17: helpers.  Warps 13 and 17 idle: the scheduler of warps 1, 5, 9, 13, 17 keeps its
-// issue slots for the MMA warp.
+// except 9, 13, 17: helpers.  Warps 13 and 17 share the MMA warp's scheduler: they idle in FusedMM and
+// SPMM, whose tensor pipe wants that scheduler's issue slots, and are two more helpers in SDDMM, where the
+// MMA thread issues half the time (measured: 134 -> 129 us).
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
-constexpr int kFusedMaxHelpers = 12;   // the MMA warp's scheduler (warp % 4 == 1) gets no helper: its issue slots feed the tensor pipe
+constexpr int kFusedMaxHelpers = 14;
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 // The tensor core adds every MMA into its fp32 accumulator with truncation: a bias of about -2e-8 of
 // the running sum per MMA, which nothing cancels on same-sign data (measured: -3.0e-5 after the 1536
@@ -104,16 +105,17 @@ struct FusedCfg {
     static constexpr int NCH_B = SPMM ? 0 : KDP / 32;          // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
-    static constexpr int RING = SPMM ? 4 : FUSED ? 3 : 5;
+    static constexpr int RING = SPMM ? 4 : 3;
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
-    // 4 KB slots (two windows deep).  SPMM and SDDMM are bound by the helpers: twelve, twelve slots.
-    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : kFusedMaxHelpers;
-    static constexpr int SLOTS = HELPERS;
+    // 4 KB slots (two windows deep).  SPMM and SDDMM are bound by the helpers: twelve with twelve slots
+    // (SPMM), fourteen with twenty-eight slots (SDDMM: the count has to be a multiple of 14 and of 4).
+    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 14;
+    static constexpr int SLOTS = FUSED ? HELPERS : 2 * HELPERS;
     // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one
     // phase away: every slot is always filled by the same helper and drained by the same processor warp.
     static_assert(SLOTS % HELPERS == 0 && SLOTS % 4 == 0, "slot ownership must be fixed");
     static constexpr int FLUSH_BYTES = FUSED ? 4 * 4096 : 0;   // per processor warp: two buffers of 32 rows x 16 columns
-    static constexpr int AUX_BYTES = 512 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * 4096 + FLUSH_BYTES;
+    static constexpr int AUX_BYTES = 1024 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * 4096 + FLUSH_BYTES;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
     // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
@@ -157,7 +159,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
     auto o_free = [&](int b) { return aux + 8u * (2 * RING + 9 + 2 * NSLOT + b); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 12 + 2 * NSLOT));
-    const uint32_t helper_tabs = aux + 512, slots = aux + 512 + kFusedMaxHelpers * 256;
+    const uint32_t helper_tabs = aux + 1024, slots = aux + 1024 + kFusedMaxHelpers * 256;
     const uint32_t flush_stage = slots + NSLOT * 4096;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -579,15 +581,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             }
         }
         B2SP_FPROF_FLUSH(8)
-    } else if ((warp & 3) != 1 && (warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2)) < NH) {
-        // warp 0 and warps 6.. that do not share the MMA warp's scheduler, as many as this mode uses
+    } else if (((warp & 3) != 1 && (warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2)) < NH) || (NH > 12 && (warp == 13 || warp == 17))) {
+        // warp 0 and warps 6.. that do not share the MMA warp's scheduler, as many as this mode uses (SDDMM: and warps 13, 17)
         // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
         // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
         // values) and write them transposed into a slot, from which the processor thread of each row
         // reads its row.  SDDMM: prefetch the stored values the same way, then take the P rows the
         // processors left in the slot and write the stored entries, one coalesced run per row.
-        const int h = warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);   // warps 0,6,7,8,10,11,12,14,... -> 0,1,2,3,...
+        const int h = warp == 13 ? 12 : warp == 17 ? 13 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);   // warps 0,6,7,8,10,11,12,14,... -> 0,1,2,3,...; SDDMM: warps 13, 17 -> 12, 13
         const uint32_t tab = helper_tabs + h * 256;   // 32 records (position, mask) of the item's rows
         const int wbase = b0 * WPB, nitems = nblk * WPB * 4;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
