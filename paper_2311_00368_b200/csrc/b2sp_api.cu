@@ -74,12 +74,12 @@ inline unsigned gated_blocks(unsigned rows, const int *gate)
 template <int U, int SPLIT>
 void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
                  const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
-                 const int *order, const int *gate)
+                 const int *order, const int *gate, int *clear)
 {
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
     spmm_row_kernel<U, SPLIT><<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                           ldo, order, gate, nrows);
+                                                           ldo, order, gate, nrows, clear);
 }
 
 // Column geometry for a width N on the float4 path: U float4 per lane, SPLIT sub-warps.
@@ -98,20 +98,20 @@ inline int pick_ku(int Kd) { return Kd <= 64 ? 2 : Kd <= 128 ? 4 : Kd <= 256 ? 8
 template <int KU>
 void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const int *col_idx,
                   const float *sv, const float *A, int64_t lda, const float *B, int64_t ldb,
-                  float *out, const int *order, const int *gate)
+                  float *out, const int *order, const int *gate, int *clear)
 {
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
     sddmm_row_kernel<KU><<<grid, kRowThreads, smem, st>>>(Kd, row_ptr, col_idx, sv, A, lda, B, ldb,
-                                                         out, order, gate, nrows);
+                                                         out, order, gate, nrows, clear);
 }
 
 template <int KU, int U, int SPLIT>
 b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
                          const int *col_idx, const float *sv, const float *A, int64_t lda,
                          const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
-                         int64_t ldo, const int *order, const int *gate)
+                         int64_t ldo, const int *order, const int *gate, int *clear)
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
@@ -125,7 +125,7 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
     kern<<<grid, kRowThreads, smem, st>>>(Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
-                                          order, gate, nrows);
+                                          order, gate, nrows, clear);
     return B2SP_OK;
 }
 
@@ -134,10 +134,10 @@ b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int K
                                 const int *row_ptr, const int *col_idx, const float *sv,
                                 const float *A, int64_t lda, const float *B, int64_t ldb,
                                 const float *D, int64_t ldd, float *O, int64_t ldo,
-                                const int *order, const int *gate)
+                                const int *order, const int *gate, int *clear)
 {
 #define B2SP_F(U_, S_) \
-    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate)
+    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear)
     if (g.SPLIT == 4) B2SP_F(1, 4);
     if (g.SPLIT == 2) B2SP_F(1, 2);
     if (g.U == 1) B2SP_F(1, 1);
@@ -231,14 +231,6 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
 int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
 
-// The workspace's device status word (read by b2sp_device_status) is 0 after a call whose kernels
-// could not fail; the binning pass and the tile family's first kernel reset it themselves.
-static b2sp_status clear_status(void *workspace, cudaStream_t st)
-{
-    return cudaMemsetAsync(static_cast<char *>(workspace) + kWsStatusOffset, 0, 64, st) == cudaSuccess ? B2SP_OK
-                                                                                                       : B2SP_ERR_CUDA;
-}
-
 // The row family under AUTO: the binning pass (two small launches, ~10 us) orders the rows longest
 // first, which only pays when the CTAs of the row kernel need several waves on the GPU.
 static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_ALGO_ROW; }
@@ -246,21 +238,21 @@ static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_AL
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
                              const float *D, long long ldd, float *O, long long ldo, const int *order,
-                             const int *gate, cudaStream_t st)
+                             const int *gate, int *clear, cudaStream_t st)
 {
     bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
     if (vec) {
         Geom g = pick_geom(N);
         dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
-        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
-        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
-        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
-        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
-        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate);
+        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
         spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                            ldo, order, gate, M);
+                                                            ldo, order, gate, M, clear);
     }
     return check_launch();
 }
@@ -298,19 +290,20 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
         if (rc != B2SP_OK) return rc;
         // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
-        rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, st);
+        rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_SPMM] = launches + 1;
         return rc;
     }
     const int *order = nullptr;
+    int *clear = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
-    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
-        return B2SP_ERR_CUDA;
+    } else {   // no binning pass: the row kernel itself resets the status word
+        clear = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsStatusOffset);
     }
-    rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, nullptr, st);
+    rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, nullptr, clear, st);
     g_last_launches[B2SP_OP_SPMM] = launches + 1;
     return rc;
 }
@@ -318,29 +311,29 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
 // Enqueues the row-family SDDMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_idx, const float *s_values,
                               const float *A, long long lda, const float *B, long long ldb,
-                              float *out_values, const int *order, const int *gate, cudaStream_t st)
+                              float *out_values, const int *order, const int *gate, int *clear, cudaStream_t st)
 {
     dim3 grid((unsigned)M);
     bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
                Kd <= 40960;
     if (vec) {
         switch (pick_ku(Kd)) {
-        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
-        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
-        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate); break;
+        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
+        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
+        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
         default: {
             size_t smem = sizeof(float) * (size_t)Kd;
             if (smem > 48 * 1024 &&
                 cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)smem) != cudaSuccess)
                 return B2SP_ERR_CUDA;
-            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate);
+            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear);
         }
         }
     } else {
         grid.x = gated_blocks(grid.x, gate);
         sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
-                                                             B, ldb, out_values, order, gate, M);
+                                                             B, ldb, out_values, order, gate, M, clear);
     }
     return check_launch();
 }
@@ -381,19 +374,20 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
                         out_values, 0, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
-        rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, nullptr, gate, st);
+        rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_SDDMM] = launches + 1;
         return rc;
     }
     const int *order = nullptr;
+    int *clear = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
-    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
-        return B2SP_ERR_CUDA;
+    } else {   // no binning pass: the row kernel itself resets the status word
+        clear = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsStatusOffset);
     }
-    rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr, st);
+    rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, nullptr, clear, st);
     g_last_launches[B2SP_OP_SDDMM] = launches + 1;
     return rc;
 }
@@ -402,7 +396,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const int *col_idx,
                               const float *s_values, const float *A, long long lda, const float *B,
                               long long ldb, const float *D, long long ldd, float *O, long long ldo,
-                              const int *order, const int *gate, cudaStream_t st)
+                              const int *order, const int *gate, int *clear, cudaStream_t st)
 {
     b2sp_status rc = B2SP_OK;
     bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
@@ -412,16 +406,16 @@ static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const in
         Geom g = pick_geom(N);
         dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
         switch (pick_ku(Kd)) {
-        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
-        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
-        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
-        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate); break;
+        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
+        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
+        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
+        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
         }
         if (rc != B2SP_OK) return rc;
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
         fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
-                                                               lda, B, ldb, D, ldd, O, ldo, order, gate, M);
+                                                               lda, B, ldb, D, ldd, O, ldo, order, gate, M, clear);
     }
     return check_launch();
 }
@@ -472,19 +466,20 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
         }
         if (rc != B2SP_OK) return rc;
         const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
-        rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, st);
+        rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
         return rc;
     }
     const int *order = nullptr;
+    int *clear = nullptr;
     if (use == B2SP_ALGO_ROW) {
         rc = bin_rows(M, row_ptr, w, st, &launches);
         if (rc != B2SP_OK) return rc;
         order = w.row_order;
-    } else if (clear_status(workspace, st) != B2SP_OK) {   // no binning pass: nothing else resets the status word
-        return B2SP_ERR_CUDA;
+    } else {   // no binning pass: the row kernel itself resets the status word
+        clear = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsStatusOffset);
     }
-    rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, st);
+    rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, clear, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
     return rc;
 }

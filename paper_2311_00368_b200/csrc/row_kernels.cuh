@@ -7,6 +7,8 @@
 // FusedMM, their partial output rows are combined through shared memory in a fixed order, so
 // results are deterministic.  Rows are visited in the order given by `row_order` (longest
 // first, produced by the binning kernels below) or in natural order when it is NULL.
+// `clear`, when not NULL, points at the workspace's status word, which the kernel resets (a call whose only
+// launch is this kernel cannot fail on the device).
 // `gate`, when not NULL, points at a device word: the kernel does nothing if that word is 0
 // (used when the row family is only the fallback of the dense-tile family).
 #pragma once
@@ -173,11 +175,12 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                 const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                 float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                const int *__restrict__ gate, int nrows)
+                const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     using G = SweepGeom<U, SPLIT>;
     __shared__ float4 red[kRowWarps * U * G::LPN];
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / G::LPN, sl = lane % G::LPN;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
@@ -225,10 +228,11 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                        const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                        float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                       const int *__restrict__ gate, int nrows)
+                       const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
@@ -327,11 +331,12 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                  const float *s_values, const float *__restrict__ A, int64_t lda,
                  const float *__restrict__ B, int64_t ldb, float *out_values,
-                 const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
+                 const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     extern __shared__ float4 dyn_smem[];
     float *a_smem = reinterpret_cast<float *>(dyn_smem);
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
@@ -355,9 +360,10 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                         const float *s_values, const float *__restrict__ A, int64_t lda,
                         const float *__restrict__ B, int64_t ldb, float *out_values,
-                        const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
+                        const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
         const int beg = row_ptr[row], end = row_ptr[row + 1];
@@ -382,11 +388,12 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
                    const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
-                   const int *__restrict__ row_order, const int *__restrict__ gate, int nrows)
+                   const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     float4 *red = dyn_smem;                                                   // kRowWarps*U*LPN
     float *a_smem = reinterpret_cast<float *>(dyn_smem + kRowWarps * U * G::LPN);  // Kd (KU == 0)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -434,10 +441,11 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
                           const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
                           int64_t ldb, const float *__restrict__ D, int64_t ldd,
                           float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                          const int *__restrict__ gate, int nrows)
+                          const int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
+    if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
