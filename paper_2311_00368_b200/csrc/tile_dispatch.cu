@@ -202,7 +202,7 @@ b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, cons
     auto kern = fused_tile_kernel<KDP, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
-    kern<<<items, kFusedThreads, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, out, a);
+    kern<<<items, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, out, a);
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 

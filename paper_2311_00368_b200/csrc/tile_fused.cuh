@@ -64,7 +64,7 @@ constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 // MMA thread issues half the time (measured: 134 -> 129 us).
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
-constexpr int kFusedMaxHelpers = 14;
+constexpr int kFusedMaxHelpers = 20;
 constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
 // The tensor core adds every MMA into its fp32 accumulator with truncation: a bias of about -2e-8 of
 // the running sum per MMA, which nothing cancels on same-sign data (measured: -3.0e-5 after the 1536
@@ -98,6 +98,17 @@ struct FusedTileArgs {
 // themselves (no A, no GEMM1).
 constexpr int kModeSddmm = 0, kModeFused = 1, kModeSpmm = 2;
 
+// Which helper a warp is (-1: none).  20-warp kernels (FusedMM, SPMM): warps 0, 6, 7, 8, 10, 11, 12, 14, ...
+// -> 0, 1, 2, ...: none on the MMA warp's scheduler (warp % 4 == 1).  28-warp kernel (SDDMM): every warp
+// but 1-5 (MMA, processors), 9 (TMA), 21 and 25.
+template <bool NARROW>
+__device__ __forceinline__ int helper_index(int warp)
+{
+    if (NARROW) return (warp & 3) == 1 || (warp >= 2 && warp < 6) ? -1 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);
+    if ((warp >= 1 && warp < 6) || warp == 9 || warp == 21 || warp == 25) return -1;
+    return warp == 0 ? 0 : 1 + (warp - 6) - (warp > 9 ? 1 : 0) - (warp > 21 ? 1 : 0) - (warp > 25 ? 1 : 0);
+}
+
 template <int KDP, int MODE>
 struct FusedCfg {
     static constexpr bool FUSED = MODE != kModeSddmm;          // has GEMM2 / O
@@ -105,17 +116,23 @@ struct FusedCfg {
     static constexpr int NCH_B = SPMM ? 0 : KDP / 32;          // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
-    static constexpr int RING = SPMM ? 4 : 3;
+    // SDDMM runs 28 warps of 72 registers (its processors only copy P, and its helpers work on items of
+    // 16 rows, so nobody needs more): twenty helpers instead of twelve.  FusedMM and SPMM: 20 warps of 96.
+    static constexpr int THREADS = FUSED ? kFusedThreads : 896;
+    static constexpr int RING = FUSED && !SPMM ? 3 : 4;
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
     // 4 KB slots (two windows deep).  SPMM and SDDMM are bound by the helpers: twelve with twelve slots
-    // (SPMM), fourteen with twenty-eight slots (SDDMM: the count has to be a multiple of 14 and of 4).
-    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 14;
+    // (SPMM), twenty with forty half-size slots (SDDMM).
+    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 20;
+    static constexpr int ITEM_ROWS = FUSED ? 32 : 16;           // rows of a helper's work item
+    static constexpr int IPW = kFusedRows / ITEM_ROWS;         // items per window
+    static constexpr int SLOT_BYTES = ITEM_ROWS * 128;
     static constexpr int SLOTS = FUSED ? HELPERS : 2 * HELPERS;
     // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one
     // phase away: every slot is always filled by the same helper and drained by the same processor warp.
-    static_assert(SLOTS % HELPERS == 0 && SLOTS % 4 == 0, "slot ownership must be fixed");
+    static_assert(SLOTS % HELPERS == 0 && SLOTS % IPW == 0, "slot ownership must be fixed");
     static constexpr int FLUSH_BYTES = FUSED ? 4 * 4096 : 0;   // per processor warp: two buffers of 32 rows x 16 columns
-    static constexpr int AUX_BYTES = 1024 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * 4096 + FLUSH_BYTES;
+    static constexpr int AUX_BYTES = 1024 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * SLOT_BYTES + FLUSH_BYTES;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
     // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
@@ -126,7 +143,7 @@ struct FusedCfg {
 };
 
 template <int KDP, int MODE>
-__global__ void __launch_bounds__(kFusedThreads, 1)
+__global__ void __launch_bounds__((FusedCfg<KDP, MODE>::THREADS), 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
                   const __grid_constant__ CUtensorMap tm_out, const FusedTileArgs a)
@@ -160,7 +177,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     auto o_free = [&](int b) { return aux + 8u * (2 * RING + 9 + 2 * NSLOT + b); };
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 12 + 2 * NSLOT));
     const uint32_t helper_tabs = aux + 1024, slots = aux + 1024 + kFusedMaxHelpers * 256;
-    const uint32_t flush_stage = slots + NSLOT * 4096;
+    const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     B2SP_FPROF_STAMP(fp_kernel_start)
@@ -197,15 +214,20 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     bool failed = false;
 
     // ---- A tile -> TMEM (hi, and lo for SDDMM) / shared memory (lo for FusedMM); thread = row ----
-    const int q = warp & 3;                 // TMEM lane quarter of warps 2..5
-    const int row = q * 32 + lane;          // row inside the tile (warps >= 2)
+    // A warp reaches the tensor-memory lanes of quarter warp % 4: all warps of a quarter but the MMA and the
+    // TMA warp share the tile's 16-column groups.
+    const int q = warp & 3;                 // TMEM lane quarter
+    const int row = q * 32 + lane;          // row inside the tile
     const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    if (!SPMM && warp >= 2 && warp < 6) {
+    constexpr int NWARP = Cfg::THREADS / 32;
+    const int pro_n = q == 1 ? NWARP / 4 - 2 : NWARP / 4;                            // warps of this quarter that take part
+    const int pro_i = q == 1 ? (warp == 5 ? 0 : (warp >> 2) - 2) : (warp >> 2);      // ... and this warp's place among them
+    if (!SPMM && warp != 1 && warp != kFusedTmaWarp) {
         const int grow = m0 + row;
         const float *arow = a.A + (long long)(grow < a.M ? grow : 0) * a.lda;
         const bool vec = (a.lda & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
 #pragma unroll 1
-        for (int c = 0; c < KDP; c += 16) {
+        for (int c = pro_i * 16; c < KDP; c += pro_n * 16) {
             uint32_t hi[16], lo[16];
             float v[16];
 #pragma unroll
@@ -390,8 +412,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         B2SP_FPROF_START
         for (int it = 0; it < nwin; ++it) {
             const int blk = it / WPB, w = it % WPB;
-            const int j = it * 4 + q, s = j % NSLOT, use = j / NSLOT;
-            const uint32_t slot = slots + s * 4096 + lane * 128;
+            // FusedMM / SPMM: one item (32 rows) per processor warp and window.  SDDMM: two items of 16 rows,
+            // lanes 0-15 and lanes 16-31 each with their own slot.
+            const int j = FUSED ? it * 4 + q : it * 8 + 2 * q + (lane >> 4);
+            const int s = j % NSLOT, use = j / NSLOT;
+            const uint32_t slot = slots + s * Cfg::SLOT_BYTES + (FUSED ? lane : (lane & 15)) * 128;
             if (FUSED) {
                 float sv[32];
                 {
@@ -576,28 +601,28 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                                  "r"(src[0]), "r"(src[1]), "r"(src[2]), "r"(src[3]) : "memory");
                 }
                 __syncwarp();
-                if (lane == 0) ptx::mbar_arrive(sl_full(s));
+                if ((lane & 15) == 0) ptx::mbar_arrive(sl_full(s));
                 B2SP_FPROF_STOP(4)
             }
         }
         B2SP_FPROF_FLUSH(8)
-    } else if (((warp & 3) != 1 && (warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2)) < NH) || (NH > 12 && (warp == 13 || warp == 17))) {
-        // warp 0 and warps 6.. that do not share the MMA warp's scheduler, as many as this mode uses (SDDMM: and warps 13, 17)
-        // ---------------- helper warps: work items (window, row quarter), round-robin ----------------
+    } else if (helper_index<FUSED>(warp) >= 0 && helper_index<FUSED>(warp) < NH) {
+        // ---------------- helper warps: work items (window, group of rows), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
         // (coalesced), densify (0 where nothing is stored; 1 for stored entries when there are no
         // values) and write them transposed into a slot, from which the processor thread of each row
-        // reads its row.  SDDMM: prefetch the stored values the same way, then take the P rows the
-        // processors left in the slot and write the stored entries, one coalesced run per row.
-        const int h = warp == 13 ? 12 : warp == 17 ? 13 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);   // warps 0,6,7,8,10,11,12,14,... -> 0,1,2,3,...; SDDMM: warps 13, 17 -> 12, 13
+        // reads its row.  SDDMM (items of 16 rows): prefetch the stored values the same way, then take the
+        // P rows the processors left in the slot and write the stored entries, one coalesced run per row.
+        const int h = helper_index<FUSED>(warp);
         const uint32_t tab = helper_tabs + h * 256;   // 32 records (position, mask) of the item's rows
-        const int wbase = b0 * WPB, nitems = nblk * WPB * 4;
+        constexpr int IR = Cfg::ITEM_ROWS, IPW = Cfg::IPW;
+        const int wbase = b0 * WPB, nitems = nblk * WPB * IPW;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
         const bool has_values = a.s_values != nullptr;
         auto load_rec = [&](int jj) {   // lane = row: window record of one row of item jj
             int2 r = make_int2(0, 0);
-            const int hrow = m0 + (jj & 3) * 32 + lane, wglob = wbase + (jj >> 2);
-            if (jj < nitems && hrow < a.M && wglob < a.Wk) r = __ldg(a.win + (size_t)hrow * a.Wk + wglob);
+            const int hrow = m0 + (jj % IPW) * IR + lane, wglob = wbase + jj / IPW;
+            if (jj < nitems && lane < IR && hrow < a.M && wglob < a.Wk) r = __ldg(a.win + (size_t)hrow * a.Wk + wglob);
             return r;
         };
         // the records of the next two items are in flight while an item is processed
@@ -612,9 +637,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             __syncwarp();   // everyone is done with the previous item's records
             ptx::sts64(tab + lane * 8, (uint32_t)rec.x, (uint32_t)rec.y);
             __syncwarp();
-            float vn[32];
-            int idx[FUSED ? 1 : 32];   // SDDMM: CSR position of the lane's entry in each row (-1: nothing stored)
-            ptx::for_each_row<32>([&](auto rc) {
+            float vn[IR];
+            int idx[FUSED ? 1 : IR];   // SDDMM: CSR position of the lane's entry in each row (-1: nothing stored)
+            ptx::for_each_row<IR>([&](auto rc) {
                 constexpr int r = decltype(rc)::value;
                 uint32_t pos, m;
                 ptx::lds64_off<r * 8>(tab, pos, m);
@@ -624,7 +649,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (present && has_values) vn[r] = __ldg(a.s_values + at);
                 if (!FUSED) idx[r] = present ? at : -1;
             });
-            const uint32_t slot = slots + s * 4096;
+            const uint32_t slot = slots + s * Cfg::SLOT_BYTES;
             B2SP_FPROF_STOP(0)
             if (FUSED) {
                 if (use > 0) {
@@ -632,7 +657,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
                 B2SP_FPROF_STOP(1)
-                ptx::for_each_row<32>([&](auto rc) {
+                ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     ptx::sts32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
                 });
@@ -646,13 +671,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 B2SP_FPROF_STOP(1)
                 // all reads of the slot first (independent loads), then the stores
-                ptx::for_each_row<32>([&](auto rc) {
+                ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     vn[r] *= __uint_as_float(ptx::lds32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4))));
                 });
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
-                ptx::for_each_row<32>([&](auto rc) {
+                ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     if (idx[FUSED ? 0 : r] >= 0) a.out[idx[FUSED ? 0 : r]] = vn[r];
                 });
