@@ -702,7 +702,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         __syncthreads();
         if (*last_flag) {
             __threadfence();
-            for (int e = threadIdx.x; e < kFusedRows * (kFusedNT / 4); e += kFusedThreads) {
+            for (int e = threadIdx.x; e < kFusedRows * (kFusedNT / 4); e += Cfg::THREADS) {
                 const int r = e / (kFusedNT / 4), c = (e % (kFusedNT / 4)) * 4;
                 const int grow = m0 + r, n = n0 + c;
                 if (grow >= a.M || n >= a.N) continue;
