@@ -10,7 +10,7 @@
 //     in chunks of 32 k (hi + lo, 32 KB); N = 128 MMAs run the tensor pipe at full rate (a 128xNx8
 //     tf32 MMA costs max(N/2, 45.6) cycles, so 32-column GEMMs would waste two thirds of it).
 //   * Four processor warps (thread = row) read P window by window (32 columns) and multiply it by the
-//     window's stored values (0 where nothing is stored), which twelve helper warps fetch with lane =
+//     window's stored values (0 where nothing is stored), which helper warps fetch with lane =
 //     column (coalesced), densify and transpose through shared-memory slots.  The sampled C of the
 //     paper (Alg. 3) exists only in these registers.  Then
 //       - FusedMM: split the result into hi/lo and write it back to TMEM as P' (two buffers); GEMM2
@@ -57,11 +57,10 @@ namespace b2sp {
 constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
-// 20 warps = 5 per scheduler (a sixth would cut the register budget from 96 to 80 per thread).
-// Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors; warp 0 and warps 6-19
-// except 9, 13, 17: helpers.  Warps 13 and 17 share the MMA warp's scheduler: they idle in FusedMM and
-// SPMM, whose tensor pipe wants that scheduler's issue slots, and are two more helpers in SDDMM, where the
-// MMA thread issues half the time (measured: 134 -> 129 us).
+// FusedMM and SPMM: 20 warps = 5 per scheduler (a sixth would cut the register budget from 96 to 80 per
+// thread).  Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors; warp 0 and warps
+// 6-19 except 9, 13, 17: helpers.  Warps 13 and 17 share the MMA warp's scheduler and idle: the tensor pipe
+// wants that scheduler's issue slots.  SDDMM: 28 warps of 72 registers, see FusedCfg.
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
 constexpr int kFusedMaxHelpers = 20;
@@ -121,8 +120,9 @@ struct FusedCfg {
     static constexpr int THREADS = FUSED ? kFusedThreads : 896;
     static constexpr int RING = FUSED && !SPMM ? 3 : 4;
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
-    // 4 KB slots (two windows deep).  SPMM and SDDMM are bound by the helpers: twelve with twelve slots
-    // (SPMM), twenty with forty half-size slots (SDDMM).
+    // 4 KB slots (two windows deep).  SPMM: twelve with twelve slots.  SDDMM: twenty with forty 2 KB slots
+    // (measured: 12 helpers 134 us, 14 helpers 129 us, 20 helpers on 28 warps 125 us; for SPMM the same
+    // layout was slower, 136-140 us against 131 us).
     static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 20;
     static constexpr int ITEM_ROWS = FUSED ? 32 : 16;           // rows of a helper's work item
     static constexpr int IPW = kFusedRows / ITEM_ROWS;         // items per window
