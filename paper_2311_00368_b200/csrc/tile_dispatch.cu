@@ -150,8 +150,9 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     p.Kp = (K + kFusedBlk - 1) / kFusedBlk * kFusedBlk;   // operand copies padded to whole 128-column blocks
     p.Kdp = Kd == 0 ? 0 : Kd <= 32 ? 32 : Kd <= 64 ? 64 : 128;   // Kd == 0: SPMM through the fused pipeline
     p.Mt = (M + kFusedRows - 1) / kFusedRows;
-    p.Nt = fused ? (N + kFusedNT - 1) / kFusedNT : 1;
-    p.Np = fused ? p.Nt * kFusedNT : 0;
+    p.NT = fused && N <= 64 ? 64 : kFusedNT;   // a 64-column GEMM2 costs 46 instead of 64 cycles per MMA
+    p.Nt = fused ? (N + p.NT - 1) / p.NT : 1;
+    p.Np = fused ? p.Nt * p.NT : 0;
     size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(p.Mt * p.Nt, p.Kp / kFusedBlk);
@@ -250,8 +251,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
                   !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
         return B2SP_ERR_CUDA;
     if (fused) {
-        if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true) ||
-            !make_blocked_map(&tm_dl, dlo, p.Kp, p.Np / 32, kFusedW, kFusedNT / 32, true))
+        if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, p.NT / 32, true) ||
+            !make_blocked_map(&tm_dl, dlo, p.Kp, p.Np / 32, kFusedW, p.NT / 32, true))
             return B2SP_ERR_CUDA;
     } else {
         tm_dh = tm_bh;   // unused by the SDDMM kernel
@@ -277,7 +278,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
 
     FusedTileArgs a;
-    a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt;
+    a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.NT = p.NT;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     a.flags = flags; a.status = status;
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);

@@ -19,6 +19,7 @@ constexpr size_t kWsHeaderBytes = 512;
 struct FusedPlan {
     bool feasible = false;
     int Kdp = 0, Nt = 1, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
+    int NT = 128;   // O columns per CTA: 64 when N <= 64
     size_t off_win = 0, off_bhi = 0, off_blo = 0, off_dhi = 0, off_dlo = 0, off_part = 0, off_cnt = 0;
     size_t bytes = 0;
 };

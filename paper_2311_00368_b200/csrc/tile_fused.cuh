@@ -64,7 +64,7 @@ constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
 constexpr int kFusedMaxHelpers = 20;
-constexpr int kFusedNT = 128;       // O columns per CTA (UMMA N of GEMM2)
+constexpr int kFusedNT = 128;       // most O columns per CTA (UMMA N of GEMM2); see FusedTileArgs::NT
 // The tensor core adds every MMA into its fp32 accumulator with truncation: a bias of about -2e-8 of
 // the running sum per MMA, which nothing cancels on same-sign data (measured: -3.0e-5 after the 1536
 // MMAs of 32 blocks, three times the 1e-5 gate).  So O is accumulated in tensor memory over at most
@@ -75,6 +75,7 @@ constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
+    int NT;                   // O columns per CTA (UMMA N of GEMM2): 128, or 64 when N <= 64
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
     const float *A;           // M x Kd
@@ -188,7 +189,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int nblk_all = (a.Wk + WPB - 1) / WPB;
     const int b0 = (int)((long long)nblk_all * ks / a.KS), b1 = (int)((long long)nblk_all * (ks + 1) / a.KS);
     const int nblk = b1 - b0;
-    const int m0 = mt * kFusedRows, n0 = nt * kFusedNT;
+    const int m0 = mt * kFusedRows, n0 = nt * a.NT;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
@@ -281,14 +282,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
                 const uint32_t dst = ring + s * kFusedChunk;
                 const int col0 = (b0 + blk) * kFusedBlk;
-                ptx::mbar_arrive_expect_tx(full(s), kFusedChunk);
+                ptx::mbar_arrive_expect_tx(full(s), is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4);   // hi + lo
                 if (is_b) {   // B rows col0..col0+127, k group i
                     ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
                     ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
                 } else {      // D rows of window i of the block
                     const int krow = col0 + i * kFusedW;
-                    ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (kFusedNT / 32));
-                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (kFusedNT / 32));
+                    ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (a.NT / 32));
+                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
                 }
                 ++c;
                 return true;
@@ -309,7 +310,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedBlk, false, false);
-            constexpr uint32_t idesc2 = ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
+            const uint32_t idesc2 = a.NT == 64 ? ptx::idesc_tf32(kFusedRows, 64, false, true) : ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
             B2SP_FPROF_DECL
             B2SP_FPROF_START
             B2SP_FPROF_STAMP(fp_loop_start)
@@ -506,7 +507,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         __syncwarp();
                         const int y = ks * a.slab_rows + m0 + q * 32;
 #pragma unroll 1
-                        for (int c = 0; c < kFusedNT / 16; ++c) {
+                        for (int c = 0; c < a.NT / 16; ++c) {
                             const uint32_t buf = stage + (uint32_t)(c & 1) * 2048;
                             if (c >= 2) {
                                 if (lane == 0) ptx::bulk_wait_read<1>();   // the buffer's previous contents have been read
@@ -515,7 +516,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                             uint32_t r[16];
                             ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
                             ptx::tmem_ld_wait();
-                            if (c == kFusedNT / 16 - 1) {
+                            if (c == a.NT / 16 - 1) {
                                 ptx::tc_fence_before_sync();
                                 __syncwarp();
                                 if (lane == 0) ptx::mbar_arrive(o_free(ob));
@@ -535,10 +536,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     } else {
                         // output rows that are not 16-byte aligned: the same through plain stores / atomics
                         float *obase = a.out + (long long)ks * a.slab + (long long)(m0 + q * 32) * a.ld_out;
-                        const int ncols = a.KS == 1 ? a.N : a.Nt * kFusedNT;   // slabs are padded to whole tiles
+                        const int ncols = a.KS == 1 ? a.N : a.Nt * a.NT;   // slabs are padded to whole tiles
                         const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
 #pragma unroll 1
-                        for (int c = 0; c < kFusedNT / 16; ++c) {
+                        for (int c = 0; c < a.NT / 16; ++c) {
                             uint32_t r[16];
                             ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
                             ptx::tmem_ld_wait();
@@ -702,8 +703,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         __syncthreads();
         if (*last_flag) {
             __threadfence();
-            for (int e = threadIdx.x; e < kFusedRows * (kFusedNT / 4); e += Cfg::THREADS) {
-                const int r = e / (kFusedNT / 4), c = (e % (kFusedNT / 4)) * 4;
+            for (int e = threadIdx.x; e < kFusedRows * (a.NT / 4); e += Cfg::THREADS) {
+                const int r = e / (a.NT / 4), c = (e % (a.NT / 4)) * 4;
                 const int grow = m0 + r, n = n0 + c;
                 if (grow >= a.M || n >= a.N) continue;
                 const float *src = a.out + (long long)grow * a.ld_out + n;
