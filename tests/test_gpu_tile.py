@@ -49,6 +49,8 @@ def spmm_tile_check(b, p, expect_algo=TILE):
     (384, 1024, 0.20, 256, "powerlaw"),  # skewed rows incl. full rows
     (256, 512, 0.20, 128, "band"),
     (200, 640, 0.05, 36, "uniform"),     # sparse windows (8 lanes per row), N = 36
+    (260, 700, 0.20, 63, "uniform"),     # widest output that still takes 64-column O tiles (odd: no TMA flush)
+    (260, 700, 0.20, 65, "uniform"),     # narrowest output on 128-column O tiles
 ])
 def test_spmm_tile_shapes(b, M, K, density, N, kind):
     p = W.small_random(2000 + M + N, M, K, density, 0, N, kind=kind)
@@ -154,6 +156,8 @@ def fused_tile_check(b, p, null_values=False, ops=("sddmm", "fusedmm")):
     (384, 1024, 0.20, 64, 128, "powerlaw"),   # skewed rows incl. full rows
     (256, 512, 0.20, 64, 64, "band"),
     (200, 640, 0.05, 36, 36, "uniform"),
+    (260, 700, 0.20, 48, 64, "powerlaw"),     # 64-column O tile, several K splits
+    (260, 700, 0.20, 48, 68, "powerlaw"),     # 128-column O tile just above the switch
 ])
 def test_fused_and_sddmm_tile_shapes(b, M, K, density, Kd, N, kind):
     p = W.small_random(3000 + M + N, M, K, density, Kd, N, kind=kind)
