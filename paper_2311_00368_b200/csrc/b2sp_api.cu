@@ -63,6 +63,26 @@ b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t
     return check_launch();
 }
 
+// Launches `kern`; a gated launch (the row family as the dense-tile family's device-side fallback) is marked as a
+// programmatic dependent of the tile kernel before it: the tile kernel lets its dependents go as soon
+// as it has read the gate's flags, which are final before it starts, so the fallback (which almost always
+// finds its gate closed and exits) runs beside the tile kernel instead of after it.
+template <class... KArgs, class... Args>
+inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStream_t st, bool gated, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(kRowThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = gated ? attr : nullptr;
+    cfg.numAttrs = gated ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
 // A gated launch (the row family as the dense-tile family's fallback) almost always finds its gate
 // closed: it gets a small grid whose blocks walk the rows, so that the usual case costs little.
 inline unsigned gated_blocks(unsigned rows, const int *gate)
@@ -78,8 +98,8 @@ void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const in
 {
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    spmm_row_kernel<U, SPLIT><<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                           ldo, order, gate, nrows, clear);
+    launch_row(spmm_row_kernel<U, SPLIT>, grid, 0, st, gate != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+               gate, nrows, clear);
 }
 
 // Column geometry for a width N on the float4 path: U float4 per lane, SPLIT sub-warps.
@@ -103,8 +123,8 @@ void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const 
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    sddmm_row_kernel<KU><<<grid, kRowThreads, smem, st>>>(Kd, row_ptr, col_idx, sv, A, lda, B, ldb,
-                                                         out, order, gate, nrows, clear);
+    launch_row(sddmm_row_kernel<KU>, grid, smem, st, gate != nullptr, Kd, row_ptr, col_idx, sv, A, lda, B, ldb, out, order,
+               gate, nrows, clear);
 }
 
 template <int KU, int U, int SPLIT>
@@ -124,8 +144,8 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     }
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    kern<<<grid, kRowThreads, smem, st>>>(Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
-                                          order, gate, nrows, clear);
+    launch_row(kern, grid, smem, st, gate != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
+               nrows, clear);
     return B2SP_OK;
 }
 
@@ -251,8 +271,8 @@ static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_id
         else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
-        spmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(N, row_ptr, col_idx, values, D, ldd, O,
-                                                            ldo, order, gate, M, clear);
+        launch_row(spmm_row_scalar_kernel, grid, 0, st, gate != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+                   gate, M, clear);
     }
     return check_launch();
 }
@@ -332,8 +352,8 @@ static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_
         }
     } else {
         grid.x = gated_blocks(grid.x, gate);
-        sddmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, row_ptr, col_idx, s_values, A, lda,
-                                                             B, ldb, out_values, order, gate, M, clear);
+        launch_row(sddmm_row_scalar_kernel, grid, 0, st, gate != nullptr, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb,
+                   out_values, order, gate, M, clear);
     }
     return check_launch();
 }
@@ -414,8 +434,8 @@ static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const in
         if (rc != B2SP_OK) return rc;
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
-        fusedmm_row_scalar_kernel<<<grid, kRowThreads, 0, st>>>(Kd, N, row_ptr, col_idx, s_values, A,
-                                                               lda, B, ldb, D, ldd, O, ldo, order, gate, M, clear);
+        launch_row(fusedmm_row_scalar_kernel, grid, 0, st, gate != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
+                   D, ldd, O, ldo, order, gate, M, clear);
     }
     return check_launch();
 }

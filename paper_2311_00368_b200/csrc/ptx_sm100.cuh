@@ -118,6 +118,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     return false;
 }
 
+// ---- programmatic dependent launch --------------------------------------------------------------------
+// Lets the grids that were launched as programmatic dependents of this one start (once every CTA has
+// called it or exited).  They see what grids that completed before this one wrote, not this grid's writes.
+__device__ __forceinline__ void launch_dependents()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ---- fences ---------------------------------------------------------------------------------------
 // Makes this thread's generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05).
 __device__ __forceinline__ void fence_proxy_async_smem()

@@ -228,7 +228,8 @@ b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &
 
 // Splits one or two dense operands (job 1 optional), clears the device status word and optionally
 // zero-fills an output matrix.
-void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int *status, cudaStream_t st)
+void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int *status, const TableCheck &chk,
+                  cudaStream_t st)
 {
     auto groups = [](const SplitJob &j) { return (long long)j.rows_p * (j.cols_p >> 2); };
     long long most = groups(j0);
@@ -236,7 +237,7 @@ void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int 
     const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
     const int njobs = j1 ? 2 : 1;
     dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(njobs + (z.out ? 1 : 0)));
-    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, njobs, z, status);
+    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, njobs, z, status, chk);
 }
 
 }  // namespace
@@ -279,9 +280,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), p.Mt * p.Nt, 1, p.Mt * p.Nt}
                                             : ZeroJob{nullptr, 0, 0, 0};
         int *clear = keep_status ? nullptr : status;
-        if (spmm) launch_split(jd, nullptr, z, clear, st);
-        else if (fused) launch_split(jb, &jd, z, clear, st);
-        else launch_split(jb, nullptr, z, clear, st);
+        // (a prepared table is checked against this call's arrays here, so that the flags are final before the tile kernel)
+        const TableCheck chk{PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx},
+                             prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags};
+        if (spmm) launch_split(jd, nullptr, z, clear, chk, st);
+        else if (fused) launch_split(jb, &jd, z, clear, chk, st);
+        else launch_split(jb, nullptr, z, clear, chk, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;

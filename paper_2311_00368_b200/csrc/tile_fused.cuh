@@ -153,11 +153,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
     constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
-    if (a.flags[0] != 0) return;  // pattern not usable for tiles: the row kernels take over
-    if (!signature_matches(a.sig_want, a.sig_have)) {   // stale or foreign table (uniform over the grid)
-        if (threadIdx.x == 0) atomicExch(&a.flags[kFlagUnsorted], 1);
-        return;
-    }
+    // The flags are final before this kernel starts (the pre-pass or, for a prepared table, the operand-split
+    // kernel's signature check wrote them): the gated row kernel launched behind this one may run beside it.
+    const bool unusable = a.flags[0] != 0;
+    ptx::launch_dependents();
+    if (unusable) return;  // pattern not usable for tiles: the row kernels take over
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;

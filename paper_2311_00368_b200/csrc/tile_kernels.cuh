@@ -169,9 +169,21 @@ struct ZeroJob {
     int cols;
 };
 
-__global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status)
+// It also compares the signature stored beside a prepared window table with the arrays of this call
+// (`sig_have` != NULL) and raises the fallback flag on a mismatch: the flags are then final before the tile
+// kernel starts, which lets the gated fallback run beside it.
+struct TableCheck {
+    PatternSignature want;
+    const PatternSignature *have;   // NULL: nothing to check (the table was built by this call)
+    int *flags;
+};
+
+__global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
 {
-    if (status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *status = 0;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        if (status) *status = 0;
+        if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
+    }
     if ((int)blockIdx.y == njobs) {   // zero-fill job
         const long long total = (long long)z.rows * z.cols;
         const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
