@@ -126,6 +126,12 @@ __device__ __forceinline__ void launch_dependents()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Waits until the grids this one programmatically depends on have completed and their writes are visible.
+__device__ __forceinline__ void wait_for_primary_grid()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // ---- fences ---------------------------------------------------------------------------------------
 // Makes this thread's generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05).
 __device__ __forceinline__ void fence_proxy_async_smem()

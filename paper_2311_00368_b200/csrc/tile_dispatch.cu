@@ -212,7 +212,18 @@ b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, cons
     auto kern = fused_tile_kernel<KDP, MODE>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
         return B2SP_ERR_CUDA;
-    kern<<<items, Cfg::THREADS, Cfg::SMEM_BYTES, st>>>(bh, bl, dh, dl, out, a);
+    // a programmatic dependent of the operand-split kernel: its CTAs are placed while that kernel still runs
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)items);
+    cfg.blockDim = dim3(Cfg::THREADS);
+    cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kern, bh, bl, dh, dl, out, a);
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 

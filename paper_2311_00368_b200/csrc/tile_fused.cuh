@@ -155,6 +155,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
     // The flags are final before this kernel starts (the pre-pass or, for a prepared table, the operand-split
     // kernel's signature check wrote them): the gated row kernel launched behind this one may run beside it.
+    ptx::wait_for_primary_grid();   // the operand-split kernel before this one: its copies and its flag
     const bool unusable = a.flags[0] != 0;
     ptx::launch_dependents();
     if (unusable) return;  // pattern not usable for tiles: the row kernels take over

@@ -180,6 +180,7 @@ struct TableCheck {
 
 __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
 {
+    ptx::launch_dependents();   // the tile kernel may take its SMs; it waits for this grid before it reads anything
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
         if (status) *status = 0;
         if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
