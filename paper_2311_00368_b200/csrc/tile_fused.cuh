@@ -153,13 +153,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
     constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
-    // The flags are final before this kernel starts (the pre-pass or, for a prepared table, the operand-split
-    // kernel's signature check wrote them): the gated row kernel launched behind this one may run beside it.
-    ptx::wait_for_primary_grid();   // the operand-split kernel before this one: its copies and its flag
-    const bool unusable = a.flags[0] != 0;
-    ptx::launch_dependents();
-    if (unusable) return;  // pattern not usable for tiles: the row kernels take over
-
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -269,6 +262,22 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
+
+    // Everything above (barriers, tensor memory, the A tile: none of it written by the kernel before) ran
+    // while the operand-split kernel, whose programmatic dependent this grid is, was still at work.  Its tf32
+    // copies and its verdict on a prepared table are needed from here on.  After it the flags are final (the
+    // pre-pass or that kernel's signature check wrote them), so the gated row kernel launched behind this
+    // grid may run beside it.
+    ptx::wait_for_primary_grid();
+    const bool unusable = a.flags[0] != 0;
+    ptx::launch_dependents();
+    if (unusable) {   // pattern not usable for tiles: the row kernels take over
+        if (warp == 1) {
+            __syncwarp();
+            ptx::tmem_dealloc(tmem, 512);
+        }
+        return;
+    }
 
     if (warp == kFusedTmaWarp) {
         // ---------------- TMA producer: per block NCH_B chunks of B rows, then NCH_D chunks of D rows ----------------
