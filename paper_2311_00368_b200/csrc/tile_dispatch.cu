@@ -248,7 +248,16 @@ void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int 
     const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
     const int njobs = j1 ? 2 : 1;
     dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(njobs + (z.out ? 1 : 0)));
-    split_dense_kernel<<<grid, 256, 0, st>>>(j0, j1 ? *j1 : j0, njobs, z, status, chk);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(256);
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = chk.after_prepass ? attr : nullptr;   // beside the pattern pre-pass of the same call, never beside foreign work
+    cfg.numAttrs = chk.after_prepass ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, split_dense_kernel, j0, j1 ? *j1 : j0, njobs, z, status, chk);
 }
 
 }  // namespace
@@ -293,7 +302,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         int *clear = keep_status ? nullptr : status;
         // (a prepared table is checked against this call's arrays here, so that the flags are final before the tile kernel)
         const TableCheck chk{PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx},
-                             prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags};
+                             prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags,
+                             prepared ? 0 : 1};
         if (spmm) launch_split(jd, nullptr, z, clear, chk, st);
         else if (fused) launch_split(jb, &jd, z, clear, chk, st);
         else launch_split(jb, nullptr, z, clear, chk, st);

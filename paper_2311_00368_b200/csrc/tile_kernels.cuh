@@ -49,6 +49,9 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
                   PatternSignature sig, PatternSignature *__restrict__ sig_out)
 {
     extern __shared__ __align__(16) unsigned mask[];     // Wk words
+    // (inside a stateless tile op the operand-split kernel is launched as a programmatic dependent of this
+    // one: the two touch different data and may overlap; that kernel waits for this grid before it ends)
+    ptx::launch_dependents();
     if (blockIdx.x == 0 && threadIdx.x == 0) *sig_out = sig;   // what the table is built from
     __shared__ int warp_total[kMasksWarps];
     constexpr unsigned kFull = 0xffffffffu;
@@ -176,6 +179,8 @@ struct TableCheck {
     PatternSignature want;
     const PatternSignature *have;   // NULL: nothing to check (the table was built by this call)
     int *flags;
+    int after_prepass;              // launched as a programmatic dependent of the pattern pre-pass of the same call:
+                                    // this grid must not complete before that one (the tile kernel waits for this grid only)
 };
 
 __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
@@ -194,6 +199,7 @@ __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob 
         } else {
             for (long long i = t0; i < total; i += step) z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
         }
+        if (chk.after_prepass) ptx::wait_for_primary_grid();
         return;
     }
     const SplitJob j = blockIdx.y ? j1 : j0;
@@ -223,6 +229,7 @@ __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob 
         reinterpret_cast<uint4 *>(j.hi)[g] = make_uint4(h[0], h[1], h[2], h[3]);
         reinterpret_cast<uint4 *>(j.lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
     }
+    if (chk.after_prepass) ptx::wait_for_primary_grid();
 }
 
 }  // namespace b2sp
