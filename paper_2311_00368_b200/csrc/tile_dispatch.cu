@@ -317,8 +317,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.flags = flags; a.status = status;
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
     a.O = out; a.ldo = ldo;
-    a.sig_want = PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx};
-    a.sig_have = reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset);
     a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }

@@ -88,8 +88,6 @@ struct FusedTileArgs {
     long long ldo;
     int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
     int *flags;                // flags[0] != 0: the table cannot be used, the row kernels take over
-    PatternSignature sig_want; // the arrays this call was given ...
-    const PatternSignature *sig_have;   // ... and what the table in the workspace was built from
     int *status;
     unsigned long long *prof;  // optional role timers (profiling builds only)
 };

@@ -173,7 +173,7 @@ struct ZeroJob {
 };
 
 // It also compares the signature stored beside a prepared window table with the arrays of this call
-// (`sig_have` != NULL) and raises the fallback flag on a mismatch: the flags are then final before the tile
+// (`chk.have` != NULL) and raises the fallback flag on a mismatch: the flags are then final before the tile
 // kernel starts, which lets the gated fallback run beside it.
 struct TableCheck {
     PatternSignature want;
