@@ -58,7 +58,18 @@ b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t
     if (cudaMemsetAsync(w.count, 0, 512, st) != cudaSuccess) return B2SP_ERR_CUDA;
     int blocks = (M + 255) / 256;
     bin_count_kernel<<<blocks, 256, 0, st>>>(M, row_ptr, w.count);
-    bin_scatter_kernel<<<blocks, 256, 0, st>>>(M, row_ptr, w.count, w.cursor, w.row_order);
+    {   // a programmatic dependent of the counting kernel (it waits for the counts where it needs them)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, bin_scatter_kernel, M, row_ptr, (const int *)w.count, w.cursor, w.row_order);
+    }
     *launches += 2;
     return check_launch();
 }
@@ -66,9 +77,10 @@ b2sp_status bin_rows(int M, const int *row_ptr, const Workspace &w, cudaStream_t
 // Launches `kern`; a gated launch (the row family as the dense-tile family's device-side fallback) is marked as a
 // programmatic dependent of the tile kernel before it: the tile kernel lets its dependents go as soon
 // as it has read the gate's flags, which are final before it starts, so the fallback (which almost always
-// finds its gate closed and exits) runs beside the tile kernel instead of after it.
+// finds its gate closed and exits) runs beside the tile kernel instead of after it.  A launch behind the binning
+// pass (`order` given) is a programmatic dependent of it too: the kernel waits for the row order at its top.
 template <class... KArgs, class... Args>
-inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStream_t st, bool gated, Args... args)
+inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStream_t st, bool dependent, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -78,8 +90,8 @@ inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStrea
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = gated ? attr : nullptr;
-    cfg.numAttrs = gated ? 1 : 0;
+    cfg.attrs = dependent ? attr : nullptr;
+    cfg.numAttrs = dependent ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
@@ -98,7 +110,7 @@ void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const in
 {
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    launch_row(spmm_row_kernel<U, SPLIT>, grid, 0, st, gate != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+    launch_row(spmm_row_kernel<U, SPLIT>, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
                gate, nrows, clear);
 }
 
@@ -123,7 +135,7 @@ void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const 
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    launch_row(sddmm_row_kernel<KU>, grid, smem, st, gate != nullptr, Kd, row_ptr, col_idx, sv, A, lda, B, ldb, out, order,
+    launch_row(sddmm_row_kernel<KU>, grid, smem, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, sv, A, lda, B, ldb, out, order,
                gate, nrows, clear);
 }
 
@@ -144,7 +156,7 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     }
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    launch_row(kern, grid, smem, st, gate != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
+    launch_row(kern, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
                nrows, clear);
     return B2SP_OK;
 }
@@ -271,7 +283,7 @@ static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_id
         else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
-        launch_row(spmm_row_scalar_kernel, grid, 0, st, gate != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+        launch_row(spmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
                    gate, M, clear);
     }
     return check_launch();
@@ -352,7 +364,7 @@ static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_
         }
     } else {
         grid.x = gated_blocks(grid.x, gate);
-        launch_row(sddmm_row_scalar_kernel, grid, 0, st, gate != nullptr, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb,
+        launch_row(sddmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb,
                    out_values, order, gate, M, clear);
     }
     return check_launch();
@@ -434,7 +446,7 @@ static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const in
         if (rc != B2SP_OK) return rc;
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
-        launch_row(fusedmm_row_scalar_kernel, grid, 0, st, gate != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
+        launch_row(fusedmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
                    D, ldd, O, ldo, order, gate, M, clear);
     }
     return check_launch();

@@ -28,9 +28,15 @@ constexpr unsigned kFull = 0xffffffffu;
 // ------------------------------------------------------------------------------------------
 __device__ __forceinline__ int bucket_of(int len) { return len <= 0 ? 0 : 32 - __clz(len); }
 
+// Programmatic dependent launches: the binning kernels and the row kernel that follows them are chained so
+// that each is placed, and does what does not need its predecessor's output, while the predecessor runs.
+__device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void grid_wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __global__ void bin_count_kernel(int M, const int *__restrict__ row_ptr, int *__restrict__ count)
 {
     __shared__ int h[kBuckets];
+    grid_release_dependents();
     if (threadIdx.x < kBuckets) h[threadIdx.x] = 0;
     __syncthreads();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
@@ -54,6 +60,8 @@ __global__ void bin_scatter_kernel(int M, const int *__restrict__ row_ptr,
         r = atomicAdd(&h[b], 1);
     }
     __syncthreads();
+    grid_wait_for_primary();     // the counts of the whole matrix (bin_count_kernel)
+    grid_release_dependents();   // the row kernel behind this one waits for this grid before it reads the order
     if (threadIdx.x < kBuckets) {
         int mine = threadIdx.x, start = 0;
         for (int j = kBuckets - 1; j > mine; --j) start += count[j];
@@ -181,6 +189,7 @@ spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ 
     __shared__ float4 red[kRowWarps * U * G::LPN];
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int sub = lane / G::LPN, sl = lane % G::LPN;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
@@ -233,6 +242,7 @@ spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__rest
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
@@ -337,6 +347,7 @@ sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict_
     float *a_smem = reinterpret_cast<float *>(dyn_smem);
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
@@ -364,6 +375,7 @@ sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__re
 {
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
         const int beg = row_ptr[row], end = row_ptr[row + 1];
@@ -394,6 +406,7 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
     extern __shared__ float4 dyn_smem[];
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     float4 *red = dyn_smem;                                                   // kRowWarps*U*LPN
     float *a_smem = reinterpret_cast<float *>(dyn_smem + kRowWarps * U * G::LPN);  // Kd (KU == 0)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -446,6 +459,7 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
     __shared__ float red[kRowWarps][128];
     if (gate && *gate == 0) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
+    if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
