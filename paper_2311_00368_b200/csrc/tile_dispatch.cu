@@ -133,13 +133,15 @@ bool tile_profitable(int op, int M, int K, int width, long long nnz)
     // 4.5% on large matrices and rises as the matrix shrinks (16% at 2048^2, never at 1024^2).
     // Operands narrower than 64 use half of a 64-wide tile at best while the row kernels lose nothing
     // (sub-warps share a row): measured at width 32 on 1k^2 ... 32k x 8k, the cross-over is about 3.5x
-    // higher for SPMM, 2x for SDDMM, 2.2x for FusedMM.  With 74 or more row tiles (no K split) the last
+    // higher for SPMM, 2x for SDDMM, 2.5x for FusedMM.  With 74 or more row tiles (no K split) the last
     // wave of CTAs is partly empty (96 tiles: 65% of the SMs; 192 tiles: two waves, 65%), which the tile
     // family pays in full: the cross-over rises by the waves' efficiency against the usual 86%.
     if (M < 256 || K < 256 || width < 16 || nnz <= 0) return false;
     const double cells = (double)M * (double)K;
     const double density = (double)nnz / cells;
-    double crossover = 0.045 + 0.5e6 / cells;
+    // (FusedMM's row kernel does the work of two ops per stored entry, its tile kernel shares the expansion of S
+    // between them: a fit over the 72 grid cases puts its cross-over lower)
+    double crossover = op == B2SP_OP_FUSEDMM ? 0.035 + 0.3e6 / cells : 0.045 + 0.5e6 / cells;
     const int tiles = (M + kFusedRows - 1) / kFusedRows;
     if (tiles >= kSMs / 2 && width <= kFusedNT) {
         const int waves = (tiles + kSMs - 1) / kSMs;
@@ -147,7 +149,7 @@ bool tile_profitable(int op, int M, int K, int width, long long nnz)
         const double factor = 0.86 / eff;
         crossover *= factor < 1.0 ? 1.0 : factor > 1.35 ? 1.35 : factor;
     }
-    const double narrow = op == B2SP_OP_SPMM ? 3.5 : op == B2SP_OP_SDDMM ? 2.0 : 2.2;
+    const double narrow = op == B2SP_OP_SPMM ? 3.5 : op == B2SP_OP_SDDMM ? 2.0 : 2.5;
     return density >= (width >= 64 ? crossover : narrow * crossover);
 }
 
