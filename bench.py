@@ -194,6 +194,111 @@ def parity_on_sample(p, rows, gpu_spmm, gpu_sddmm, gpu_fused):
     return out
 
 
+def time_calls(torch, stream, flush, fn, reps):
+    """Mean and minimum device time (ms) of `fn` over `reps` calls, L2 flushed (untimed) before each."""
+    ev = []
+    for _ in range(reps):
+        flush.fill_(1)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        fn()
+        e1.record(stream)
+        ev.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(z) for a, z in ev]
+    return float(np.mean(ms)), float(np.min(ms))
+
+
+def measure_problems(torch, b, device, flush, problems, ops, fp32_peak_gflops, hbm_gbs, reps, check=True):
+    """One entry of the bench line's `configs` object: the given ops on a list of independent problems of one
+    configuration (eight for the attention-shaped one, else one), per op summed over the problems.  Same
+    protocol as the headline: L2 flushed before every call, CUDA events on the launching stream.  Three
+    timings per op: the window table of S prepared once and reused (`ms`), a stateless call that rebuilds it
+    (`stateless_ms`), and the CUDA-core row family (`row_ms`).  Every output of the prepared calls is
+    checked against the oracle, every element."""
+    import oracle
+    stream = torch.cuda.current_stream()
+    dev = lambda x: None if x is None else torch.from_numpy(np.ascontiguousarray(x)).to(device)
+    out = {"problems": len(problems), "ops": {}}
+    acc = {op: {"ms": 0.0, "ms_min": 0.0, "stateless_ms": 0.0, "row_ms": 0.0, "flops": 0, "bytes": 0, "worst": 0.0,
+                "ok": True, "algo": None, "launches": 0} for op in ops}
+    for p in problems:
+        rp, ci, v, A, B, D = map(dev, (p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D))
+        O = torch.empty((p.M, max(p.N, 1)), dtype=torch.float32, device=device)
+        C = torch.empty(p.nnz, dtype=torch.float32, device=device)
+        ws = torch.empty(max(b.workspace_bytes(i, p.M, p.K, p.Kd, p.N, p.nnz) for i in range(3)),
+                         dtype=torch.uint8, device=device)
+        calls = {"spmm": lambda a: b.spmm(rp, ci, v, D, K=p.K, out=O, workspace=ws, algo=a),
+                 "sddmm": lambda a: b.sddmm(rp, ci, v, A, B, out=C, workspace=ws, algo=a),
+                 "fusedmm": lambda a: b.fusedmm(rp, ci, v, A, B, D, out=O, workspace=ws, algo=a)}
+        for op in ops:
+            i = OPS.index(op)
+            calls[op](b.ALGO_AUTO)
+            torch.cuda.synchronize()
+            auto = b.last_algo(i)
+            a = acc[op]
+            a["algo"] = b.ALGO_NAMES[auto]
+            if auto == b.ALGO_TILE:
+                b.prepare_pattern(rp, ci, p.K, ws)
+                fn = lambda: calls[op](b.ALGO_TILE_PREPARED)
+            else:
+                fn = lambda: calls[op](b.ALGO_AUTO)
+            for _ in range(3):
+                fn()
+            mean, mn = time_calls(torch, stream, flush, fn, reps)
+            a["launches"] += b.last_launches(i)
+            a["ms"] += mean
+            a["ms_min"] += mn
+            if check:
+                got = (C if op == "sddmm" else O).cpu().numpy()
+                if op == "spmm":
+                    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+                elif op == "sddmm":
+                    ref, T = oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B)
+                else:
+                    ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)
+                ok, ratio = oracle.within_tolerance(got, ref, T)
+                a["ok"] = a["ok"] and bool(ok) and b.device_status(ws) == 0
+                a["worst"] = max(a["worst"], float(ratio))
+            fn = lambda: calls[op](b.ALGO_AUTO)
+            for _ in range(3):
+                fn()
+            a["stateless_ms"] += time_calls(torch, stream, flush, fn, reps)[0]
+            fn = lambda: calls[op](b.ALGO_ROW)
+            fn()
+            a["row_ms"] += time_calls(torch, stream, flush, fn, max(3, reps // 4))[0]
+            a["flops"] += W.flops(op, p.nnz, p.Kd, p.N)
+            a["bytes"] += W.compulsory_bytes(op, p.M, p.K, p.nnz, p.Kd, p.N)
+        del rp, ci, v, A, B, D, O, C, ws
+    for op, a in acc.items():
+        t_alu = a["flops"] / (fp32_peak_gflops * 1e9)
+        t_hbm = a["bytes"] / (hbm_gbs * 1e9)
+        t_roof = max(t_alu, t_hbm)
+        out["ops"][op] = {"ms": round(a["ms"], 4), "ms_min": round(a["ms_min"], 4),
+                          "roofline_frac": round(t_roof / (a["ms"] * 1e-3), 4),
+                          "roofline_bound": "alu" if t_alu >= t_hbm else "hbm",
+                          "gflops": round(a["flops"] / a["ms"] / 1e6, 1),
+                          "algo": a["algo"] + (" (window table prepared once)" if a["algo"] == "tile" else ""),
+                          "launches": a["launches"],
+                          "stateless_ms": round(a["stateless_ms"], 4),
+                          "stateless_roofline_frac": round(t_roof / (a["stateless_ms"] * 1e-3), 4),
+                          "row_family_ms": round(a["row_ms"], 4),
+                          "parity_ok": a["ok"] if check else None,
+                          "parity_worst_error_over_allowed": round(a["worst"], 4) if check else None}
+    return out
+
+
+# The "largest configurations" besides the headline workload: SPMM config, SDDMM config, the eight
+# attention-shaped problems, and the 30% sweep points at the wider outputs.
+EXTRA_CONFIGS = (
+    ("spmm_2048_d20_n256", lambda: [W.spmm_case()], ("spmm",)),
+    ("sddmm_4096_d10_kd128", lambda: [W.sddmm_case()], ("sddmm",)),
+    ("attention_8x4096_d20_hd64", lambda: [W.attention_case(i) for i in range(8)], ("fusedmm", "sddmm", "spmm")),
+    ("sweep_d30_n256", lambda: [W.sweep_case(0.3, 256)], OPS),
+    ("sweep_d30_n512", lambda: [W.sweep_case(0.3, 512)], OPS),
+)
+
+
 def run_reference(args):
     rank, _, world = replicas.env_world()
     if rank != 0:
@@ -320,7 +425,7 @@ def run_grid(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=400)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="sweep_d30_n128")
     ap.add_argument("--impl", default="b200", choices=["b200", "reference"])
@@ -329,6 +434,9 @@ def main():
                     help="every op rebuilds S's window table itself instead of sharing one per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the `configs` object (the other large configurations, timed beside the headline workload)")
+    ap.add_argument("--config-reps", type=int, default=50, help="timed calls per op of the `configs` object")
     ap.add_argument("--min-warmup", type=int, default=3,
                     help="lower bound on warm-up steps (only profiler captures go below 3)")
     ap.add_argument("--grid", action="store_true",
@@ -460,6 +568,19 @@ def main():
         warm = [a.elapsed_time(z) for a, z in ev]
         per_op[op]["warm_ms_min"] = round(float(np.min(warm)), 4)
         per_op[op]["warm_ms_median"] = round(float(np.median(warm)), 4)
+    # the same ops as stateless calls (each builds S's window table itself), L2 flushed before every call
+    if shared_table:
+        for i, op in enumerate(OPS):
+            fn = lambda op=op: probe[op](b.ALGO_AUTO)
+            for _ in range(3):
+                fn()
+            mean, mn = time_calls(torch, stream, flush, fn, 20)
+            t_roof = max(fl[op] / (fp32_peak_gflops * 1e9), by[op] / (hbm_gbs * 1e9))
+            per_op[op]["stateless_ms"] = round(mean, 4)
+            per_op[op]["stateless_roofline_frac"] = round(t_roof / (mean * 1e-3), 4)
+            per_op[op]["stateless_launches"] = b.last_launches(i)
+        step()   # the outputs the parity check reads come from the timed configuration (prepared table)
+        torch.cuda.synchronize()
     sep_ms = per_op["sddmm"]["ms"] + per_op["spmm"]["ms"]
     fused_vs_separate = sep_ms / per_op["fusedmm"]["ms"]
 
@@ -484,6 +605,11 @@ def main():
     roof["fp32_fma_probe"] = {"tflops": probe_gflops / 1e3, "achieved_over_probe": fl[dom] / dom_ms / 1e6 / probe_gflops,
                               "how": "b2sp_probe_fp32_peak: 8 FMA chains x 2048 threads x every SM, CUDA events, best of 10"}
     roof["traffic"] = MEASURED_TRAFFIC_BYTES.get((args.workload, algos[dom]))
+    roof["traffic_source"] = ("one ncu capture of this kernel on this workload (dram__bytes_read.sum + dram__bytes_write.sum, "
+                              "summary under profiles/), not measured in this run" if roof["traffic"] else None)
+    roof["variant"] = ("window table of S prepared once per step and shared by the three ops (its pass is timed inside the "
+                       "step and listed under ops.prepare_pattern); ops.*.stateless_* = the same op building the table itself"
+                       if shared_table else "stateless calls")
     roof["algorithmic_bytes"] = by[dom]
     roof["algorithmic_flops"] = fl[dom]
 
@@ -520,6 +646,22 @@ def main():
                "d2h_bytes_per_step": d2h, "ms_per_step": t_e2e * 1e3, "steps": e2e_steps,
                "timer": "host wall clock around synchronous C-ABI calls"}
 
+    # the other large configurations, same protocol
+    configs, configs_clocks = None, None
+    if rank == 0 and world == 1 and not args.no_configs:
+        sampler2 = ClockSampler(local_rank)
+        sampler2.start()
+        configs = {}
+        for cname, make, cops in EXTRA_CONFIGS:
+            configs[cname] = measure_problems(torch, b, device, flush, make(), cops, fp32_peak_gflops, hbm_gbs,
+                                              args.config_reps, check=not args.no_cpu_baseline)
+            if set(("sddmm", "spmm", "fusedmm")) <= set(cops):
+                o = configs[cname]["ops"]
+                configs[cname]["fused_speedup_over_separate_launches"] = round(
+                    (o["sddmm"]["ms"] + o["spmm"]["ms"]) / o["fusedmm"]["ms"], 3)
+            torch.cuda.empty_cache()
+        configs_clocks = sampler2.stop()
+
     cpu_baseline, parity = None, None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_baseline, _ = oracle_sample(p, 15.0)
@@ -530,13 +672,15 @@ def main():
         line = {"metric": "SPMM+SDDMM+FusedMM GFLOP/s (2*nnz*width per stage)", "value": value,
                 "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, args.min_warmup),
                 "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-                "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "vs_baseline": None, "dtype": ("f32 in/out, 3xTF32 products, fp32 accumulate"
+                                              if any(a == "tile" for a in algos.values()) else "f32"),
+                "data": "synthetic",
                 "config": dict(workload_config(p, args.workload),
                                pattern_table="built once per step, shared by the ops" if shared_table
                                else "built inside each op that needs it"),
                 "roofline": roof, "cpu_baseline": cpu_baseline, "parity": parity,
                 "e2e": e2e, "gpu_launches": int((sum(launches.values()) + (1 if shared_table else 0)) * args.steps),
-                "clocks": clocks, "ops": per_op,
+                "clocks": clocks, "ops": per_op, "configs": configs, "configs_clocks": configs_clocks,
                 "fused_speedup_over_separate_launches": round(fused_vs_separate, 3),
                 "paper_context": "Intel Max 1550 (1 stack), 8k/8k/128/70%: SDDMM 9732, SPMM 11482, "
                                  "FusedMM 12647 GFLOP/s (other hardware; context only)"}

@@ -43,6 +43,16 @@
  *                      earlier b2sp_prepare_pattern call for the same S left it (see there).
  * Floating-point results of the families differ in summation order only; all stay within
  * |x - exact| <= 1e-5 * sum|terms| + 1e-6.
+ *
+ * Non-finite inputs.  The row kernels touch exactly the entries Eq. 1-3 name and follow IEEE
+ * propagation.  The dense-tile kernels multiply whole windows of S, positions without a stored entry
+ * included (by zero), so they only run when every element of A, B and D -- referenced by a stored
+ * entry or not -- is finite and small enough for its tf32 hi part to be finite (|x| below about
+ * 3.4e38 * (1 - 2^-11)): the operand pre-pass of every call checks this on the device, and otherwise
+ * the row kernels produce that call's result (the check is per call and costs no extra launch).
+ * Not checked, and undefined (NaN or Inf) on the dense-tile kernels: stored values s_p that are not
+ * finite, and inputs so large that a dot product A_i . B_j overflows fp32 at ANY position (i, j) of
+ * a 128 x 128 tile of S that holds a stored entry, stored there or not.
  */
 #ifndef B2SP_H
 #define B2SP_H
@@ -88,16 +98,6 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz);
  * family's (0 if these sizes are outside that family).  Returns 0 on invalid arguments.
  */
 size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz);
-
-/*
- * Measurement aid with no counterpart in the paper: the FP32 FMA rate the current device sustains
- * right now (8 independent register-only FMA chains per thread, 2048 threads on every SM, best of 10
- * launches timed with CUDA events), in GFLOP/s, for the denominator of a roofline fraction.
- * `iters` = chain length in units of 64 FMAs per thread (4096 takes about a millisecond);
- * `scratch` = DEVICE pointer to at least one float (never written in practice); `gflops_host` =
- * HOST pointer for the result.  Synchronises `stream`.  B2SP_ERR_INVALID_ARG / B2SP_ERR_CUDA.
- */
-b2sp_status b2sp_probe_fp32_peak(int iters, float *scratch, double *gflops_host, void *stream);
 
 /*
  * Pattern analysis shared by the dense-tile kernels of all three ops (work assignment and index
@@ -164,8 +164,11 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz,
  * makes the copies asynchronous and faster, pageable memory also works).  Each call copies
  * its inputs to the device, runs the device entry point above with algo = B2SP_ALGO_AUTO,
  * copies the result back and synchronises `stream` before returning.  Device memory comes
- * from the stream-ordered CUDA memory pool (cudaMallocAsync) and is returned to it before the
- * call ends.  Dense operands are contiguous (ld = number of columns).
+ * from a stream-ordered memory pool that the library creates for itself on each device at first
+ * use (the process's default pool and its settings are not touched) and is returned to that pool
+ * before the call ends; the pool keeps freed blocks for the next call.  Dense operands are
+ * contiguous (ld = number of columns).  The workspace's device status word is read back with the
+ * result: B2SP_ERR_TIMEOUT if a bounded wait inside a kernel gave up (outputs undefined).
  */
 b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz,
                            const int *row_ptr, const int *col_idx, const float *values,
@@ -194,11 +197,14 @@ b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz,
  * Limits and rules:
  *   - M <= B2SP_STATIC_SCRATCH_MAX_ROWS, otherwise B2SP_ERR_TOO_LARGE and nothing is enqueued.
  *     K, N and nnz are unrestricted.
- *   - The array (512 bytes + 4 bytes per row of the limit, about 257 KiB) occupies device memory on
- *     every GPU that loads the library, until the process exits, used or not.
- *   - The first call on each device looks up the array's device address (a host-side runtime
- *     query, no allocation).  Make that first call with the device current and before starting any
- *     stream capture on it.
+ *   - The array (512 bytes + 4 bytes per row of the limit, about 257 KiB) is part of the library's
+ *     device image: every GPU on which the image gets loaded holds it until the process exits.
+ *   - The first call on each device looks up the array's device address.  With CUDA's lazy module
+ *     loading that look-up is also what loads the library's device image on that GPU, and the
+ *     driver reserves room for the array (and the code) at that moment; it may synchronise the
+ *     device.  So make the first call at start-up: with the device current, BEFORE the host
+ *     process's arena takes the remaining device memory, outside any latency-critical loop and
+ *     before starting any stream capture.  Later calls on that device do no such work.
  *   - All calls on a device share the one array, and it keeps whatever the previous call left.  The
  *     part that must start from zero is cleared at the start of each call, so back-to-back calls on
  *     one stream are fine; two calls that can overlap on the GPU (different streams, or different
@@ -227,14 +233,6 @@ b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, c
  * kernel gave up (the outputs of that call are then undefined).
  */
 b2sp_status b2sp_device_status(const void *workspace, void *stream);
-
-/*
- * Which kernel family the most recent call of the given op on this host thread resolved
- * B2SP_ALGO_AUTO (or its explicit request) to: one of B2SP_ALGO_ROW, _ROW_NAT, _TILE; -1 if the
- * op has not been called.  Number of kernels that call enqueued: b2sp_last_launches(op).
- */
-int b2sp_last_algo(int op);
-int b2sp_last_launches(int op);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,45 @@
+/*
+ * b2sp -- measurement, test and tuning aids.  Not part of the method of the paper (no passage of it
+ * corresponds to anything here) and not needed to use the three ops of b2sp.h; exported by the same
+ * library.
+ */
+#ifndef B2SP_DEBUG_H
+#define B2SP_DEBUG_H
+
+#include "b2sp.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/*
+ * The FP32 FMA rate the current device sustains right now (8 independent register-only FMA chains
+ * per thread, 2048 threads on every SM, best of 10 launches timed with CUDA events), in GFLOP/s, for
+ * the denominator of a roofline fraction.
+ * `iters` = chain length in units of 64 FMAs per thread (4096 takes about a millisecond);
+ * `scratch` = DEVICE pointer to at least one float (never written in practice); `gflops_host` =
+ * HOST pointer for the result.  Synchronises `stream`.  B2SP_ERR_INVALID_ARG / B2SP_ERR_CUDA.
+ */
+b2sp_status b2sp_probe_fp32_peak(int iters, float *scratch, double *gflops_host, void *stream);
+
+/*
+ * Which kernel family the most recent call of the given op (B2SP_OP_*) on this host thread resolved
+ * B2SP_ALGO_AUTO (or its explicit request) to: one of B2SP_ALGO_ROW, _ROW_NAT, _TILE; -1 if the
+ * op has not been called.  Number of kernels that call enqueued: b2sp_last_launches(op).
+ */
+int b2sp_last_algo(int op);
+int b2sp_last_launches(int op);
+
+/*
+ * Overrides, process-wide, the number of K splits the dense-tile planner picks (how many CTAs share
+ * one tile of the output along the columns of S); 0 gives the choice back to the planner.  A value
+ * larger than the number of 128-column blocks of S is ignored.  It changes b2sp_workspace_bytes for
+ * the dense-tile family and the order of the floating-point sums, so set it before sizing the
+ * workspace.  For tests of the K-split epilogues and for tuning only.
+ */
+void b2sp_debug_force_k_splits(int k_splits);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* B2SP_DEBUG_H */

@@ -6,7 +6,7 @@ raises on a non-zero status.  There is no CPU fallback: importing this module ra
 ``ImportError`` if the library has not been built, and calling an op without a CUDA device
 fails in the library.
 
-Function names and argument order follow ``include/b2sp.h``.
+Function names and argument order follow ``include/b2sp.h`` (and ``include/b2sp_debug.h``).
 """
 from __future__ import annotations
 
@@ -65,6 +65,8 @@ lib.b2sp_last_algo.restype = _i
 lib.b2sp_last_algo.argtypes = [_i]
 lib.b2sp_last_launches.restype = _i
 lib.b2sp_last_launches.argtypes = [_i]
+lib.b2sp_debug_force_k_splits.restype = None
+lib.b2sp_debug_force_k_splits.argtypes = [_i]
 
 
 class B2spError(RuntimeError):
@@ -139,6 +141,11 @@ def last_algo(op: int) -> int:
 
 def last_launches(op: int) -> int:
     return int(lib.b2sp_last_launches(op))
+
+
+def debug_force_k_splits(k_splits: int) -> None:
+    """b2sp_debug_force_k_splits: override the dense-tile planner's K split (0 = planner's choice)."""
+    lib.b2sp_debug_force_k_splits(int(k_splits))
 
 
 def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALGO_AUTO):

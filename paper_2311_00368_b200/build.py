@@ -25,8 +25,9 @@ def sources():
 
 
 def _deps():
-    return sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + [
-        os.path.join(os.path.dirname(HERE), "include", "b2sp.h"), os.path.abspath(__file__)]
+    return sources() + glob.glob(os.path.join(CSRC, "*.cuh")) + glob.glob(os.path.join(CSRC, "*.h")) + [
+        os.path.join(os.path.dirname(HERE), "include", "b2sp.h"),
+        os.path.join(os.path.dirname(HERE), "include", "b2sp_debug.h"), os.path.abspath(__file__)]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

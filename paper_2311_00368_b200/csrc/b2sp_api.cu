@@ -1,10 +1,11 @@
 // C-ABI entry points of libb2sp: argument checks, workspace carving, kernel dispatch.
-// See include/b2sp.h for the contract of every function.
-#include "../../include/b2sp.h"
+// See include/b2sp.h (and include/b2sp_debug.h) for the contract of every function.
+#include "../../include/b2sp_debug.h"
 
 #include <climits>
 #include <cstdlib>
 #include <cstdint>
+#include <mutex>
 
 #include "row_kernels.cuh"
 #include "tile_dispatch.h"
@@ -97,7 +98,7 @@ inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStrea
 
 // A gated launch (the row family as the dense-tile family's fallback) almost always finds its gate
 // closed: it gets a small grid whose blocks walk the rows, so that the usual case costs little.
-inline unsigned gated_blocks(unsigned rows, const int *gate)
+inline unsigned gated_blocks(unsigned rows, int *gate)
 {
     const unsigned cap = 148u * 4u;
     return gate && rows > cap ? cap : rows;
@@ -106,7 +107,7 @@ inline unsigned gated_blocks(unsigned rows, const int *gate)
 template <int U, int SPLIT>
 void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
                  const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
-                 const int *order, const int *gate, int *clear)
+                 const int *order, int *gate, int *clear)
 {
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
@@ -130,7 +131,7 @@ inline int pick_ku(int Kd) { return Kd <= 64 ? 2 : Kd <= 128 ? 4 : Kd <= 256 ? 8
 template <int KU>
 void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const int *col_idx,
                   const float *sv, const float *A, int64_t lda, const float *B, int64_t ldb,
-                  float *out, const int *order, const int *gate, int *clear)
+                  float *out, const int *order, int *gate, int *clear)
 {
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     const int nrows = (int)grid.x;
@@ -143,7 +144,7 @@ template <int KU, int U, int SPLIT>
 b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
                          const int *col_idx, const float *sv, const float *A, int64_t lda,
                          const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
-                         int64_t ldo, const int *order, const int *gate, int *clear)
+                         int64_t ldo, const int *order, int *gate, int *clear)
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
@@ -166,7 +167,7 @@ b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int K
                                 const int *row_ptr, const int *col_idx, const float *sv,
                                 const float *A, int64_t lda, const float *B, int64_t ldb,
                                 const float *D, int64_t ldd, float *O, int64_t ldo,
-                                const int *order, const int *gate, int *clear)
+                                const int *order, int *gate, int *clear)
 {
 #define B2SP_F(U_, S_) \
     return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear)
@@ -270,7 +271,7 @@ static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_AL
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
                              const float *D, long long ldd, float *O, long long ldo, const int *order,
-                             const int *gate, int *clear, cudaStream_t st)
+                             int *gate, int *clear, cudaStream_t st)
 {
     bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
     if (vec) {
@@ -321,7 +322,7 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
                         O, ldo, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
         // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
-        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
         rc = spmm_rows(M, N, row_ptr, col_idx, values, D, ldd, O, ldo, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_SPMM] = launches + 1;
         return rc;
@@ -343,7 +344,7 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
 // Enqueues the row-family SDDMM.  `gate` != NULL makes it a device-side fallback.
 static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_idx, const float *s_values,
                               const float *A, long long lda, const float *B, long long ldb,
-                              float *out_values, const int *order, const int *gate, int *clear, cudaStream_t st)
+                              float *out_values, const int *order, int *gate, int *clear, cudaStream_t st)
 {
     dim3 grid((unsigned)M);
     bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
@@ -405,7 +406,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
         rc = fused_tile(plan, prepared, 0, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
                         out_values, 0, workspace, st, &launches);
         if (rc != B2SP_OK) return rc;
-        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
         rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_SDDMM] = launches + 1;
         return rc;
@@ -428,7 +429,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const int *col_idx,
                               const float *s_values, const float *A, long long lda, const float *B,
                               long long ldb, const float *D, long long ldd, float *O, long long ldo,
-                              const int *order, const int *gate, int *clear, cudaStream_t st)
+                              const int *order, int *gate, int *clear, cudaStream_t st)
 {
     b2sp_status rc = B2SP_OK;
     bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
@@ -497,7 +498,7 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
                             workspace, st, &launches);
         }
         if (rc != B2SP_OK) return rc;
-        const int *gate = reinterpret_cast<const int *>(static_cast<const char *>(workspace) + kWsTileFlagsOffset);
+        int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
         rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, nullptr, st);
         g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
         return rc;
@@ -568,31 +569,45 @@ b2sp_status b2sp_device_status(const void *workspace, void *stream)
 // ---- host-buffer forms ------------------------------------------------------------------------
 namespace {
 
+// Device memory of one host-buffer call.  It comes from a stream-ordered pool that the library owns (one
+// per device, created at first use, release threshold "never": freed blocks stay in it across calls, so a
+// call does not pay for fresh allocations).  The process's default pool is left as it is.
+cudaMemPool_t library_pool()
+{
+    constexpr int kMaxDevices = 64;
+    static std::mutex mu;
+    static cudaMemPool_t pools[kMaxDevices] = {};
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return nullptr;
+    std::lock_guard<std::mutex> lock(mu);
+    if (!pools[dev]) {
+        cudaMemPoolProps props = {};
+        props.allocType = cudaMemAllocationTypePinned;
+        props.handleTypes = cudaMemHandleTypeNone;
+        props.location.type = cudaMemLocationTypeDevice;
+        props.location.id = dev;
+        cudaMemPool_t pool = nullptr;
+        if (cudaMemPoolCreate(&pool, &props) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+        unsigned long long keep = ~0ull;
+        cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
+        pools[dev] = pool;
+    }
+    return pools[dev];
+}
+
 struct DevArena {
     cudaStream_t st;
+    cudaMemPool_t pool;
     void *ptrs[16];
     int n = 0;
     bool ok = true;
-    explicit DevArena(cudaStream_t s) : st(s)
-    {
-        // keep freed blocks in the stream-ordered pool across calls (the default returns them to the
-        // driver at every synchronisation, which makes each call pay for fresh allocations)
-        static thread_local int tuned_device = -1;
-        int dev = -1;
-        if (cudaGetDevice(&dev) == cudaSuccess && dev != tuned_device) {
-            cudaMemPool_t pool;
-            if (cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
-                unsigned long long keep = ~0ull;
-                cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &keep);
-            }
-            tuned_device = dev;
-        }
-    }
+    int device_word = 0;   // the workspace's status word, copied back with the result
+    explicit DevArena(cudaStream_t s) : st(s), pool(library_pool()) { ok = pool != nullptr; }
     void *alloc(size_t bytes)
     {
         void *p = nullptr;
         if (bytes == 0) bytes = 16;
-        if (!ok || cudaMallocAsync(&p, bytes, st) != cudaSuccess) { ok = false; return nullptr; }
+        if (!ok || cudaMallocFromPoolAsync(&p, bytes, pool, st) != cudaSuccess) { ok = false; return nullptr; }
         ptrs[n++] = p;
         return p;
     }
@@ -604,11 +619,20 @@ struct DevArena {
             ok = false;
         return d;
     }
+    // Queues the read-back of the status word that device code left in `ws` (a bounded wait that gave up).
+    void fetch_status(const void *ws)
+    {
+        if (ok && ws &&
+            cudaMemcpyAsync(&device_word, static_cast<const char *>(ws) + b2sp::kWsStatusOffset, sizeof(int),
+                            cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            ok = false;
+    }
     b2sp_status finish(b2sp_status rc)
     {
         for (int i = 0; i < n; ++i) cudaFreeAsync(ptrs[i], st);
         if (cudaStreamSynchronize(st) != cudaSuccess && rc == B2SP_OK) rc = B2SP_ERR_CUDA;
         if (!ok && rc == B2SP_OK) rc = B2SP_ERR_CUDA;
+        if (rc == B2SP_OK && device_word != 0) rc = B2SP_ERR_TIMEOUT;   // the outputs are undefined
         return rc;
     }
 };
@@ -632,11 +656,13 @@ b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_pt
     size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_SPMM, B2SP_ALGO_AUTO, M, K, 0, N, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
+    const bool launched_work = M > 0 && N > 0 && nnz > 0;   // otherwise no kernel ran and the status word is unset
     if (a.ok) {
         rc = b2sp_spmm(M, K, N, nnz, d_rp, d_ci, d_v, d_D, N, d_O, N, ws, wsb, B2SP_ALGO_AUTO, stream);
         if (rc == B2SP_OK && (size_t)M * N > 0 &&
             cudaMemcpyAsync(O, d_O, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
             rc = B2SP_ERR_CUDA;
+        if (rc == B2SP_OK && launched_work) a.fetch_status(ws);
     }
     return a.finish(rc);
 }
@@ -657,11 +683,13 @@ b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_
     size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_SDDMM, B2SP_ALGO_AUTO, M, K, Kd, 0, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
+    const bool launched_work = M > 0 && Kd > 0 && nnz > 0;
     if (a.ok) {
         rc = b2sp_sddmm(M, K, Kd, nnz, d_rp, d_ci, d_v, d_A, Kd, d_B, Kd, d_C, ws, wsb, B2SP_ALGO_AUTO, stream);
         if (rc == B2SP_OK && nnz > 0 &&
             cudaMemcpyAsync(out_values, d_C, sizeof(float) * (size_t)nnz, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
             rc = B2SP_ERR_CUDA;
+        if (rc == B2SP_OK && launched_work) a.fetch_status(ws);
     }
     return a.finish(rc);
 }
@@ -684,12 +712,14 @@ b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const 
     size_t wsb = b2sp_workspace_bytes_algo(B2SP_OP_FUSEDMM, B2SP_ALGO_AUTO, M, K, Kd, N, nnz);
     void *ws = a.alloc(wsb);
     b2sp_status rc = B2SP_ERR_CUDA;
+    const bool launched_work = M > 0 && N > 0 && Kd > 0 && nnz > 0;
     if (a.ok) {
         rc = b2sp_fusedmm(M, K, Kd, N, nnz, d_rp, d_ci, d_v, d_A, Kd, d_B, Kd, d_D, N, d_O, N, ws, wsb,
                           B2SP_ALGO_AUTO, stream);
         if (rc == B2SP_OK && (size_t)M * N > 0 &&
             cudaMemcpyAsync(O, d_O, sizeof(float) * (size_t)M * N, cudaMemcpyDeviceToHost, a.st) != cudaSuccess)
             rc = B2SP_ERR_CUDA;
+        if (rc == B2SP_OK && launched_work) a.fetch_status(ws);
     }
     return a.finish(rc);
 }

@@ -7,8 +7,11 @@
 // nowhere to get the row-binning workspace the regular entry point asks for.  This file gives
 // that workspace a permanent home: a fixed array in the library's own device image.
 //
-// The array costs kScratchBytes of device memory on every GPU that loads the library, from load
-// until the process exits, whether or not this entry point is ever called.
+// The array is part of the library's device image and costs kScratchBytes of device memory on every
+// GPU where that image gets loaded, until the process exits.  With CUDA's lazy module loading the
+// first cudaGetSymbolAddress on a device is what loads the image there: the driver reserves the
+// array (and the code) at that moment and may synchronise the device.  That first call therefore
+// belongs at start-up, before the host's arena takes the rest of the memory.
 #include "../../include/b2sp.h"
 
 #include <cuda_runtime.h>

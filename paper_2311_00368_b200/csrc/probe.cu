@@ -2,7 +2,7 @@
 // SM), for the denominator of the roofline fraction.  Not part of the method.
 #include <cuda_runtime.h>
 
-#include "../../include/b2sp.h"
+#include "../../include/b2sp_debug.h"
 
 namespace {
 

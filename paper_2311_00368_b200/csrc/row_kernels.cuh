@@ -9,8 +9,11 @@
 // first, produced by the binning kernels below) or in natural order when it is NULL.
 // `clear`, when not NULL, points at the workspace's status word, which the kernel resets (a call whose only
 // launch is this kernel cannot fail on the device).
-// `gate`, when not NULL, points at a device word: the kernel does nothing if that word is 0
-// (used when the row family is only the fallback of the dense-tile family).
+// `gate`, when not NULL, points at three device words (used when the row family is only the fallback of
+// the dense-tile family): the kernel does nothing if words 0 and 1 are both 0.  Word 0 says that the
+// window table cannot be used and stays as it is; word 1 says that a dense operand of this call holds a
+// non-finite value and is per call: the last CTA of this grid to have read it clears it (word 2 counts
+// the readers), so that the next call on the workspace starts clean without a launch of its own.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,6 +35,25 @@ __device__ __forceinline__ int bucket_of(int len) { return len <= 0 ? 0 : 32 - _
 // that each is placed, and does what does not need its predecessor's output, while the predecessor runs.
 __device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// True when a gated launch has nothing to do (see the top of this file).  Called by every thread of the CTA.
+__device__ __forceinline__ bool gate_closed(int *gate)
+{
+    if (!gate) return false;
+    __shared__ int gate_word;
+    if (threadIdx.x == 0) {
+        volatile int *g = gate;
+        gate_word = g[0] | g[1];
+        __threadfence();   // the read above is performed before this CTA is counted as a reader
+        const unsigned readers = gridDim.x * gridDim.y * gridDim.z;
+        if ((unsigned)atomicAdd(gate + 2, 1) == readers - 1) {
+            g[2] = 0;
+            g[1] = 0;
+        }
+    }
+    __syncthreads();
+    return gate_word == 0;
+}
 
 __global__ void bin_count_kernel(int M, const int *__restrict__ row_ptr, int *__restrict__ count)
 {
@@ -183,11 +205,11 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                 const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                 float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     using G = SweepGeom<U, SPLIT>;
     __shared__ float4 red[kRowWarps * U * G::LPN];
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -237,10 +259,10 @@ __global__ void __launch_bounds__(kRowThreads)
 spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                        const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
                        float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                       const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                       int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     __shared__ float red[kRowWarps][128];
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -341,11 +363,11 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                  const float *s_values, const float *__restrict__ A, int64_t lda,
                  const float *__restrict__ B, int64_t ldb, float *out_values,
-                 const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                 const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     extern __shared__ float4 dyn_smem[];
     float *a_smem = reinterpret_cast<float *>(dyn_smem);
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -371,9 +393,9 @@ __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                         const float *s_values, const float *__restrict__ A, int64_t lda,
                         const float *__restrict__ B, int64_t ldb, float *out_values,
-                        const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                        const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
@@ -400,11 +422,11 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
                    const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
-                   const int *__restrict__ row_order, const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                   const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     float4 *red = dyn_smem;                                                   // kRowWarps*U*LPN
@@ -454,10 +476,10 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
                           const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
                           int64_t ldb, const float *__restrict__ D, int64_t ldd,
                           float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                          const int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                          int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     __shared__ float red[kRowWarps][128];
-    if (gate && *gate == 0) return;
+    if (gate_closed(gate)) return;
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

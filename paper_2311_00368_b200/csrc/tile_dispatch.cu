@@ -4,7 +4,7 @@
 
 #include <cuda.h>
 
-#include <cstdlib>
+#include <atomic>
 #include <mutex>
 
 #include "tile_kernels.cuh"
@@ -15,6 +15,9 @@ namespace b2sp {
 namespace {
 
 constexpr int kSMs = 148;
+
+// 0 = the planner decides; set through b2sp_debug_force_k_splits (tests of the K-split epilogues, tuning).
+std::atomic<int> g_forced_k_splits{0};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -57,7 +60,6 @@ bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, 
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// K splits of a tile; `blocks` = 128-column blocks of S.
 // fp32 matrix [rows][cols] with row stride `ld` elements, as the target of the tile kernel's flush:
 // boxes of 16 columns x 32 rows, 64-byte swizzle.  Needs a 16-byte aligned base and row stride.
 bool make_output_map(CUtensorMap *tm, float *base, long long rows, int cols, long long ld)
@@ -73,11 +75,25 @@ bool make_output_map(CUtensorMap *tm, float *base, long long rows, int cols, lon
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Raises a kernel's dynamic shared-memory limit once per kernel (TAG) and device instead of on every launch.
+template <int TAG>
+bool allow_dynamic_smem(const void *kernel, int bytes)
+{
+    static std::atomic<unsigned long long> done{0};   // one bit per device
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    const unsigned long long bit = 1ull << (dev & 63);
+    if (done.load(std::memory_order_acquire) & bit) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+    done.fetch_or(bit, std::memory_order_release);
+    return true;
+}
+
+// K splits of a tile; `blocks` = 128-column blocks of S.
 int pick_split(int base_tiles, int blocks)
 {
-    if (const char *e = getenv("B2SP_FORCE_KS")) {   // tuning aid
-        int ks = atoi(e);
-        if (ks >= 1 && ks <= blocks) return ks;
+    if (const int forced = g_forced_k_splits.load(std::memory_order_relaxed)) {   // b2sp_debug_force_k_splits
+        if (forced >= 1 && forced <= blocks) return forced;
     }
     // One wave of long-lived CTAs beats several waves of short ones (each CTA pays a prologue, an
     // epilogue and a partial-output slab): take the largest split that still fits one wave, as long
@@ -117,8 +133,7 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     if (cudaMemsetAsync(ws, 0, kWsHeaderBytes, st) != cudaSuccess) return B2SP_ERR_CUDA;
     int2 *win = reinterpret_cast<int2 *>(ws + pattern_table_offset(M));
     if (Wk > kMasksMaxWk) return B2SP_ERR_UNSUPPORTED;
-    if (cudaFuncSetAttribute(tile_masks_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMasksMaxWk * 4) != cudaSuccess)
-        return B2SP_ERR_CUDA;
+    if (!allow_dynamic_smem<-1>(reinterpret_cast<const void *>(tile_masks_kernel), kMasksMaxWk * 4)) return B2SP_ERR_CUDA;
     const int cap = kSMs * 64;
     tile_masks_kernel<<<M < cap ? M : cap, kMasksWarps * 32, (size_t)Wk * 4, st>>>(M, K, Wk, nnz, row_ptr, col_idx, win, flags, sig, sig_dev);
     *launches += 1;
@@ -212,8 +227,7 @@ b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, cons
 {
     using Cfg = FusedCfg<KDP, MODE>;
     auto kern = fused_tile_kernel<KDP, MODE>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) != cudaSuccess)
-        return B2SP_ERR_CUDA;
+    if (!allow_dynamic_smem<KDP * 4 + MODE>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
     // a programmatic dependent of the operand-split kernel: its CTAs are placed while that kernel still runs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)items);
@@ -239,17 +253,17 @@ b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &
     return launch_fused_tile<128, MODE>(bh, bl, dh, dl, out, a, items, st);
 }
 
-// Splits one or two dense operands (job 1 optional), clears the device status word and optionally
-// zero-fills an output matrix.
-void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int *status, const TableCheck &chk,
-                  cudaStream_t st)
+// Splits (or only checks) up to three dense operands, clears the device status word and optionally
+// zero-fills an array.
+void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const TableCheck &chk, cudaStream_t st)
 {
-    auto groups = [](const SplitJob &j) { return (long long)j.rows_p * (j.cols_p >> 2); };
-    long long most = groups(j0);
-    if (j1 && groups(*j1) > most) most = groups(*j1);
+    long long most = 1;
+    for (int i = 0; i < jobs.n; ++i) {
+        const long long g = (long long)jobs.j[i].batch * jobs.j[i].rows_p * (jobs.j[i].cols_p >> 2);
+        if (g > most) most = g;
+    }
     const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
-    const int njobs = j1 ? 2 : 1;
-    dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(njobs + (z.out ? 1 : 0)));
+    dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(jobs.n + (z.out ? 1 : 0)));
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(256);
@@ -259,7 +273,7 @@ void launch_split(const SplitJob &j0, const SplitJob *j1, const ZeroJob &z, int 
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = chk.after_prepass ? attr : nullptr;   // beside the pattern pre-pass of the same call, never beside foreign work
     cfg.numAttrs = chk.after_prepass ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, split_dense_kernel, j0, j1 ? *j1 : j0, njobs, z, status, chk);
+    cudaLaunchKernelEx(&cfg, split_dense_kernel, jobs, z, status, chk);
 }
 
 }  // namespace
@@ -296,7 +310,16 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         if (prc != B2SP_OK) return prc;
     }
     {
-        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp}, jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np};
+        // B and D are split into tf32 hi/lo copies; A, which the tile kernel splits itself, is only checked
+        // for non-finite values (see split_dense_kernel).
+        const int a_rows_p = (M + 3) & ~3, a_cols_p = (Kd + 31) & ~31;
+        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, 1, 0, kDenseF32, 0};
+        const SplitJob jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np, 1, 0, kDenseF32, 0};
+        const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, 1, 0, kDenseF32, 1};
+        SplitJobs jobs;
+        jobs.n = 0;
+        if (!spmm) { jobs.j[jobs.n++] = jb; jobs.j[jobs.n++] = ja; }
+        if (fused) jobs.j[jobs.n++] = jd;
         // With several K splits the CTA that finishes an output tile last sums the splits' slabs: the
         // per-tile arrival counters start at zero.
         const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), p.Mt * p.Nt, 1, p.Mt * p.Nt}
@@ -306,9 +329,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         const TableCheck chk{PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx},
                              prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags,
                              prepared ? 0 : 1};
-        if (spmm) launch_split(jd, nullptr, z, clear, chk, st);
-        else if (fused) launch_split(jb, &jd, z, clear, chk, st);
-        else launch_split(jb, nullptr, z, clear, chk, st);
+        launch_split(jobs, z, clear, chk, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
@@ -319,7 +340,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.flags = flags; a.status = status;
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
     a.O = out; a.ldo = ldo;
-    a.prof = reinterpret_cast<unsigned long long *>(ws + kWsStatusOffset + 128);  // profiling builds only
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
     else { a.out = part; a.ld_out = p.Np; a.slab = (long long)p.Mt * kFusedRows * p.Np; }
@@ -350,17 +370,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 
 }  // namespace b2sp
 
-#ifdef B2SP_TILE_PROFILE
-// Profiling builds only: copies the fused tile kernel's role timers to the host and clears them.
-extern "C" int b2sp_prof_fetch(unsigned long long *host32)
+// Debug / tuning hook declared in include/b2sp_debug.h.
+extern "C" void b2sp_debug_force_k_splits(int k_splits)
 {
-    unsigned long long zero[32] = {};
-    if (cudaMemcpyFromSymbol(host32, b2sp::g_fused_prof, sizeof(zero)) != cudaSuccess) return 1;
-    return cudaMemcpyToSymbol(b2sp::g_fused_prof, zero, sizeof(zero)) != cudaSuccess;
+    b2sp::g_forced_k_splits.store(k_splits > 0 ? k_splits : 0, std::memory_order_relaxed);
 }
-// Profiling builds only: per CTA the global-timer stamps (start, end of the MMA loop, end) and the SM id.
-extern "C" int b2sp_prof_cta_times(unsigned long long *host4096)
-{
-    return cudaMemcpyFromSymbol(host4096, b2sp::g_fused_cta, 4096 * sizeof(unsigned long long)) != cudaSuccess;
-}
-#endif

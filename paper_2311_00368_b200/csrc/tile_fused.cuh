@@ -31,26 +31,6 @@
 #include "ptx_sm100.cuh"
 #include "tile_kernels.cuh"
 
-#ifdef B2SP_TILE_PROFILE
-#define B2SP_FPROF_DECL long long fp_t0 = 0, fp_acc[6] = {0, 0, 0, 0, 0, 0};
-#define B2SP_FPROF_START fp_t0 = clock64();
-#define B2SP_FPROF_STOP(i) { long long t_ = clock64(); fp_acc[i] += t_ - fp_t0; fp_t0 = t_; }
-#define B2SP_FPROF_FLUSH(base) { if (lane == 0) { for (int i_ = 0; i_ < 6; ++i_) atomicAdd(b2sp::g_fused_prof + (base) + i_, (unsigned long long)fp_acc[i_]); } }
-#define B2SP_FPROF_STAMP(var) const long long var = clock64();
-#define B2SP_FPROF_ADD(i, v) { atomicAdd(b2sp::g_fused_prof + (i), (unsigned long long)(v)); }
-namespace b2sp { __device__ unsigned long long g_fused_prof[32]; __device__ unsigned long long g_fused_cta[1024 * 4]; }
-__device__ __forceinline__ unsigned long long b2sp_gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-__device__ __forceinline__ unsigned b2sp_smid() { unsigned t; asm volatile("mov.u32 %0, %smid;" : "=r"(t)); return t; }
-#define B2SP_FPROF_CTA(i) { if (threadIdx.x == 32 && blockIdx.x < 1024) { b2sp::g_fused_cta[blockIdx.x * 4 + (i)] = b2sp_gtime(); b2sp::g_fused_cta[blockIdx.x * 4 + 3] = b2sp_smid(); } }
-#else
-#define B2SP_FPROF_CTA(i) {}
-#define B2SP_FPROF_STAMP(var)
-#define B2SP_FPROF_ADD(i, v) {}
-#define B2SP_FPROF_DECL
-#define B2SP_FPROF_START
-#define B2SP_FPROF_STOP(i) {}
-#define B2SP_FPROF_FLUSH(base) {}
-#endif
 
 namespace b2sp {
 
@@ -87,9 +67,8 @@ struct FusedTileArgs {
     float *O;                 // FusedMM / SPMM with several K splits: the output the slabs are summed into ...
     long long ldo;
     int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
-    int *flags;                // flags[0] != 0: the table cannot be used, the row kernels take over
+    int *flags;                // flags[kFlagUnsorted] or flags[kFlagNotFinite] != 0: the row kernels take over
     int *status;
-    unsigned long long *prof;  // optional role timers (profiling builds only)
 };
 
 // MODE: which op the kernel runs.  SPMM reuses the FusedMM pipeline with P' = the stored values
@@ -173,8 +152,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    B2SP_FPROF_STAMP(fp_kernel_start)
-    B2SP_FPROF_CTA(0)
     const int ks = blockIdx.x % a.KS;
     const int tile = blockIdx.x / a.KS;
     const int nt = tile % a.Nt, mt = tile / a.Nt;
@@ -267,7 +244,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     // pre-pass or that kernel's signature check wrote them), so the gated row kernel launched behind this
     // grid may run beside it.
     ptx::wait_for_primary_grid();
-    const bool unusable = a.flags[0] != 0;
+    const bool unusable = (a.flags[kFlagUnsorted] | a.flags[kFlagNotFinite]) != 0;
     ptx::launch_dependents();
     if (unusable) {   // pattern not usable for tiles: the row kernels take over
         if (warp == 1) {
@@ -319,20 +296,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedBlk, false, false);
             const uint32_t idesc2 = a.NT == 64 ? ptx::idesc_tf32(kFusedRows, 64, false, true) : ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
-            B2SP_FPROF_DECL
-            B2SP_FPROF_START
-            B2SP_FPROF_STAMP(fp_loop_start)
             int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
             auto gemm1 = [&](int b) -> bool {   // P = A_tile * B_block^T over NCH_B chunks
                 const int pb = FUSED ? 0 : (b & 1);
                 const int puse = FUSED ? b : (b >> 1);
                 if (puse > 0 && !ptx::mbar_wait(p_free(pb), (puse - 1) & 1)) return false;   // P drained?
-                B2SP_FPROF_STOP(0)
                 const uint32_t pacc = tmem + Cfg::COL_P + pb * kFusedBlk;
                 for (int i = 0; i < NCH_B; ++i, ++c) {
                     const int s = c % RING;
                     if (!ptx::mbar_wait(full(s), (c / RING) & 1)) return false;
-                    B2SP_FPROF_STOP(1)
                     ptx::tc_fence_after_sync();
                     const uint32_t b_hi = ring + s * kFusedChunk, b_lo = b_hi + kFusedChunk / 2;
 #pragma unroll
@@ -350,7 +322,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         }
                     }
                     ptx::mma_commit(empty(s));
-                    B2SP_FPROF_STOP(2)
                 }
                 ptx::mma_commit(p_full(pb));
                 return true;
@@ -358,9 +329,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             auto gemm2 = [&](int b, int w) -> bool {   // O += P'_window * D_window
                 const int s = c % RING, ppb = ppu & 1;
                 if (!ptx::mbar_wait(pp_full(ppb), (ppu >> 1) & 1)) return false;
-                B2SP_FPROF_STOP(3)
                 if (!ptx::mbar_wait(full(s), (c / RING) & 1)) return false;
-                B2SP_FPROF_STOP(1)
                 ptx::tc_fence_after_sync();
                 const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
                 const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
@@ -379,7 +348,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::mma_commit(empty(s));
                 ++c;
                 ++ppu;
-                B2SP_FPROF_STOP(4)
                 return true;
             };
             // GEMM1 of block b+1 is issued between the second and third GEMM2 of block b: by then the
@@ -391,9 +359,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 // previous partial sum out of tensor memory
                 if (FUSED && b % kFusedFlushBlocks == 0 && b / kFusedFlushBlocks >= NOB) {
                     const int ch = b / kFusedFlushBlocks;   // chunk ch reuses the accumulator of chunk ch - NOB
-                    B2SP_FPROF_STOP(4)
                     failed = !ptx::mbar_wait(o_free(ch % NOB), (ch / NOB - 1) & 1);
-                    B2SP_FPROF_STOP(5)
                 }
                 // At the end of a chunk GEMM1 of the next block is issued after the chunk's last GEMM2, so that
                 // the tensor core works on it while the processors take O out of tensor memory.
@@ -405,10 +371,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     ptx::mma_commit(o_full((b / kFusedFlushBlocks) % NOB));
                 if (!SPMM && b + 1 < nblk && late_b && !failed) failed = !gemm1(b + 1);
             }
-            B2SP_FPROF_FLUSH(0)
-            B2SP_FPROF_ADD(26, fp_loop_start - fp_kernel_start)
-            B2SP_FPROF_ADD(27, clock64() - fp_loop_start)
-            B2SP_FPROF_CTA(1)
         }
     } else if (warp >= 2 && warp < 6) {
         // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
@@ -417,8 +379,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // SPMM), split to hi/lo and write P' to tensor memory.
         // SDDMM: per window, copy the row of P into a slot; a helper warp writes the stored entries.
         const int nwin = nblk * WPB;
-        B2SP_FPROF_DECL
-        B2SP_FPROF_START
         for (int it = 0; it < nwin; ++it) {
             const int blk = it / WPB, w = it % WPB;
             // FusedMM / SPMM: one item (32 rows) per processor warp and window.  SDDMM: two items of 16 rows,
@@ -432,7 +392,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     bool ok = ptx::mbar_wait(sl_full(s), use & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
-                B2SP_FPROF_STOP(0)
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
                     uint32_t x0, x1, x2, x3;
@@ -444,7 +403,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
-                B2SP_FPROF_STOP(1)
                 uint32_t p0[16], p1[16];
                 if (SPMM) {
 #pragma unroll
@@ -465,14 +423,12 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         if (lane == 0) ptx::mbar_arrive(p_free(0));
                     }
                 }
-                B2SP_FPROF_STOP(2)
                 const int ppb = it & 1, ppuse = it >> 1;
                 if (ppuse > 0) {
                     bool ok = ptx::mbar_wait(pp_free(ppb), (ppuse - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     ptx::tc_fence_after_sync();
                 }
-                B2SP_FPROF_STOP(3)
                 uint32_t hi[16], lo[16];
                 const uint32_t pph = tmem + lane_addr + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
 #pragma unroll
@@ -487,7 +443,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::tc_fence_before_sync();
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(pp_full(ppb));
-                B2SP_FPROF_STOP(4)
                 // ---- flush: after every kFusedFlushBlocks-th block (and after the last block) the partial O
                 // leaves tensor memory: each thread adds its row into the output (or
                 // its K split's slab): the first partial sum is stored, the later ones are added with fp32
@@ -597,12 +552,10 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     __syncwarp();
                     if (lane == 0) ptx::mbar_arrive(p_free(pb));
                 }
-                B2SP_FPROF_STOP(2)
                 if (use > 0) {
                     bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
-                B2SP_FPROF_STOP(0)
 #pragma unroll
                 for (int jj = 0; jj < 8; ++jj) {
                     const uint32_t *src = jj < 4 ? &p0[4 * jj] : &p1[4 * (jj - 4)];
@@ -611,10 +564,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 __syncwarp();
                 if ((lane & 15) == 0) ptx::mbar_arrive(sl_full(s));
-                B2SP_FPROF_STOP(4)
             }
         }
-        B2SP_FPROF_FLUSH(8)
     } else if (helper_index<FUSED>(warp) >= 0 && helper_index<FUSED>(warp) < NH) {
         // ---------------- helper warps: work items (window, group of rows), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
@@ -636,8 +587,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         };
         // the records of the next two items are in flight while an item is processed
         int2 rec_next = load_rec(h), rec_next2 = load_rec(h + NH);
-        B2SP_FPROF_DECL
-        B2SP_FPROF_START
         for (int j = h; j < nitems; j += NH) {
             const int s = j % NSLOT, use = j / NSLOT;
             const int2 rec = rec_next;
@@ -659,26 +608,22 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (!FUSED) idx[r] = present ? at : -1;
             });
             const uint32_t slot = slots + s * Cfg::SLOT_BYTES;
-            B2SP_FPROF_STOP(0)
             if (FUSED) {
                 if (use > 0) {
                     bool ok = ptx::mbar_wait(sl_empty(s), (use - 1) & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
-                B2SP_FPROF_STOP(1)
                 ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
                     ptx::sts32_off<r * 128>(slot + (uint32_t)((lane << 2) ^ ((r & 7) << 4)), __float_as_uint(vn[r]));
                 });
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(sl_full(s));
-                B2SP_FPROF_STOP(2)
             } else {
                 {
                     bool ok = ptx::mbar_wait(sl_full(s), use & 1);
                     if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 }
-                B2SP_FPROF_STOP(1)
                 // all reads of the slot first (independent loads), then the stores
                 ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
@@ -690,10 +635,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     constexpr int r = decltype(rc)::value;
                     if (idx[FUSED ? 0 : r] >= 0) a.out[idx[FUSED ? 0 : r]] = vn[r];
                 });
-                B2SP_FPROF_STOP(2)
             }
         }
-        B2SP_FPROF_FLUSH(16)
     }
     if (failed) atomicExch(a.status, 1);
     if (FUSED && warp >= 2 && warp < 6 && lane == 0) {   // this warp's TMA stores / reductions have been performed
@@ -737,8 +680,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         __syncwarp();
         ptx::tmem_dealloc(tmem, 512);
     }
-    if (threadIdx.x == 32) B2SP_FPROF_ADD(28, clock64() - fp_kernel_start)
-    B2SP_FPROF_CTA(2)
 }
 
 }  // namespace b2sp

@@ -19,7 +19,11 @@
 namespace b2sp {
 
 constexpr int kTileKC = 32;       // columns of S per pipeline stage (one 128-byte swizzle row of tf32)
-constexpr int kFlagUnsorted = 0;  // flags[0] != 0: some row's columns are not strictly increasing
+// Flag words of the tile pre-passes (the gate of the row-kernel fallback reads the first two, see row_kernels.cuh):
+constexpr int kFlagUnsorted = 0;   // != 0: the window table is unusable (a row's columns are not strictly increasing,
+                                   // or the table belongs to other arrays); stays set until the table is rebuilt
+constexpr int kFlagNotFinite = 1;  // != 0: a dense operand of this call holds a non-finite value; cleared by the fallback
+constexpr int kFlagGateReaders = 2;  // CTAs of the gated fallback that have read the flags so far
 
 // ---- table signature ------------------------------------------------------------------------------------
 struct PatternSignature {
@@ -153,16 +157,33 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // ((c/32)*rows_p + r)*32 + c%32, i.e. [cols_p/32][rows_p][32] floats, zero in the padding
 // (rows_p >= rows, cols_p >= cols, cols_p % 32 == 0).  One 32-float group of a row is one
 // 128-byte swizzle row for TMA, and the whole thing is a plain packed 3-D tensor.
-// One launch splits up to two operands (blockIdx.y picks the job) and, being the first kernel of
+// A batch of `batch` equally sized operands, `batch_stride` elements apart, is stacked along the rows:
+// [cols_p/32][batch * rows_p][32].
+// bf16 operands (dtype 1) are exact in tf32: hi is the value itself and no lo copy is written.
+// One launch handles up to three jobs (blockIdx.y picks the job) and, being the first kernel of
 // every tile op, also clears the workspace's device status word (unless `status` is NULL: the second
 // kernel of a two-phase op keeps what the first one reported) and, when asked to, zero-fills an
 // array (the last blockIdx.y): the per-tile arrival counters of a FusedMM / SPMM with several K splits.
+//
+// The dense-tile kernels multiply whole windows of S, positions without a stored entry included (by
+// zero), so an Inf or NaN anywhere in a dense operand -- also in a row no stored entry refers to -- or a
+// value so close to FLT_MAX that its tf32 hi part rounds to Inf would turn into NaN in outputs that
+// Eq. 1-3 leave finite.  Every job therefore also looks at what it reads, and a job with `check_only`
+// (the A operand, which the tile kernel splits itself) does nothing else: a non-finite hi part raises
+// the fallback flag, and the row kernels, which touch exactly the entries the equations name, produce
+// the result.
+constexpr int kDenseF32 = 0, kDenseBf16 = 1;
+
 struct SplitJob {
-    const float *X;
+    const void *X;
     long long ld;
     int rows, cols;
     float *hi, *lo;
     int rows_p, cols_p;
+    int batch;                // operands stacked along the rows (1: a single operand)
+    long long batch_stride;   // elements between consecutive operands of the batch
+    int dtype;                // kDenseF32 / kDenseBf16
+    int check_only;           // look for non-finite values, write nothing
 };
 
 struct ZeroJob {
@@ -183,14 +204,21 @@ struct TableCheck {
                                     // this grid must not complete before that one (the tile kernel waits for this grid only)
 };
 
-__global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
+struct SplitJobs {
+    SplitJob j[3];
+    int n;
+};
+
+__device__ __forceinline__ bool tf32_hi_not_finite(uint32_t hi) { return (hi & 0x7f800000u) == 0x7f800000u; }
+
+__global__ void split_dense_kernel(SplitJobs jobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
 {
     ptx::launch_dependents();   // the tile kernel may take its SMs; it waits for this grid before it reads anything
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
         if (status) *status = 0;
         if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
     }
-    if ((int)blockIdx.y == njobs) {   // zero-fill job
+    if ((int)blockIdx.y == jobs.n) {   // zero-fill job
         const long long total = (long long)z.rows * z.cols;
         const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
         if (z.ld == z.cols && (total & 3) == 0 && (reinterpret_cast<uintptr_t>(z.out) & 15) == 0) {
@@ -202,33 +230,59 @@ __global__ void split_dense_kernel(SplitJob j0, SplitJob j1, int njobs, ZeroJob 
         if (chk.after_prepass) ptx::wait_for_primary_grid();
         return;
     }
-    const SplitJob j = blockIdx.y ? j1 : j0;
-    const bool vec = (j.ld & 3) == 0 && (reinterpret_cast<uintptr_t>(j.X) & 15) == 0;
-    const long long groups = (long long)j.rows_p * (j.cols_p >> 2);  // float4 groups
+    const SplitJob j = jobs.j[blockIdx.y];
+    const bool bf16 = j.dtype == kDenseBf16;
+    // 16-byte loads of four fp32 (or 8-byte loads of four bf16) need the alignment for every operand of the batch
+    const bool vec = (j.ld & 3) == 0 && (j.batch_stride & 3) == 0 &&
+                     (reinterpret_cast<uintptr_t>(j.X) & (bf16 ? 7 : 15)) == 0;
+    const long long rows_all = (long long)j.batch * j.rows_p;
+    const long long groups = rows_all * (j.cols_p >> 2);  // float4 groups
+    bool bad = false;
     for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
          g += (long long)gridDim.x * blockDim.x) {
         const int q = (int)(g & 7);                 // float4 inside the 32-float group
-        const long long rg = g >> 3;                // (column group, row) pair
-        const int r = (int)(rg % j.rows_p);
-        const int c = (int)(rg / j.rows_p) * 32 + q * 4;
+        const long long rg = g >> 3;                // (column group, stacked row) pair
+        const long long rs = rg % rows_all;
+        const int b = (int)(rs / j.rows_p), r = (int)(rs % j.rows_p);
+        const int c = (int)(rg / rows_all) * 32 + q * 4;
         uint32_t h[4] = {0, 0, 0, 0}, l[4] = {0, 0, 0, 0};
         if (r < j.rows && c < j.cols) {
-            const float *src = j.X + (long long)r * j.ld + c;
-            if (vec && c + 3 < j.cols) {
-                const float4 f = __ldg(reinterpret_cast<const float4 *>(src));
-                ptx::split_tf32(f.x, h[0], l[0]);
-                ptx::split_tf32(f.y, h[1], l[1]);
-                ptx::split_tf32(f.z, h[2], l[2]);
-                ptx::split_tf32(f.w, h[3], l[3]);
-            } else {
+            const long long at = (long long)b * j.batch_stride + (long long)r * j.ld + c;
+            float x[4] = {0.f, 0.f, 0.f, 0.f};
+            if (bf16) {
+                const unsigned short *src = static_cast<const unsigned short *>(j.X) + at;
+                if (vec && c + 3 < j.cols) {
+                    const uint2 u = __ldg(reinterpret_cast<const uint2 *>(src));
+                    x[0] = __uint_as_float(u.x << 16); x[1] = __uint_as_float(u.x & 0xffff0000u);
+                    x[2] = __uint_as_float(u.y << 16); x[3] = __uint_as_float(u.y & 0xffff0000u);
+                } else {
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (c + i < j.cols) ptx::split_tf32(__ldg(src + i), h[i], l[i]);
+                    for (int i = 0; i < 4; ++i)
+                        if (c + i < j.cols) x[i] = __uint_as_float((uint32_t)__ldg(src + i) << 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) h[i] = __float_as_uint(x[i]);   // bf16 is exact in tf32
+            } else {
+                const float *src = static_cast<const float *>(j.X) + at;
+                if (vec && c + 3 < j.cols) {
+                    const float4 f = __ldg(reinterpret_cast<const float4 *>(src));
+                    x[0] = f.x; x[1] = f.y; x[2] = f.z; x[3] = f.w;
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (c + i < j.cols) x[i] = __ldg(src + i);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) ptx::split_tf32(x[i], h[i], l[i]);
             }
+            bad |= tf32_hi_not_finite(h[0]) || tf32_hi_not_finite(h[1]) || tf32_hi_not_finite(h[2]) || tf32_hi_not_finite(h[3]);
         }
-        reinterpret_cast<uint4 *>(j.hi)[g] = make_uint4(h[0], h[1], h[2], h[3]);
-        reinterpret_cast<uint4 *>(j.lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
+        if (!j.check_only) {
+            reinterpret_cast<uint4 *>(j.hi)[g] = make_uint4(h[0], h[1], h[2], h[3]);
+            if (j.lo) reinterpret_cast<uint4 *>(j.lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
+        }
     }
+    if (bad) atomicExch(&chk.flags[kFlagNotFinite], 1);
     if (chk.after_prepass) ptx::wait_for_primary_grid();
 }
 

@@ -230,45 +230,6 @@ def test_host_buffer_entry_points(b):
 
 # ---- the named full-size workloads -------------------------------------------------------------
 
-def _sample_rows(p, count=48):
-    """Row ranges to spot-check on big problems: spread rows plus the longest and shortest."""
-    lens = np.diff(p.row_ptr)
-    rows = set(np.linspace(0, p.M - 1, count).astype(int).tolist())
-    rows |= set(np.argsort(lens)[-4:].tolist()) | set(np.argsort(lens)[:4].tolist())
-    return sorted(rows)
-
-
-def check_sampled(b, p, algos, ops, null_values=False):
-    d = DevProblem(p)
-    sv_np = None if null_values else p.values
-    sv = None if null_values else d.values
-    rows = _sample_rows(p)
-    for algo in algos:
-        res = {}
-        if "spmm" in ops:
-            res["spmm"] = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, algo=algo).cpu().numpy()
-        if "sddmm" in ops:
-            res["sddmm"] = b.sddmm(d.row_ptr, d.col_idx, sv, d.A, d.B, algo=algo).cpu().numpy()
-        if "fusedmm" in ops:
-            res["fusedmm"] = b.fusedmm(d.row_ptr, d.col_idx, sv, d.A, d.B, d.D, algo=algo).cpu().numpy()
-        for name, out in res.items():
-            assert np.all(np.isfinite(out)), f"{name}: non-finite output"
-            for r in rows:
-                if name == "spmm":
-                    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D, rows=(r, r + 1))
-                    got = out[r:r + 1]
-                elif name == "sddmm":
-                    ref, T = oracle.sddmm(p.row_ptr, p.col_idx, sv_np, p.A, p.B, rows=(r, r + 1))
-                    got = out[p.row_ptr[r]:p.row_ptr[r + 1]]
-                else:
-                    ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, sv_np, p.A, p.B, p.D, rows=(r, r + 1))
-                    got = out[r:r + 1]
-                ok, ratio = oracle.within_tolerance(got, ref, T, RTOL, ATOL)
-                assert ok, f"{name} algo={algo} {p.name} row {r}: err/bound {ratio:.3g}"
-    torch.cuda.synchronize()
-    assert d.pattern_untouched()
-
-
 def test_config_spmm_full(b):
     p = W.spmm_case()
     d = DevProblem(p)
@@ -286,11 +247,9 @@ def test_config_sddmm_full(b):
     gate(b.sddmm(d.row_ptr, d.col_idx, None, d.A, d.B), ref, T, "sddmm config, NULL values")
 
 
-def test_config_attention_full(b):
-    for prob in (0, 7):
+def test_config_attention_fused_equals_separate_launches(b):
+    for prob in (0, 7):   # (every element of all eight problems: tests/test_gpu_configs.py)
         p = W.attention_case(prob)
-        assert abs(p.nnz / 4096 ** 2 - 0.20) < 0.002
-        check_sampled(b, p, (0,), ("fusedmm", "sddmm", "spmm"))
         # fused == separate launches on the GPU too (C rounded to fp32 in between)
         d = DevProblem(p)
         C = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B)
@@ -298,13 +257,6 @@ def test_config_attention_full(b):
         O1 = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D)
         scale = float(O1.abs().max())
         assert float((O1 - O2).abs().max()) <= 1e-4 * scale
-
-
-@pytest.mark.parametrize("density,N", [(0.1, 128), (0.3, 512), (0.2, 256)])
-def test_config_sweep_sampled(b, density, N):
-    p = W.sweep_case(density, N)
-    assert p.nnz == round(density * 8192 * 8192)
-    check_sampled(b, p, (0,), ("spmm", "sddmm", "fusedmm"))
 
 
 def test_device_status_is_reset_by_every_family(b):

@@ -278,11 +278,18 @@ def test_prepared_pattern_is_shared_by_all_ops_and_stale_tables_are_detected(b):
 
 @pytest.mark.parametrize("width", [100, 101])
 @pytest.mark.parametrize("ks", [1, 2, 3])
-def test_k_split_epilogues(b, ks, width, monkeypatch):
+def test_k_split_epilogues(b, ks, width):
     """One K split stores O, two splits add their tiles into a zero-filled O, more go through slabs
     and the fixed-order sum: all three must give the same result, also for a ragged width, an output
     whose rows are padded, and an output that held NaNs before the call; repeated calls are bit-equal."""
-    monkeypatch.setenv("B2SP_FORCE_KS", str(ks))
+    b.debug_force_k_splits(ks)
+    try:
+        _k_split_epilogues(b, ks, width)
+    finally:
+        b.debug_force_k_splits(0)
+
+
+def _k_split_epilogues(b, ks, width):
     p = W.small_random(4100 + ks, 300, 1024, 0.2, 48, width)
     d = DevProblem(p)
     ws = _ws(b, b.OP_FUSEDMM, p)
@@ -347,3 +354,69 @@ def test_entry_points_can_be_captured_in_a_cuda_graph(b):
         assert b.device_status(ws) == 0
         for name, out, (ref, T) in zip(("spmm", "sddmm", "fusedmm"), (O1, C, O2), refs):
             gate(out, ref, T, f"{name} replayed from a CUDA graph, algo={algo}")
+
+
+def test_non_finite_values_in_rows_nobody_refers_to(b):
+    """Eq. 1-3 only touch the rows of B and D that a stored entry names.  The dense-tile kernels multiply
+    whole windows (by zero where nothing is stored), so an Inf or NaN in an unreferenced row -- for instance
+    uninitialised padding -- would leak into every output; the operand pre-pass detects non-finite values
+    and the row kernels produce the result of that call.  The detection is per call: the next call on the
+    same (prepared) workspace with clean operands runs on the tile kernels again."""
+    p = W.small_random(4400, 300, 700, 0.2, 64, 128)
+    dead = np.array([5, 77, 699])
+    keep = ~np.isin(p.col_idx, dead)
+    lens = np.add.reduceat(keep.astype(np.int64), p.row_ptr[:-1].astype(np.int64))
+    rp = np.zeros(p.M + 1, dtype=np.int32)
+    rp[1:] = np.cumsum(lens)
+    q = W.Problem("holes", p.M, p.K, rp, p.col_idx[keep], p.values[keep], p.Kd, p.N, p.A.copy(), p.B.copy(), p.D.copy())
+    refs = (oracle.spmm(q.row_ptr, q.col_idx, q.values, q.D),
+            oracle.sddmm(q.row_ptr, q.col_idx, q.values, q.A, q.B),
+            oracle.fusedmm(q.row_ptr, q.col_idx, q.values, q.A, q.B, q.D))
+    dirty = W.Problem("holes", q.M, q.K, q.row_ptr, q.col_idx, q.values, q.Kd, q.N, q.A, q.B.copy(), q.D.copy())
+    dirty.D[5, :] = np.nan
+    dirty.D[699, 3] = np.inf
+    dirty.B[77, :] = -np.inf
+    dirty.B[5, 0] = np.nan
+    ref_d = (oracle.spmm(dirty.row_ptr, dirty.col_idx, dirty.values, dirty.D),
+             oracle.sddmm(dirty.row_ptr, dirty.col_idx, dirty.values, dirty.A, dirty.B),
+             oracle.fusedmm(dirty.row_ptr, dirty.col_idx, dirty.values, dirty.A, dirty.B, dirty.D))
+    for r_clean, r_dirty in zip(refs, ref_d):   # the oracle never reads those rows
+        assert np.array_equal(r_clean[0], r_dirty[0]) and np.all(np.isfinite(r_dirty[0]))
+    dc, dd = DevProblem(q), DevProblem(dirty)
+    n = max(b.workspace_bytes(op, q.M, q.K, q.Kd, q.N, q.nnz) for op in range(3))
+    ws = torch.empty(max(n, 1 << 20), dtype=torch.uint8, device="cuda")
+
+    def run(d, algo, tag):
+        out = b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=algo)
+        gate(out, *refs[0], f"spmm {tag}")
+        out = b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=algo)
+        gate(out, *refs[1], f"sddmm {tag}")
+        out = b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=algo)
+        gate(out, *refs[2], f"fusedmm {tag}")
+        assert b.device_status(ws) == 0
+        flags = ws[320:332].view(torch.int32).cpu().numpy()
+        assert flags[1] == 0 and flags[2] == 0, "the per-call flag and its reader count are reset by the fallback"
+        return int(flags[0])
+
+    run(dd, TILE, "tile, NaN / Inf in unreferenced rows")
+    run(dc, TILE, "tile, clean operands afterwards")
+    b.prepare_pattern(dc.row_ptr, dc.col_idx, q.K, ws)
+    assert run(dc, 4, "prepared table, clean") == 0
+    b.prepare_pattern(dd.row_ptr, dd.col_idx, q.K, ws)
+    assert run(dd, 4, "prepared table, NaN / Inf in unreferenced rows") == 0   # the table itself stays usable
+    b.prepare_pattern(dc.row_ptr, dc.col_idx, q.K, ws)
+    assert run(dc, 4, "prepared table, clean again") == 0
+    # a row of A without stored entries may hold anything as well
+    lens = np.diff(q.row_ptr)
+    empty = W.Problem("empty-row", q.M, q.K, q.row_ptr.copy(), q.col_idx, q.values, q.Kd, q.N, q.A.copy(), q.B, q.D)
+    a, e = empty.row_ptr[10], empty.row_ptr[11]
+    ci = np.concatenate([q.col_idx[:a], q.col_idx[e:]])
+    v = np.concatenate([q.values[:a], q.values[e:]])
+    empty.row_ptr[11:] -= (e - a)
+    empty = W.Problem("empty-row", q.M, q.K, empty.row_ptr, ci, v, q.Kd, q.N, empty.A, q.B, q.D)
+    empty.A[10, :] = np.nan
+    de = DevProblem(empty)
+    ref, T = oracle.fusedmm(empty.row_ptr, empty.col_idx, empty.values, empty.A, empty.B, empty.D)
+    assert np.all(ref[10] == 0) and np.all(np.isfinite(ref))
+    out = b.fusedmm(de.row_ptr, de.col_idx, de.values, de.A, de.B, de.D, workspace=ws, algo=TILE)
+    gate(out, ref, T, "fusedmm tile, NaN in the A row of an empty row of S")
