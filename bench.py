@@ -288,6 +288,60 @@ def measure_problems(torch, b, device, flush, problems, ops, fp32_peak_gflops, h
     return out
 
 
+def measure_batched(torch, b, device, flush, problems, fp32_peak_gflops, hbm_gbs, reps, check=True):
+    """The attention-shaped configuration through b2sp_fusedmm_batched: all problems in ONE call (one pattern
+    pre-pass, one operand pre-pass, one tile launch).  Same protocol and fields as measure_problems."""
+    import oracle
+    stream = torch.cuda.current_stream()
+    nb, p0 = len(problems), problems[0]
+    stride = (max(p.nnz for p in problems) + 3) // 4 * 4
+    ci = np.zeros((nb, stride), dtype=np.int32)
+    sv = np.zeros((nb, stride), dtype=np.float32)
+    for i, p in enumerate(problems):
+        ci[i, :p.nnz], sv[i, :p.nnz] = p.col_idx, p.values
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(device)
+    rp, ci, sv = dev(np.stack([p.row_ptr for p in problems])), dev(ci), dev(sv)
+    A, B, D = (dev(np.stack([getattr(p, k) for p in problems])) for k in "ABD")
+    O = torch.empty((nb, p0.M, p0.N), dtype=torch.float32, device=device)
+    ws = torch.empty(b.workspace_bytes_batched(nb, p0.M, p0.K, p0.Kd, p0.N, stride), dtype=torch.uint8, device=device)
+    call = lambda a: b.fusedmm_batched(rp, ci, sv, A, B, D, out=O, workspace=ws, algo=a)
+    call(b.ALGO_AUTO)
+    torch.cuda.synchronize()
+    auto = b.last_algo(2)
+    if auto == b.ALGO_TILE:
+        b.prepare_pattern_batched(rp, ci, p0.K, ws)
+        fn = lambda: call(b.ALGO_TILE_PREPARED)
+    else:
+        fn = lambda: call(b.ALGO_AUTO)
+    for _ in range(3):
+        fn()
+    mean, mn = time_calls(torch, stream, flush, fn, reps)
+    launches = b.last_launches(2)
+    ok, worst = True, 0.0
+    if check:
+        got = O.cpu().numpy()
+        for i, p in enumerate(problems):
+            ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D)
+            k, ratio = oracle.within_tolerance(got[i], ref, T)
+            ok, worst = ok and bool(k), max(worst, float(ratio))
+        ok = ok and b.device_status(ws) == 0
+    fn = lambda: call(b.ALGO_AUTO)
+    for _ in range(3):
+        fn()
+    stateless = time_calls(torch, stream, flush, fn, reps)[0]
+    flops = sum(W.flops("fusedmm", p.nnz, p.Kd, p.N) for p in problems)
+    nbytes = sum(W.compulsory_bytes("fusedmm", p.M, p.K, p.nnz, p.Kd, p.N) for p in problems)
+    t_alu, t_hbm = flops / (fp32_peak_gflops * 1e9), nbytes / (hbm_gbs * 1e9)
+    t_roof = max(t_alu, t_hbm)
+    return {"ms": round(mean, 4), "ms_min": round(mn, 4), "roofline_frac": round(t_roof / (mean * 1e-3), 4),
+            "roofline_bound": "alu" if t_alu >= t_hbm else "hbm", "gflops": round(flops / mean / 1e6, 1),
+            "algo": b.ALGO_NAMES[auto] + (" (window tables prepared once)" if auto == b.ALGO_TILE else ""),
+            "launches": launches, "stateless_ms": round(stateless, 4),
+            "stateless_roofline_frac": round(t_roof / (stateless * 1e-3), 4),
+            "call": f"b2sp_fusedmm_batched, {nb} problems in one call",
+            "parity_ok": ok if check else None, "parity_worst_error_over_allowed": round(worst, 4) if check else None}
+
+
 # The "largest configurations" besides the headline workload: SPMM config, SDDMM config, the eight
 # attention-shaped problems, and the 30% sweep points at the wider outputs.
 EXTRA_CONFIGS = (
@@ -655,6 +709,13 @@ def main():
         for cname, make, cops in EXTRA_CONFIGS:
             configs[cname] = measure_problems(torch, b, device, flush, make(), cops, fp32_peak_gflops, hbm_gbs,
                                               args.config_reps, check=not args.no_cpu_baseline)
+            if cname.startswith("attention"):
+                probs = make()
+                o = configs[cname]["ops"]
+                o["fusedmm_one_call_each"] = o["fusedmm"]
+                o["fusedmm"] = measure_batched(torch, b, device, flush, probs, fp32_peak_gflops, hbm_gbs,
+                                               args.config_reps, check=not args.no_cpu_baseline)
+                del probs
             if set(("sddmm", "spmm", "fusedmm")) <= set(cops):
                 o = configs[cname]["ops"]
                 configs[cname]["fused_speedup_over_separate_launches"] = round(

@@ -160,6 +160,43 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz,
                          void *workspace, size_t workspace_bytes, int algo, void *stream);
 
 /*
+ * FusedMM (Eq. 3 / Alg. 3) on a batch of independent problems of the same sizes in one call -- the rows
+ * of Alg. 3 are independent work units, and so are whole problems: e.g. the (batch x heads) problems of
+ * sparse attention, O_b = (S_b .* (Q_b * K_b^T)) * V_b.  One pattern pre-pass, one operand pre-pass and one
+ * kernel launch cover all problems (CTAs of all problems are in flight together).
+ *   batch            number of problems (>= 1)
+ *   M, K, Kd, N      sizes of every problem, as for b2sp_fusedmm
+ *   row_ptr, row_ptr_stride   problem b's row pointers are row_ptr + b * row_ptr_stride (M + 1 of them,
+ *                    starting at 0: positions count inside the problem's own col_idx array);
+ *                    row_ptr_stride >= M + 1, or 0 when all problems share one pattern
+ *   col_idx, s_values, nnz_stride   problem b's column indices (and stored values, if s_values is not
+ *                    NULL) are col_idx + b * nnz_stride (s_values + b * nnz_stride); nnz_stride is at least
+ *                    every problem's entry count (row_ptr_b[M]); with a shared pattern pass nnz_stride = that
+ *                    count for the size queries and the family choice -- then s_values is shared too
+ *                    (stride 0 is taken when row_ptr_stride is 0)
+ *   A, lda, stride_a (and B, D, O likewise)   problem b's operand is A + b * stride_a, row-major with
+ *                    leading dimension lda; an input's stride may be 0 (operand shared by all problems);
+ *                    outputs must not overlap: stride_o >= (M - 1) * ldo + N
+ * Workspace: b2sp_workspace_bytes_batched(...) bytes.  algo as for b2sp_fusedmm; B2SP_ALGO_ROW and
+ * B2SP_ALGO_ROW_NAT both take the rows in natural order; B2SP_ALGO_TILE_PREPARED needs a table built by
+ * b2sp_prepare_pattern_batched with the same batch, M, K, nnz_stride, row_ptr, row_ptr_stride and col_idx.
+ * B2SP_ALGO_AUTO chooses the family from the density nnz_stride / (M * K).  Outputs wider than 256
+ * columns (where a single problem takes two phases, see b2sp_fusedmm) run on the row kernels.
+ * Every other convention (device pointers, asynchronous on `stream`, outputs overwritten, patterns that
+ * are not strictly sorted handled by the row kernels inside the same call) is b2sp_fusedmm's.
+ */
+size_t b2sp_workspace_bytes_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride);
+b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, long long nnz_stride, const int *row_ptr,
+                                         long long row_ptr_stride, const int *col_idx, void *workspace,
+                                         size_t workspace_bytes, void *stream);
+b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                 const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                 const float *s_values, const float *A, long long lda, long long stride_a,
+                                 const float *B, long long ldb, long long stride_b, const float *D, long long ldd,
+                                 long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
+                                 size_t workspace_bytes, int algo, void *stream);
+
+/*
  * Host-buffer forms of the three ops: every data pointer is a HOST pointer (pinned memory
  * makes the copies asynchronous and faster, pageable memory also works).  Each call copies
  * its inputs to the device, runs the device entry point above with algo = B2SP_ALGO_AUTO,

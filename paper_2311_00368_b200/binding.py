@@ -53,6 +53,13 @@ lib.b2sp_fusedmm_host.restype = _i
 lib.b2sp_fusedmm_host.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.b2sp_spmm_static_scratch.restype = _i
 lib.b2sp_spmm_static_scratch.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp]
+lib.b2sp_workspace_bytes_batched.restype = _sz
+lib.b2sp_workspace_bytes_batched.argtypes = [_i, _i, _i, _i, _i, _ll]
+lib.b2sp_prepare_pattern_batched.restype = _i
+lib.b2sp_prepare_pattern_batched.argtypes = [_i, _i, _i, _ll, _vp, _ll, _vp, _vp, _sz, _vp]
+lib.b2sp_fusedmm_batched.restype = _i
+lib.b2sp_fusedmm_batched.argtypes = [_i, _i, _i, _i, _i, _ll, _vp, _ll, _vp, _vp, _vp, _ll, _ll, _vp, _ll, _ll,
+                                     _vp, _ll, _ll, _vp, _ll, _ll, _vp, _sz, _i, _vp]
 lib.b2sp_prepare_pattern.restype = _i
 lib.b2sp_prepare_pattern.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_validate_csr.restype = _i
@@ -216,6 +223,61 @@ def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=
     _check(lib.b2sp_fusedmm(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
                             _ld(A), _ptr(B), _ld(B), _ptr(D), _ld(D), _ptr(out), _ld(out), _ptr(ws), wsb,
                             algo, _stream()), "b2sp_fusedmm")
+    return out
+
+
+def _batch_dims(row_ptr, col_idx):
+    """[batch, M + 1] row pointers and [batch, nnz_stride] column indices (a 1-D row_ptr: one shared pattern)."""
+    if row_ptr.dim() == 1:
+        return None, row_ptr.numel() - 1, 0, col_idx.shape[-1]
+    assert row_ptr.stride(1) == 1 and col_idx.dim() == 2 and col_idx.stride(1) == 1
+    return row_ptr.shape[0], row_ptr.shape[1] - 1, row_ptr.stride(0), col_idx.stride(0)
+
+
+def _batch_stride(t, batch):
+    """Element stride between the problems of a [batch, rows, cols] operand (0 for a shared [rows, cols] one)."""
+    if t.dim() == 2:
+        return 0
+    assert t.dim() == 3 and t.shape[0] == batch and (t.shape[2] <= 1 or t.stride(2) == 1)
+    return t.stride(0)
+
+
+def workspace_bytes_batched(batch: int, M: int, K: int, Kd: int, N: int, nnz_stride: int) -> int:
+    return int(lib.b2sp_workspace_bytes_batched(batch, M, K, Kd, N, nnz_stride))
+
+
+def prepare_pattern_batched(row_ptr, col_idx, K, workspace, batch=None):
+    """b2sp_prepare_pattern_batched: the window tables of a batch of patterns (row_ptr [batch, M + 1],
+    col_idx [batch, nnz_stride]; 1-D tensors with `batch`: one pattern shared by all problems)."""
+    nb, M, rps, nzs = _batch_dims(row_ptr, col_idx)
+    nb = batch if nb is None else nb
+    _check(lib.b2sp_prepare_pattern_batched(nb, M, K, nzs, _ptr(row_ptr), rps, _ptr(col_idx), _ptr(workspace),
+                                            workspace.numel(), _stream()), "b2sp_prepare_pattern_batched")
+
+
+def fusedmm_batched(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO):
+    """b2sp_fusedmm_batched: O[b] = (S[b] .* (A[b] @ B[b].T)) @ D[b] for all problems of a batch in one
+    call.  row_ptr [batch, M + 1] (each problem's positions start at 0), col_idx / s_values
+    [batch, nnz_stride] (rows padded to a common length), A [batch, M, Kd], B [batch, K, Kd],
+    D [batch, K, N]; a 1-D row_ptr / col_idx / s_values or a 2-D dense operand is shared by all problems."""
+    _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
+    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
+    _want(D, torch.float32, "D")
+    nb, M, rps, nzs = _batch_dims(row_ptr, col_idx)
+    if nb is None:
+        nb = max(t.shape[0] if t.dim() == 3 else 1 for t in (A, B, D))
+    K, Kd, N = B.shape[-2], B.shape[-1], D.shape[-1]
+    if out is None:
+        out = torch.empty((nb, M, N), dtype=torch.float32, device=D.device)
+    assert out.dim() == 3 and out.shape[0] == nb and out.stride(2) == 1
+    if workspace is None:
+        workspace = torch.empty(max(workspace_bytes_batched(nb, M, K, Kd, N, nzs), 1 << 20), dtype=torch.uint8,
+                                device=D.device)
+    ld = lambda t: t.stride(-2) if t.shape[-2] > 1 else max(t.shape[-1], t.stride(-2))
+    _check(lib.b2sp_fusedmm_batched(nb, M, K, Kd, N, nzs, _ptr(row_ptr), rps, _ptr(col_idx), _ptr(s_values),
+                                    _ptr(A), ld(A), _batch_stride(A, nb), _ptr(B), ld(B), _batch_stride(B, nb),
+                                    _ptr(D), ld(D), _batch_stride(D, nb), _ptr(out), ld(out), out.stride(0),
+                                    _ptr(workspace), workspace.numel(), algo, _stream()), "b2sp_fusedmm_batched")
     return out
 
 

@@ -144,7 +144,7 @@ template <int KU, int U, int SPLIT>
 b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
                          const int *col_idx, const float *sv, const float *A, int64_t lda,
                          const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
-                         int64_t ldo, const int *order, int *gate, int *clear)
+                         int64_t ldo, const int *order, int *gate, int *clear, const RowBatch &rb)
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
@@ -158,7 +158,7 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
     launch_row(kern, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
-               nrows, clear);
+               nrows, clear, rb);
     return B2SP_OK;
 }
 
@@ -167,10 +167,10 @@ b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int K
                                 const int *row_ptr, const int *col_idx, const float *sv,
                                 const float *A, int64_t lda, const float *B, int64_t ldb,
                                 const float *D, int64_t ldd, float *O, int64_t ldo,
-                                const int *order, int *gate, int *clear)
+                                const int *order, int *gate, int *clear, const RowBatch &rb)
 {
 #define B2SP_F(U_, S_) \
-    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear)
+    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb)
     if (g.SPLIT == 4) B2SP_F(1, 4);
     if (g.SPLIT == 2) B2SP_F(1, 2);
     if (g.U == 1) B2SP_F(1, 1);
@@ -429,26 +429,27 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const int *col_idx,
                               const float *s_values, const float *A, long long lda, const float *B,
                               long long ldb, const float *D, long long ldd, float *O, long long ldo,
-                              const int *order, int *gate, int *clear, cudaStream_t st)
+                              const int *order, int *gate, int *clear, cudaStream_t st,
+                              int nbatch = 1, const RowBatch &rb = RowBatch{0, 0, 0, 0, 0, 0})
 {
     b2sp_status rc = B2SP_OK;
     bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
                Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
-               Kd <= 40960;
+               Kd <= 40960 && ((rb.A | rb.B | rb.D | rb.O) & 3) == 0;
     if (vec) {
         Geom g = pick_geom(N);
-        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
+        dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab), (unsigned)nbatch);
         switch (pick_ku(Kd)) {
-        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
-        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
-        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
-        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear); break;
+        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
         }
         if (rc != B2SP_OK) return rc;
     } else {
-        dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
+        dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128), (unsigned)nbatch);
         launch_row(fusedmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
-                   D, ldd, O, ldo, order, gate, M, clear);
+                   D, ldd, O, ldo, order, gate, M, clear, rb);
     }
     return check_launch();
 }
@@ -514,6 +515,112 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     }
     rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, clear, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
+    return rc;
+}
+
+// ---- batched FusedMM --------------------------------------------------------------------------------
+namespace {
+
+bool bad_batch_args(int batch, int M, int K, long long nnz_stride, const int *row_ptr, long long row_ptr_stride,
+                    const int *col_idx)
+{
+    if (batch < 1 || M < 0 || K < 0 || nnz_stride < 0 || nnz_stride > (long long)INT_MAX) return true;
+    if (M > 0 && !row_ptr) return true;
+    if (row_ptr_stride != 0 && row_ptr_stride < (long long)M + 1) return true;
+    if (nnz_stride > 0 && (!col_idx || K == 0 || M == 0)) return true;
+    return false;
+}
+
+FusedPlan plan_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride)
+{
+    if (fusedmm_two_phase(N)) return FusedPlan();   // wide outputs: not on the dense-tile family in a batch
+    return plan_fused_tile(M, K, Kd, N, nnz_stride, row_workspace_bytes(M), true, batch);
+}
+
+}  // namespace
+
+size_t b2sp_workspace_bytes_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride)
+{
+    if (batch < 1 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz_stride < 0) return 0;
+    const size_t rows = row_workspace_bytes(M);
+    const FusedPlan p = plan_batched(batch, M, K, Kd, N, nnz_stride);
+    return p.feasible && p.bytes > rows ? p.bytes : rows;
+}
+
+b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, long long nnz_stride, const int *row_ptr,
+                                         long long row_ptr_stride, const int *col_idx, void *workspace,
+                                         size_t workspace_bytes, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_batch_args(batch, M, K, nnz_stride, row_ptr, row_ptr_stride, col_idx) || M == 0 || K == 0 || nnz_stride == 0)
+        return B2SP_ERR_INVALID_ARG;
+    const size_t need = pattern_table_offset(M) + pattern_table_bytes(M, K, batch);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, need);
+    if (rc != B2SP_OK) return rc;
+    int launches = 0;
+    BatchDesc bd;
+    bd.count = batch; bd.rp = row_ptr_stride; bd.nz = row_ptr_stride == 0 ? 0 : nnz_stride;   // a shared pattern
+    return pattern_pass(false, M, K, nnz_stride, row_ptr, col_idx, workspace, st, &launches, bd);
+}
+
+b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                 const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                 const float *s_values, const float *A, long long lda, long long stride_a,
+                                 const float *B, long long ldb, long long stride_b, const float *D, long long ldd,
+                                 long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
+                                 size_t workspace_bytes, int algo, void *stream)
+{
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (bad_batch_args(batch, M, K, nnz_stride, row_ptr, row_ptr_stride, col_idx) || Kd < 0 || N < 0)
+        return B2SP_ERR_INVALID_ARG;
+    if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return B2SP_ERR_INVALID_ARG;
+    const bool prepared = algo == B2SP_ALGO_TILE_PREPARED;
+    if (prepared) algo = B2SP_ALGO_TILE;
+    if (stride_a < 0 || stride_b < 0 || stride_d < 0) return B2SP_ERR_INVALID_ARG;
+    if (M > 0 && N > 0 && (!O || ldo < N || (batch > 1 && stride_o < (long long)(M - 1) * ldo + N))) return B2SP_ERR_INVALID_ARG;
+    if (nnz_stride > 0 && N > 0 && (!D || ldd < N)) return B2SP_ERR_INVALID_ARG;
+    if (nnz_stride > 0 && N > 0 && Kd > 0 && (!A || !B || lda < Kd || ldb < Kd)) return B2SP_ERR_INVALID_ARG;
+    const size_t row_bytes = row_workspace_bytes(M);
+    b2sp_status rc = check_workspace(workspace, workspace_bytes, row_bytes);
+    if (rc != B2SP_OK) return rc;
+    FusedPlan plan;
+    // (the family is chosen from nnz_stride, an upper bound of every problem's entry count)
+    if (algo == B2SP_ALGO_TILE ||
+        (algo == B2SP_ALGO_AUTO && tile_profitable(B2SP_OP_FUSEDMM, M, K, Kd < N ? Kd : N, nnz_stride)))
+        plan = plan_batched(batch, M, K, Kd, N, nnz_stride);
+    int use = B2SP_ALGO_ROW_NAT;   // the row family takes the problems' rows in natural order
+    if (plan.feasible && workspace_bytes >= plan.bytes) use = B2SP_ALGO_TILE;
+    else if (algo == B2SP_ALGO_TILE) return plan.feasible ? B2SP_ERR_WORKSPACE : B2SP_ERR_UNSUPPORTED;
+    g_last_algo[B2SP_OP_FUSEDMM] = use;
+    int launches = 0;
+    g_last_launches[B2SP_OP_FUSEDMM] = 0;
+    if (M == 0 || N == 0) return B2SP_OK;
+    if (nnz_stride == 0 || Kd == 0) {   // empty patterns or empty dot products: zero outputs
+        for (int b = 0; b < batch; ++b) {
+            rc = zero_rows(O + (long long)b * stride_o, ldo, M, N, st);
+            if (rc != B2SP_OK) return rc;
+        }
+        return B2SP_OK;
+    }
+    const long long nz_step = row_ptr_stride == 0 ? 0 : nnz_stride;   // a shared pattern shares its arrays
+    const RowBatch rb{row_ptr_stride, nz_step, stride_a, stride_b, stride_d, stride_o};
+    if (use == B2SP_ALGO_TILE) {
+        BatchDesc bd;
+        bd.count = batch; bd.rp = row_ptr_stride; bd.nz = nz_step;
+        bd.A = stride_a; bd.B = stride_b; bd.D = stride_d; bd.O = stride_o;
+        rc = fused_tile(plan, prepared, 1, M, K, Kd, N, nnz_stride, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd,
+                        O, ldo, workspace, st, &launches, false, bd);
+        if (rc != B2SP_OK) return rc;
+        int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
+        rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, nullptr, st,
+                        batch, rb);
+        g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
+        return rc;
+    }
+    int *clear = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsStatusOffset);
+    rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, nullptr, clear, st,
+                    batch, rb);
+    g_last_launches[B2SP_OP_FUSEDMM] = 1;
     return rc;
 }
 

@@ -36,6 +36,12 @@ __device__ __forceinline__ int bucket_of(int len) { return len <= 0 ? 0 : 32 - _
 __device__ __forceinline__ void grid_release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void grid_wait_for_primary() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
+// A batch of independent problems of the same sizes in one launch (FusedMM only): blockIdx.z is the problem,
+// whose arrays start `*` elements after those of problem 0.  All zero for a single problem.
+struct RowBatch {
+    long long rp, nz, A, B, D, O;
+};
+
 // True when a gated launch has nothing to do (see the top of this file).  Called by every thread of the CTA.
 __device__ __forceinline__ bool gate_closed(int *gate)
 {
@@ -422,11 +428,17 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
                    const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
                    const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
-                   const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                   const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear,
+                   RowBatch batch)
 {
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
     if (gate_closed(gate)) return;
+    {   // this problem's arrays
+        const long long pb = blockIdx.z;
+        row_ptr += pb * batch.rp; col_idx += pb * batch.nz; if (s_values) s_values += pb * batch.nz;
+        A += pb * batch.A; B += pb * batch.B; D += pb * batch.D; O += pb * batch.O;
+    }
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     float4 *red = dyn_smem;                                                   // kRowWarps*U*LPN
@@ -476,10 +488,15 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
                           const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
                           int64_t ldb, const float *__restrict__ D, int64_t ldd,
                           float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
-                          int *__restrict__ gate, int nrows, int *__restrict__ clear)
+                          int *__restrict__ gate, int nrows, int *__restrict__ clear, RowBatch batch)
 {
     __shared__ float red[kRowWarps][128];
     if (gate_closed(gate)) return;
+    {   // this problem's arrays
+        const long long pb = blockIdx.z;
+        row_ptr += pb * batch.rp; col_idx += pb * batch.nz; if (s_values) s_values += pb * batch.nz;
+        A += pb * batch.A; B += pb * batch.B; D += pb * batch.D; O += pb * batch.O;
+    }
     if (clear && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *clear = 0;
     if (row_order) grid_wait_for_primary();   // launched behind the binning pass: its row order
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;

@@ -62,15 +62,16 @@ bool make_blocked_map(CUtensorMap *tm, const float *base, int rows, int groups, 
 
 // fp32 matrix [rows][cols] with row stride `ld` elements, as the target of the tile kernel's flush:
 // boxes of 16 columns x 32 rows, 64-byte swizzle.  Needs a 16-byte aligned base and row stride.
-bool make_output_map(CUtensorMap *tm, float *base, long long rows, int cols, long long ld)
+// `count` such matrices `stride` elements apart (a multiple of four) form the third dimension.
+bool make_output_map(CUtensorMap *tm, float *base, long long rows, int cols, long long ld, int count, long long stride)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
-    cuuint32_t box[2] = {16, 32};
-    cuuint32_t estr[2] = {1, 1};
-    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)count};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)(count > 1 ? stride : rows * ld) * 4};
+    cuuint32_t box[3] = {16, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -114,19 +115,28 @@ size_t pattern_table_offset(int M)
 {
     return align_up(align_up(kWsHeaderBytes + sizeof(int) * (size_t)M, 256), 1024);
 }
-size_t pattern_table_bytes(int M, int K)
+size_t pattern_table_bytes(int M, int K, int batch)
 {
-    return sizeof(int2) * (size_t)M * (size_t)((K + kTileKC - 1) / kTileKC);
+    return sizeof(int2) * (size_t)batch * (size_t)M * (size_t)((K + kTileKC - 1) / kTileKC);
 }
 
+namespace {
+// What a window table is built from (for a batch, `nnz` is the distance between the problems' col_idx arrays).
+PatternSignature make_signature(int M, int K, int Wk, long long nnz, const int *row_ptr, const int *col_idx,
+                                const BatchDesc &batch)
+{
+    return PatternSignature{kPatternMagic, M, K, Wk, nnz, row_ptr, col_idx, batch.count, batch.rp, batch.nz};
+}
+}  // namespace
+
 b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
-                         void *workspace, cudaStream_t st, int *launches)
+                         void *workspace, cudaStream_t st, int *launches, const BatchDesc &batch)
 {
     char *ws = static_cast<char *>(workspace);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
     PatternSignature *sig_dev = reinterpret_cast<PatternSignature *>(ws + kWsSignatureOffset);
     const int Wk = (K + kTileKC - 1) / kTileKC;
-    PatternSignature sig{kPatternMagic, M, K, Wk, nnz, row_ptr, col_idx};
+    const PatternSignature sig = make_signature(M, K, Wk, nnz, row_ptr, col_idx, batch);
     // A prepared table is used as it is: the tile kernel itself compares the signature stored beside
     // the table with these arrays and raises the fallback flag on a mismatch.
     if (prepared) return B2SP_OK;
@@ -134,8 +144,9 @@ b2sp_status pattern_pass(bool prepared, int M, int K, long long nnz, const int *
     int2 *win = reinterpret_cast<int2 *>(ws + pattern_table_offset(M));
     if (Wk > kMasksMaxWk) return B2SP_ERR_UNSUPPORTED;
     if (!allow_dynamic_smem<-1>(reinterpret_cast<const void *>(tile_masks_kernel), kMasksMaxWk * 4)) return B2SP_ERR_CUDA;
-    const int cap = kSMs * 64;
-    tile_masks_kernel<<<M < cap ? M : cap, kMasksWarps * 32, (size_t)Wk * 4, st>>>(M, K, Wk, nnz, row_ptr, col_idx, win, flags, sig, sig_dev);
+    const long long cap = kSMs * 64, rows_all = (long long)M * batch.count;
+    tile_masks_kernel<<<(unsigned)(rows_all < cap ? rows_all : cap), kMasksWarps * 32, (size_t)Wk * 4, st>>>(
+        M, K, Wk, nnz, row_ptr, col_idx, win, flags, sig, sig_dev);
     *launches += 1;
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
@@ -168,9 +179,10 @@ bool tile_profitable(int op, int M, int K, int width, long long nnz)
     return density >= (width >= 64 ? crossover : narrow * crossover);
 }
 
-FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused)
+FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused, int batch)
 {
     FusedPlan p;
+    if (batch < 1 || (long long)batch * ((K + kFusedBlk - 1) / kFusedBlk * kFusedBlk) > 0x7fffff00ll) return p;   // stacked operand rows are int coordinates
     if (M <= 0 || K <= 0 || Kd < 0 || Kd > 128 || nnz <= 0 || (fused && N <= 0) || (!fused && Kd == 0)) return p;
     p.Wk = (K + kFusedW - 1) / kFusedW;
     p.Kp = (K + kFusedBlk - 1) / kFusedBlk * kFusedBlk;   // operand copies padded to whole 128-column blocks
@@ -179,27 +191,27 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     p.NT = fused && N <= 64 ? 64 : kFusedNT;   // a 64-column GEMM2 costs 46 instead of 64 cycles per MMA
     p.Nt = fused ? (N + p.NT - 1) / p.NT : 1;
     p.Np = fused ? p.Nt * p.NT : 0;
-    size_t win_bytes = sizeof(int2) * (size_t)M * (size_t)p.Wk;
+    size_t win_bytes = sizeof(int2) * (size_t)batch * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
-    p.KS = pick_split(p.Mt * p.Nt, p.Kp / kFusedBlk);
+    p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
     off = align_up(off + win_bytes, 1024);
-    size_t bbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Kdp;
+    size_t bbytes = sizeof(float) * (size_t)batch * (size_t)p.Kp * (size_t)p.Kdp;
     p.off_bhi = off;
     off = align_up(off + bbytes, 1024);
     p.off_blo = off;
     off = align_up(off + bbytes, 1024);
     if (fused) {
-        size_t dbytes = sizeof(float) * (size_t)p.Kp * (size_t)p.Np;
+        size_t dbytes = sizeof(float) * (size_t)batch * (size_t)p.Kp * (size_t)p.Np;
         p.off_dhi = off;
         off = align_up(off + dbytes, 1024);
         p.off_dlo = off;
         off = align_up(off + dbytes, 1024);
         p.off_part = off;
-        if (p.KS > 1) off += sizeof(float) * (size_t)p.KS * (size_t)p.Mt * kFusedRows * (size_t)p.Np;
+        if (p.KS > 1) off += sizeof(float) * (size_t)batch * (size_t)p.KS * (size_t)p.Mt * kFusedRows * (size_t)p.Np;
         p.off_cnt = off;   // one arrival counter per output tile (more than one K split only)
-        if (p.KS > 1) off = align_up(off + sizeof(int) * (size_t)p.Mt * (size_t)p.Nt, 256);
+        if (p.KS > 1) off = align_up(off + sizeof(int) * (size_t)batch * (size_t)p.Mt * (size_t)p.Nt, 256);
     }
     p.bytes = align_up(off, 256);
     p.feasible = true;
@@ -220,14 +232,14 @@ TwoPhasePlan plan_two_phase(int M, int K, int Kd, int N, long long nnz, size_t b
 
 namespace {
 
-template <int KDP, int MODE>
+template <int KDP, int MODE, bool BATCHED>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                               const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                               cudaStream_t st)
 {
     using Cfg = FusedCfg<KDP, MODE>;
-    auto kern = fused_tile_kernel<KDP, MODE>;
-    if (!allow_dynamic_smem<KDP * 4 + MODE>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
+    auto kern = fused_tile_kernel<KDP, MODE, BATCHED>;
+    if (!allow_dynamic_smem<KDP * 8 + MODE * 2 + (BATCHED ? 1 : 0)>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
     // a programmatic dependent of the operand-split kernel: its CTAs are placed while that kernel still runs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)items);
@@ -248,9 +260,14 @@ b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE>(bh, bl, dh, dl, out, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, MODE>(bh, bl, dh, dl, out, a, items, st);
-    return launch_fused_tile<128, MODE>(bh, bl, dh, dl, out, a, items, st);
+    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
+        if (kdp == 32) return launch_fused_tile<32, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
+    }
+    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false>(bh, bl, dh, dl, out, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, MODE, false>(bh, bl, dh, dl, out, a, items, st);
+    return launch_fused_tile<128, MODE, false>(bh, bl, dh, dl, out, a, items, st);
 }
 
 // Splits (or only checks) up to three dense operands, clears the device status word and optionally
@@ -281,8 +298,10 @@ void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const Ta
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
                        const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
                        long long lda, const float *B, long long ldb, const float *D, long long ldd,
-                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches, bool keep_status)
+                       float *out, long long ldo, void *workspace, cudaStream_t st, int *launches, bool keep_status,
+                       const BatchDesc &batch)
 {
+    const int nb = batch.count;
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
@@ -293,12 +312,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 
     const bool fused = mode != kModeSddmm, spmm = mode == kModeSpmm;
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
-    if (!spmm && (!make_blocked_map(&tm_bh, bhi, p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
-                  !make_blocked_map(&tm_bl, blo, p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
+    if (!spmm && (!make_blocked_map(&tm_bh, bhi, nb * p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
+                  !make_blocked_map(&tm_bl, blo, nb * p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
         return B2SP_ERR_CUDA;
     if (fused) {
-        if (!make_blocked_map(&tm_dh, dhi, p.Kp, p.Np / 32, kFusedW, p.NT / 32, true) ||
-            !make_blocked_map(&tm_dl, dlo, p.Kp, p.Np / 32, kFusedW, p.NT / 32, true))
+        if (!make_blocked_map(&tm_dh, dhi, nb * p.Kp, p.Np / 32, kFusedW, p.NT / 32, true) ||
+            !make_blocked_map(&tm_dl, dlo, nb * p.Kp, p.Np / 32, kFusedW, p.NT / 32, true))
             return B2SP_ERR_CUDA;
     } else {
         tm_dh = tm_bh;   // unused by the SDDMM kernel
@@ -306,27 +325,27 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     }
     if (spmm) { tm_bh = tm_dh; tm_bl = tm_dl; }   // unused by the SPMM mode
     {
-        b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches);
+        b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches, batch);
         if (prc != B2SP_OK) return prc;
     }
     {
         // B and D are split into tf32 hi/lo copies; A, which the tile kernel splits itself, is only checked
         // for non-finite values (see split_dense_kernel).
         const int a_rows_p = (M + 3) & ~3, a_cols_p = (Kd + 31) & ~31;
-        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, 1, 0, kDenseF32, 0};
-        const SplitJob jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np, 1, 0, kDenseF32, 0};
-        const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, 1, 0, kDenseF32, 1};
+        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, nb, batch.B, kDenseF32, 0};
+        const SplitJob jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np, nb, batch.D, kDenseF32, 0};
+        const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, nb, batch.A, kDenseF32, 1};
         SplitJobs jobs;
         jobs.n = 0;
         if (!spmm) { jobs.j[jobs.n++] = jb; jobs.j[jobs.n++] = ja; }
         if (fused) jobs.j[jobs.n++] = jd;
         // With several K splits the CTA that finishes an output tile last sums the splits' slabs: the
         // per-tile arrival counters start at zero.
-        const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), p.Mt * p.Nt, 1, p.Mt * p.Nt}
+        const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), nb * p.Mt * p.Nt, 1, nb * p.Mt * p.Nt}
                                             : ZeroJob{nullptr, 0, 0, 0};
         int *clear = keep_status ? nullptr : status;
         // (a prepared table is checked against this call's arrays here, so that the flags are final before the tile kernel)
-        const TableCheck chk{PatternSignature{kPatternMagic, M, K, p.Wk, nnz, row_ptr, col_idx},
+        const TableCheck chk{make_signature(M, K, p.Wk, nnz, row_ptr, col_idx, batch),
                              prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags,
                              prepared ? 0 : 1};
         launch_split(jobs, z, clear, chk, st);
@@ -336,6 +355,8 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 
     FusedTileArgs a;
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.NT = p.NT;
+    a.batch = nb; a.ctas_per_problem = p.Mt * p.Nt * p.KS; a.Kp = p.Kp;
+    a.stride_sv = batch.nz; a.stride_A = batch.A; a.stride_O = fused ? batch.O : batch.nz;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     a.flags = flags; a.status = status;
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
@@ -351,15 +372,17 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         // (TMA clips out-of-range columns in units of 16 bytes: a width that is not a multiple of four
         // would let it write up to three floats past the end of every row of O)
         const bool aligned = (reinterpret_cast<uintptr_t>(a.out) & 15) == 0 && (a.ld_out & 3) == 0 &&
-                             (p.KS > 1 || (N & 3) == 0);
+                             (p.KS > 1 || ((N & 3) == 0 && (batch.O & 3) == 0));
         if (aligned) {
-            const long long rows = p.KS == 1 ? M : (long long)p.KS * a.slab_rows;
+            // one K split: the caller's outputs, one per problem along the third dimension; several: the slabs
+            // of all problems and splits, stacked along the rows
+            const long long rows = p.KS == 1 ? M : (long long)nb * p.KS * a.slab_rows;
             const int cols = p.KS == 1 ? N : p.Np;
-            if (!make_output_map(&tm_out, a.out, rows, cols, a.ld_out)) return B2SP_ERR_CUDA;
+            if (!make_output_map(&tm_out, a.out, rows, cols, a.ld_out, p.KS == 1 ? nb : 1, batch.O)) return B2SP_ERR_CUDA;
             a.out_tma = 1;
         }
     }
-    const int items = p.Mt * p.Nt * p.KS;
+    const int items = nb * p.Mt * p.Nt * p.KS;
     b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
                      : fused ? launch_fused_kdp<kModeFused>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
                              : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st);

@@ -55,6 +55,11 @@ constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
+    // A batch of `batch` independent problems of the same sizes in one launch: CTA blockIdx.x works on problem
+    // blockIdx.x / ctas_per_problem.  Window tables, tf32 operand copies (rows b*Kp ...), slabs and arrival
+    // counters of the problems are stacked; the caller's arrays are `stride_*` elements apart.
+    int batch, ctas_per_problem, Kp;
+    long long stride_sv, stride_A, stride_O;
     int NT;                   // O columns per CTA (UMMA N of GEMM2): 128, or 64 when N <= 64
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
@@ -120,7 +125,9 @@ struct FusedCfg {
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
 
-template <int KDP, int MODE>
+// BATCHED: the launch covers several problems (FusedTileArgs::batch); without it the problem index is the
+// constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to spare).
+template <int KDP, int MODE, bool BATCHED = false>
 __global__ void __launch_bounds__((FusedCfg<KDP, MODE>::THREADS), 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
@@ -152,13 +159,17 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int ks = blockIdx.x % a.KS;
-    const int tile = blockIdx.x / a.KS;
+    const int prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;            // problem of the batch
+    const int cta = BATCHED ? blockIdx.x % a.ctas_per_problem : blockIdx.x;
+    const int ks = cta % a.KS;
+    const int tile = cta / a.KS;
     const int nt = tile % a.Nt, mt = tile / a.Nt;
     const int nblk_all = (a.Wk + WPB - 1) / WPB;
     const int b0 = (int)((long long)nblk_all * ks / a.KS), b1 = (int)((long long)nblk_all * (ks + 1) / a.KS);
     const int nblk = b1 - b0;
     const int m0 = mt * kFusedRows, n0 = nt * a.NT;
+    const int tiles_pp = a.ctas_per_problem / a.KS;            // output tiles per problem
+    const int krow0 = prob * a.Kp;                               // first row of this problem in the stacked operand copies
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
@@ -194,8 +205,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int pro_i = q == 1 ? (warp == 5 ? 0 : (warp >> 2) - 2) : (warp >> 2);      // ... and this warp's place among them
     if (!SPMM && warp != 1 && warp != kFusedTmaWarp) {
         const int grow = m0 + row;
-        const float *arow = a.A + (long long)(grow < a.M ? grow : 0) * a.lda;
-        const bool vec = (a.lda & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
+        const float *arow = a.A + prob * a.stride_A + (long long)(grow < a.M ? grow : 0) * a.lda;
+        const bool vec = (a.lda & 3) == 0 && (a.stride_A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
 #pragma unroll 1
         for (int c = pro_i * 16; c < KDP; c += pro_n * 16) {
             uint32_t hi[16], lo[16];
@@ -266,7 +277,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 const int s = c % RING;
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
                 const uint32_t dst = ring + s * kFusedChunk;
-                const int col0 = (b0 + blk) * kFusedBlk;
+                const int col0 = krow0 + (b0 + blk) * kFusedBlk;
                 ptx::mbar_arrive_expect_tx(full(s), is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4);   // hi + lo
                 if (is_b) {   // B rows col0..col0+127, k group i
                     ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
@@ -468,7 +479,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     if (a.out_tma) {
                         if (lane == 0) ptx::bulk_wait<0>();   // the previous flush's reductions are complete (order of the sums)
                         __syncwarp();
-                        const int y = ks * a.slab_rows + m0 + q * 32;
+                        // one K split: the output itself, problem = third coordinate; several: the slabs, stacked
+                        const int y = (a.KS == 1 ? 0 : (prob * a.KS + ks) * a.slab_rows) + m0 + q * 32;
+                        const int z = a.KS == 1 ? prob : 0;
 #pragma unroll 1
                         for (int c = 0; c < a.NT / 16; ++c) {
                             const uint32_t buf = stage + (uint32_t)(c & 1) * 2048;
@@ -491,14 +504,15 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) {
-                                if (chunk == 0) ptx::tma_store_2d(&tm_out, buf, n0 + c * 16, y);
-                                else ptx::tma_reduce_add_2d(&tm_out, buf, n0 + c * 16, y);
+                                if (chunk == 0) ptx::tma_store_3d(&tm_out, buf, n0 + c * 16, y, z);
+                                else ptx::tma_reduce_add_3d(&tm_out, buf, n0 + c * 16, y, z);
                                 ptx::bulk_commit();
                             }
                         }
                     } else {
                         // output rows that are not 16-byte aligned: the same through plain stores / atomics
-                        float *obase = a.out + (long long)ks * a.slab + (long long)(m0 + q * 32) * a.ld_out;
+                        float *obase = a.out + (a.KS == 1 ? prob * a.stride_O : (long long)(prob * a.KS + ks) * a.slab) +
+                                       (long long)(m0 + q * 32) * a.ld_out;
                         const int ncols = a.KS == 1 ? a.N : a.Nt * a.NT;   // slabs are padded to whole tiles
                         const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
 #pragma unroll 1
@@ -579,10 +593,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         const int wbase = b0 * WPB, nitems = nblk * WPB * IPW;
         const unsigned lane_bit = 1u << lane, lt_mask = lane_bit - 1u;
         const bool has_values = a.s_values != nullptr;
+        const float *s_values = a.s_values + prob * a.stride_sv;           // this problem's stored values,
+        const int2 *win = a.win + (size_t)prob * a.M * a.Wk;               // window table
+        float *out_values = a.out + prob * a.stride_O;                     // and (SDDMM) output values
         auto load_rec = [&](int jj) {   // lane = row: window record of one row of item jj
             int2 r = make_int2(0, 0);
             const int hrow = m0 + (jj % IPW) * IR + lane, wglob = wbase + jj / IPW;
-            if (jj < nitems && lane < IR && hrow < a.M && wglob < a.Wk) r = __ldg(a.win + (size_t)hrow * a.Wk + wglob);
+            if (jj < nitems && lane < IR && hrow < a.M && wglob < a.Wk) r = __ldg(win + (size_t)hrow * a.Wk + wglob);
             return r;
         };
         // the records of the next two items are in flight while an item is processed
@@ -604,7 +621,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 const bool present = (m & lane_bit) != 0;
                 const int at = (int)pos + __popc(m & lt_mask);
                 vn[r] = (present && (!FUSED || !has_values)) ? 1.f : 0.f;
-                if (present && has_values) vn[r] = __ldg(a.s_values + at);
+                if (present && has_values) vn[r] = __ldg(s_values + at);
                 if (!FUSED) idx[r] = present ? at : -1;
             });
             const uint32_t slot = slots + s * Cfg::SLOT_BYTES;
@@ -633,7 +650,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (lane == 0) ptx::mbar_arrive(sl_empty(s));
                 ptx::for_each_row<IR>([&](auto rc) {
                     constexpr int r = decltype(rc)::value;
-                    if (idx[FUSED ? 0 : r] >= 0) a.out[idx[FUSED ? 0 : r]] = vn[r];
+                    if (idx[FUSED ? 0 : r] >= 0) out_values[idx[FUSED ? 0 : r]] = vn[r];
                 });
             }
         }
@@ -650,7 +667,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         // The CTA that arrives last at its output tile's counter sums the K splits' slabs, always in
         // the order of the splits, into O: no CTA waits for another and the result is reproducible.
         int *last_flag = reinterpret_cast<int *>(smem_gen + (helper_tabs - smem_base));   // the record tables are idle now
-        if (threadIdx.x == 0) *last_flag = atomicAdd(a.tile_arrivals + tile, 1) == a.KS - 1;
+        if (threadIdx.x == 0) *last_flag = atomicAdd(a.tile_arrivals + prob * tiles_pp + tile, 1) == a.KS - 1;
         __syncthreads();
         if (*last_flag) {
             __threadfence();
@@ -658,14 +675,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 const int r = e / (a.NT / 4), c = (e % (a.NT / 4)) * 4;
                 const int grow = m0 + r, n = n0 + c;
                 if (grow >= a.M || n >= a.N) continue;
-                const float *src = a.out + (long long)grow * a.ld_out + n;
+                const float *src = a.out + (long long)prob * a.KS * a.slab + (long long)grow * a.ld_out + n;
                 float4 acc = __ldcg(reinterpret_cast<const float4 *>(src));
                 for (int k = 1; k < a.KS; ++k) {
                     const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + (long long)k * a.slab));
                     acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
                 }
-                float *dst = a.O + (long long)grow * a.ldo + n;
-                if (n + 3 < a.N && (a.ldo & 3) == 0 && (reinterpret_cast<uintptr_t>(a.O) & 15) == 0) {
+                float *dst = a.O + prob * a.stride_O + (long long)grow * a.ldo + n;
+                if (n + 3 < a.N && (a.ldo & 3) == 0 && (a.stride_O & 3) == 0 && (reinterpret_cast<uintptr_t>(a.O) & 15) == 0) {
                     *reinterpret_cast<float4 *>(dst) = acc;
                 } else {
                     dst[0] = acc.x;

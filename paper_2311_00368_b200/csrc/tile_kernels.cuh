@@ -30,6 +30,7 @@ struct PatternSignature {
     int magic, M, K, Wk;
     long long nnz;
     const int *row_ptr, *col_idx;
+    long long batch, rp_stride, nz_stride;   // a batch of patterns (see tile_masks_kernel); 1, 0, 0 for a single one
 };
 constexpr int kPatternMagic = 0x62327370;
 
@@ -47,9 +48,12 @@ constexpr int kPatternMagic = 0x62327370;
 constexpr int kMasksWarps = 4;
 constexpr int kMasksMaxWk = 24 * 1024;   // the mask row must fit in the shared memory a block may ask for (96 KB)
 
+// A batch of `sig.batch` patterns of the same M and K (row_ptr arrays `sig.rp_stride` elements apart, each
+// starting at 0; col_idx arrays `sig.nz_stride` elements apart) gives one table per pattern, stacked:
+// T[(b*M + r)*Wk + w], positions relative to the pattern's own col_idx array.
 __global__ void __launch_bounds__(kMasksWarps * 32)
-tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ row_ptr,
-                  const int *__restrict__ col_idx, int2 *__restrict__ T, int *__restrict__ flags,
+tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ row_ptr0,
+                  const int *__restrict__ col_idx0, int2 *__restrict__ T, int *__restrict__ flags,
                   PatternSignature sig, PatternSignature *__restrict__ sig_out)
 {
     extern __shared__ __align__(16) unsigned mask[];     // Wk words
@@ -60,10 +64,14 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
     __shared__ int warp_total[kMasksWarps];
     constexpr unsigned kFull = 0xffffffffu;
     constexpr int NT = kMasksWarps * 32;
-    const bool vec = (reinterpret_cast<uintptr_t>(col_idx) & 15) == 0;
     const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
     bool bad = false;
-    for (int row = blockIdx.x; row < M; row += gridDim.x) {
+    const long long rows_all = (long long)M * sig.batch;
+    for (long long rowg = blockIdx.x; rowg < rows_all; rowg += gridDim.x) {
+        const int pb = (int)(rowg / M), row = (int)(rowg % M);
+        const int *__restrict__ row_ptr = row_ptr0 + pb * sig.rp_stride;
+        const int *__restrict__ col_idx = col_idx0 + pb * sig.nz_stride;
+        const bool vec = (reinterpret_cast<uintptr_t>(col_idx) & 15) == 0;
         for (int w = threadIdx.x; w < Wk; w += NT) mask[w] = 0u;
         __syncthreads();
         const int beg = __ldg(row_ptr + row), end = __ldg(row_ptr + row + 1);
@@ -136,7 +144,7 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
                 if (i < wib) before += t;
                 all += t;
             }
-            if (w < Wk) T[(size_t)row * Wk + w] = make_int2(run + before + incl - cnt, (int)m);
+            if (w < Wk) T[(size_t)rowg * Wk + w] = make_int2(run + before + incl - cnt, (int)m);
             run += all;
             __syncthreads();   // warp_total and mask are reused
         }
@@ -149,7 +157,8 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 {
     const PatternSignature h = *have;
     return h.magic == want.magic && h.M == want.M && h.K == want.K && h.Wk == want.Wk && h.nnz == want.nnz &&
-           h.row_ptr == want.row_ptr && h.col_idx == want.col_idx;
+           h.row_ptr == want.row_ptr && h.col_idx == want.col_idx && h.batch == want.batch &&
+           h.rp_stride == want.rp_stride && h.nz_stride == want.nz_stride;
 }
 
 // ---- dense operand split ----------------------------------------------------------------------------
