@@ -496,6 +496,8 @@ def main():
     ap.add_argument("--grid", action="store_true",
                     help="run the paper's 72-case grid (uniform-random stand-ins), one JSON line per case")
     ap.add_argument("--grid-filter", default="", help="only grid cases whose name contains this text")
+    ap.add_argument("--only-config", default="",
+                    help="time just this entry of the `configs` object (for profiler captures) and print it")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -513,6 +515,19 @@ def main():
     replicas.init("nccl", device)
     hbm_gbs, sm_max_mhz, peak_src = peaks()
     fp32_peak_gflops = SM_COUNT * FP32_LANES_PER_SM * 2 * sm_max_mhz / 1e3
+
+    if args.only_config:
+        flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=device)
+        for cname, make, cops in EXTRA_CONFIGS:
+            if cname != args.only_config:
+                continue
+            probs = make()
+            if cname.startswith("attention"):
+                res = measure_batched(torch, b, device, flush, probs, fp32_peak_gflops, hbm_gbs, args.config_reps, check=False)
+            else:
+                res = measure_problems(torch, b, device, flush, probs, cops, fp32_peak_gflops, hbm_gbs, args.config_reps, check=False)
+            print(json.dumps({"config": cname, "result": res}))
+        return 0
 
     p = make_workload(args.workload, rank)
     dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(device)

@@ -148,7 +148,8 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
-    auto kern = fusedmm_row_kernel<KU, U, SPLIT>;
+    const bool batched = grid.z > 1;
+    auto kern = batched ? fusedmm_row_kernel<KU, U, SPLIT, true> : fusedmm_row_kernel<KU, U, SPLIT, false>;
     if (smem > 48 * 1024) {
         if (smem > 200 * 1024) return B2SP_ERR_UNSUPPORTED;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=

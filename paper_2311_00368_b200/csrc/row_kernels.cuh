@@ -422,7 +422,7 @@ sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__re
 // FusedMM  (Alg. 3): per chunk, the SDDMM values stay in registers (one per lane) and are the
 // scalars of the SAXPY sweep over the same staged column indices; C never reaches memory.
 // ------------------------------------------------------------------------------------------
-template <int KU, int U, int SPLIT>
+template <int KU, int U, int SPLIT, bool BATCHED = false>
 __global__ void __launch_bounds__(kRowThreads)
 fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
                    const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
@@ -434,7 +434,7 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
     if (gate_closed(gate)) return;
-    {   // this problem's arrays
+    if (BATCHED) {   // this problem's arrays
         const long long pb = blockIdx.z;
         row_ptr += pb * batch.rp; col_idx += pb * batch.nz; if (s_values) s_values += pb * batch.nz;
         A += pb * batch.A; B += pb * batch.B; D += pb * batch.D; O += pb * batch.O;

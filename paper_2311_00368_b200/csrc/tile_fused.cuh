@@ -107,6 +107,11 @@ struct FusedCfg {
     // (measured: 12 helpers 134 us, 14 helpers 129 us, 20 helpers on 28 warps 125 us; for SPMM the same
     // layout was slower, 136-140 us against 131 us).
     static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 20;
+    // FusedMM runs two sets of processor warps (warps 2-5 and 16-19) that take alternate windows: a window is a
+    // chain of long-latency steps for its processor (slot, tensor-memory load, arithmetic, tensor-memory store,
+    // hand-over), about 2 k cycles, and with a single set that chain, not the tensor core, paced the kernel
+    // wherever a window holds less than 2 k cycles of MMAs.  The second set (odd windows) also does the flushes.
+    static constexpr int PSETS = (FUSED && !SPMM) ? 2 : 1;
     static constexpr int ITEM_ROWS = FUSED ? 32 : 16;           // rows of a helper's work item
     static constexpr int IPW = kFusedRows / ITEM_ROWS;         // items per window
     static constexpr int SLOT_BYTES = ITEM_ROWS * 128;
@@ -175,7 +180,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
         for (int b = 0; b < 2; ++b) {
             ptx::mbar_init(p_full(b), 1);
-            ptx::mbar_init(p_free(b), 4);
+            ptx::mbar_init(p_free(b), FUSED ? 4 * Cfg::PSETS : 4);
             ptx::mbar_init(pp_full(b), 4);
             ptx::mbar_init(pp_free(b), 1);
         }
@@ -383,14 +388,16 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (!SPMM && b + 1 < nblk && late_b && !failed) failed = !gemm1(b + 1);
             }
         }
-    } else if (warp >= 2 && warp < 6) {
+    } else if ((warp >= 2 && warp < 6) || (Cfg::PSETS == 2 && warp >= 16)) {
         // ---------------- processor warps (thread = row; TMEM lane quarter q) ----------------
         // FusedMM / SPMM: per window, take the row's stored values (densified and transposed by a
         // helper warp into a shared-memory slot), multiply them into P (or use them as they are for
         // SPMM), split to hi/lo and write P' to tensor memory.
         // SDDMM: per window, copy the row of P into a slot; a helper warp writes the stored entries.
         const int nwin = nblk * WPB;
-        for (int it = 0; it < nwin; ++it) {
+        constexpr int PSETS = Cfg::PSETS;
+        const int pset = warp >= 16 ? 1 : 0;   // which set of processor warps this one belongs to
+        for (int it = FUSED ? pset : 0; it < nwin; it += FUSED ? PSETS : 1) {
             const int blk = it / WPB, w = it % WPB;
             // FusedMM / SPMM: one item (32 rows) per processor warp and window.  SDDMM: two items of 16 rows,
             // lanes 0-15 and lanes 16-31 each with their own slot.
@@ -419,7 +426,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 #pragma unroll
                     for (int c = 0; c < 16; ++c) { p0[c] = 0x3f800000u; p1[c] = 0x3f800000u; }
                 } else {
-                    if (w == 0) {
+                    if (w < PSETS) {   // this set's first window of the block
                         bool ok = ptx::mbar_wait(p_full(0), blk & 1);
                         if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                         ptx::tc_fence_after_sync();
@@ -428,7 +435,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     ptx::tmem_ld_32x16(pcol, p0);
                     ptx::tmem_ld_32x16(pcol + 16, p1);
                     ptx::tmem_ld_wait();
-                    if (w == WPB - 1) {   // the whole block has been read: GEMM1 may overwrite P
+                    if (w + PSETS >= WPB) {   // this set has read its share of the block: GEMM1 may overwrite P once every set has
                         ptx::tc_fence_before_sync();
                         __syncwarp();
                         if (lane == 0) ptx::mbar_arrive(p_free(0));
@@ -656,7 +663,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         }
     }
     if (failed) atomicExch(a.status, 1);
-    if (FUSED && warp >= 2 && warp < 6 && lane == 0) {   // this warp's TMA stores / reductions have been performed
+    if (FUSED && (Cfg::PSETS == 2 ? warp >= 16 : (warp >= 2 && warp < 6)) && lane == 0) {   // this warp's TMA stores / reductions have been performed
         ptx::bulk_wait<0>();
         ptx::fence_proxy_async_all();
     }
