@@ -650,6 +650,46 @@ def main():
             per_op[op]["stateless_launches"] = b.last_launches(i)
         step()   # the outputs the parity check reads come from the timed configuration (prepared table)
         torch.cuda.synchronize()
+    # the same workload with bfloat16 dense operands and fp32 accumulation (b2sp_*_bf16), beside the fp32 ops
+    bf16 = None
+    if shared_table:
+        A16, B16, D16 = (t.to(torch.bfloat16) for t in (A, B, D))
+        O16 = torch.empty_like(O)
+        C16 = torch.empty_like(C)
+        b.prepare_pattern(rp, ci, p.K, ws)
+        bcalls = {"spmm": lambda: b.spmm(rp, ci, v, D16, K=p.K, out=O16, workspace=ws, algo=b.ALGO_TILE_PREPARED, dtype=torch.bfloat16),
+                  "sddmm": lambda: b.sddmm(rp, ci, v, A16, B16, out=C16, workspace=ws, algo=b.ALGO_TILE_PREPARED, dtype=torch.bfloat16),
+                  "fusedmm": lambda: b.fusedmm(rp, ci, v, A16, B16, D16, out=O16, workspace=ws, algo=b.ALGO_TILE_PREPARED, dtype=torch.bfloat16)}
+        bf16 = {"dtype": "bf16 A/B/D, fp32 S values, one tf32 MMA per exact product, fp32 accumulate", "ops": {}}
+        rows16 = min(p.M, 256)
+        nnz16 = int(p.row_ptr[rows16])
+        for op in OPS:
+            for _ in range(3):
+                bcalls[op]()
+            mean, mn = time_calls(torch, stream, flush, bcalls[op], 20)
+            t_roof = max(fl[op] / (fp32_peak_gflops * 1e9), by[op] / (hbm_gbs * 1e9))
+            bf16["ops"][op] = {"ms": round(mean, 4), "ms_min": round(mn, 4),
+                               "fp32_roofline_frac": round(t_roof / (mean * 1e-3), 4),
+                               "speedup_over_fp32": round(per_op[op]["ms"] / mean, 3)}
+            if not args.no_cpu_baseline and rank == 0:
+                import oracle
+                r16 = lambda t: t.to(torch.float32).cpu().numpy()
+                if op == "spmm":
+                    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, r16(D16), rows=(0, rows16))
+                    got = O16[:rows16]
+                elif op == "sddmm":
+                    ref, T = oracle.sddmm(p.row_ptr, p.col_idx, p.values, r16(A16), r16(B16), rows=(0, rows16))
+                    got = C16[:nnz16]
+                else:
+                    ref, T = oracle.fusedmm(p.row_ptr, p.col_idx, p.values, r16(A16), r16(B16), r16(D16), rows=(0, rows16))
+                    got = O16[:rows16]
+                ok, ratio = oracle.within_tolerance(got.cpu().numpy(), ref, T)
+                bf16["ops"][op]["parity_ok"] = bool(ok)
+                bf16["ops"][op]["parity_worst_error_over_allowed"] = round(float(ratio), 4)
+                bf16["ops"][op]["parity_rows"] = rows16
+        bf16["fused_speedup_over_separate_launches"] = round(
+            (bf16["ops"]["sddmm"]["ms"] + bf16["ops"]["spmm"]["ms"]) / bf16["ops"]["fusedmm"]["ms"], 3)
+        del A16, B16, D16, O16, C16
     sep_ms = per_op["sddmm"]["ms"] + per_op["spmm"]["ms"]
     fused_vs_separate = sep_ms / per_op["fusedmm"]["ms"]
 
@@ -756,7 +796,7 @@ def main():
                                else "built inside each op that needs it"),
                 "roofline": roof, "cpu_baseline": cpu_baseline, "parity": parity,
                 "e2e": e2e, "gpu_launches": int((sum(launches.values()) + (1 if shared_table else 0)) * args.steps),
-                "clocks": clocks, "ops": per_op, "configs": configs, "configs_clocks": configs_clocks,
+                "clocks": clocks, "ops": per_op, "bf16": bf16, "configs": configs, "configs_clocks": configs_clocks,
                 "fused_speedup_over_separate_launches": round(fused_vs_separate, 3),
                 "paper_context": "Intel Max 1550 (1 stack), 8k/8k/128/70%: SDDMM 9732, SPMM 11482, "
                                  "FusedMM 12647 GFLOP/s (other hardware; context only)"}

@@ -160,6 +160,34 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz,
                          void *workspace, size_t workspace_bytes, int algo, void *stream);
 
 /*
+ * The three ops with bfloat16 dense operands and fp32 accumulation -- the variant the paper's conclusion
+ * names as its next step.  A, B and D are bfloat16 (the upper 16 bits of an fp32 value; pointers passed as
+ * const void*, leading dimensions in elements); the stored values of S, all sums and the outputs stay fp32.
+ * Everything else (CSR conventions, workspace from b2sp_workspace_bytes, algo, prepared pattern tables,
+ * stream, error behaviour) is as for the fp32 entry points above.  Results satisfy the same bound against
+ * Eq. 1-3 evaluated exactly on the bfloat16 values: every product of two bfloat16 numbers is exact in
+ * fp32, only the order of the fp32 sums differs.  The row kernels gather half the bytes per dense row;
+ * the dense-tile kernels need no lo halves for operands that are exact in tf32, i.e. one tensor-core
+ * product per GEMM1 term instead of three and two per GEMM2 term.  The four-element loads of the vector
+ * kernels want 8-byte aligned operands and leading dimensions that are multiples of 4 (16 bytes and
+ * multiples of 8 for A on the dense-tile kernels); other shapes take the scalar paths.
+ */
+b2sp_status b2sp_spmm_bf16(int M, int K, int N, long long nnz,
+                           const int *row_ptr, const int *col_idx, const float *values,
+                           const void *D, long long ldd, float *O, long long ldo,
+                           void *workspace, size_t workspace_bytes, int algo, void *stream);
+b2sp_status b2sp_sddmm_bf16(int M, int K, int Kd, long long nnz,
+                            const int *row_ptr, const int *col_idx, const float *s_values,
+                            const void *A, long long lda, const void *B, long long ldb,
+                            float *out_values,
+                            void *workspace, size_t workspace_bytes, int algo, void *stream);
+b2sp_status b2sp_fusedmm_bf16(int M, int K, int Kd, int N, long long nnz,
+                              const int *row_ptr, const int *col_idx, const float *s_values,
+                              const void *A, long long lda, const void *B, long long ldb,
+                              const void *D, long long ldd, float *O, long long ldo,
+                              void *workspace, size_t workspace_bytes, int algo, void *stream);
+
+/*
  * FusedMM (Eq. 3 / Alg. 3) on a batch of independent problems of the same sizes in one call -- the rows
  * of Alg. 3 are independent work units, and so are whole problems: e.g. the (batch x heads) problems of
  * sparse attention, O_b = (S_b .* (Q_b * K_b^T)) * V_b.  One pattern pre-pass, one operand pre-pass and one

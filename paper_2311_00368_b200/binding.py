@@ -45,6 +45,12 @@ lib.b2sp_sddmm.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _
 lib.b2sp_fusedmm.restype = _i
 lib.b2sp_fusedmm.argtypes = [_i, _i, _i, _i, _ll, _vp, _vp, _vp, _vp, _ll, _vp, _ll, _vp, _ll, _vp, _ll,
                              _vp, _sz, _i, _vp]
+lib.b2sp_spmm_bf16.restype = _i
+lib.b2sp_spmm_bf16.argtypes = lib.b2sp_spmm.argtypes
+lib.b2sp_sddmm_bf16.restype = _i
+lib.b2sp_sddmm_bf16.argtypes = lib.b2sp_sddmm.argtypes
+lib.b2sp_fusedmm_bf16.restype = _i
+lib.b2sp_fusedmm_bf16.argtypes = lib.b2sp_fusedmm.argtypes
 lib.b2sp_spmm_host.restype = _i
 lib.b2sp_spmm_host.argtypes = [_i, _i, _i, _ll, _vp, _vp, _vp, _vp, _vp, _vp]
 lib.b2sp_sddmm_host.restype = _i
@@ -155,18 +161,20 @@ def debug_force_k_splits(k_splits: int) -> None:
     lib.b2sp_debug_force_k_splits(int(k_splits))
 
 
-def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALGO_AUTO):
-    """b2sp_spmm: O = S @ D.  CSR tensors int32/fp32 on the GPU; D [K, N] fp32 row-major."""
+def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALGO_AUTO, dtype=torch.float32):
+    """b2sp_spmm: O = S @ D.  CSR tensors int32/fp32 on the GPU; D [K, N] fp32 row-major
+    (dtype=torch.bfloat16: b2sp_spmm_bf16, D in bfloat16)."""
     _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
-    _want(values, torch.float32, "values"); _want(D, torch.float32, "D")
+    _want(values, torch.float32, "values"); _want(D, dtype, "D")
     M, nnz = row_ptr.numel() - 1, col_idx.numel()
     K = D.shape[0] if K is None else K
     N = D.shape[1]
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=D.device)
     ws, wsb = _workspace(OP_SPMM, M, K, 0, N, nnz, D.device, workspace, algo)
-    _check(lib.b2sp_spmm(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D), _ld(D),
-                         _ptr(out), _ld(out), _ptr(ws), wsb, algo, _stream()), "b2sp_spmm")
+    fn, name = (lib.b2sp_spmm, "b2sp_spmm") if dtype == torch.float32 else (lib.b2sp_spmm_bf16, "b2sp_spmm_bf16")
+    _check(fn(M, K, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(values), _ptr(D), _ld(D),
+                         _ptr(out), _ld(out), _ptr(ws), wsb, algo, _stream()), name)
     return out
 
 
@@ -191,10 +199,11 @@ def spmm_static_scratch(row_ptr, col_idx, values, D, K=None, out=None):
     return out
 
 
-def sddmm(row_ptr, col_idx, s_values, A, B, out=None, workspace=None, algo=ALGO_AUTO):
-    """b2sp_sddmm: out[p] = s_p * <A[i], B[j]> on S's pattern; s_values=None means all ones."""
+def sddmm(row_ptr, col_idx, s_values, A, B, out=None, workspace=None, algo=ALGO_AUTO, dtype=torch.float32):
+    """b2sp_sddmm: out[p] = s_p * <A[i], B[j]> on S's pattern; s_values=None means all ones
+    (dtype=torch.bfloat16: b2sp_sddmm_bf16, A and B in bfloat16)."""
     _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
-    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
+    _want(s_values, torch.float32, "s_values"); _want(A, dtype, "A"); _want(B, dtype, "B")
     M, nnz = row_ptr.numel() - 1, col_idx.numel()
     K, Kd = B.shape
     if A.shape != (M, Kd):
@@ -202,16 +211,18 @@ def sddmm(row_ptr, col_idx, s_values, A, B, out=None, workspace=None, algo=ALGO_
     if out is None:
         out = torch.empty(nnz, dtype=torch.float32, device=A.device)
     ws, wsb = _workspace(OP_SDDMM, M, K, Kd, 0, nnz, A.device, workspace, algo)
-    _check(lib.b2sp_sddmm(M, K, Kd, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A), _ld(A),
-                          _ptr(B), _ld(B), _ptr(out), _ptr(ws), wsb, algo, _stream()), "b2sp_sddmm")
+    fn, name = (lib.b2sp_sddmm, "b2sp_sddmm") if dtype == torch.float32 else (lib.b2sp_sddmm_bf16, "b2sp_sddmm_bf16")
+    _check(fn(M, K, Kd, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A), _ld(A),
+                          _ptr(B), _ld(B), _ptr(out), _ptr(ws), wsb, algo, _stream()), name)
     return out
 
 
-def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO):
-    """b2sp_fusedmm: O = (S .* (A @ B.T)) @ D in one pass; the sampled values never reach HBM."""
+def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO, dtype=torch.float32):
+    """b2sp_fusedmm: O = (S .* (A @ B.T)) @ D in one pass; the sampled values never reach HBM
+    (dtype=torch.bfloat16: b2sp_fusedmm_bf16, A, B and D in bfloat16)."""
     _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
-    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
-    _want(D, torch.float32, "D")
+    _want(s_values, torch.float32, "s_values"); _want(A, dtype, "A"); _want(B, dtype, "B")
+    _want(D, dtype, "D")
     M, nnz = row_ptr.numel() - 1, col_idx.numel()
     K, Kd = B.shape
     N = D.shape[1]
@@ -220,9 +231,10 @@ def fusedmm(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=D.device)
     ws, wsb = _workspace(OP_FUSEDMM, M, K, Kd, N, nnz, D.device, workspace, algo)
-    _check(lib.b2sp_fusedmm(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
+    fn, name = (lib.b2sp_fusedmm, "b2sp_fusedmm") if dtype == torch.float32 else (lib.b2sp_fusedmm_bf16, "b2sp_fusedmm_bf16")
+    _check(fn(M, K, Kd, N, nnz, _ptr(row_ptr), _ptr(col_idx), _ptr(s_values), _ptr(A),
                             _ld(A), _ptr(B), _ld(B), _ptr(D), _ld(D), _ptr(out), _ld(out), _ptr(ws), wsb,
-                            algo, _stream()), "b2sp_fusedmm")
+                            algo, _stream()), name)
     return out
 
 

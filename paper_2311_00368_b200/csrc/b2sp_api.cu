@@ -41,6 +41,9 @@ thread_local int g_last_algo[3] = {-1, -1, -1};
 thread_local int g_last_launches[3] = {0, 0, 0};
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+// alignment a dense operand needs for the four-element loads of the vector kernels (16 bytes of fp32, 8 of bf16)
+template <typename DT> inline bool aligned_vec(const DT *p) { return (reinterpret_cast<uintptr_t>(p) & (4 * sizeof(DT) - 1)) == 0; }
+template <typename DT> constexpr int dense_dtype() { return sizeof(DT) == 2 ? kDenseBf16 : kDenseF32; }
 
 inline b2sp_status check_launch()
 {
@@ -104,14 +107,14 @@ inline unsigned gated_blocks(unsigned rows, int *gate)
     return gate && rows > cap ? cap : rows;
 }
 
-template <int U, int SPLIT>
+template <int U, int SPLIT, typename DT>
 void launch_spmm(dim3 grid, cudaStream_t st, int N, const int *row_ptr, const int *col_idx,
-                 const float *values, const float *D, int64_t ldd, float *O, int64_t ldo,
+                 const float *values, const DT *D, int64_t ldd, float *O, int64_t ldo,
                  const int *order, int *gate, int *clear)
 {
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    launch_row(spmm_row_kernel<U, SPLIT>, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+    launch_row(spmm_row_kernel<U, SPLIT, DT>, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
                gate, nrows, clear);
 }
 
@@ -128,28 +131,28 @@ inline Geom pick_geom(int N)
 
 inline int pick_ku(int Kd) { return Kd <= 64 ? 2 : Kd <= 128 ? 4 : Kd <= 256 ? 8 : 0; }
 
-template <int KU>
+template <int KU, typename DT>
 void launch_sddmm(dim3 grid, cudaStream_t st, int Kd, const int *row_ptr, const int *col_idx,
-                  const float *sv, const float *A, int64_t lda, const float *B, int64_t ldb,
+                  const float *sv, const DT *A, int64_t lda, const DT *B, int64_t ldb,
                   float *out, const int *order, int *gate, int *clear)
 {
     size_t smem = KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0;
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate);
-    launch_row(sddmm_row_kernel<KU>, grid, smem, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, sv, A, lda, B, ldb, out, order,
+    launch_row(sddmm_row_kernel<KU, DT>, grid, smem, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, sv, A, lda, B, ldb, out, order,
                gate, nrows, clear);
 }
 
-template <int KU, int U, int SPLIT>
+template <int KU, int U, int SPLIT, typename DT>
 b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *row_ptr,
-                         const int *col_idx, const float *sv, const float *A, int64_t lda,
-                         const float *B, int64_t ldb, const float *D, int64_t ldd, float *O,
+                         const int *col_idx, const float *sv, const DT *A, int64_t lda,
+                         const DT *B, int64_t ldb, const DT *D, int64_t ldd, float *O,
                          int64_t ldo, const int *order, int *gate, int *clear, const RowBatch &rb)
 {
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
     const bool batched = grid.z > 1;
-    auto kern = batched ? fusedmm_row_kernel<KU, U, SPLIT, true> : fusedmm_row_kernel<KU, U, SPLIT, false>;
+    auto kern = batched ? fusedmm_row_kernel<KU, U, SPLIT, true, DT> : fusedmm_row_kernel<KU, U, SPLIT, false, DT>;
     if (smem > 48 * 1024) {
         if (smem > 200 * 1024) return B2SP_ERR_UNSUPPORTED;
         if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
@@ -163,15 +166,15 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     return B2SP_OK;
 }
 
-template <int KU>
+template <int KU, typename DT>
 b2sp_status dispatch_fused_geom(const Geom &g, dim3 grid, cudaStream_t st, int Kd, int N,
                                 const int *row_ptr, const int *col_idx, const float *sv,
-                                const float *A, int64_t lda, const float *B, int64_t ldb,
-                                const float *D, int64_t ldd, float *O, int64_t ldo,
+                                const DT *A, int64_t lda, const DT *B, int64_t ldb,
+                                const DT *D, int64_t ldd, float *O, int64_t ldo,
                                 const int *order, int *gate, int *clear, const RowBatch &rb)
 {
 #define B2SP_F(U_, S_) \
-    return launch_fused<KU, U_, S_>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb)
+    return launch_fused<KU, U_, S_, DT>(grid, st, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb)
     if (g.SPLIT == 4) B2SP_F(1, 4);
     if (g.SPLIT == 2) B2SP_F(1, 2);
     if (g.U == 1) B2SP_F(1, 1);
@@ -201,11 +204,9 @@ bool bad_csr_args(int M, int K, long long nnz, const int *row_ptr, const int *co
 
 using namespace b2sp;
 
-extern "C" {
+extern "C" int b2sp_version(void) { return 100; }
 
-int b2sp_version(void) { return 100; }
-
-const char *b2sp_status_string(b2sp_status s)
+extern "C" const char *b2sp_status_string(b2sp_status s)
 {
     switch (s) {
     case B2SP_OK: return "ok";
@@ -243,7 +244,7 @@ static size_t tile_workspace_bytes(int op, int M, int K, int Kd, int N, long lon
 
 static int tile_width(int op, int Kd, int N) { return op == B2SP_OP_SPMM ? N : op == B2SP_OP_SDDMM ? Kd : (Kd < N ? Kd : N); }
 
-size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz)
+extern "C" size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, long long nnz)
 {
     if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
     if (algo < B2SP_ALGO_AUTO || algo > B2SP_ALGO_TILE_PREPARED) return 0;
@@ -254,7 +255,7 @@ size_t b2sp_workspace_bytes_algo(int op, int algo, int M, int K, int Kd, int N, 
     return tile > rows && tile_profitable(op, M, K, tile_width(op, Kd, N), nnz) ? tile : rows;
 }
 
-size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
+extern "C" size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
 {
     if (op < 0 || op > 2 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz < 0) return 0;
     const size_t rows = row_workspace_bytes(M);
@@ -262,38 +263,40 @@ size_t b2sp_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz)
     return tile > rows ? tile : rows;
 }
 
-int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
-int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
+extern "C" int b2sp_last_algo(int op) { return op >= 0 && op < 3 ? g_last_algo[op] : -1; }
+extern "C" int b2sp_last_launches(int op) { return op >= 0 && op < 3 ? g_last_launches[op] : 0; }
 
 // The row family under AUTO: the binning pass (two small launches, ~10 us) orders the rows longest
 // first, which only pays when the CTAs of the row kernel need several waves on the GPU.
 static int auto_row_algo(int M) { return M <= 4096 ? B2SP_ALGO_ROW_NAT : B2SP_ALGO_ROW; }
 
 // Enqueues the row-family SPMM.  `gate` != NULL makes it a device-side fallback.
+template <typename DT>
 static b2sp_status spmm_rows(int M, int N, const int *row_ptr, const int *col_idx, const float *values,
-                             const float *D, long long ldd, float *O, long long ldo, const int *order,
+                             const DT *D, long long ldd, float *O, long long ldo, const int *order,
                              int *gate, int *clear, cudaStream_t st)
 {
-    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O);
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned_vec(D) && aligned16(O);
     if (vec) {
         Geom g = pick_geom(N);
         dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab));
-        if (g.SPLIT == 4) launch_spmm<1, 4>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
-        else if (g.SPLIT == 2) launch_spmm<1, 2>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
-        else if (g.U == 1) launch_spmm<1, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
-        else if (g.U == 2) launch_spmm<2, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
-        else launch_spmm<4, 1>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        if (g.SPLIT == 4) launch_spmm<1, 4, DT>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.SPLIT == 2) launch_spmm<1, 2, DT>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.U == 1) launch_spmm<1, 1, DT>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else if (g.U == 2) launch_spmm<2, 1, DT>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
+        else launch_spmm<4, 1, DT>(grid, st, N, row_ptr, col_idx, values, D, ldd, O, ldo, order, gate, clear);
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128));
-        launch_row(spmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
+        launch_row(spmm_row_scalar_kernel<DT>, grid, 0, st, gate != nullptr || order != nullptr, N, row_ptr, col_idx, values, D, ldd, O, ldo, order,
                    gate, M, clear);
     }
     return check_launch();
 }
 
-b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
-                      const float *values, const float *D, long long ldd, float *O, long long ldo,
-                      void *workspace, size_t workspace_bytes, int algo, void *stream)
+template <typename DT>
+static b2sp_status spmm_impl(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
+                             const float *values, const DT *D, long long ldd, float *O, long long ldo,
+                             void *workspace, size_t workspace_bytes, int algo, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || N < 0) return B2SP_ERR_INVALID_ARG;
@@ -320,7 +323,7 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
         rc = fused_tile(plan, prepared, 2, M, K, 0, N, nnz, row_ptr, col_idx, values, nullptr, 0, nullptr, 0, D, ldd,
-                        O, ldo, workspace, st, &launches);
+                        O, ldo, workspace, st, &launches, false, BatchDesc(), dense_dtype<DT>());
         if (rc != B2SP_OK) return rc;
         // device-side fallback: runs only if the pre-pass found rows that are not strictly sorted
         int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
@@ -343,39 +346,41 @@ b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, co
 }
 
 // Enqueues the row-family SDDMM.  `gate` != NULL makes it a device-side fallback.
+template <typename DT>
 static b2sp_status sddmm_rows(int M, int Kd, const int *row_ptr, const int *col_idx, const float *s_values,
-                              const float *A, long long lda, const float *B, long long ldb,
+                              const DT *A, long long lda, const DT *B, long long ldb,
                               float *out_values, const int *order, int *gate, int *clear, cudaStream_t st)
 {
     dim3 grid((unsigned)M);
-    bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+    bool vec = Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned_vec(A) && aligned_vec(B) &&
                Kd <= 40960;
     if (vec) {
         switch (pick_ku(Kd)) {
-        case 2: launch_sddmm<2>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
-        case 4: launch_sddmm<4>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
-        case 8: launch_sddmm<8>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
+        case 2: launch_sddmm<2, DT>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
+        case 4: launch_sddmm<4, DT>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
+        case 8: launch_sddmm<8, DT>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear); break;
         default: {
             size_t smem = sizeof(float) * (size_t)Kd;
             if (smem > 48 * 1024 &&
-                cudaFuncSetAttribute(sddmm_row_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                cudaFuncSetAttribute(sddmm_row_kernel<0, DT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)smem) != cudaSuccess)
                 return B2SP_ERR_CUDA;
-            launch_sddmm<0>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear);
+            launch_sddmm<0, DT>(grid, st, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, order, gate, clear);
         }
         }
     } else {
         grid.x = gated_blocks(grid.x, gate);
-        launch_row(sddmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb,
+        launch_row(sddmm_row_scalar_kernel<DT>, grid, 0, st, gate != nullptr || order != nullptr, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb,
                    out_values, order, gate, M, clear);
     }
     return check_launch();
 }
 
-b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
-                       const float *s_values, const float *A, long long lda, const float *B,
-                       long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
-                       int algo, void *stream)
+template <typename DT>
+static b2sp_status sddmm_impl(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
+                              const float *s_values, const DT *A, long long lda, const DT *B,
+                              long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
+                              int algo, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0) return B2SP_ERR_INVALID_ARG;
@@ -405,7 +410,7 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
         rc = fused_tile(plan, prepared, 0, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
-                        out_values, 0, workspace, st, &launches);
+                        out_values, 0, workspace, st, &launches, false, BatchDesc(), dense_dtype<DT>());
         if (rc != B2SP_OK) return rc;
         int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
         rc = sddmm_rows(M, Kd, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, nullptr, gate, nullptr, st);
@@ -427,39 +432,41 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, 
 }
 
 // Enqueues the row-family FusedMM.  `gate` != NULL makes it a device-side fallback.
+template <typename DT>
 static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const int *col_idx,
-                              const float *s_values, const float *A, long long lda, const float *B,
-                              long long ldb, const float *D, long long ldd, float *O, long long ldo,
+                              const float *s_values, const DT *A, long long lda, const DT *B,
+                              long long ldb, const DT *D, long long ldd, float *O, long long ldo,
                               const int *order, int *gate, int *clear, cudaStream_t st,
                               int nbatch = 1, const RowBatch &rb = RowBatch{0, 0, 0, 0, 0, 0})
 {
     b2sp_status rc = B2SP_OK;
-    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned16(D) && aligned16(O) &&
-               Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned16(A) && aligned16(B) &&
+    bool vec = N % 4 == 0 && ldd % 4 == 0 && ldo % 4 == 0 && aligned_vec(D) && aligned16(O) &&
+               Kd % 4 == 0 && lda % 4 == 0 && ldb % 4 == 0 && aligned_vec(A) && aligned_vec(B) &&
                Kd <= 40960 && ((rb.A | rb.B | rb.D | rb.O) & 3) == 0;
     if (vec) {
         Geom g = pick_geom(N);
         dim3 grid((unsigned)M, (unsigned)((N + g.slab - 1) / g.slab), (unsigned)nbatch);
         switch (pick_ku(Kd)) {
-        case 2: rc = dispatch_fused_geom<2>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
-        case 4: rc = dispatch_fused_geom<4>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
-        case 8: rc = dispatch_fused_geom<8>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
-        default: rc = dispatch_fused_geom<0>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        case 2: rc = dispatch_fused_geom<2, DT>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        case 4: rc = dispatch_fused_geom<4, DT>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        case 8: rc = dispatch_fused_geom<8, DT>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
+        default: rc = dispatch_fused_geom<0, DT>(g, grid, st, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, gate, clear, rb); break;
         }
         if (rc != B2SP_OK) return rc;
     } else {
         dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128), (unsigned)nbatch);
-        launch_row(fusedmm_row_scalar_kernel, grid, 0, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
+        launch_row(fusedmm_row_scalar_kernel<DT>, grid, 0, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
                    D, ldd, O, ldo, order, gate, M, clear, rb);
     }
     return check_launch();
 }
 
-b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
-                         const int *col_idx, const float *s_values, const float *A, long long lda,
-                         const float *B, long long ldb, const float *D, long long ldd, float *O,
-                         long long ldo, void *workspace, size_t workspace_bytes, int algo,
-                         void *stream)
+template <typename DT>
+static b2sp_status fusedmm_impl(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+                                const int *col_idx, const float *s_values, const DT *A, long long lda,
+                                const DT *B, long long ldb, const DT *D, long long ldd, float *O,
+                                long long ldo, void *workspace, size_t workspace_bytes, int algo,
+                                void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_csr_args(M, K, nnz, row_ptr, col_idx) || Kd < 0 || N < 0) return B2SP_ERR_INVALID_ARG;
@@ -491,13 +498,13 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
         if (two.feasible && workspace_bytes >= two.bytes) {
             float *C = reinterpret_cast<float *>(static_cast<char *>(workspace) + two.off_c);
             rc = fused_tile(two.sddmm, prepared, 0, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
-                            C, 0, workspace, st, &launches);
+                            C, 0, workspace, st, &launches, false, BatchDesc(), dense_dtype<DT>());
             if (rc != B2SP_OK) return rc;
             rc = fused_tile(two.spmm, true, 2, M, K, 0, N, nnz, row_ptr, col_idx, C, nullptr, 0, nullptr, 0, D, ldd, O, ldo,
-                            workspace, st, &launches, /*keep_status=*/true);
+                            workspace, st, &launches, /*keep_status=*/true, BatchDesc(), dense_dtype<DT>());
         } else {
             rc = fused_tile(plan, prepared, 1, M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo,
-                            workspace, st, &launches);
+                            workspace, st, &launches, false, BatchDesc(), dense_dtype<DT>());
         }
         if (rc != B2SP_OK) return rc;
         int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
@@ -517,6 +524,56 @@ b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *
     rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, order, nullptr, clear, st);
     g_last_launches[B2SP_OP_FUSEDMM] = launches + 1;
     return rc;
+}
+
+// ---- the entry points: fp32 and bfloat16 dense operands -------------------------------------------------
+extern "C" b2sp_status b2sp_spmm(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
+                                 const float *values, const float *D, long long ldd, float *O, long long ldo,
+                                 void *workspace, size_t workspace_bytes, int algo, void *stream)
+{
+    return spmm_impl<float>(M, K, N, nnz, row_ptr, col_idx, values, D, ldd, O, ldo, workspace, workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
+                                  const float *s_values, const float *A, long long lda, const float *B,
+                                  long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
+                                  int algo, void *stream)
+{
+    return sddmm_impl<float>(M, K, Kd, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, out_values, workspace,
+                             workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+                                    const int *col_idx, const float *s_values, const float *A, long long lda,
+                                    const float *B, long long ldb, const float *D, long long ldd, float *O,
+                                    long long ldo, void *workspace, size_t workspace_bytes, int algo,
+                                    void *stream)
+{
+    return fusedmm_impl<float>(M, K, Kd, N, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, workspace,
+                               workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_spmm_bf16(int M, int K, int N, long long nnz, const int *row_ptr, const int *col_idx,
+                                      const float *values, const void *D, long long ldd, float *O, long long ldo,
+                                      void *workspace, size_t workspace_bytes, int algo, void *stream)
+{
+    return spmm_impl<bf16_t>(M, K, N, nnz, row_ptr, col_idx, values, static_cast<const bf16_t *>(D), ldd, O, ldo,
+                             workspace, workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_sddmm_bf16(int M, int K, int Kd, long long nnz, const int *row_ptr, const int *col_idx,
+                                       const float *s_values, const void *A, long long lda, const void *B,
+                                       long long ldb, float *out_values, void *workspace, size_t workspace_bytes,
+                                       int algo, void *stream)
+{
+    return sddmm_impl<bf16_t>(M, K, Kd, nnz, row_ptr, col_idx, s_values, static_cast<const bf16_t *>(A), lda,
+                              static_cast<const bf16_t *>(B), ldb, out_values, workspace, workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_fusedmm_bf16(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+                                         const int *col_idx, const float *s_values, const void *A, long long lda,
+                                         const void *B, long long ldb, const void *D, long long ldd, float *O,
+                                         long long ldo, void *workspace, size_t workspace_bytes, int algo,
+                                         void *stream)
+{
+    return fusedmm_impl<bf16_t>(M, K, Kd, N, nnz, row_ptr, col_idx, s_values, static_cast<const bf16_t *>(A), lda,
+                                static_cast<const bf16_t *>(B), ldb, static_cast<const bf16_t *>(D), ldd, O, ldo,
+                                workspace, workspace_bytes, algo, stream);
 }
 
 // ---- batched FusedMM --------------------------------------------------------------------------------
@@ -540,7 +597,7 @@ FusedPlan plan_batched(int batch, int M, int K, int Kd, int N, long long nnz_str
 
 }  // namespace
 
-size_t b2sp_workspace_bytes_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride)
+extern "C" size_t b2sp_workspace_bytes_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride)
 {
     if (batch < 1 || M < 0 || K < 0 || Kd < 0 || N < 0 || nnz_stride < 0) return 0;
     const size_t rows = row_workspace_bytes(M);
@@ -548,7 +605,7 @@ size_t b2sp_workspace_bytes_batched(int batch, int M, int K, int Kd, int N, long
     return p.feasible && p.bytes > rows ? p.bytes : rows;
 }
 
-b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, long long nnz_stride, const int *row_ptr,
+extern "C" b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, long long nnz_stride, const int *row_ptr,
                                          long long row_ptr_stride, const int *col_idx, void *workspace,
                                          size_t workspace_bytes, void *stream)
 {
@@ -564,7 +621,7 @@ b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, long long nnz_
     return pattern_pass(false, M, K, nnz_stride, row_ptr, col_idx, workspace, st, &launches, bd);
 }
 
-b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+extern "C" b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
                                  const int *row_ptr, long long row_ptr_stride, const int *col_idx,
                                  const float *s_values, const float *A, long long lda, long long stride_a,
                                  const float *B, long long ldb, long long stride_b, const float *D, long long ldd,
@@ -625,7 +682,7 @@ b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long lo
     return rc;
 }
 
-b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+extern "C" b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
                                  void *workspace, size_t workspace_bytes, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -637,7 +694,7 @@ b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr
     return pattern_pass(false, M, K, nnz, row_ptr, col_idx, workspace, st, &launches);
 }
 
-b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
+extern "C" b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,
                               void *workspace, size_t workspace_bytes, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -660,7 +717,7 @@ b2sp_status b2sp_validate_csr(int M, int K, long long nnz, const int *row_ptr, c
     return h ? B2SP_ERR_BAD_CSR : B2SP_OK;
 }
 
-b2sp_status b2sp_device_status(const void *workspace, void *stream)
+extern "C" b2sp_status b2sp_device_status(const void *workspace, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!workspace) return B2SP_ERR_WORKSPACE;
@@ -672,7 +729,6 @@ b2sp_status b2sp_device_status(const void *workspace, void *stream)
     return h == 0 ? B2SP_OK : B2SP_ERR_TIMEOUT;
 }
 
-}  // extern "C"
 
 // ---- host-buffer forms ------------------------------------------------------------------------
 namespace {
@@ -747,9 +803,7 @@ struct DevArena {
 
 }  // namespace
 
-extern "C" {
-
-b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_ptr,
+extern "C" b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_ptr,
                            const int *col_idx, const float *values, const float *D, float *O,
                            void *stream)
 {
@@ -775,7 +829,7 @@ b2sp_status b2sp_spmm_host(int M, int K, int N, long long nnz, const int *row_pt
     return a.finish(rc);
 }
 
-b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_ptr,
+extern "C" b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_ptr,
                             const int *col_idx, const float *s_values, const float *A,
                             const float *B, float *out_values, void *stream)
 {
@@ -802,7 +856,7 @@ b2sp_status b2sp_sddmm_host(int M, int K, int Kd, long long nnz, const int *row_
     return a.finish(rc);
 }
 
-b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
+extern "C" b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const int *row_ptr,
                               const int *col_idx, const float *s_values, const float *A,
                               const float *B, const float *D, float *O, void *stream)
 {
@@ -832,4 +886,3 @@ b2sp_status b2sp_fusedmm_host(int M, int K, int Kd, int N, long long nnz, const 
     return a.finish(rc);
 }
 
-}  // extern "C"

@@ -102,7 +102,21 @@ __global__ void bin_scatter_kernel(int M, const int *__restrict__ row_ptr,
 // ------------------------------------------------------------------------------------------
 // helpers
 // ------------------------------------------------------------------------------------------
+// Dense operands are fp32 or bfloat16 (DT below); sums and outputs are always fp32.  A bf16 value is the top
+// half of the fp32 value it stands for, so widening it is exact.
+struct bf16_t { unsigned short bits; };
 __device__ __forceinline__ float4 ldg4(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+__device__ __forceinline__ float4 ldg4(const bf16_t *p)   // four consecutive elements, 8-byte aligned
+{
+    const uint2 u = __ldg(reinterpret_cast<const uint2 *>(p));
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xffff0000u),
+                       __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xffff0000u));
+}
+__device__ __forceinline__ float ldg1(const float *p) { return __ldg(p); }
+__device__ __forceinline__ float ldg1(const bf16_t *p)
+{
+    return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short *>(p)) << 16);
+}
 
 __device__ __forceinline__ void fma4(float4 &acc, float s, const float4 &v)
 {
@@ -131,9 +145,9 @@ struct SweepGeom {
 
 // One chunk (up to 32 entries, lane l holds entry l: column k, scalar s) of the Alg. 2 SAXPY
 // sweep.  SRC(j) gives the lane that holds entry j's scalar.
-template <int U, int SPLIT, bool PERMUTED>
+template <int U, int SPLIT, bool PERMUTED, typename DT>
 __device__ __forceinline__ void saxpy_chunk(float4 (&acc)[U], int k, float s, int cnt,
-                                            const float *__restrict__ Dcol, int64_t ldd,
+                                            const DT *__restrict__ Dcol, int64_t ldd,
                                             bool (&live)[U], int sub)
 {
     constexpr int LPN = 32 / SPLIT;
@@ -145,7 +159,7 @@ __device__ __forceinline__ void saxpy_chunk(float4 (&acc)[U], int k, float s, in
             int src = PERMUTED ? ((j & 3) * 8 + (j >> 2)) : j;
             int kk = __shfl_sync(kFull, k, j);
             float ss = __shfl_sync(kFull, s, src);
-            const float *d = Dcol + (int64_t)kk * ldd;
+            const DT *d = Dcol + (int64_t)kk * ldd;
 #pragma unroll
             for (int u = 0; u < U; ++u)
                 if (live[u]) fma4(acc[u], ss, ldg4(d + u * LPN * 4));
@@ -157,7 +171,7 @@ __device__ __forceinline__ void saxpy_chunk(float4 (&acc)[U], int k, float s, in
             int kk = __shfl_sync(kFull, k, j);
             float ss = __shfl_sync(kFull, s, src);
             if (j < cnt) {
-                const float *d = Dcol + (int64_t)kk * ldd;
+                const DT *d = Dcol + (int64_t)kk * ldd;
 #pragma unroll
                 for (int u = 0; u < U; ++u)
                     if (live[u]) fma4(acc[u], ss, ldg4(d + u * LPN * 4));
@@ -206,10 +220,10 @@ __device__ __forceinline__ void reduce_and_store_row(float4 (&acc)[U], float4 *r
 // ------------------------------------------------------------------------------------------
 // SPMM  (Alg. 2; float4 path: N, ldd, ldo multiples of 4, D and O 16-byte aligned)
 // ------------------------------------------------------------------------------------------
-template <int U, int SPLIT>
+template <int U, int SPLIT, typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
-                const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
+                const float *__restrict__ values, const DT *__restrict__ D, int64_t ldd,
                 float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
                 int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
@@ -231,7 +245,7 @@ spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ 
             acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         const int beg = row_ptr[row], end = row_ptr[row + 1];
-        const float *Dcol = D + col0;
+        const DT *Dcol = D + col0;
         // the next chunk's indices and values are fetched before the current chunk is consumed
         // (the role of the paper's prefetch of the next ja/avalues block)
         int k = 0;
@@ -251,7 +265,7 @@ spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ 
                 kn = __ldg(col_idx + pn);
                 sn = __ldg(values + pn);
             }
-            saxpy_chunk<U, SPLIT, false>(acc, k, s, min(32, end - c), Dcol, ldd, live, sub);
+            saxpy_chunk<U, SPLIT, false, DT>(acc, k, s, min(32, end - c), Dcol, ldd, live, sub);
             k = kn;
             s = sn;
         }
@@ -261,9 +275,10 @@ spmm_row_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ 
 }
 
 // Scalar path for any N / ld / alignment: a lane owns columns col0 + lane + 32u (u < 4).
+template <typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
-                       const float *__restrict__ values, const float *__restrict__ D, int64_t ldd,
+                       const float *__restrict__ values, const DT *__restrict__ D, int64_t ldd,
                        float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
                        int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
@@ -289,10 +304,10 @@ spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__rest
             for (int j = 0; j < cnt; ++j) {
                 int kk = __shfl_sync(kFull, k, j);
                 float ss = __shfl_sync(kFull, s, j);
-                const float *d = D + (int64_t)kk * ldd + col0;
+                const DT *d = D + (int64_t)kk * ldd + col0;
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, ldg1(d + 32 * u), acc[u]);
             }
         }
 #pragma unroll
@@ -320,17 +335,17 @@ spmm_row_scalar_kernel(int N, const int *__restrict__ row_ptr, const int *__rest
 // group g takes entries 4r + g (r = 0..7); after the 3-step butterfly every lane of the
 // group has the sum and lane t keeps round t's, so lane 8g + t ends up holding entry 4t + g.
 // ------------------------------------------------------------------------------------------
-template <int KU>
+template <int KU, typename DT>
 __device__ __forceinline__ float sddmm_chunk(const float4 (&areg)[KU > 0 ? KU : 1],
                                              const float *__restrict__ a_smem, int Kd, int k,
-                                             const float *__restrict__ B, int64_t ldb, int lane)
+                                             const DT *__restrict__ B, int64_t ldb, int lane)
 {
     const int g = lane >> 3, t = lane & 7;
     float mine = 0.f;
 #pragma unroll 4
     for (int r = 0; r < 8; ++r) {
         int kq = __shfl_sync(kFull, k, 4 * r + g);
-        const float *b = B + (int64_t)kq * ldb + t * 4;
+        const DT *b = B + (int64_t)kq * ldb + t * 4;
         float part = 0.f;
         if (KU > 0) {
 #pragma unroll
@@ -348,9 +363,9 @@ __device__ __forceinline__ float sddmm_chunk(const float4 (&areg)[KU > 0 ? KU : 
     return mine;  // lane 8g+t: dot product of entry 4t+g
 }
 
-template <int KU>
+template <int KU, typename DT>
 __device__ __forceinline__ void load_a_row(float4 (&areg)[KU > 0 ? KU : 1], float *a_smem,
-                                           const float *__restrict__ Arow, int Kd, int lane)
+                                           const DT *__restrict__ Arow, int Kd, int lane)
 {
     if (KU > 0) {
         const int t = lane & 7;
@@ -364,11 +379,11 @@ __device__ __forceinline__ void load_a_row(float4 (&areg)[KU > 0 ? KU : 1], floa
     }
 }
 
-template <int KU>
+template <int KU, typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
-                 const float *s_values, const float *__restrict__ A, int64_t lda,
-                 const float *__restrict__ B, int64_t ldb, float *out_values,
+                 const float *s_values, const DT *__restrict__ A, int64_t lda,
+                 const DT *__restrict__ B, int64_t ldb, float *out_values,
                  const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     extern __shared__ float4 dyn_smem[];
@@ -381,12 +396,12 @@ sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict_
         const int row = row_order ? row_order[rb] : rb;
         const int beg = row_ptr[row], end = row_ptr[row + 1];
         float4 areg[KU > 0 ? KU : 1];
-        load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+        load_a_row<KU, DT>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
         const int slot = (lane & 7) * 4 + (lane >> 3);  // entry of the chunk this lane ends up holding
         for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
             int p = c + lane;
             int k = p < end ? __ldg(col_idx + p) : 0;
-            float dp = sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
+            float dp = sddmm_chunk<KU, DT>(areg, a_smem, Kd, k, B, ldb, lane);
             int q = c + slot;
             if (q < end) out_values[q] = s_values ? s_values[q] * dp : dp;
         }
@@ -395,10 +410,11 @@ sddmm_row_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict_
 }
 
 // Scalar path for any Kd / ld / alignment: one lane per entry, serial dot product.
+template <typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
-                        const float *s_values, const float *__restrict__ A, int64_t lda,
-                        const float *__restrict__ B, int64_t ldb, float *out_values,
+                        const float *s_values, const DT *__restrict__ A, int64_t lda,
+                        const DT *__restrict__ B, int64_t ldb, float *out_values,
                         const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear)
 {
     if (gate_closed(gate)) return;
@@ -407,11 +423,11 @@ sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__re
     for (int rb = blockIdx.x; rb < nrows; rb += gridDim.x) {
         const int row = row_order ? row_order[rb] : rb;
         const int beg = row_ptr[row], end = row_ptr[row + 1];
-        const float *a = A + (int64_t)row * lda;
+        const DT *a = A + (int64_t)row * lda;
         for (int p = beg + threadIdx.x; p < end; p += kRowThreads) {
-            const float *b = B + (int64_t)__ldg(col_idx + p) * ldb;
+            const DT *b = B + (int64_t)__ldg(col_idx + p) * ldb;
             float dp = 0.f;
-            for (int l = 0; l < Kd; ++l) dp = fmaf(__ldg(a + l), __ldg(b + l), dp);
+            for (int l = 0; l < Kd; ++l) dp = fmaf(ldg1(a + l), ldg1(b + l), dp);
             out_values[p] = s_values ? s_values[p] * dp : dp;
         }
         __syncthreads();   // shared memory is reused by the next row
@@ -422,11 +438,11 @@ sddmm_row_scalar_kernel(int Kd, const int *__restrict__ row_ptr, const int *__re
 // FusedMM  (Alg. 3): per chunk, the SDDMM values stay in registers (one per lane) and are the
 // scalars of the SAXPY sweep over the same staged column indices; C never reaches memory.
 // ------------------------------------------------------------------------------------------
-template <int KU, int U, int SPLIT, bool BATCHED = false>
+template <int KU, int U, int SPLIT, bool BATCHED, typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__restrict__ col_idx,
-                   const float *__restrict__ s_values, const float *__restrict__ A, int64_t lda,
-                   const float *__restrict__ B, int64_t ldb, const float *__restrict__ D,
+                   const float *__restrict__ s_values, const DT *__restrict__ A, int64_t lda,
+                   const DT *__restrict__ B, int64_t ldb, const DT *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
                    const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear,
                    RowBatch batch)
@@ -457,9 +473,9 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
         }
         const int beg = row_ptr[row], end = row_ptr[row + 1];
         float4 areg[KU > 0 ? KU : 1];
-        load_a_row<KU>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
+        load_a_row<KU, DT>(areg, a_smem, A + (int64_t)row * lda, Kd, lane);
         const int slot = (lane & 7) * 4 + (lane >> 3);
-        const float *Dcol = D + col0;
+        const DT *Dcol = D + col0;
         int k = 0;
         float sv = 1.f;
         {
@@ -471,8 +487,8 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
             int pn = c + kRowWarps * 32 + lane, qn = c + kRowWarps * 32 + slot;
             int kn = pn < end ? __ldg(col_idx + pn) : 0;
             float svn = (s_values && qn < end) ? __ldg(s_values + qn) : 1.f;
-            float cv = sv * sddmm_chunk<KU>(areg, a_smem, Kd, k, B, ldb, lane);
-            saxpy_chunk<U, SPLIT, true>(acc, k, cv, min(32, end - c), Dcol, ldd, live, sub);
+            float cv = sv * sddmm_chunk<KU, DT>(areg, a_smem, Kd, k, B, ldb, lane);
+            saxpy_chunk<U, SPLIT, true, DT>(acc, k, cv, min(32, end - c), Dcol, ldd, live, sub);
             k = kn;
             sv = svn;
         }
@@ -482,11 +498,12 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
 }
 
 // Scalar path for any widths / alignment: lane-per-entry dot products, then a scalar sweep.
+template <typename DT>
 __global__ void __launch_bounds__(kRowThreads)
 fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
                           const int *__restrict__ col_idx, const float *__restrict__ s_values,
-                          const float *__restrict__ A, int64_t lda, const float *__restrict__ B,
-                          int64_t ldb, const float *__restrict__ D, int64_t ldd,
+                          const DT *__restrict__ A, int64_t lda, const DT *__restrict__ B,
+                          int64_t ldb, const DT *__restrict__ D, int64_t ldd,
                           float *__restrict__ O, int64_t ldo, const int *__restrict__ row_order,
                           int *__restrict__ gate, int nrows, int *__restrict__ clear, RowBatch batch)
 {
@@ -505,25 +522,25 @@ fusedmm_row_scalar_kernel(int Kd, int N, const int *__restrict__ row_ptr,
         const int col0 = blockIdx.y * 128 + lane;
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         const int beg = row_ptr[row], end = row_ptr[row + 1];
-        const float *a = A + (int64_t)row * lda;
+        const DT *a = A + (int64_t)row * lda;
         for (int c = beg + warp * 32; c < end; c += kRowWarps * 32) {
             int p = c + lane;
             int k = 0;
             float cv = 0.f;
             if (p < end) {
                 k = __ldg(col_idx + p);
-                const float *b = B + (int64_t)k * ldb;
-                for (int l = 0; l < Kd; ++l) cv = fmaf(__ldg(a + l), __ldg(b + l), cv);
+                const DT *b = B + (int64_t)k * ldb;
+                for (int l = 0; l < Kd; ++l) cv = fmaf(ldg1(a + l), ldg1(b + l), cv);
                 if (s_values) cv *= __ldg(s_values + p);
             }
             int cnt = min(32, end - c);
             for (int j = 0; j < cnt; ++j) {
                 int kk = __shfl_sync(kFull, k, j);
                 float ss = __shfl_sync(kFull, cv, j);
-                const float *d = D + (int64_t)kk * ldd + col0;
+                const DT *d = D + (int64_t)kk * ldd + col0;
 #pragma unroll
                 for (int u = 0; u < 4; ++u)
-                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, __ldg(d + 32 * u), acc[u]);
+                    if (col0 + 32 * u < N) acc[u] = fmaf(ss, ldg1(d + 32 * u), acc[u]);
             }
         }
 #pragma unroll

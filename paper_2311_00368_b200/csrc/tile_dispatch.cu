@@ -232,14 +232,14 @@ TwoPhasePlan plan_two_phase(int M, int K, int Kd, int N, long long nnz, size_t b
 
 namespace {
 
-template <int KDP, int MODE, bool BATCHED>
+template <int KDP, int MODE, bool BATCHED, bool EXACT>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                               const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                               cudaStream_t st)
 {
-    using Cfg = FusedCfg<KDP, MODE>;
-    auto kern = fused_tile_kernel<KDP, MODE, BATCHED>;
-    if (!allow_dynamic_smem<KDP * 8 + MODE * 2 + (BATCHED ? 1 : 0)>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
+    using Cfg = FusedCfg<KDP, MODE, EXACT>;
+    auto kern = fused_tile_kernel<KDP, MODE, BATCHED, EXACT>;
+    if (!allow_dynamic_smem<KDP * 16 + MODE * 4 + (BATCHED ? 2 : 0) + (EXACT ? 1 : 0)>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
     // a programmatic dependent of the operand-split kernel: its CTAs are placed while that kernel still runs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)items);
@@ -256,18 +256,23 @@ b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, cons
 }
 
 template <int MODE>
-b2sp_status launch_fused_kdp(int kdp, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
+b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
-        if (kdp == 32) return launch_fused_tile<32, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, kModeFused, true>(bh, bl, dh, dl, out, a, items, st);
+    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM on fp32 operands is offered on batches)
+        if (kdp == 32) return launch_fused_tile<32, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
     }
-    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false>(bh, bl, dh, dl, out, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, MODE, false>(bh, bl, dh, dl, out, a, items, st);
-    return launch_fused_tile<128, MODE, false>(bh, bl, dh, dl, out, a, items, st);
+    if (exact) {
+        if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
+    }
+    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
+    return launch_fused_tile<128, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
 }
 
 // Splits (or only checks) up to three dense operands, clears the device status word and optionally
@@ -296,12 +301,13 @@ void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const Ta
 }  // namespace
 
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
-                       const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
-                       long long lda, const float *B, long long ldb, const float *D, long long ldd,
+                       const int *row_ptr, const int *col_idx, const float *s_values, const void *A,
+                       long long lda, const void *B, long long ldb, const void *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches, bool keep_status,
-                       const BatchDesc &batch)
+                       const BatchDesc &batch, int dtype)
 {
     const int nb = batch.count;
+    const bool exact = dtype == kDenseBf16;   // operands exact in tf32: no lo halves anywhere
     char *ws = static_cast<char *>(workspace);
     int *status = reinterpret_cast<int *>(ws + kWsStatusOffset);
     int *flags = reinterpret_cast<int *>(ws + kWsTileFlagsOffset);
@@ -313,17 +319,18 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     const bool fused = mode != kModeSddmm, spmm = mode == kModeSpmm;
     CUtensorMap tm_bh, tm_bl, tm_dh, tm_dl;
     if (!spmm && (!make_blocked_map(&tm_bh, bhi, nb * p.Kp, p.Kdp / 32, kFusedBlk, 1, false) ||
-                  !make_blocked_map(&tm_bl, blo, nb * p.Kp, p.Kdp / 32, kFusedBlk, 1, false)))
+                  (!exact && !make_blocked_map(&tm_bl, blo, nb * p.Kp, p.Kdp / 32, kFusedBlk, 1, false))))
         return B2SP_ERR_CUDA;
     if (fused) {
         if (!make_blocked_map(&tm_dh, dhi, nb * p.Kp, p.Np / 32, kFusedW, p.NT / 32, true) ||
-            !make_blocked_map(&tm_dl, dlo, nb * p.Kp, p.Np / 32, kFusedW, p.NT / 32, true))
+            (!exact && !make_blocked_map(&tm_dl, dlo, nb * p.Kp, p.Np / 32, kFusedW, p.NT / 32, true)))
             return B2SP_ERR_CUDA;
     } else {
         tm_dh = tm_bh;   // unused by the SDDMM kernel
-        tm_dl = tm_bl;
     }
-    if (spmm) { tm_bh = tm_dh; tm_bl = tm_dl; }   // unused by the SPMM mode
+    if (spmm) tm_bh = tm_dh;   // unused by the SPMM mode
+    if (exact || !fused) tm_dl = tm_dh;   // (maps the kernel never touches still have to be valid objects)
+    if (exact || spmm) tm_bl = tm_bh;
     {
         b2sp_status prc = pattern_pass(prepared, M, K, nnz, row_ptr, col_idx, workspace, st, launches, batch);
         if (prc != B2SP_OK) return prc;
@@ -332,9 +339,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         // B and D are split into tf32 hi/lo copies; A, which the tile kernel splits itself, is only checked
         // for non-finite values (see split_dense_kernel).
         const int a_rows_p = (M + 3) & ~3, a_cols_p = (Kd + 31) & ~31;
-        const SplitJob jb{B, ldb, K, Kd, bhi, blo, p.Kp, p.Kdp, nb, batch.B, kDenseF32, 0};
-        const SplitJob jd{D, ldd, K, N, dhi, dlo, p.Kp, p.Np, nb, batch.D, kDenseF32, 0};
-        const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, nb, batch.A, kDenseF32, 1};
+        const SplitJob jb{B, ldb, K, Kd, bhi, exact ? nullptr : blo, p.Kp, p.Kdp, nb, batch.B, dtype, 0};
+        const SplitJob jd{D, ldd, K, N, dhi, exact ? nullptr : dlo, p.Kp, p.Np, nb, batch.D, dtype, 0};
+        const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, nb, batch.A, dtype, 1};
         SplitJobs jobs;
         jobs.n = 0;
         if (!spmm) { jobs.j[jobs.n++] = jb; jobs.j[jobs.n++] = ja; }
@@ -358,6 +365,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.batch = nb; a.ctas_per_problem = p.Mt * p.Nt * p.KS; a.Kp = p.Kp;
     a.stride_sv = batch.nz; a.stride_A = batch.A; a.stride_O = fused ? batch.O : batch.nz;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
+    if (exact && nb > 1) return B2SP_ERR_UNSUPPORTED;
     a.flags = flags; a.status = status;
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
     a.O = out; a.ldo = ldo;
@@ -383,9 +391,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         }
     }
     const int items = nb * p.Mt * p.Nt * p.KS;
-    b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
-                     : fused ? launch_fused_kdp<kModeFused>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
-                             : launch_fused_kdp<kModeSddmm>(p.Kdp, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st);
+    b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
+                     : fused ? launch_fused_kdp<kModeFused>(p.Kdp, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
+                             : launch_fused_kdp<kModeSddmm>(p.Kdp, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
     return B2SP_OK;

@@ -13,6 +13,9 @@ constexpr size_t kWsTileFlagsOffset = 320;   // int[..]: flags written by the ti
 constexpr size_t kWsSignatureOffset = 448;   // int[16]: which CSR arrays the window table was built from
 constexpr size_t kWsHeaderBytes = 512;
 
+// Element type of the dense operands A, B, D.
+constexpr int kDenseF32 = 0, kDenseBf16 = 1;
+
 // A batch of independent problems of the same sizes handled by one set of launches: `count` problems, the
 // caller's arrays of consecutive problems `*` elements apart (rp: row_ptr; nz: col_idx, stored values and
 // SDDMM output values; A, B, D, O: the dense operands and the output).  Every problem's row_ptr starts at 0.
@@ -37,11 +40,13 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
 // The tile kernel leaves immediately if the pre-pass found a row whose columns are not strictly increasing
 // (flag at kWsTileFlagsOffset).
 // mode: 0 = SDDMM, 1 = FusedMM, 2 = SPMM through the FusedMM pipeline (P' = the stored values)
+// A, B, D: fp32 (dtype 0) or bfloat16 (dtype 1) -- the latter are exact in tf32, so their lo halves (copies,
+// loads, MMAs) are left out.
 b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K, int Kd, int N, long long nnz,
-                       const int *row_ptr, const int *col_idx, const float *s_values, const float *A,
-                       long long lda, const float *B, long long ldb, const float *D, long long ldd,
+                       const int *row_ptr, const int *col_idx, const float *s_values, const void *A,
+                       long long lda, const void *B, long long ldb, const void *D, long long ldd,
                        float *out, long long ldo, void *workspace, cudaStream_t st, int *launches,
-                       bool keep_status = false, const BatchDesc &batch = BatchDesc());
+                       bool keep_status = false, const BatchDesc &batch = BatchDesc(), int dtype = 0);
 
 // FusedMM with an output wider than two 128-column tiles runs as SDDMM into a scratch C followed by SPMM
 // on C (see b2sp_fusedmm): the plans of the two phases and where C sits in the workspace.

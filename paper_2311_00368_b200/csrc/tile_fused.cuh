@@ -63,7 +63,7 @@ struct FusedTileArgs {
     int NT;                   // O columns per CTA (UMMA N of GEMM2): 128, or 64 when N <= 64
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
-    const float *A;           // M x Kd
+    const void *A;            // M x Kd, fp32 (bfloat16 in the EXACT kernels)
     long long lda;
     float *out;               // FusedMM / SPMM: O (one K split) or the K splits' slabs; SDDMM: out_values
     long long ld_out, slab;
@@ -91,22 +91,30 @@ __device__ __forceinline__ int helper_index(int warp)
     return warp == 0 ? 0 : 1 + (warp - 6) - (warp > 9 ? 1 : 0) - (warp > 21 ? 1 : 0) - (warp > 25 ? 1 : 0);
 }
 
-template <int KDP, int MODE>
+// EXACT: the dense operands A, B, D are exact in tf32 (bfloat16 inputs): their lo halves are zero, so the lo
+// copies are neither loaded nor multiplied -- GEMM1 is one MMA per product instead of three, GEMM2 two (P' still
+// has a hi and a lo part).
+template <int KDP, int MODE, bool EXACT = false>
 struct FusedCfg {
     static constexpr bool FUSED = MODE != kModeSddmm;          // has GEMM2 / O
     static constexpr bool SPMM = MODE == kModeSpmm;
     static constexpr int NCH_B = SPMM ? 0 : KDP / 32;          // B chunks per block
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
-    static constexpr int ALO_BYTES = (FUSED && !SPMM) ? kFusedRows * KDP * 4 : 0;
+    static constexpr int ALO_BYTES = (FUSED && !SPMM && !EXACT) ? kFusedRows * KDP * 4 : 0;
     // SDDMM runs 28 warps of 72 registers (its processors only copy P, and its helpers work on items of
     // 16 rows, so nobody needs more): twenty helpers instead of twelve.  FusedMM and SPMM: 20 warps of 96.
-    static constexpr int THREADS = FUSED ? kFusedThreads : 896;
+    // SPMM has four flusher warps (16-19) of its own: it has two O accumulators so that the tensor core can go on
+    // while a partial sum leaves tensor memory, which only helps if the processors, who make its next operands,
+    // are not the ones doing the flush (measured with role timers: a third of the processors' time).
+    static constexpr bool DEDICATED_FLUSH = SPMM;
+    static constexpr int THREADS = !FUSED ? 896 : kFusedThreads;
+    static constexpr int FLUSH_WARP0 = 16;   // the flusher warps: 16-19 (SPMM: dedicated; FusedMM: the second processor set)
     static constexpr int RING = FUSED && !SPMM ? 3 : 4;
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
     // 4 KB slots (two windows deep).  SPMM: twelve with twelve slots.  SDDMM: twenty with forty 2 KB slots
     // (measured: 12 helpers 134 us, 14 helpers 129 us, 20 helpers on 28 warps 125 us; for SPMM the same
     // layout was slower, 136-140 us against 131 us).
-    static constexpr int HELPERS = (FUSED && !SPMM) ? 8 : SPMM ? 12 : 20;
+    static constexpr int HELPERS = FUSED ? 8 : 20;
     // FusedMM runs two sets of processor warps (warps 2-5 and 16-19) that take alternate windows: a window is a
     // chain of long-latency steps for its processor (slot, tensor-memory load, arithmetic, tensor-memory store,
     // hand-over), about 2 k cycles, and with a single set that chain, not the tensor core, paced the kernel
@@ -132,13 +140,13 @@ struct FusedCfg {
 
 // BATCHED: the launch covers several problems (FusedTileArgs::batch); without it the problem index is the
 // constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to spare).
-template <int KDP, int MODE, bool BATCHED = false>
-__global__ void __launch_bounds__((FusedCfg<KDP, MODE>::THREADS), 1)
+template <int KDP, int MODE, bool BATCHED = false, bool EXACT = false>
+__global__ void __launch_bounds__((FusedCfg<KDP, MODE, EXACT>::THREADS), 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
                   const __grid_constant__ CUtensorMap tm_out, const FusedTileArgs a)
 {
-    using Cfg = FusedCfg<KDP, MODE>;
+    using Cfg = FusedCfg<KDP, MODE, EXACT>;
     constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
     constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
     constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
@@ -210,8 +218,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int pro_i = q == 1 ? (warp == 5 ? 0 : (warp >> 2) - 2) : (warp >> 2);      // ... and this warp's place among them
     if (!SPMM && warp != 1 && warp != kFusedTmaWarp) {
         const int grow = m0 + row;
-        const float *arow = a.A + prob * a.stride_A + (long long)(grow < a.M ? grow : 0) * a.lda;
-        const bool vec = (a.lda & 3) == 0 && (a.stride_A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0;
+        const long long aoff = prob * a.stride_A + (long long)(grow < a.M ? grow : 0) * a.lda;
+        const float *arow = static_cast<const float *>(a.A) + aoff;
+        const unsigned short *arow16 = static_cast<const unsigned short *>(a.A) + aoff;
+        const bool vec = (a.lda & 3) == 0 && (a.stride_A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0 &&
+                         (!EXACT || (a.lda & 7) == 0);   // (16-byte loads of eight bf16)
 #pragma unroll 1
         for (int c = pro_i * 16; c < KDP; c += pro_n * 16) {
             uint32_t hi[16], lo[16];
@@ -219,7 +230,24 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] = 0.f;
             if (grow < a.M) {
-                if (vec && c + 16 <= a.Kd) {
+                if (EXACT) {
+                    if (vec && c + 16 <= a.Kd) {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 8) {
+                            const uint4 u = __ldg(reinterpret_cast<const uint4 *>(arow16 + c + i));
+                            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                v[i + 2 * j] = __uint_as_float(w[j] << 16);
+                                v[i + 2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (c + i < a.Kd) v[i] = __uint_as_float((uint32_t)__ldg(arow16 + c + i) << 16);
+                    }
+                } else if (vec && c + 16 <= a.Kd) {
 #pragma unroll
                     for (int i = 0; i < 16; i += 4) {
                         const float4 f = __ldg(reinterpret_cast<const float4 *>(arow + c + i));
@@ -231,6 +259,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         if (c + i < a.Kd) v[i] = __ldg(arow + c + i);
                 }
             }
+            if constexpr (EXACT) {   // the value is its own hi part
+#pragma unroll
+                for (int i = 0; i < 16; ++i) hi[i] = __float_as_uint(v[i]);
+                ptx::tmem_st_32x16(tmem + lane_addr + Cfg::COL_AHI + c, hi);
+            } else {
 #pragma unroll
             for (int i = 0; i < 16; ++i) ptx::split_tf32_fast(v[i], hi[i], lo[i]);
             ptx::tmem_st_32x16(tmem + lane_addr + Cfg::COL_AHI + c, hi);
@@ -245,6 +278,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
             } else {
                 ptx::tmem_st_32x16(tmem + lane_addr + Cfg::COL_ALO + c, lo);
+            }
             }
         }
         ptx::tmem_st_wait();
@@ -270,11 +304,102 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         return;
     }
 
+    // ---- flush of one chunk of blocks: the partial O leaves tensor memory.  Called by the four warps (one per
+    // tensor-memory lane quarter q) that do the flushes: each thread adds its row into the output (or its K
+    // split's slab): the first partial sum is stored, the later ones are added with fp32 reductions (round to
+    // nearest).  A given element is only ever touched by the same lane of the same warp, in program order, so
+    // the sum is reproducible.  false: a bounded wait gave up.
+    auto flush_chunk = [&](int chunk) -> bool {
+        const int ob = chunk % NOB;
+        bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
+        if (!__all_sync(0xffffffffu, ok)) return false;
+        ptx::tc_fence_after_sync();
+        // 16 columns at a time go through shared memory (per warp two buffers of 32 rows x 16
+        // columns, 64-byte swizzle: 16-byte piece j of row r at piece j ^ ((r >> 1) & 3)).  From
+        // there one TMA store (first partial sum) or fp32 add-reduction per buffer moves whole
+        // 64-byte row pieces; rows and columns outside the output are clipped by TMA.  O is free
+        // for the tensor core again as soon as its last columns have been read.
+        const uint32_t stage = flush_stage + (uint32_t)q * 4096;
+        if (a.out_tma) {
+            if (lane == 0) ptx::bulk_wait<0>();   // the previous flush's reductions are complete (order of the sums)
+            __syncwarp();
+            // one K split: the output itself, problem = third coordinate; several: the slabs, stacked
+            const int y = (a.KS == 1 ? 0 : (prob * a.KS + ks) * a.slab_rows) + m0 + q * 32;
+            const int z = a.KS == 1 ? prob : 0;
+#pragma unroll 1
+            for (int c = 0; c < a.NT / 16; ++c) {
+                const uint32_t buf = stage + (uint32_t)(c & 1) * 2048;
+                if (c >= 2) {
+                    if (lane == 0) ptx::bulk_wait_read<1>();   // the buffer's previous contents have been read
+                    __syncwarp();
+                }
+                uint32_t r[16];
+                ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                ptx::tmem_ld_wait();
+                if (c == a.NT / 16 - 1) {
+                    ptx::tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(o_free(ob));
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
+                                 "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                ptx::fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (chunk == 0) ptx::tma_store_3d(&tm_out, buf, n0 + c * 16, y, z);
+                    else ptx::tma_reduce_add_3d(&tm_out, buf, n0 + c * 16, y, z);
+                    ptx::bulk_commit();
+                }
+            }
+        } else {
+            // output rows that are not 16-byte aligned: the same through plain stores / atomics
+            float *obase = a.out + (a.KS == 1 ? prob * a.stride_O : (long long)(prob * a.KS + ks) * a.slab) +
+                           (long long)(m0 + q * 32) * a.ld_out;
+            const int ncols = a.KS == 1 ? a.N : a.Nt * a.NT;   // slabs are padded to whole tiles
+            const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
+#pragma unroll 1
+            for (int c = 0; c < a.NT / 16; ++c) {
+                uint32_t r[16];
+                ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
+                                 "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
+                __syncwarp();
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const int rr = t * 8 + (lane >> 2), pc = lane & 3;
+                    uint32_t x[4];
+                    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
+                                 : "r"(stage + (uint32_t)rr * 64 + (uint32_t)((pc ^ ((rr >> 1) & 3)) << 4)) : "memory");
+                    const int n = n0 + c * 16 + pc * 4;
+                    if (m0 + q * 32 + rr < nrows) {
+                        float *dst = obase + (long long)rr * a.ld_out + n;
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            if (n + e >= ncols) continue;
+                            if (chunk == 0) dst[e] = __uint_as_float(x[e]);   // the first partial sum initialises the target
+                            else atomicAdd(dst + e, __uint_as_float(x[e]));
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(o_free(ob));
+        }
+        return true;
+    };
+
     if (warp == kFusedTmaWarp) {
         // ---------------- TMA producer: per block NCH_B chunks of B rows, then NCH_D chunks of D rows ----------------
         if (lane == 0) {
-            if (!SPMM) { ptx::tma_prefetch_desc(&tm_bhi); ptx::tma_prefetch_desc(&tm_blo); }
-            if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); ptx::tma_prefetch_desc(&tm_dlo); }
+            if (!SPMM) { ptx::tma_prefetch_desc(&tm_bhi); if (!EXACT) ptx::tma_prefetch_desc(&tm_blo); }
+            if (FUSED) { ptx::tma_prefetch_desc(&tm_dhi); if (!EXACT) ptx::tma_prefetch_desc(&tm_dlo); }
             // Chunk order = the order the MMA thread consumes them: B(0); then per block b:
             // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only; last block of a chunk: B(b+1) last).
             int c = 0;
@@ -283,14 +408,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
                 const uint32_t dst = ring + s * kFusedChunk;
                 const int col0 = krow0 + (b0 + blk) * kFusedBlk;
-                ptx::mbar_arrive_expect_tx(full(s), is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4);   // hi + lo
+                ptx::mbar_arrive_expect_tx(full(s), (is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4) / (EXACT ? 2 : 1));   // hi (+ lo)
                 if (is_b) {   // B rows col0..col0+127, k group i
                     ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
-                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
+                    if (!EXACT) ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
                 } else {      // D rows of window i of the block
                     const int krow = col0 + i * kFusedW;
                     ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (a.NT / 32));
-                    ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
+                    if (!EXACT) ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
                 }
                 ++c;
                 return true;
@@ -329,6 +454,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                         const uint64_t dbl = ptx::smem_desc(b_lo + k8 * 32, 16, 1024, ptx::kLayoutSw128);
                         const uint32_t acol = i * 32 + k8 * 8;
                         ptx::mma_tf32_ts(pacc, tmem + Cfg::COL_AHI + acol, dbh, idesc1, (i | k8) != 0);
+                        if (EXACT) continue;   // A and B exact in tf32: no lo terms
                         ptx::mma_tf32_ts(pacc, tmem + Cfg::COL_AHI + acol, dbl, idesc1, 1);
                         if (FUSED) {
                             const uint64_t dal = ptx::smem_desc(alo_smem + i * (kFusedRows * 128) + k8 * 32, 16, 1024, ptx::kLayoutSw128);
@@ -358,7 +484,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
                     ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
                     ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
-                    ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
+                    if (!EXACT) ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
                 }
                 ptx::mma_commit(pp_free(ppb));
                 ptx::mma_commit(empty(s));
@@ -471,90 +597,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 // FusedMM: right away; the tensor core runs GEMM1 of the next block meanwhile.
                 const bool chunk_ended = SPMM ? (w == 0 && blk > 0 && blk % kFusedFlushBlocks == 0)
                                               : (w == WPB - 1 && blk % kFusedFlushBlocks == kFusedFlushBlocks - 1);
-                if (chunk_ended || it == nwin - 1) {
+                if (!Cfg::DEDICATED_FLUSH && (chunk_ended || it == nwin - 1)) {
                     const int chunk = (chunk_ended && SPMM) ? blk / kFusedFlushBlocks - 1 : blk / kFusedFlushBlocks;
-                    const int ob = chunk % NOB;
-                    bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
-                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                    ptx::tc_fence_after_sync();
-                    // 16 columns at a time go through shared memory (per warp two buffers of 32 rows x 16
-                    // columns, 64-byte swizzle: 16-byte piece j of row r at piece j ^ ((r >> 1) & 3)).  From
-                    // there one TMA store (first partial sum) or fp32 add-reduction per buffer moves whole
-                    // 64-byte row pieces; rows and columns outside the output are clipped by TMA.  O is free
-                    // for the tensor core again as soon as its last columns have been read.
-                    const uint32_t stage = flush_stage + (uint32_t)q * 4096;
-                    if (a.out_tma) {
-                        if (lane == 0) ptx::bulk_wait<0>();   // the previous flush's reductions are complete (order of the sums)
-                        __syncwarp();
-                        // one K split: the output itself, problem = third coordinate; several: the slabs, stacked
-                        const int y = (a.KS == 1 ? 0 : (prob * a.KS + ks) * a.slab_rows) + m0 + q * 32;
-                        const int z = a.KS == 1 ? prob : 0;
-#pragma unroll 1
-                        for (int c = 0; c < a.NT / 16; ++c) {
-                            const uint32_t buf = stage + (uint32_t)(c & 1) * 2048;
-                            if (c >= 2) {
-                                if (lane == 0) ptx::bulk_wait_read<1>();   // the buffer's previous contents have been read
-                                __syncwarp();
-                            }
-                            uint32_t r[16];
-                            ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
-                            ptx::tmem_ld_wait();
-                            if (c == a.NT / 16 - 1) {
-                                ptx::tc_fence_before_sync();
-                                __syncwarp();
-                                if (lane == 0) ptx::mbar_arrive(o_free(ob));
-                            }
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(buf + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
-                                             "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
-                            ptx::fence_proxy_async_smem();
-                            __syncwarp();
-                            if (lane == 0) {
-                                if (chunk == 0) ptx::tma_store_3d(&tm_out, buf, n0 + c * 16, y, z);
-                                else ptx::tma_reduce_add_3d(&tm_out, buf, n0 + c * 16, y, z);
-                                ptx::bulk_commit();
-                            }
-                        }
-                    } else {
-                        // output rows that are not 16-byte aligned: the same through plain stores / atomics
-                        float *obase = a.out + (a.KS == 1 ? prob * a.stride_O : (long long)(prob * a.KS + ks) * a.slab) +
-                                       (long long)(m0 + q * 32) * a.ld_out;
-                        const int ncols = a.KS == 1 ? a.N : a.Nt * a.NT;   // slabs are padded to whole tiles
-                        const int nrows = a.KS == 1 ? a.M : a.M + kFusedRows;   // ... and to whole row tiles
-#pragma unroll 1
-                        for (int c = 0; c < a.NT / 16; ++c) {
-                            uint32_t r[16];
-                            ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
-                            ptx::tmem_ld_wait();
-#pragma unroll
-                            for (int j = 0; j < 4; ++j)
-                                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + (uint32_t)lane * 64 + (uint32_t)((j ^ ((lane >> 1) & 3)) << 4)),
-                                             "r"(r[4 * j]), "r"(r[4 * j + 1]), "r"(r[4 * j + 2]), "r"(r[4 * j + 3]) : "memory");
-                            __syncwarp();
-#pragma unroll
-                            for (int t = 0; t < 4; ++t) {
-                                const int rr = t * 8 + (lane >> 2), pc = lane & 3;
-                                uint32_t x[4];
-                                asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x[0]), "=r"(x[1]), "=r"(x[2]), "=r"(x[3])
-                                             : "r"(stage + (uint32_t)rr * 64 + (uint32_t)((pc ^ ((rr >> 1) & 3)) << 4)) : "memory");
-                                const int n = n0 + c * 16 + pc * 4;
-                                if (m0 + q * 32 + rr < nrows) {
-                                    float *dst = obase + (long long)rr * a.ld_out + n;
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e) {
-                                        if (n + e >= ncols) continue;
-                                        if (chunk == 0) dst[e] = __uint_as_float(x[e]);   // the first partial sum initialises the target
-                                        else atomicAdd(dst + e, __uint_as_float(x[e]));
-                                    }
-                                }
-                            }
-                            __syncwarp();
-                        }
-                        ptx::tc_fence_before_sync();
-                        __syncwarp();
-                        if (lane == 0) ptx::mbar_arrive(o_free(ob));
-                    }
+                    if (!flush_chunk(chunk)) { failed = true; break; }
                 }
             } else {
                 const int pb = blk & 1;
@@ -587,6 +632,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if ((lane & 15) == 0) ptx::mbar_arrive(sl_full(s));
             }
         }
+    } else if (Cfg::DEDICATED_FLUSH && warp >= Cfg::FLUSH_WARP0) {
+        // ---------------- flusher warps (SPMM): take every chunk's partial sum out of tensor memory ----------------
+        const int nchunks = (nblk + kFusedFlushBlocks - 1) / kFusedFlushBlocks;
+        for (int chunk = 0; chunk < nchunks; ++chunk)
+            if (!flush_chunk(chunk)) { failed = true; break; }
     } else if (helper_index<FUSED>(warp) >= 0 && helper_index<FUSED>(warp) < NH) {
         // ---------------- helper warps: work items (window, group of rows), round-robin ----------------
         // FusedMM / SPMM: fetch the stored values of the item's 32 rows x 32 columns with lane = column
@@ -663,7 +713,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         }
     }
     if (failed) atomicExch(a.status, 1);
-    if (FUSED && (Cfg::PSETS == 2 ? warp >= 16 : (warp >= 2 && warp < 6)) && lane == 0) {   // this warp's TMA stores / reductions have been performed
+    if (FUSED && (Cfg::DEDICATED_FLUSH ? warp >= Cfg::FLUSH_WARP0 : Cfg::PSETS == 2 ? warp >= 16 : (warp >= 2 && warp < 6)) && lane == 0) {   // this warp's TMA stores / reductions have been performed
         ptx::bulk_wait<0>();
         ptx::fence_proxy_async_all();
     }

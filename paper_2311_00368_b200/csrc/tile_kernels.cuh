@@ -15,6 +15,7 @@
 #include <stdint.h>
 
 #include "ptx_sm100.cuh"
+#include "tile_dispatch.h"
 
 namespace b2sp {
 
@@ -181,8 +182,6 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // (the A operand, which the tile kernel splits itself) does nothing else: a non-finite hi part raises
 // the fallback flag, and the row kernels, which touch exactly the entries the equations name, produce
 // the result.
-constexpr int kDenseF32 = 0, kDenseBf16 = 1;
-
 struct SplitJob {
     const void *X;
     long long ld;
