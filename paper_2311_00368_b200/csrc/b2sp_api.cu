@@ -101,9 +101,10 @@ inline void launch_row(void (*kern)(KArgs...), dim3 grid, size_t smem, cudaStrea
 
 // A gated launch (the row family as the dense-tile family's fallback) almost always finds its gate
 // closed: it gets a small grid whose blocks walk the rows, so that the usual case costs little.
-inline unsigned gated_blocks(unsigned rows, int *gate)
+inline unsigned gated_blocks(unsigned rows, int *gate, unsigned nbatch = 1)
 {
-    const unsigned cap = 148u * 4u;
+    unsigned cap = 148u * 4u / (nbatch ? nbatch : 1);   // (every CTA of a gated grid counts itself at the gate: keep them few)
+    if (cap < 16u) cap = 16u;
     return gate && rows > cap ? cap : rows;
 }
 
@@ -160,7 +161,7 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
             return B2SP_ERR_CUDA;
     }
     const int nrows = (int)grid.x;
-    grid.x = gated_blocks(grid.x, gate);
+    grid.x = gated_blocks(grid.x, gate, grid.z);
     launch_row(kern, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
                nrows, clear, rb);
     return B2SP_OK;
@@ -454,7 +455,7 @@ static b2sp_status fused_rows(int M, int Kd, int N, const int *row_ptr, const in
         }
         if (rc != B2SP_OK) return rc;
     } else {
-        dim3 grid(gated_blocks((unsigned)M, gate), (unsigned)((N + 127) / 128), (unsigned)nbatch);
+        dim3 grid(gated_blocks((unsigned)M, gate, (unsigned)nbatch), (unsigned)((N + 127) / 128), (unsigned)nbatch);
         launch_row(fusedmm_row_scalar_kernel<DT>, grid, 0, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb,
                    D, ldd, O, ldo, order, gate, M, clear, rb);
     }
