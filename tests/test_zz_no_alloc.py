@@ -61,3 +61,25 @@ def test_static_scratch_rejects_oversized_problems():
         b.spmm_static_scratch(rp, e_i, e_f, D)
     assert e.value.status == 7
     assert "scratch" in str(e.value)
+
+
+def test_static_scratch_takes_the_largest_problem_it_promises():
+    """M equal to the limit is the one size at which the built-in array is exactly as large as the
+    workspace the regular entry point would ask for; most rows are empty, a few carry entries."""
+    from paper_2311_00368_b200 import binding as b
+    M, K, N = b.STATIC_SCRATCH_MAX_ROWS, 64, 32
+    rng = np.random.default_rng(11)
+    lens = np.zeros(M, dtype=np.int64)
+    busy = rng.choice(M, size=500, replace=False)
+    lens[busy] = rng.integers(1, K + 1, size=busy.size)
+    lens[M - 1] = K                       # the last row too
+    row_ptr = np.zeros(M + 1, dtype=np.int32)
+    row_ptr[1:] = np.cumsum(lens)
+    col_idx = np.concatenate([np.sort(rng.choice(K, size=l, replace=False)) for l in lens[lens > 0]]).astype(np.int32)
+    values = W.values_uniform(rng, int(row_ptr[-1]))
+    D = W.dense_normal(rng, K, N)
+    out = torch.full((M, N), float("nan"), device="cuda")
+    b.spmm_static_scratch(_dev(row_ptr), _dev(col_idx), _dev(values), _dev(D), K=K, out=out)   # B2SP_OK or it raises
+    ref, T = oracle.spmm(row_ptr, col_idx, values, D)
+    ok, ratio = oracle.within_tolerance(out.cpu().numpy(), ref, T, RTOL, ATOL)
+    assert ok, f"static-scratch SPMM at the size limit differs from the oracle by {ratio:.3g} x the tolerance"
