@@ -86,7 +86,7 @@ constexpr int kModeSddmm = 0, kModeFused = 1, kModeSpmm = 2;
 template <bool NARROW>
 __device__ __forceinline__ int helper_index(int warp)
 {
-    if (NARROW) return (warp & 3) == 1 || (warp >= 2 && warp < 6) ? -1 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);
+    if (NARROW) return warp == 13 ? 9 : (warp & 3) == 1 || (warp >= 2 && warp < 6) ? -1 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);
     if ((warp >= 1 && warp < 6) || warp == 9 || warp == 21 || warp == 25) return -1;
     return warp == 0 ? 0 : 1 + (warp - 6) - (warp > 9 ? 1 : 0) - (warp > 21 ? 1 : 0) - (warp > 25 ? 1 : 0);
 }
@@ -109,12 +109,12 @@ struct FusedCfg {
     static constexpr bool DEDICATED_FLUSH = SPMM;
     static constexpr int THREADS = !FUSED ? 896 : kFusedThreads;
     static constexpr int FLUSH_WARP0 = 16;   // the flusher warps: 16-19 (SPMM: dedicated; FusedMM: the second processor set)
-    static constexpr int RING = FUSED && !SPMM ? 3 : 4;
+    static constexpr int RING = FUSED ? 3 : 4;
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
     // 4 KB slots (two windows deep).  SPMM: twelve with twelve slots.  SDDMM: twenty with forty 2 KB slots
     // (measured: 12 helpers 134 us, 14 helpers 129 us, 20 helpers on 28 warps 125 us; for SPMM the same
     // layout was slower, 136-140 us against 131 us).
-    static constexpr int HELPERS = FUSED ? 8 : 20;
+    static constexpr int HELPERS = SPMM ? 10 : FUSED ? 8 : 20;
     // FusedMM runs two sets of processor warps (warps 2-5 and 16-19) that take alternate windows: a window is a
     // chain of long-latency steps for its processor (slot, tensor-memory load, arithmetic, tensor-memory store,
     // hand-over), about 2 k cycles, and with a single set that chain, not the tensor core, paced the kernel
@@ -123,7 +123,7 @@ struct FusedCfg {
     static constexpr int ITEM_ROWS = FUSED ? 32 : 16;           // rows of a helper's work item
     static constexpr int IPW = kFusedRows / ITEM_ROWS;         // items per window
     static constexpr int SLOT_BYTES = ITEM_ROWS * 128;
-    static constexpr int SLOTS = FUSED ? HELPERS : 2 * HELPERS;
+    static constexpr int SLOTS = SPMM ? 20 : FUSED ? HELPERS : 2 * HELPERS;
     // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one
     // phase away: every slot is always filled by the same helper and drained by the same processor warp.
     static_assert(SLOTS % HELPERS == 0 && SLOTS % IPW == 0, "slot ownership must be fixed");
