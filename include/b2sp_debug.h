@@ -39,6 +39,18 @@ int b2sp_last_launches(int op);
  */
 void b2sp_debug_force_k_splits(int k_splits);
 
+/*
+ * Test hook for the bounded waits of the dense-tile kernels.  Every wait inside those kernels gives up after a
+ * time limit (0.3 s), sets the workspace's device status word and lets its CTA leave through the normal
+ * teardown; b2sp_device_status and the host-buffer entry points then report B2SP_ERR_TIMEOUT.  To let a test see
+ * that path without stalling a GPU for long, this call (a) makes the TMA producer of every CTA of the dense-tile
+ * kernels launched afterwards leave out its `chunk`-th operand chunk, whose barrier therefore never completes,
+ * and (b) sets the time limit of the current device to `limit_ns` nanoseconds (a few milliseconds).  No wait is
+ * unbounded at any time.  chunk < 0 switches the hook off and restores the 0.3 s limit; call that before any
+ * other work.  Process-wide, synchronises the device (a copy to constant memory), not for production use.
+ */
+b2sp_status b2sp_debug_inject_wait_timeout(int chunk, unsigned long long limit_ns);
+
 #ifdef __cplusplus
 }
 #endif

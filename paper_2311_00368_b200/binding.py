@@ -80,6 +80,8 @@ lib.b2sp_last_launches.restype = _i
 lib.b2sp_last_launches.argtypes = [_i]
 lib.b2sp_debug_force_k_splits.restype = None
 lib.b2sp_debug_force_k_splits.argtypes = [_i]
+lib.b2sp_debug_inject_wait_timeout.restype = _i
+lib.b2sp_debug_inject_wait_timeout.argtypes = [_i, ctypes.c_ulonglong]
 
 
 class B2spError(RuntimeError):
@@ -159,6 +161,12 @@ def last_launches(op: int) -> int:
 def debug_force_k_splits(k_splits: int) -> None:
     """b2sp_debug_force_k_splits: override the dense-tile planner's K split (0 = planner's choice)."""
     lib.b2sp_debug_force_k_splits(int(k_splits))
+
+
+def debug_inject_wait_timeout(chunk: int, limit_ns: int = 0) -> None:
+    """b2sp_debug_inject_wait_timeout: make the dense-tile kernels' bounded waits run out (chunk >= 0) with a
+    short limit, or switch the hook off again (chunk < 0)."""
+    _check(lib.b2sp_debug_inject_wait_timeout(int(chunk), int(limit_ns)), "b2sp_debug_inject_wait_timeout")
 
 
 def spmm(row_ptr, col_idx, values, D, K=None, out=None, workspace=None, algo=ALGO_AUTO, dtype=torch.float32):

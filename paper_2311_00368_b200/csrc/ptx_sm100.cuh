@@ -2,7 +2,7 @@
 // TMA tensor loads (never multicast), tensor memory (TMEM) management, tcgen05.mma / commit /
 // ld, proxy fences, and the fp32 -> (tf32 hi, tf32 lo) split.
 //
-// Every wait is bounded: mbar_wait() gives up after kWaitLimitNs (and at most kWaitPolls tries) and
+// Every wait is bounded: mbar_wait() gives up after c_wait_limit_ns (0.3 s; and at most kWaitPolls tries) and
 // returns false, so a kernel can record the failure and leave instead of waiting forever.
 #pragma once
 #include <cuda_runtime.h>
@@ -16,6 +16,8 @@ namespace ptx {
 constexpr uint32_t kWaitPolls = 1u << 22;      // hard cap on tries
 constexpr uint32_t kWaitHintNs = 20000;        // per-try suspend hint
 constexpr uint64_t kWaitLimitNs = 300000000ull; // give up after 0.3 s
+// The limit in force (constant memory; kWaitLimitNs unless a test shortened it through b2sp_debug_inject_wait_timeout).
+__constant__ unsigned long long c_wait_limit_ns = kWaitLimitNs;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
@@ -113,7 +115,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
     const uint64_t t0 = global_timer_ns();
     for (uint32_t i = 0; i < kWaitPolls; ++i) {
         if (mbar_try_wait(bar, parity, kWaitHintNs)) return true;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (global_timer_ns() - t0 > c_wait_limit_ns) return false;
     }
     return false;
 }

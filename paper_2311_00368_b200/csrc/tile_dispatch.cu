@@ -18,6 +18,8 @@ constexpr int kSMs = 148;
 
 // 0 = the planner decides; set through b2sp_debug_force_k_splits (tests of the K-split epilogues, tuning).
 std::atomic<int> g_forced_k_splits{0};
+// -1 = off; set through b2sp_debug_inject_wait_timeout (the test of the bounded waits).
+std::atomic<int> g_drop_chunk{-1};
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -367,6 +369,7 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     if (exact && nb > 1) return B2SP_ERR_UNSUPPORTED;
     a.flags = flags; a.status = status;
+    a.debug_drop_chunk = g_drop_chunk.load(std::memory_order_relaxed);
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
     a.O = out; a.ldo = ldo;
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
@@ -405,4 +408,13 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 extern "C" void b2sp_debug_force_k_splits(int k_splits)
 {
     b2sp::g_forced_k_splits.store(k_splits > 0 ? k_splits : 0, std::memory_order_relaxed);
+}
+
+// Debug hook declared in include/b2sp_debug.h.
+extern "C" b2sp_status b2sp_debug_inject_wait_timeout(int chunk, unsigned long long limit_ns)
+{
+    const unsigned long long limit = chunk >= 0 && limit_ns > 0 ? limit_ns : b2sp::ptx::kWaitLimitNs;
+    if (cudaMemcpyToSymbol(b2sp::ptx::c_wait_limit_ns, &limit, sizeof(limit)) != cudaSuccess) return B2SP_ERR_CUDA;
+    b2sp::g_drop_chunk.store(chunk >= 0 ? chunk : -1, std::memory_order_relaxed);
+    return B2SP_OK;
 }

@@ -74,6 +74,8 @@ struct FusedTileArgs {
     int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
     int *flags;                // flags[kFlagUnsorted] or flags[kFlagNotFinite] != 0: the row kernels take over
     int *status;
+    int debug_drop_chunk;      // test hook: the TMA producer leaves out this chunk of every CTA (-1: none), so that the
+                               // waits for it run out and the CTA reports B2SP_ERR_TIMEOUT through the status word
 };
 
 // MODE: which op the kernel runs.  SPMM reuses the FusedMM pipeline with P' = the stored values
@@ -406,6 +408,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             auto put = [&](bool is_b, int blk, int i) -> bool {
                 const int s = c % RING;
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
+                if (c == a.debug_drop_chunk) { ++c; return true; }   // (test hook: nobody will ever complete this chunk's barrier)
                 const uint32_t dst = ring + s * kFusedChunk;
                 const int col0 = krow0 + (b0 + blk) * kFusedBlk;
                 ptx::mbar_arrive_expect_tx(full(s), (is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4) / (EXACT ? 2 : 1));   // hi (+ lo)

@@ -420,3 +420,34 @@ def test_non_finite_values_in_rows_nobody_refers_to(b):
     assert np.all(ref[10] == 0) and np.all(np.isfinite(ref))
     out = b.fusedmm(de.row_ptr, de.col_idx, de.values, de.A, de.B, de.D, workspace=ws, algo=TILE)
     gate(out, ref, T, "fusedmm tile, NaN in the A row of an empty row of S")
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_gpu_stays_usable(b):
+    """Every wait inside the dense-tile kernels is bounded.  The debug hook withholds one operand chunk in every
+    CTA and shortens the limit to 2 ms: the waits run out, the CTAs leave through their normal teardown, the
+    status word says B2SP_ERR_TIMEOUT (6) -- through b2sp_device_status and through the host-buffer form -- and the
+    next call on the same workspace is correct again."""
+    p = W.small_random(4500, 384, 1024, 0.2, 64, 128)
+    d = DevProblem(p)
+    ws = _ws(b, b.OP_FUSEDMM, p)
+    big = W.spmm_case()     # large enough for the host form's automatic choice to be the dense-tile family
+    t = lambda x: torch.from_numpy(x).pin_memory()
+    hO = torch.empty((big.M, big.N), dtype=torch.float32).pin_memory()
+    b.debug_inject_wait_timeout(1, 2_000_000)
+    try:
+        b.spmm(d.row_ptr, d.col_idx, d.values, d.D, workspace=ws, algo=TILE)
+        assert b.device_status(ws) == 6
+        b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, workspace=ws, algo=TILE)
+        assert b.device_status(ws) == 6
+        b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, workspace=ws, algo=TILE)
+        assert b.device_status(ws) == 6
+        with pytest.raises(b.B2spError) as e:
+            b.spmm_host(t(big.row_ptr), t(big.col_idx), t(big.values), t(big.D), hO)
+        assert e.value.status == 6
+    finally:
+        b.debug_inject_wait_timeout(-1)
+    torch.cuda.synchronize()
+    spmm_tile_check(b, p)
+    fused_tile_check(b, p)
+    ref, T = oracle.spmm(big.row_ptr, big.col_idx, big.values, big.D)
+    gate(b.spmm_host(t(big.row_ptr), t(big.col_idx), t(big.values), t(big.D), hO), ref, T, "spmm_host after the hook")
