@@ -153,17 +153,22 @@ b2sp_status launch_fused(dim3 grid, cudaStream_t st, int Kd, int N, const int *r
     size_t smem = sizeof(float4) * kRowWarps * U * (32 / SPLIT) +
                   (KU == 0 ? sizeof(float) * (size_t)((Kd + 3) & ~3) : 0);
     const bool batched = grid.z > 1;
-    auto kern = batched ? fusedmm_row_kernel<KU, U, SPLIT, true, DT> : fusedmm_row_kernel<KU, U, SPLIT, false, DT>;
+    auto kern_b = fusedmm_row_kernel<KU, U, SPLIT, true, DT>;
+    auto kern_1 = fusedmm_row_kernel<KU, U, SPLIT, false, DT>;
     if (smem > 48 * 1024) {
         if (smem > 200 * 1024) return B2SP_ERR_UNSUPPORTED;
-        if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-            cudaSuccess)
+        if (cudaFuncSetAttribute(batched ? reinterpret_cast<const void *>(kern_b) : reinterpret_cast<const void *>(kern_1),
+                                 cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
             return B2SP_ERR_CUDA;
     }
     const int nrows = (int)grid.x;
     grid.x = gated_blocks(grid.x, gate, grid.z);
-    launch_row(kern, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo, order, gate,
-               nrows, clear, rb);
+    if (batched)
+        launch_row(kern_b, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
+                   order, gate, nrows, clear, rb);
+    else
+        launch_row(kern_1, grid, smem, st, gate != nullptr || order != nullptr, Kd, N, row_ptr, col_idx, sv, A, lda, B, ldb, D, ldd, O, ldo,
+                   order, gate, nrows, clear, NoBatch{});
     return B2SP_OK;
 }
 

@@ -41,6 +41,9 @@ __device__ __forceinline__ void grid_wait_for_primary() { asm volatile("griddepc
 struct RowBatch {
     long long rp, nz, A, B, D, O;
 };
+struct NoBatch {};   // what a single-problem kernel takes in RowBatch's place (no parameter bytes, no arithmetic)
+template <bool BATCHED> struct BatchArg { using type = NoBatch; };
+template <> struct BatchArg<true> { using type = RowBatch; };
 
 // True when a gated launch has nothing to do (see the top of this file).  Called by every thread of the CTA.
 __device__ __forceinline__ bool gate_closed(int *gate)
@@ -445,12 +448,12 @@ fusedmm_row_kernel(int Kd, int N, const int *__restrict__ row_ptr, const int *__
                    const DT *__restrict__ B, int64_t ldb, const DT *__restrict__ D,
                    int64_t ldd, float *__restrict__ O, int64_t ldo,
                    const int *__restrict__ row_order, int *__restrict__ gate, int nrows, int *__restrict__ clear,
-                   RowBatch batch)
+                   typename BatchArg<BATCHED>::type batch)
 {
     using G = SweepGeom<U, SPLIT>;
     extern __shared__ float4 dyn_smem[];
     if (gate_closed(gate)) return;
-    if (BATCHED) {   // this problem's arrays
+    if constexpr (BATCHED) {   // this problem's arrays
         const long long pb = blockIdx.z;
         row_ptr += pb * batch.rp; col_idx += pb * batch.nz; if (s_values) s_values += pb * batch.nz;
         A += pb * batch.A; B += pb * batch.B; D += pb * batch.D; O += pb * batch.O;
