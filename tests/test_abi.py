@@ -79,3 +79,28 @@ def test_binding_refuses_to_run_without_the_library(tmp_path, monkeypatch):
     except ImportError:
         raised = True
     assert raised
+
+
+def test_batched_and_bf16_entry_points_check_arguments_without_a_gpu():
+    lib = ctypes.CDLL(b2sp_build.build())
+    i, ll, vp, sz = ctypes.c_int, ctypes.c_longlong, ctypes.c_void_p, ctypes.c_size_t
+    lib.b2sp_workspace_bytes_batched.restype = sz
+    lib.b2sp_workspace_bytes_batched.argtypes = [i, i, i, i, i, ll]
+    one = lib.b2sp_workspace_bytes_batched(1, 4096, 4096, 64, 64, 3_400_000)
+    eight = lib.b2sp_workspace_bytes_batched(8, 4096, 4096, 64, 64, 3_400_000)
+    assert one % 256 == 0 and eight > 4 * one > 0            # tables and operand copies are per problem (a single problem also holds K-split slabs)
+    assert lib.b2sp_workspace_bytes_batched(0, 4096, 4096, 64, 64, 3_400_000) == 0
+    wide = lib.b2sp_workspace_bytes_batched(8, 4096, 4096, 64, 512, 3_400_000)
+    assert 0 < wide < 1 << 20                                # wider than 256 columns: the row kernels' few bytes per row
+    lib.b2sp_fusedmm_batched.restype = i
+    lib.b2sp_fusedmm_batched.argtypes = [i, i, i, i, i, ll, vp, ll, vp, vp, vp, ll, ll, vp, ll, ll, vp, ll, ll, vp, ll, ll,
+                                         vp, sz, i, vp]
+    args = [2, 64, 64, 16, 16, 100, None, 65, None, None, None, 16, 1024, None, 16, 1024, None, 16, 1024, None, 16, 1024,
+            None, 0, 0, None]
+    assert lib.b2sp_fusedmm_batched(*args) == 1              # NULL row_ptr
+    args[0] = 0
+    assert lib.b2sp_fusedmm_batched(*args) == 1              # empty batch
+    lib.b2sp_spmm_bf16.restype = i
+    lib.b2sp_spmm_bf16.argtypes = [i, i, i, ll, vp, vp, vp, vp, ll, vp, ll, vp, sz, i, vp]
+    assert lib.b2sp_spmm_bf16(-1, 4, 4, 0, None, None, None, None, 4, None, 4, None, 0, 0, None) == 1
+    assert lib.b2sp_spmm_bf16(4, 4, 4, 3, None, None, None, None, 4, None, 4, None, 0, 0, None) == 1
