@@ -168,3 +168,23 @@ def test_bf16_configs_every_element(b):
     d, ws = every_family(b, W.sweep_case(0.3, 128))
     w = run(b, d, d.refs(("spmm", "sddmm", "fusedmm")), 0, ws, (TILE,), tag="auto")
     assert w < 0.5
+
+
+def test_bf16_non_finite_values_in_unreferenced_rows(b):
+    """As for fp32 operands: an Inf or NaN in a row of B or D that no stored entry names must not reach the
+    outputs; the operand pre-pass sees it and the bf16 row kernels produce the call's result."""
+    p = W.small_random(6300, 300, 700, 0.2, 64, 128)
+    dead = np.array([5, 77])
+    keep = ~np.isin(p.col_idx, dead)
+    lens = np.add.reduceat(keep.astype(np.int64), p.row_ptr[:-1].astype(np.int64))
+    rp = np.zeros(p.M + 1, dtype=np.int32)
+    rp[1:] = np.cumsum(lens)
+    q = W.Problem("holes", p.M, p.K, rp, p.col_idx[keep], p.values[keep], p.Kd, p.N, p.A, p.B.copy(), p.D.copy())
+    d = Bf16Problem(q)
+    refs = d.refs(("spmm", "sddmm", "fusedmm"))        # from the clean operands
+    d.D[5, :] = float("nan")
+    d.B[77, :] = float("inf")
+    ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    run(b, d, refs, TILE, ws, (TILE,), tag="NaN / Inf in unreferenced rows")
+    flags = ws[320:332].view(torch.int32).cpu().numpy()
+    assert flags[1] == 0 and flags[2] == 0
