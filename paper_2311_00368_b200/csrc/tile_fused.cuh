@@ -38,9 +38,10 @@ constexpr int kFusedRows = 128;     // rows per CTA (UMMA M)
 constexpr int kFusedW = 32;         // S columns per window
 constexpr int kFusedBlk = 128;      // S columns per block (UMMA N of GEMM1)
 // FusedMM and SPMM: 20 warps = 5 per scheduler (a sixth would cut the register budget from 96 to 80 per
-// thread).  Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors; warp 0 and warps
-// 6-19 except 9, 13, 17: helpers.  Warps 13 and 17 share the MMA warp's scheduler and idle: the tensor pipe
-// wants that scheduler's issue slots.  SDDMM: 28 warps of 72 registers, see FusedCfg.
+// thread; measured slower).  Warp 1: MMA issue + TMEM owner; warp 9: TMA producer; warps 2-5: processors;
+// warps 16-19: second processor set (FusedMM) or flusher warps (SPMM); helpers among warps 0, 6-8, 10-15
+// (FusedMM: eight, none on the MMA warp's scheduler, warps 13 and 15 idle; SPMM: ten, warp 13 included).
+// SDDMM: 28 warps of 72 registers, see FusedCfg.
 constexpr int kFusedThreads = 640;
 constexpr int kFusedTmaWarp = 9;
 constexpr int kFusedMaxHelpers = 20;
@@ -82,13 +83,13 @@ struct FusedTileArgs {
 // themselves (no A, no GEMM1).
 constexpr int kModeSddmm = 0, kModeFused = 1, kModeSpmm = 2;
 
-// Which helper a warp is (-1: none).  20-warp kernels (FusedMM, SPMM): warps 0, 6, 7, 8, 10, 11, 12, 14, ...
-// -> 0, 1, 2, ...: none on the MMA warp's scheduler (warp % 4 == 1).  28-warp kernel (SDDMM): every warp
-// but 1-5 (MMA, processors), 9 (TMA), 21 and 25.
+// Which helper a warp is (-1: none).  20-warp kernels (FusedMM, SPMM): warps 0, 6, 7, 8, 10, 11, 12, 14, 15
+// -> 0 .. 8 (none on the MMA warp's scheduler, warp % 4 == 1), then warp 13 -> 9; warps 16-19 have other roles.
+// 28-warp kernel (SDDMM): every warp but 1-5 (MMA, processors), 9 (TMA), 21 and 25.
 template <bool NARROW>
 __device__ __forceinline__ int helper_index(int warp)
 {
-    if (NARROW) return warp == 13 ? 9 : (warp & 3) == 1 || (warp >= 2 && warp < 6) ? -1 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);
+    if (NARROW) return warp == 13 ? 9 : (warp & 3) == 1 || (warp >= 2 && warp < 6) || warp >= 16 ? -1 : warp == 0 ? 0 : 1 + (warp - 6) - ((warp - 5) >> 2);
     if ((warp >= 1 && warp < 6) || warp == 9 || warp == 21 || warp == 25) return -1;
     return warp == 0 ? 0 : 1 + (warp - 6) - (warp > 9 ? 1 : 0) - (warp > 21 ? 1 : 0) - (warp > 25 ? 1 : 0);
 }
@@ -104,18 +105,18 @@ struct FusedCfg {
     static constexpr int NCH_D = FUSED ? kFusedBlk / kFusedW : 0;  // D chunks per block
     static constexpr int ALO_BYTES = (FUSED && !SPMM && !EXACT) ? kFusedRows * KDP * 4 : 0;
     // SDDMM runs 28 warps of 72 registers (its processors only copy P, and its helpers work on items of
-    // 16 rows, so nobody needs more): twenty helpers instead of twelve.  FusedMM and SPMM: 20 warps of 96.
+    // 16 rows, so nobody needs more) with twenty helpers.  FusedMM and SPMM: 20 warps of 96.
     // SPMM has four flusher warps (16-19) of its own: it has two O accumulators so that the tensor core can go on
     // while a partial sum leaves tensor memory, which only helps if the processors, who make its next operands,
     // are not the ones doing the flush (measured with role timers: a third of the processors' time).
     static constexpr bool DEDICATED_FLUSH = SPMM;
     static constexpr int THREADS = !FUSED ? 896 : kFusedThreads;
     static constexpr int FLUSH_WARP0 = 16;   // the flusher warps: 16-19 (SPMM: dedicated; FusedMM: the second processor set)
-    static constexpr int RING = FUSED ? 3 : 4;
+    static constexpr int RING = FUSED ? 3 : 4;   // TMA chunks in flight (32 KB each)
     // FusedMM is bound by the tensor pipe and its helpers are mostly idle: eight of them, with eight
-    // 4 KB slots (two windows deep).  SPMM: twelve with twelve slots.  SDDMM: twenty with forty 2 KB slots
-    // (measured: 12 helpers 134 us, 14 helpers 129 us, 20 helpers on 28 warps 125 us; for SPMM the same
-    // layout was slower, 136-140 us against 131 us).
+    // 4 KB slots (two windows deep).  SPMM, whose helpers are the bound: the ten warps left beside the flusher
+    // warps, with twenty slots.  SDDMM: twenty with forty 2 KB slots (measured: 12 helpers 134 us, 14 helpers
+    // 129 us, 20 helpers on 28 warps 125 us; for SPMM the 28-warp layout was slower, 136-140 us against 131 us).
     static constexpr int HELPERS = SPMM ? 10 : FUSED ? 8 : 20;
     // FusedMM runs two sets of processor warps (warps 2-5 and 16-19) that take alternate windows: a window is a
     // chain of long-latency steps for its processor (slot, tensor-memory load, arithmetic, tensor-memory store,
@@ -129,7 +130,7 @@ struct FusedCfg {
     // A slot's mbarriers are waited on by parity, which is only sound when the waiter is at most one
     // phase away: every slot is always filled by the same helper and drained by the same processor warp.
     static_assert(SLOTS % HELPERS == 0 && SLOTS % IPW == 0, "slot ownership must be fixed");
-    static constexpr int FLUSH_BYTES = FUSED ? 4 * 4096 : 0;   // per processor warp: two buffers of 32 rows x 16 columns
+    static constexpr int FLUSH_BYTES = FUSED ? 4 * 4096 : 0;   // per flushing warp: two buffers of 32 rows x 16 columns
     static constexpr int AUX_BYTES = 1024 /*barriers*/ + kFusedMaxHelpers * 256 /*record tables*/ + SLOTS * SLOT_BYTES + FLUSH_BYTES;
     static constexpr int SMEM_BYTES = RING * kFusedChunk + ALO_BYTES + 1024 + AUX_BYTES;
     // tensor-memory columns
