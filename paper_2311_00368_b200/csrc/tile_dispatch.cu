@@ -346,7 +346,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         const SplitJob ja{A, lda, M, Kd, nullptr, nullptr, a_rows_p, a_cols_p, nb, batch.A, dtype, 1};
         SplitJobs jobs;
         jobs.n = 0;
-        if (!spmm) { jobs.j[jobs.n++] = jb; jobs.j[jobs.n++] = ja; }
+        jobs.has_check = 0;
+        jobs.check = ja;
+        if (!spmm) { jobs.j[jobs.n++] = jb; jobs.has_check = 1; }
         if (fused) jobs.j[jobs.n++] = jd;
         // With several K splits the CTA that finishes an output tile last sums the splits' slabs: the
         // per-tile arrival counters start at zero.

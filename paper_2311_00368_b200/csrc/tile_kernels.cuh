@@ -213,32 +213,17 @@ struct TableCheck {
 };
 
 struct SplitJobs {
-    SplitJob j[3];
+    SplitJob j[2];    // operands to split (blockIdx.y picks one)
     int n;
+    SplitJob check;   // a check_only job done on the side by the blocks of job 0 (no blocks of its own: the launch
+    int has_check;    // stays one wave of blocks, and the tile kernel behind it waits for this grid to end)
 };
 
 __device__ __forceinline__ bool tf32_hi_not_finite(uint32_t hi) { return (hi & 0x7f800000u) == 0x7f800000u; }
 
-__global__ void split_dense_kernel(SplitJobs jobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
+// One job of split_dense_kernel, walked by the blocks (gridDim.x of them) of one blockIdx.y.  True: a non-finite hi part was seen.
+__device__ __forceinline__ bool split_job(const SplitJob &j)
 {
-    ptx::launch_dependents();   // the tile kernel may take its SMs; it waits for this grid before it reads anything
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
-        if (status) *status = 0;
-        if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
-    }
-    if ((int)blockIdx.y == jobs.n) {   // zero-fill job
-        const long long total = (long long)z.rows * z.cols;
-        const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
-        if (z.ld == z.cols && (total & 3) == 0 && (reinterpret_cast<uintptr_t>(z.out) & 15) == 0) {
-            for (long long i = t0; i < total / 4; i += step)
-                reinterpret_cast<float4 *>(z.out)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        } else {
-            for (long long i = t0; i < total; i += step) z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
-        }
-        if (chk.after_prepass) ptx::wait_for_primary_grid();
-        return;
-    }
-    const SplitJob j = jobs.j[blockIdx.y];
     const bool bf16 = j.dtype == kDenseBf16;
     // 16-byte loads of four fp32 (or 8-byte loads of four bf16) need the alignment for every operand of the batch
     const bool vec = (j.ld & 3) == 0 && (j.batch_stride & 3) == 0 &&
@@ -290,6 +275,30 @@ __global__ void split_dense_kernel(SplitJobs jobs, ZeroJob z, int *__restrict__ 
             if (j.lo) reinterpret_cast<uint4 *>(j.lo)[g] = make_uint4(l[0], l[1], l[2], l[3]);
         }
     }
+    return bad;
+}
+
+__global__ void split_dense_kernel(SplitJobs jobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
+{
+    ptx::launch_dependents();   // the tile kernel may take its SMs; it waits for this grid before it reads anything
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
+        if (status) *status = 0;
+        if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
+    }
+    if ((int)blockIdx.y == jobs.n) {   // zero-fill job
+        const long long total = (long long)z.rows * z.cols;
+        const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
+        if (z.ld == z.cols && (total & 3) == 0 && (reinterpret_cast<uintptr_t>(z.out) & 15) == 0) {
+            for (long long i = t0; i < total / 4; i += step)
+                reinterpret_cast<float4 *>(z.out)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        } else {
+            for (long long i = t0; i < total; i += step) z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
+        }
+        if (chk.after_prepass) ptx::wait_for_primary_grid();
+        return;
+    }
+    bool bad = split_job(jobs.j[blockIdx.y]);
+    if (jobs.has_check && blockIdx.y == 0) bad |= split_job(jobs.check);
     if (bad) atomicExch(&chk.flags[kFlagNotFinite], 1);
     if (chk.after_prepass) ptx::wait_for_primary_grid();
 }
