@@ -329,6 +329,17 @@ def measure_batched(torch, b, device, flush, problems, fp32_peak_gflops, hbm_gbs
     for _ in range(3):
         fn()
     stateless = time_calls(torch, stream, flush, fn, reps)[0]
+    # the same batch with bfloat16 Q, K, V (fp32 accumulation), prepared tables
+    bf16_ms = None
+    if auto == b.ALGO_TILE:
+        A16, B16, D16 = (t.to(torch.bfloat16) for t in (A, B, D))
+        b.prepare_pattern_batched(rp, ci, p0.K, ws)
+        fn = lambda: b.fusedmm_batched(rp, ci, sv, A16, B16, D16, out=O, workspace=ws, algo=b.ALGO_TILE_PREPARED,
+                                       dtype=torch.bfloat16)
+        for _ in range(3):
+            fn()
+        bf16_ms = time_calls(torch, stream, flush, fn, reps)[0]
+        del A16, B16, D16
     flops = sum(W.flops("fusedmm", p.nnz, p.Kd, p.N) for p in problems)
     nbytes = sum(W.compulsory_bytes("fusedmm", p.M, p.K, p.nnz, p.Kd, p.N) for p in problems)
     t_alu, t_hbm = flops / (fp32_peak_gflops * 1e9), nbytes / (hbm_gbs * 1e9)
@@ -339,6 +350,7 @@ def measure_batched(torch, b, device, flush, problems, fp32_peak_gflops, hbm_gbs
             "launches": launches, "stateless_ms": round(stateless, 4),
             "stateless_roofline_frac": round(t_roof / (stateless * 1e-3), 4),
             "call": f"b2sp_fusedmm_batched, {nb} problems in one call",
+            "bf16_operands_ms": None if bf16_ms is None else round(bf16_ms, 4),
             "parity_ok": ok if check else None, "parity_worst_error_over_allowed": round(worst, 4) if check else None}
 
 

@@ -223,6 +223,13 @@ b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long lo
                                  const float *B, long long ldb, long long stride_b, const float *D, long long ldd,
                                  long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
                                  size_t workspace_bytes, int algo, void *stream);
+/* The same with bfloat16 A, B, D (see b2sp_fusedmm_bf16): e.g. sparse attention on bfloat16 Q, K, V. */
+b2sp_status b2sp_fusedmm_batched_bf16(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                      const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                      const float *s_values, const void *A, long long lda, long long stride_a,
+                                      const void *B, long long ldb, long long stride_b, const void *D, long long ldd,
+                                      long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
+                                      size_t workspace_bytes, int algo, void *stream);
 
 /*
  * Host-buffer forms of the three ops: every data pointer is a HOST pointer (pinned memory

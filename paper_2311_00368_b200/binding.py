@@ -66,6 +66,8 @@ lib.b2sp_prepare_pattern_batched.argtypes = [_i, _i, _i, _ll, _vp, _ll, _vp, _vp
 lib.b2sp_fusedmm_batched.restype = _i
 lib.b2sp_fusedmm_batched.argtypes = [_i, _i, _i, _i, _i, _ll, _vp, _ll, _vp, _vp, _vp, _ll, _ll, _vp, _ll, _ll,
                                      _vp, _ll, _ll, _vp, _ll, _ll, _vp, _sz, _i, _vp]
+lib.b2sp_fusedmm_batched_bf16.restype = _i
+lib.b2sp_fusedmm_batched_bf16.argtypes = lib.b2sp_fusedmm_batched.argtypes
 lib.b2sp_prepare_pattern.restype = _i
 lib.b2sp_prepare_pattern.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_validate_csr.restype = _i
@@ -275,14 +277,15 @@ def prepare_pattern_batched(row_ptr, col_idx, K, workspace, batch=None):
                                             workspace.numel(), _stream()), "b2sp_prepare_pattern_batched")
 
 
-def fusedmm_batched(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO):
+def fusedmm_batched(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=None, algo=ALGO_AUTO, dtype=torch.float32):
     """b2sp_fusedmm_batched: O[b] = (S[b] .* (A[b] @ B[b].T)) @ D[b] for all problems of a batch in one
     call.  row_ptr [batch, M + 1] (each problem's positions start at 0), col_idx / s_values
     [batch, nnz_stride] (rows padded to a common length), A [batch, M, Kd], B [batch, K, Kd],
-    D [batch, K, N]; a 1-D row_ptr / col_idx / s_values or a 2-D dense operand is shared by all problems."""
+    D [batch, K, N]; a 1-D row_ptr / col_idx / s_values or a 2-D dense operand is shared by all problems.
+    dtype=torch.bfloat16: b2sp_fusedmm_batched_bf16 (A, B, D in bfloat16)."""
     _want(row_ptr, torch.int32, "row_ptr"); _want(col_idx, torch.int32, "col_idx")
-    _want(s_values, torch.float32, "s_values"); _want(A, torch.float32, "A"); _want(B, torch.float32, "B")
-    _want(D, torch.float32, "D")
+    _want(s_values, torch.float32, "s_values"); _want(A, dtype, "A"); _want(B, dtype, "B")
+    _want(D, dtype, "D")
     nb, M, rps, nzs = _batch_dims(row_ptr, col_idx)
     if nb is None:
         nb = max(t.shape[0] if t.dim() == 3 else 1 for t in (A, B, D))
@@ -294,10 +297,12 @@ def fusedmm_batched(row_ptr, col_idx, s_values, A, B, D, out=None, workspace=Non
         workspace = torch.empty(max(workspace_bytes_batched(nb, M, K, Kd, N, nzs), 1 << 20), dtype=torch.uint8,
                                 device=D.device)
     ld = lambda t: t.stride(-2) if t.shape[-2] > 1 else max(t.shape[-1], t.stride(-2))
-    _check(lib.b2sp_fusedmm_batched(nb, M, K, Kd, N, nzs, _ptr(row_ptr), rps, _ptr(col_idx), _ptr(s_values),
+    fn, name = ((lib.b2sp_fusedmm_batched, "b2sp_fusedmm_batched") if dtype == torch.float32
+                else (lib.b2sp_fusedmm_batched_bf16, "b2sp_fusedmm_batched_bf16"))
+    _check(fn(nb, M, K, Kd, N, nzs, _ptr(row_ptr), rps, _ptr(col_idx), _ptr(s_values),
                                     _ptr(A), ld(A), _batch_stride(A, nb), _ptr(B), ld(B), _batch_stride(B, nb),
                                     _ptr(D), ld(D), _batch_stride(D, nb), _ptr(out), ld(out), out.stride(0),
-                                    _ptr(workspace), workspace.numel(), algo, _stream()), "b2sp_fusedmm_batched")
+                                    _ptr(workspace), workspace.numel(), algo, _stream()), name)
     return out
 
 

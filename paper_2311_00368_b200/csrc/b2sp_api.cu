@@ -627,12 +627,13 @@ extern "C" b2sp_status b2sp_prepare_pattern_batched(int batch, int M, int K, lon
     return pattern_pass(false, M, K, nnz_stride, row_ptr, col_idx, workspace, st, &launches, bd);
 }
 
-extern "C" b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
-                                 const int *row_ptr, long long row_ptr_stride, const int *col_idx,
-                                 const float *s_values, const float *A, long long lda, long long stride_a,
-                                 const float *B, long long ldb, long long stride_b, const float *D, long long ldd,
-                                 long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
-                                 size_t workspace_bytes, int algo, void *stream)
+template <typename DT>
+static b2sp_status fusedmm_batched_impl(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                        const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                        const float *s_values, const DT *A, long long lda, long long stride_a,
+                                        const DT *B, long long ldb, long long stride_b, const DT *D, long long ldd,
+                                        long long stride_d, float *O, long long ldo, long long stride_o, void *workspace,
+                                        size_t workspace_bytes, int algo, void *stream)
 {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (bad_batch_args(batch, M, K, nnz_stride, row_ptr, row_ptr_stride, col_idx) || Kd < 0 || N < 0)
@@ -673,7 +674,7 @@ extern "C" b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int
         bd.count = batch; bd.rp = row_ptr_stride; bd.nz = nz_step;
         bd.A = stride_a; bd.B = stride_b; bd.D = stride_d; bd.O = stride_o;
         rc = fused_tile(plan, prepared, 1, M, K, Kd, N, nnz_stride, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd,
-                        O, ldo, workspace, st, &launches, false, bd);
+                        O, ldo, workspace, st, &launches, false, bd, dense_dtype<DT>());
         if (rc != B2SP_OK) return rc;
         int *gate = reinterpret_cast<int *>(static_cast<char *>(workspace) + kWsTileFlagsOffset);
         rc = fused_rows(M, Kd, N, row_ptr, col_idx, s_values, A, lda, B, ldb, D, ldd, O, ldo, nullptr, gate, nullptr, st,
@@ -686,6 +687,32 @@ extern "C" b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int
                     batch, rb);
     g_last_launches[B2SP_OP_FUSEDMM] = 1;
     return rc;
+}
+
+extern "C" b2sp_status b2sp_fusedmm_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                            const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                            const float *s_values, const float *A, long long lda, long long stride_a,
+                                            const float *B, long long ldb, long long stride_b, const float *D,
+                                            long long ldd, long long stride_d, float *O, long long ldo,
+                                            long long stride_o, void *workspace, size_t workspace_bytes, int algo,
+                                            void *stream)
+{
+    return fusedmm_batched_impl<float>(batch, M, K, Kd, N, nnz_stride, row_ptr, row_ptr_stride, col_idx, s_values, A, lda,
+                                       stride_a, B, ldb, stride_b, D, ldd, stride_d, O, ldo, stride_o, workspace,
+                                       workspace_bytes, algo, stream);
+}
+extern "C" b2sp_status b2sp_fusedmm_batched_bf16(int batch, int M, int K, int Kd, int N, long long nnz_stride,
+                                                 const int *row_ptr, long long row_ptr_stride, const int *col_idx,
+                                                 const float *s_values, const void *A, long long lda, long long stride_a,
+                                                 const void *B, long long ldb, long long stride_b, const void *D,
+                                                 long long ldd, long long stride_d, float *O, long long ldo,
+                                                 long long stride_o, void *workspace, size_t workspace_bytes, int algo,
+                                                 void *stream)
+{
+    return fusedmm_batched_impl<bf16_t>(batch, M, K, Kd, N, nnz_stride, row_ptr, row_ptr_stride, col_idx, s_values,
+                                        static_cast<const bf16_t *>(A), lda, stride_a, static_cast<const bf16_t *>(B), ldb,
+                                        stride_b, static_cast<const bf16_t *>(D), ldd, stride_d, O, ldo, stride_o,
+                                        workspace, workspace_bytes, algo, stream);
 }
 
 extern "C" b2sp_status b2sp_prepare_pattern(int M, int K, long long nnz, const int *row_ptr, const int *col_idx,

@@ -262,7 +262,12 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM on fp32 operands is offered on batches)
+    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
+        if (exact) {
+            if (kdp == 32) return launch_fused_tile<32, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
+            if (kdp == 64) return launch_fused_tile<64, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
+            return launch_fused_tile<128, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
+        }
         if (kdp == 32) return launch_fused_tile<32, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
         if (kdp == 64) return launch_fused_tile<64, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
         return launch_fused_tile<128, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
@@ -369,7 +374,6 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     a.batch = nb; a.ctas_per_problem = p.Mt * p.Nt * p.KS; a.Kp = p.Kp;
     a.stride_sv = batch.nz; a.stride_A = batch.A; a.stride_O = fused ? batch.O : batch.nz;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
-    if (exact && nb > 1) return B2SP_ERR_UNSUPPORTED;
     a.flags = flags; a.status = status;
     a.debug_drop_chunk = g_drop_chunk.load(std::memory_order_relaxed);
     a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);

@@ -191,3 +191,23 @@ def test_batched_call_can_be_captured_in_a_cuda_graph(b):
         torch.cuda.synchronize()
         assert b.device_status(ws) == 0
         s.check(out, f"batched call replayed from a CUDA graph, algo {algo}")
+
+
+def test_batched_bf16_operands(b):
+    """b2sp_fusedmm_batched_bf16: bfloat16 A, B, D, fp32 accumulation; the oracle runs on the rounded values."""
+    probs = [W.small_random(5600 + i, 300, 700, d, 64, 64, kind="uniform") for i, d in enumerate((0.2, 0.1, 0.3))]
+    bf = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16)
+    rounded = []
+    for p in probs:
+        A, B, D = bf(p.A), bf(p.B), bf(p.D)
+        rounded.append(W.Problem(p.name, p.M, p.K, p.row_ptr, p.col_idx, p.values, p.Kd, p.N,
+                                 A.float().numpy(), B.float().numpy(), D.float().numpy()))
+    s = Stacked(rounded)            # references from the bf16-rounded operands
+    A16, B16, D16 = s.A.to(torch.bfloat16), s.B.to(torch.bfloat16), s.D.to(torch.bfloat16)   # exact: already rounded
+    ws = s.workspace(b)
+    for algo, expect in ((TILE, TILE), (ROW, 2)):
+        out = torch.full((s.nb, s.M, s.N), float("nan"), device="cuda")
+        b.fusedmm_batched(s.row_ptr, s.col_idx, s.values, A16, B16, D16, out=out, workspace=ws, algo=algo,
+                          dtype=torch.bfloat16)
+        assert b.last_algo(b.OP_FUSEDMM) == expect and b.device_status(ws) == 0
+        s.check(out, f"batched bf16, algo {algo}")
