@@ -52,7 +52,7 @@
  * the row kernels produce that call's result (the check is per call and costs no extra launch).
  * Not checked, and undefined (NaN or Inf) on the dense-tile kernels: stored values s_p that are not
  * finite, and inputs so large that a dot product A_i . B_j overflows fp32 at ANY position (i, j) of
- * a 128 x 128 tile of S that holds a stored entry, stored there or not.
+ * S, stored or not (the dense-tile kernels form all of them).
  */
 #ifndef B2SP_H
 #define B2SP_H
