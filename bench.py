@@ -811,9 +811,9 @@ def main():
                 "vs_baseline": None, "dtype": ("f32 in/out, 3xTF32 products, fp32 accumulate"
                                               if any(a == "tile" for a in algos.values()) else "f32"),
                 "data": "synthetic",
-                "config": dict(workload_config(p, args.workload),
-                               pattern_table="built once per step, shared by the ops" if shared_table
-                               else "built inside each op that needs it"),
+                "config": workload_config(p, args.workload),
+                "pattern_table": ("built once per step, shared by the ops" if shared_table
+                                  else "built inside each op that needs it"),
                 "roofline": roof, "cpu_baseline": cpu_baseline, "parity": parity,
                 "e2e": e2e, "gpu_launches": int((sum(launches.values()) + (1 if shared_table else 0)) * args.steps),
                 "clocks": clocks, "ops": per_op, "bf16": bf16, "configs": configs, "configs_clocks": configs_clocks,
