@@ -314,6 +314,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     // the sum is reproducible.  false: a bounded wait gave up.
     auto flush_chunk = [&](int chunk) -> bool {
         const int ob = chunk % NOB;
+        const bool cat_halves = !EXACT && a.NT == 64;
         bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
         if (!__all_sync(0xffffffffu, ok)) return false;
         ptx::tc_fence_after_sync();
@@ -338,6 +339,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 }
                 uint32_t r[16];
                 ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                if (cat_halves) {   // hi * lo part of a 64-column tile (see GEMM2)
+                    uint32_t r2[16];
+                    ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + 64 + c * 16, r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+                }
                 ptx::tmem_ld_wait();
                 if (c == a.NT / 16 - 1) {
                     ptx::tc_fence_before_sync();
@@ -366,6 +374,13 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             for (int c = 0; c < a.NT / 16; ++c) {
                 uint32_t r[16];
                 ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + c * 16, r);
+                if (cat_halves) {
+                    uint32_t r2[16];
+                    ptx::tmem_ld_32x16(tmem + lane_addr + Cfg::COL_O + ob * kFusedNT + 64 + c * 16, r2);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) + __uint_as_float(r2[i]));
+                }
                 ptx::tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
@@ -419,7 +434,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 } else {      // D rows of window i of the block
                     const int krow = col0 + i * kFusedW;
                     ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (a.NT / 32));
-                    if (!EXACT) ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
+                    // (64-column O tiles: the lo copy sits right behind the 8 KB hi copy, so that [hi | lo] is one
+                    // MN-major operand of 128 columns, see GEMM2)
+                    if (!EXACT) ptx::tma_load_3d(dst + (a.NT == 64 ? kFusedW * 64 * 4 : kFusedChunk / 2), &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
                 }
                 ++c;
                 return true;
@@ -441,6 +458,12 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         if (lane == 0) {
             constexpr uint32_t idesc1 = ptx::idesc_tf32(kFusedRows, kFusedBlk, false, false);
             const uint32_t idesc2 = a.NT == 64 ? ptx::idesc_tf32(kFusedRows, 64, false, true) : ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
+            constexpr uint32_t idesc2_cat = ptx::idesc_tf32(kFusedRows, kFusedNT, false, true);
+            // 64-column O tiles (N <= 64): a 64-column MMA would leave half of the tensor core's width unused (it takes 46
+            // cycles, not 32), so P'_hi is multiplied by [D_hi | D_lo] in ONE 128-column MMA whose two halves land in
+            // columns 0-63 and 64-127 of the accumulator, P'_lo by D_hi in a 64-column one: two MMAs per K step instead
+            // of three; the flush adds the two halves.
+            const bool cat = !EXACT && a.NT == 64;
             int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
             auto gemm1 = [&](int b) -> bool {   // P = A_tile * B_block^T over NCH_B chunks
                 const int pb = FUSED ? 0 : (b & 1);
@@ -486,6 +509,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                     // groups 512 B apart, +1 KB per K step of 8 rows
                     const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
                     const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                    if (cat) {
+                        ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2_cat, ((b % kFusedFlushBlocks) | w | k8) != 0);
+                        ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
+                        continue;
+                    }
                     ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
                     ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
                     if (!EXACT) ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
