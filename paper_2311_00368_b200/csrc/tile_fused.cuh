@@ -503,20 +503,26 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 const uint32_t d_hi = ring + s * kFusedChunk, d_lo = d_hi + kFusedChunk / 2;
                 const uint32_t pph = tmem + Cfg::COL_PP + ppb * 64, ppl = pph + 32;
                 const uint32_t oacc = tmem + Cfg::COL_O + ((b / kFusedFlushBlocks) % NOB) * kFusedNT;
+                // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K groups 512 B apart,
+                // +1 KB per K step of 8 rows.  (Two copies of the loop: a test inside it costs the issuing thread, whose
+                // instruction stream paces the tensor pipe, several percent.)
+                const uint32_t first = ((b % kFusedFlushBlocks) | w) != 0;   // 0: this MMA starts a new partial sum
+                if (cat) {
 #pragma unroll
-                for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
-                    // D window: MN-major tf32 (32-byte-atom swizzle): column groups 4 KB apart, 4-row K
-                    // groups 512 B apart, +1 KB per K step of 8 rows
-                    const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                    const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
-                    if (cat) {
-                        ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2_cat, ((b % kFusedFlushBlocks) | w | k8) != 0);
+                    for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
+                        const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                        ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2_cat, k8 == 0 ? first : 1u);
                         ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
-                        continue;
                     }
-                    ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2, ((b % kFusedFlushBlocks) | w | k8) != 0);
-                    ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
-                    if (!EXACT) ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
+                } else {
+#pragma unroll
+                    for (int k8 = 0; k8 < kFusedW / 8; ++k8) {
+                        const uint64_t ddh = ptx::smem_desc(d_hi + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                        const uint64_t ddl = ptx::smem_desc(d_lo + k8 * 1024, kFusedW * 128, 512, ptx::kLayoutSw128Base32);
+                        ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddh, idesc2, k8 == 0 ? first : 1u);
+                        ptx::mma_tf32_ts(oacc, ppl + k8 * 8, ddh, idesc2, 1);
+                        if (!EXACT) ptx::mma_tf32_ts(oacc, pph + k8 * 8, ddl, idesc2, 1);
+                    }
                 }
                 ptx::mma_commit(pp_free(ppb));
                 ptx::mma_commit(empty(s));
