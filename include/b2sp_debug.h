@@ -40,6 +40,18 @@ int b2sp_last_launches(int op);
 void b2sp_debug_force_k_splits(int k_splits);
 
 /*
+ * Overrides, process-wide, how the dense-tile planner deals the work of an op to CTAs.  The planner knows two
+ * partitions: "tiles x K splits" (every CTA owns one 128-row tile of the output and one of equal ranges of the
+ * columns of S) and "balanced" (the 4-block accumulation granules of all output tiles, in tile order, dealt evenly
+ * to one CTA per SM, so that a CTA may end one tile and begin the next; offered where the kernel mode supports it
+ * and the number of 128-column blocks of S is a multiple of four).  partition = 0: the planner chooses (balanced
+ * where its longest CTA is at least 6% shorter); 1: tiles x K splits only; 2: balanced wherever it is offered.
+ * Like b2sp_debug_force_k_splits it changes b2sp_workspace_bytes and the order of the sums: set it before sizing
+ * the workspace.  For tests and tuning only.
+ */
+void b2sp_debug_force_partition(int partition);
+
+/*
  * Test hook for the bounded waits of the dense-tile kernels.  Every wait inside those kernels gives up after a
  * time limit (0.3 s), sets the workspace's device status word and lets its CTA leave through the normal
  * teardown; b2sp_device_status and the host-buffer entry points then report B2SP_ERR_TIMEOUT.  To let a test see

@@ -82,6 +82,8 @@ lib.b2sp_last_launches.restype = _i
 lib.b2sp_last_launches.argtypes = [_i]
 lib.b2sp_debug_force_k_splits.restype = None
 lib.b2sp_debug_force_k_splits.argtypes = [_i]
+lib.b2sp_debug_force_partition.restype = None
+lib.b2sp_debug_force_partition.argtypes = [_i]
 lib.b2sp_debug_inject_wait_timeout.restype = _i
 lib.b2sp_debug_inject_wait_timeout.argtypes = [_i, ctypes.c_ulonglong]
 
@@ -163,6 +165,11 @@ def last_launches(op: int) -> int:
 def debug_force_k_splits(k_splits: int) -> None:
     """b2sp_debug_force_k_splits: override the dense-tile planner's K split (0 = planner's choice)."""
     lib.b2sp_debug_force_k_splits(int(k_splits))
+
+
+def debug_force_partition(partition: int) -> None:
+    """b2sp_debug_force_partition: 0 = planner's choice, 1 = tiles x K splits only, 2 = balanced wherever offered."""
+    lib.b2sp_debug_force_partition(int(partition))
 
 
 def debug_inject_wait_timeout(chunk: int, limit_ns: int = 0) -> None:

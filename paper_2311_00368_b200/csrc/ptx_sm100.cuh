@@ -29,6 +29,12 @@ __device__ __forceinline__ void sts32(uint32_t addr, uint32_t v)
 {
     asm volatile("st.shared.b32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
 }
+__device__ __forceinline__ uint32_t lds32(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+    return v;
+}
 template <int OFF>
 __device__ __forceinline__ void sts32_off(uint32_t addr, uint32_t v)
 {
@@ -200,6 +206,15 @@ template <int N>
 __device__ __forceinline__ void bulk_wait() { asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory"); }
 // Orders async-proxy and generic-proxy accesses of this thread (all state spaces).
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// a + b as the fp32 add-reduction units of the memory system compute it: round to nearest even, subnormal inputs
+// and results flushed to zero
+__device__ __forceinline__ float add_like_reduction(float a, float b)
+{
+    float r;
+    asm("add.rn.ftz.f32 %0, %1, %2;" : "=f"(r) : "f"(a), "f"(b));
+    return r;
+}
 
 __device__ __forceinline__ void prefetch_l2(const void *p)
 {

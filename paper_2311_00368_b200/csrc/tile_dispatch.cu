@@ -18,6 +18,7 @@ constexpr int kSMs = 148;
 
 // 0 = the planner decides; set through b2sp_debug_force_k_splits (tests of the K-split epilogues, tuning).
 std::atomic<int> g_forced_k_splits{0};
+std::atomic<int> g_forced_partition{0};   // 0: the library chooses; 1: tiles x K splits only; 2: balanced wherever it is legal
 // -1 = off; set through b2sp_debug_inject_wait_timeout (the test of the bounded waits).
 std::atomic<int> g_drop_chunk{-1};
 
@@ -111,6 +112,35 @@ int pick_split(int base_tiles, int blocks)
     return ks;
 }
 
+// The balanced partition (see tile_fused.cuh) of `units` row tiles of `blocks` 128-column blocks each, for an output
+// of `nt` column tiles: groups of nt CTAs, the 4-block flush granules of all row tiles dealt evenly to the groups,
+// one CTA per SM.  Returns the number of CTAs (0: the plain partition, tiles x K splits, stays) and the slabs a tile
+// needs (= the most groups that share a row tile).
+int pick_balanced(long long units, int nt, int blocks, int ks, int *slabs)
+{
+    const int forced = g_forced_partition.load(std::memory_order_relaxed);   // b2sp_debug_force_partition
+    if (forced == 1 || blocks % kFusedFlushBlocks != 0 || nt > kSMs) return 0;
+    const long long gpt = blocks / kFusedFlushBlocks, gtot = units * gpt;
+    const long long groups = gtot < kSMs / nt ? gtot : kSMs / nt;
+    const long long gmax = (gtot + groups - 1) / groups;
+    if ((gmax + gpt - 2) / gpt + 1 > kFusedMaxSegs) return 0;   // a CTA would touch too many row tiles
+    if (forced != 2) {
+        // Worth it when the longest CTA gets clearly shorter than in the plain partition (whose CTAs come in waves).
+        // Measured on SPMM: the time falls by about 0.6 of what the lengths promise (more CTAs at work slow each
+        // other down), and slabs where the plain partition writes straight into O (one K split) cost a few percent:
+        // at 7/8 of the length 8192^2 x 128 gains 4%, x 256 (one K split) 0.5%, x 512 (one K split, two waves) 3%.
+        const long long plain = (units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks);
+        if (gmax * kFusedFlushBlocks * 100 > plain * (ks > 1 ? 94 : 88)) return 0;
+    }
+    int most = 1;
+    for (long long u = 0; u < units; ++u) {
+        const long long n = balanced_group_of(u * gpt + gpt - 1, gtot, groups) - balanced_group_of(u * gpt, gtot, groups) + 1;
+        if (n > most) most = (int)n;
+    }
+    *slabs = most < 2 ? 2 : most;   // (the kernel reads "one slab" as "straight into the output")
+    return (int)(groups * nt);
+}
+
 }  // namespace
 
 size_t pattern_table_offset(int M)
@@ -196,6 +226,11 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     size_t win_bytes = sizeof(int2) * (size_t)batch * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
+    if (fused && Kd == 0 && batch == 1) {   // (SPMM)
+        int slabs = 0;
+        p.bal_ctas = pick_balanced(p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, &slabs);
+        if (p.bal_ctas) p.KS = slabs;
+    }
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
     off = align_up(off + win_bytes, 1024);
@@ -212,8 +247,6 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
         off = align_up(off + dbytes, 1024);
         p.off_part = off;
         if (p.KS > 1) off += sizeof(float) * (size_t)batch * (size_t)p.KS * (size_t)p.Mt * kFusedRows * (size_t)p.Np;
-        p.off_cnt = off;   // one arrival counter per output tile (more than one K split only)
-        if (p.KS > 1) off = align_up(off + sizeof(int) * (size_t)batch * (size_t)p.Mt * (size_t)p.Nt, 256);
     }
     p.bytes = align_up(off, 256);
     p.feasible = true;
@@ -234,14 +267,14 @@ TwoPhasePlan plan_two_phase(int M, int K, int Kd, int N, long long nnz, size_t b
 
 namespace {
 
-template <int KDP, int MODE, bool BATCHED, bool EXACT>
+template <int KDP, int MODE, int PART, bool EXACT>
 b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                               const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                               cudaStream_t st)
 {
     using Cfg = FusedCfg<KDP, MODE, EXACT>;
-    auto kern = fused_tile_kernel<KDP, MODE, BATCHED, EXACT>;
-    if (!allow_dynamic_smem<KDP * 16 + MODE * 4 + (BATCHED ? 2 : 0) + (EXACT ? 1 : 0)>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
+    auto kern = fused_tile_kernel<KDP, MODE, PART, EXACT>;
+    if (!allow_dynamic_smem<KDP * 32 + MODE * 8 + PART * 2 + (EXACT ? 1 : 0)>(reinterpret_cast<const void *>(kern), Cfg::SMEM_BYTES)) return B2SP_ERR_CUDA;
     // a programmatic dependent of the operand-split kernel: its CTAs are placed while that kernel still runs
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)items);
@@ -264,27 +297,32 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
 {
     if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
         if (exact) {
-            if (kdp == 32) return launch_fused_tile<32, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
-            if (kdp == 64) return launch_fused_tile<64, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
-            return launch_fused_tile<128, kModeFused, true, true>(bh, bl, dh, dl, out, a, items, st);
+            if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
+            if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
+            return launch_fused_tile<128, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
         }
-        if (kdp == 32) return launch_fused_tile<32, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, kModeFused, true, false>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
+    }
+    if constexpr (MODE == kModeSpmm) {
+        if (a.bal_ctas > 0) {
+            if (exact) return launch_fused_tile<32, kModeSpmm, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
+            return launch_fused_tile<32, kModeSpmm, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
+        }
     }
     if (exact) {
-        if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, MODE, false, true>(bh, bl, dh, dl, out, a, items, st);
+        if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
     }
-    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
-    return launch_fused_tile<128, MODE, false, false>(bh, bl, dh, dl, out, a, items, st);
+    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
+    if (kdp == 64) return launch_fused_tile<64, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
+    return launch_fused_tile<128, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
 }
 
-// Splits (or only checks) up to three dense operands, clears the device status word and optionally
-// zero-fills an array.
-void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const TableCheck &chk, cudaStream_t st)
+// Splits (or only checks) up to three dense operands and clears the device status word.
+void launch_split(const SplitJobs &jobs, int *status, const TableCheck &chk, cudaStream_t st)
 {
     long long most = 1;
     for (int i = 0; i < jobs.n; ++i) {
@@ -292,7 +330,7 @@ void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const Ta
         if (g > most) most = g;
     }
     const long long want = (most + 255) / 256, cap = (long long)kSMs * 8;
-    dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)(jobs.n + (z.out ? 1 : 0)));
+    dim3 grid((unsigned)(want < cap ? want : cap), (unsigned)jobs.n);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = dim3(256);
@@ -302,7 +340,7 @@ void launch_split(const SplitJobs &jobs, const ZeroJob &z, int *status, const Ta
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = chk.after_prepass ? attr : nullptr;   // beside the pattern pre-pass of the same call, never beside foreign work
     cfg.numAttrs = chk.after_prepass ? 1 : 0;
-    cudaLaunchKernelEx(&cfg, split_dense_kernel, jobs, z, status, chk);
+    cudaLaunchKernelEx(&cfg, split_dense_kernel, jobs, status, chk);
 }
 
 }  // namespace
@@ -355,16 +393,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         jobs.check = ja;
         if (!spmm) { jobs.j[jobs.n++] = jb; jobs.has_check = 1; }
         if (fused) jobs.j[jobs.n++] = jd;
-        // With several K splits the CTA that finishes an output tile last sums the splits' slabs: the
-        // per-tile arrival counters start at zero.
-        const ZeroJob z = fused && p.KS > 1 ? ZeroJob{reinterpret_cast<float *>(ws + p.off_cnt), nb * p.Mt * p.Nt, 1, nb * p.Mt * p.Nt}
-                                            : ZeroJob{nullptr, 0, 0, 0};
         int *clear = keep_status ? nullptr : status;
         // (a prepared table is checked against this call's arrays here, so that the flags are final before the tile kernel)
         const TableCheck chk{make_signature(M, K, p.Wk, nnz, row_ptr, col_idx, batch),
                              prepared ? reinterpret_cast<const PatternSignature *>(ws + kWsSignatureOffset) : nullptr, flags,
                              prepared ? 0 : 1};
-        launch_split(jobs, z, clear, chk, st);
+        launch_split(jobs, clear, chk, st);
         *launches += 1;
     }
     if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
@@ -372,11 +406,11 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
     FusedTileArgs a;
     a.M = M; a.K = K; a.Kd = Kd; a.Kdp = p.Kdp; a.N = N; a.Wk = p.Wk; a.KS = p.KS; a.Nt = p.Nt; a.NT = p.NT;
     a.batch = nb; a.ctas_per_problem = p.Mt * p.Nt * p.KS; a.Kp = p.Kp;
+    a.tiles_pp = p.Mt * p.Nt; a.bal_ctas = p.bal_ctas;
     a.stride_sv = batch.nz; a.stride_A = batch.A; a.stride_O = fused ? batch.O : batch.nz;
     a.win = win; a.s_values = s_values; a.A = A; a.lda = lda;
     a.flags = flags; a.status = status;
     a.debug_drop_chunk = g_drop_chunk.load(std::memory_order_relaxed);
-    a.tile_arrivals = reinterpret_cast<int *>(ws + p.off_cnt);
     a.O = out; a.ldo = ldo;
     if (!fused) { a.out = out; a.ld_out = 0; a.slab = 0; }
     else if (p.KS == 1) { a.out = out; a.ld_out = ldo; a.slab = 0; }
@@ -399,12 +433,35 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
             a.out_tma = 1;
         }
     }
-    const int items = nb * p.Mt * p.Nt * p.KS;
+    const int items = p.bal_ctas ? p.bal_ctas : nb * p.Mt * p.Nt * p.KS;
     b2sp_status rc = spmm    ? launch_fused_kdp<kModeSpmm>(32, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
                      : fused ? launch_fused_kdp<kModeFused>(p.Kdp, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st)
                              : launch_fused_kdp<kModeSddmm>(p.Kdp, exact, tm_bh, tm_bl, tm_dh, tm_dl, tm_out, a, items, st);
     *launches += 1;
     if (rc != B2SP_OK) return rc;
+    if (fused && p.KS > 1) {
+        // several slabs per output tile: a kernel of its own, behind the tile kernel, adds them into O (slab_sum.cuh)
+        SlabSumArgs sa;
+        sa.slabs = part; sa.slab = a.slab; sa.ld = p.Np; sa.KS = p.KS;
+        sa.O = out; sa.ldo = ldo; sa.stride_O = batch.O;
+        sa.M = M; sa.N = N; sa.batch = nb; sa.Mt = p.Mt; sa.Nt = p.Nt; sa.NT = p.NT;
+        sa.gpt = p.Kp / kFusedBlk / kFusedFlushBlocks; sa.bal_ctas = p.bal_ctas;
+        sa.flags = flags;
+        const long long threads = (long long)nb * M * ((N + 3) / 4);
+        const long long want = (threads + 255) / 256, cap = (long long)kSMs * 8;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)(want < cap ? want : cap));
+        cfg.blockDim = dim3(256);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, slab_sum_kernel, sa);
+        *launches += 1;
+        if (cudaGetLastError() != cudaSuccess) return B2SP_ERR_CUDA;
+    }
     return B2SP_OK;
 }
 
@@ -414,6 +471,12 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
 extern "C" void b2sp_debug_force_k_splits(int k_splits)
 {
     b2sp::g_forced_k_splits.store(k_splits > 0 ? k_splits : 0, std::memory_order_relaxed);
+}
+
+// Debug / tuning hook declared in include/b2sp_debug.h.
+extern "C" void b2sp_debug_force_partition(int partition)
+{
+    b2sp::g_forced_partition.store(partition == 1 || partition == 2 ? partition : 0, std::memory_order_relaxed);
 }
 
 // Debug hook declared in include/b2sp_debug.h.

@@ -31,7 +31,8 @@ struct FusedPlan {
     bool feasible = false;
     int Kdp = 0, Nt = 1, Mt = 0, Wk = 0, KS = 1, Np = 0, Kp = 0;
     int NT = 128;   // O columns per CTA: 64 when N <= 64
-    size_t off_win = 0, off_bhi = 0, off_blo = 0, off_dhi = 0, off_dlo = 0, off_part = 0, off_cnt = 0;
+    int bal_ctas = 0;   // > 0: the balanced partition over this many CTAs (KS = slabs per output tile then)
+    size_t off_win = 0, off_bhi = 0, off_blo = 0, off_dhi = 0, off_dlo = 0, off_part = 0;
     size_t bytes = 0;
 };
 FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t base_off, bool fused, int batch = 1);

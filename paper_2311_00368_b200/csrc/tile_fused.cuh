@@ -29,6 +29,7 @@
 #include <stdint.h>
 
 #include "ptx_sm100.cuh"
+#include "slab_sum.cuh"
 #include "tile_kernels.cuh"
 
 
@@ -53,6 +54,14 @@ constexpr int kFusedNT = 128;       // most O columns per CTA (UMMA N of GEMM2);
 // round-to-nearest fp32 reductions and restarted from zero.
 constexpr int kFusedFlushBlocks = 4;
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
+// The balanced partition (FusedTileArgs::bal_ctas): the CTAs form groups of Nt (one CTA per column tile of O), and
+// the 4-block flush granules of all row tiles, in the order (problem, row tile, granule), are dealt evenly to the
+// groups -- group c of n gets granules [c * G / n, (c + 1) * G / n) of G -- so a CTA may finish one output tile and go
+// on with the next row tile's: at most kFusedMaxSegs segments, each with a slab of its own (the tile's first, second,
+// ... segment writes slab 0, 1, ...).  The CTAs of a group work on the same blocks of S at the same time, so S is
+// fetched from memory once per group.
+constexpr int kFusedMaxSegs = 4;
+// (balanced_group_of, in slab_sum.cuh, tells which group holds a granule.)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
@@ -62,6 +71,9 @@ struct FusedTileArgs {
     int batch, ctas_per_problem, Kp;
     long long stride_sv, stride_A, stride_O;
     int NT;                   // O columns per CTA (UMMA N of GEMM2): 128, or 64 when N <= 64
+    int tiles_pp;             // output tiles per problem (row tiles x column tiles)
+    int bal_ctas;             // > 0: the balanced partition over this many CTAs (KS = slabs per tile then); 0: every
+                              // CTA has one tile and one of its KS equal K splits
     const int2 *win;          // [M][Wk] window records (position, mask)
     const float *s_values;    // NULL = all ones
     const void *A;            // M x Kd, fp32 (bfloat16 in the EXACT kernels)
@@ -70,9 +82,8 @@ struct FusedTileArgs {
     long long ld_out, slab;
     int out_tma;              // the flush may use TMA on `out` (tm_out covers it; 16-byte aligned rows)
     int slab_rows;            // rows of one slab (TMA y coordinate of slab ks = ks * slab_rows)
-    float *O;                 // FusedMM / SPMM with several K splits: the output the slabs are summed into ...
+    float *O;                 // the caller's output (several slabs per tile: the grid behind this one adds them into it, see slab_sum.cuh)
     long long ldo;
-    int *tile_arrivals;       // ... by the CTA that arrives last at the tile's counter (zeroed before the launch)
     int *flags;                // flags[kFlagUnsorted] or flags[kFlagNotFinite] != 0: the row kernels take over
     int *status;
     int debug_drop_chunk;      // test hook: the TMA producer leaves out this chunk of every CTA (-1: none), so that the
@@ -137,13 +148,18 @@ struct FusedCfg {
     // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
     // chunk of blocks while the previous partial sum is flushed.
     static constexpr int NOB = SPMM ? 2 : 1;
+    static constexpr bool BALANCED = SPMM;   // the mode knows the balanced partition
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
 
-// BATCHED: the launch covers several problems (FusedTileArgs::batch); without it the problem index is the
-// constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to spare).
-template <int KDP, int MODE, bool BATCHED = false, bool EXACT = false>
+// PART: how the work is dealt to CTAs.  kPartTiles: every CTA has one output tile and one of its KS equal K splits.
+// kPartBatched: the same over several problems (FusedTileArgs::batch) -- a template parameter because without it the
+// problem index is the constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to
+// spare).  kPartBalanced: the balanced partition (see kFusedMaxSegs); a template parameter too: with the choice made
+// at run time the SPMM kernel was 5% slower on either partition.
+constexpr int kPartTiles = 0, kPartBatched = 1, kPartBalanced = 2;
+template <int KDP, int MODE, int PART = kPartTiles, bool EXACT = false>
 __global__ void __launch_bounds__((FusedCfg<KDP, MODE, EXACT>::THREADS), 1)
 fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
                   const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
@@ -175,17 +191,54 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr bool BATCHED = PART == kPartBatched, bal = PART == kPartBalanced;
+    static_assert(!bal || Cfg::BALANCED, "this mode does not know the balanced partition");
     const int prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;            // problem of the batch
     const int cta = BATCHED ? blockIdx.x % a.ctas_per_problem : blockIdx.x;
     const int ks = cta % a.KS;
     const int tile = cta / a.KS;
     const int nt = tile % a.Nt, mt = tile / a.Nt;
     const int nblk_all = (a.Wk + WPB - 1) / WPB;
-    const int b0 = (int)((long long)nblk_all * ks / a.KS), b1 = (int)((long long)nblk_all * (ks + 1) / a.KS);
-    const int nblk = b1 - b0;
-    const int m0 = mt * kFusedRows, n0 = nt * a.NT;
-    const int tiles_pp = a.ctas_per_problem / a.KS;            // output tiles per problem
+    const int m0 = mt * kFusedRows;
+    const int tiles_pp = a.tiles_pp;                             // output tiles per problem
     const int krow0 = prob * a.Kp;                               // first row of this problem in the stacked operand copies
+    // Balanced partition: this CTA's granules [g0, g1) of the batch's units * gpt, and its segments (one per
+    // output tile it touches) in shared memory, read by the roles through seg_at().
+    // segment records of eight ints (first block counted from the CTA's first, first row of the tile, column tile,
+    // first block within the tile's row of blocks, slab, problem, -, -); their number at segtab - 8
+    const uint32_t segtab = aux + 896;
+    constexpr uint32_t kSegStart = 0, kSegM0 = 4, kSegNt = 8, kSegBt0 = 12, kSegOrd = 16, kSegProb = 20;
+    const int gpt = nblk_all / kFusedFlushBlocks;
+    const int groups = bal ? a.bal_ctas / a.Nt : 1, grp = (int)blockIdx.x / a.Nt;   // (CTA blockIdx.x: group grp, column tile blockIdx.x % Nt)
+    const int mtiles = tiles_pp / a.Nt;                                               // row tiles per problem
+    const long long gtot = (long long)a.batch * mtiles * gpt;
+    const long long g0 = bal ? grp * gtot / groups : 0, g1 = bal ? (grp + 1ll) * gtot / groups : 0;
+    const int b0 = bal ? 0 : (int)((long long)nblk_all * ks / a.KS);
+    const int nblk = bal ? (int)(g1 - g0) * kFusedFlushBlocks : (int)((long long)nblk_all * (ks + 1) / a.KS) - b0;
+    if (bal && threadIdx.x == 0) {
+        int n = 0;
+        for (long long g = g0; g < g1 && n < kFusedMaxSegs; ++n) {
+            const int unit = (int)(g / gpt);                    // problem * row tiles + row tile
+            const long long gfirst = (long long)unit * gpt;
+            const uint32_t rec = segtab + n * 32;
+            ptx::sts32(rec + kSegStart, (uint32_t)((int)(g - g0) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegM0, (uint32_t)(unit % mtiles * kFusedRows));
+            ptx::sts32(rec + kSegNt, (uint32_t)((int)blockIdx.x % a.Nt));
+            ptx::sts32(rec + kSegBt0, (uint32_t)((int)(g - gfirst) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegOrd, (uint32_t)(grp - (int)balanced_group_of(gfirst, gtot, groups)));
+            ptx::sts32(rec + kSegProb, (uint32_t)(unit / mtiles));
+            g = gfirst + gpt < g1 ? gfirst + gpt : g1;
+        }
+        ptx::sts32(segtab - 8, (uint32_t)n);
+    }
+    // the record (shared-memory address) of the segment that holds block blk of this CTA, and a field of a record
+    auto seg_at = [&](int blk) -> uint32_t {
+        const int n = (int)ptx::lds32(segtab - 8);
+        uint32_t rec = segtab;
+        for (int i = 1; i < n; ++i) rec += blk >= (int)ptx::lds32(segtab + i * 32) ? 32u : 0u;
+        return rec;
+    };
+    auto seg_f = [&](uint32_t rec, uint32_t field) -> int { return (int)ptx::lds32(rec + field); };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
@@ -314,6 +367,14 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     // the sum is reproducible.  false: a bounded wait gave up.
     auto flush_chunk = [&](int chunk) -> bool {
         const int ob = chunk % NOB;
+        // the tile the chunk belongs to, its slab, and whether the chunk is the first partial sum that goes there
+        int m0 = mt * kFusedRows, n0 = nt * a.NT, ks = cta % a.KS, prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;
+        bool first_sum = chunk == 0;
+        if (bal) {
+            const uint32_t sg = seg_at(chunk * kFusedFlushBlocks);
+            m0 = seg_f(sg, kSegM0); n0 = seg_f(sg, kSegNt) * a.NT; ks = seg_f(sg, kSegOrd); prob = seg_f(sg, kSegProb);
+            first_sum = chunk * kFusedFlushBlocks == seg_f(sg, kSegStart);
+        }
         const bool cat_halves = !EXACT && a.NT == 64;
         bool ok = ptx::mbar_wait(o_full(ob), (chunk / NOB) & 1);
         if (!__all_sync(0xffffffffu, ok)) return false;
@@ -359,7 +420,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 ptx::fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) {
-                    if (chunk == 0) ptx::tma_store_3d(&tm_out, buf, n0 + c * 16, y, z);
+                    if (first_sum) ptx::tma_store_3d(&tm_out, buf, n0 + c * 16, y, z);
                     else ptx::tma_reduce_add_3d(&tm_out, buf, n0 + c * 16, y, z);
                     ptx::bulk_commit();
                 }
@@ -399,7 +460,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 #pragma unroll
                         for (int e = 0; e < 4; ++e) {
                             if (n + e >= ncols) continue;
-                            if (chunk == 0) dst[e] = __uint_as_float(x[e]);   // the first partial sum initialises the target
+                            if (first_sum) dst[e] = __uint_as_float(x[e]);   // the first partial sum initialises the target
                             else atomicAdd(dst + e, __uint_as_float(x[e]));
                         }
                     }
@@ -426,17 +487,22 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
                 if (c == a.debug_drop_chunk) { ++c; return true; }   // (test hook: nobody will ever complete this chunk's barrier)
                 const uint32_t dst = ring + s * kFusedChunk;
-                const int col0 = krow0 + (b0 + blk) * kFusedBlk;
+                int col0 = krow0 + (b0 + blk) * kFusedBlk, ntile = nt;
+                if (bal) {
+                    const uint32_t sg = seg_at(blk);
+                    col0 = seg_f(sg, kSegProb) * a.Kp + (seg_f(sg, kSegBt0) + blk - seg_f(sg, kSegStart)) * kFusedBlk;
+                    ntile = seg_f(sg, kSegNt);
+                }
                 ptx::mbar_arrive_expect_tx(full(s), (is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4) / (EXACT ? 2 : 1));   // hi (+ lo)
                 if (is_b) {   // B rows col0..col0+127, k group i
                     ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
                     if (!EXACT) ptx::tma_load_3d(dst + kFusedChunk / 2, &tm_blo, full(s), 0, col0, i);
                 } else {      // D rows of window i of the block
                     const int krow = col0 + i * kFusedW;
-                    ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, nt * (a.NT / 32));
+                    ptx::tma_load_3d(dst, &tm_dhi, full(s), 0, krow, ntile * (a.NT / 32));
                     // (64-column O tiles: the lo copy sits right behind the 8 KB hi copy, so that [hi | lo] is one
                     // MN-major operand of 128 columns, see GEMM2)
-                    if (!EXACT) ptx::tma_load_3d(dst + (a.NT == 64 ? kFusedW * 64 * 4 : kFusedChunk / 2), &tm_dlo, full(s), 0, krow, nt * (a.NT / 32));
+                    if (!EXACT) ptx::tma_load_3d(dst + (a.NT == 64 ? kFusedW * 64 * 4 : kFusedChunk / 2), &tm_dlo, full(s), 0, krow, ntile * (a.NT / 32));
                 }
                 ++c;
                 return true;
@@ -691,9 +757,18 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         const float *s_values = a.s_values + prob * a.stride_sv;           // this problem's stored values,
         const int2 *win = a.win + (size_t)prob * a.M * a.Wk;               // window table
         float *out_values = a.out + prob * a.stride_O;                     // and (SDDMM) output values
+        // (balanced partition: the tile and the first window of the segment that holds the items load_rec is asked
+        // for, which come in increasing order; single problem, so `win` and `s_values` are the problem's)
+        int seg_m0 = m0, seg_w0 = wbase, seg_end = bal ? 0 : nitems;
         auto load_rec = [&](int jj) {   // lane = row: window record of one row of item jj
             int2 r = make_int2(0, 0);
-            const int hrow = m0 + (jj % IPW) * IR + lane, wglob = wbase + jj / IPW;
+            if (bal && jj >= seg_end && jj < nitems) {   // the item is in a later segment than the one before: read its record
+                const uint32_t sg = seg_at(jj / (IPW * WPB));
+                seg_m0 = seg_f(sg, kSegM0);
+                seg_w0 = (seg_f(sg, kSegBt0) - seg_f(sg, kSegStart)) * WPB;
+                seg_end = sg + 32 < segtab + 32 * (uint32_t)ptx::lds32(segtab - 8) ? seg_f(sg + 32, kSegStart) * (IPW * WPB) : nitems;
+            }
+            const int hrow = seg_m0 + (jj % IPW) * IR + lane, wglob = seg_w0 + jj / IPW;
             if (jj < nitems && lane < IR && hrow < a.M && wglob < a.Wk) r = __ldg(win + (size_t)hrow * a.Wk + wglob);
             return r;
         };
@@ -755,39 +830,9 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         ptx::bulk_wait<0>();
         ptx::fence_proxy_async_all();
     }
-    if (FUSED && a.KS > 1) __threadfence();   // this CTA's slab is complete before its arrival is counted
+    // (Several slabs per output tile: the grid launched behind this one adds them into O, see slab_sum.cuh.)
     ptx::tc_fence_before_sync();
     __syncthreads();
-    if (FUSED && a.KS > 1) {
-        // The CTA that arrives last at its output tile's counter sums the K splits' slabs, always in
-        // the order of the splits, into O: no CTA waits for another and the result is reproducible.
-        int *last_flag = reinterpret_cast<int *>(smem_gen + (helper_tabs - smem_base));   // the record tables are idle now
-        if (threadIdx.x == 0) *last_flag = atomicAdd(a.tile_arrivals + prob * tiles_pp + tile, 1) == a.KS - 1;
-        __syncthreads();
-        if (*last_flag) {
-            __threadfence();
-            for (int e = threadIdx.x; e < kFusedRows * (a.NT / 4); e += Cfg::THREADS) {
-                const int r = e / (a.NT / 4), c = (e % (a.NT / 4)) * 4;
-                const int grow = m0 + r, n = n0 + c;
-                if (grow >= a.M || n >= a.N) continue;
-                const float *src = a.out + (long long)prob * a.KS * a.slab + (long long)grow * a.ld_out + n;
-                float4 acc = __ldcg(reinterpret_cast<const float4 *>(src));
-                for (int k = 1; k < a.KS; ++k) {
-                    const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + (long long)k * a.slab));
-                    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-                }
-                float *dst = a.O + prob * a.stride_O + (long long)grow * a.ldo + n;
-                if (n + 3 < a.N && (a.ldo & 3) == 0 && (a.stride_O & 3) == 0 && (reinterpret_cast<uintptr_t>(a.O) & 15) == 0) {
-                    *reinterpret_cast<float4 *>(dst) = acc;
-                } else {
-                    dst[0] = acc.x;
-                    if (n + 1 < a.N) dst[1] = acc.y;
-                    if (n + 2 < a.N) dst[2] = acc.z;
-                    if (n + 3 < a.N) dst[3] = acc.w;
-                }
-            }
-        }
-    }
     if (warp == 1) {
         __syncwarp();
         ptx::tmem_dealloc(tmem, 512);

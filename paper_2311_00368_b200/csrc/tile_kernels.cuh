@@ -172,8 +172,7 @@ __device__ __forceinline__ bool signature_matches(const PatternSignature &want, 
 // bf16 operands (dtype 1) are exact in tf32: hi is the value itself and no lo copy is written.
 // One launch handles up to three jobs (blockIdx.y picks the job) and, being the first kernel of
 // every tile op, also clears the workspace's device status word (unless `status` is NULL: the second
-// kernel of a two-phase op keeps what the first one reported) and, when asked to, zero-fills an
-// array (the last blockIdx.y): the per-tile arrival counters of a FusedMM / SPMM with several K splits.
+// kernel of a two-phase op keeps what the first one reported).
 //
 // The dense-tile kernels multiply whole windows of S, positions without a stored entry included (by
 // zero), so an Inf or NaN anywhere in a dense operand -- also in a row no stored entry refers to -- or a
@@ -194,12 +193,6 @@ struct SplitJob {
     int check_only;           // look for non-finite values, write nothing
 };
 
-struct ZeroJob {
-    float *out;      // NULL: nothing to clear
-    long long ld;
-    long long rows;
-    int cols;
-};
 
 // It also compares the signature stored beside a prepared window table with the arrays of this call
 // (`chk.have` != NULL) and raises the fallback flag on a mismatch: the flags are then final before the tile
@@ -278,24 +271,12 @@ __device__ __forceinline__ bool split_job(const SplitJob &j)
     return bad;
 }
 
-__global__ void split_dense_kernel(SplitJobs jobs, ZeroJob z, int *__restrict__ status, TableCheck chk)
+__global__ void split_dense_kernel(SplitJobs jobs, int *__restrict__ status, TableCheck chk)
 {
     ptx::launch_dependents();   // the tile kernel may take its SMs; it waits for this grid before it reads anything
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {
         if (status) *status = 0;
         if (chk.have && !signature_matches(chk.want, chk.have)) atomicExch(&chk.flags[kFlagUnsorted], 1);
-    }
-    if ((int)blockIdx.y == jobs.n) {   // zero-fill job
-        const long long total = (long long)z.rows * z.cols;
-        const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
-        if (z.ld == z.cols && (total & 3) == 0 && (reinterpret_cast<uintptr_t>(z.out) & 15) == 0) {
-            for (long long i = t0; i < total / 4; i += step)
-                reinterpret_cast<float4 *>(z.out)[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        } else {
-            for (long long i = t0; i < total; i += step) z.out[(i / z.cols) * z.ld + i % z.cols] = 0.f;
-        }
-        if (chk.after_prepass) ptx::wait_for_primary_grid();
-        return;
     }
     bool bad = split_job(jobs.j[blockIdx.y]);
     if (jobs.has_check && blockIdx.y == 0) bad |= split_job(jobs.check);

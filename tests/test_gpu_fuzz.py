@@ -1,6 +1,6 @@
 """Seeded random shapes through every entry point and family: sizes that are not multiples of the tile, odd
 widths, several densities and row-length laws, fp32 and bfloat16 operands, NULL values, batches of one to four
-problems, prepared and stateless calls.  Everything is checked element by element against the CPU oracle
+problems, prepared and stateless calls, either partition of the dense-tile work.  Everything is checked element by element against the CPU oracle
 (|gpu - ref| <= 1e-5 * T + 1e-6) and the device status word must stay clear."""
 import numpy as np
 import pytest
@@ -26,7 +26,18 @@ def _one_case(b, rng):
         return
     algo = int(rng.choice([0, 1, 3, 4]))
     use_bf, null = bool(rng.integers(0, 2)), bool(rng.random() < 0.25)
-    what = f"M={M} K={K} d={dens} Kd={Kd} N={N} nb={nb} {kind} algo={algo} bf16={use_bf} null={null}"
+    part = int(rng.choice([0, 1, 2]))   # the dense-tile planner's partition: its choice, tiles x K splits, balanced
+    what = f"M={M} K={K} d={dens} Kd={Kd} N={N} nb={nb} {kind} algo={algo} bf16={use_bf} null={null} partition={part}"
+    b.debug_force_partition(part)
+    try:
+        _run_case(b, rng, M, K, Kd, N, nb, probs, algo, use_bf, null, what)
+    finally:
+        b.debug_force_partition(0)
+
+
+def _run_case(b, rng, M, K, Kd, N, nb, probs, algo, use_bf, null, what):
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    bf = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16)
     if use_bf:                      # the bfloat16 values are the inputs: the oracle sees the rounded operands
         for p in probs:
             p.A, p.B, p.D = (bf(x).float().numpy() for x in (p.A, p.B, p.D))

@@ -10,7 +10,7 @@ from tests.test_gpu_parity import DevProblem, _custom_rows, gate
 
 pytestmark = pytest.mark.gpu
 
-TILE = 3
+TILE, PREPARED = 3, 4
 
 
 @pytest.fixture(scope="module")
@@ -308,6 +308,72 @@ def _k_split_epilogues(b, ks, width):
         again = torch.full((p.M, p.N), float("nan"), device="cuda")
         call(again)
         assert torch.equal(again, out.contiguous()), f"{name}: two runs differ ({ks} K splits)"
+
+
+@pytest.mark.parametrize("M,K,N,kind", [
+    (256, 512, 128, "uniform"),      # two row tiles, one granule each
+    (1000, 2048, 200, "uniform"),    # ragged last row tile, two column tiles (CTAs in groups of two), ragged width
+    (130, 4096, 300, "powerlaw"),    # three column tiles: 49 groups of three CTAs, eight granules per row tile
+    (5000, 512, 128, "uniform"),     # 40 row tiles of one granule: several whole tiles per CTA
+    (2049, 1536, 96, "band"),        # 17 row tiles of three granules: segments begin and end inside tiles
+    (700, 8192, 64, "uniform"),      # six row tiles of sixteen granules, one per CTA: sixteen slabs per tile
+])
+def test_balanced_partition_matches_plain(b, M, K, N, kind):
+    """SPMM on the balanced partition (granules of all row tiles dealt evenly to the CTAs, a slab per segment, the
+    slab-sum kernel behind) against the oracle, for bfloat16 operands too, on an output whose rows are padded and held
+    NaNs; twice, bit-equal; and the plain partition on the same workspace size rules afterwards."""
+    p = W.small_random(4300 + M, M, K, 0.15, 32, N, kind=kind)
+    d = DevProblem(p)
+    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
+    D16 = d.D.to(torch.bfloat16)
+    ref16, T16 = oracle.spmm(p.row_ptr, p.col_idx, p.values, D16.float().cpu().numpy())
+    outs = {}
+    for part in (2, 1):
+        b.debug_force_partition(part)
+        try:
+            ws = _ws(b, b.OP_SPMM, p)
+            b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
+            for pad in (4, 3):
+                padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
+                out = padded[:, :p.N]
+                b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=out, workspace=ws, algo=PREPARED)
+                assert b.last_algo(b.OP_SPMM) == TILE and b.device_status(ws) == 0
+                gate(out, ref, T, f"spmm partition {part}, rows padded by {pad}")
+                assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
+            again = torch.full((p.M, p.N), float("nan"), device="cuda")
+            b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=again, workspace=ws, algo=TILE)
+            assert torch.equal(again, out.contiguous()), f"two runs differ (partition {part})"
+            outs[part] = again
+            o16 = torch.full((p.M, p.N), float("nan"), device="cuda")
+            b.spmm(d.row_ptr, d.col_idx, d.values, D16, K=p.K, out=o16, workspace=ws, algo=TILE, dtype=torch.bfloat16)
+            assert b.device_status(ws) == 0
+            gate(o16, ref16, T16, f"spmm bf16 partition {part}")
+        finally:
+            b.debug_force_partition(0)
+    assert d.pattern_untouched()
+
+
+def test_balanced_partition_falls_back_on_non_finite_operand(b):
+    """The slab-sum kernel must not touch O when the row kernels produced it (a NaN in an unreferenced row of D)."""
+    p = W.small_random(4400, 600, 2048, 0.2, 32, 128)
+    keep = p.col_idx != 9
+    lens = np.add.reduceat(keep.astype(np.int64), p.row_ptr[:-1].astype(np.int64))
+    rp = np.zeros(p.M + 1, dtype=np.int32)
+    rp[1:] = np.cumsum(lens)
+    q = W.Problem("hole", p.M, p.K, rp, p.col_idx[keep], p.values[keep], p.Kd, p.N, p.A, p.B, p.D.copy())
+    ref, T = oracle.spmm(q.row_ptr, q.col_idx, q.values, q.D)
+    d = DevProblem(q)
+    d.D[9, :] = float("nan")
+    b.debug_force_partition(2)
+    try:
+        ws = _ws(b, b.OP_SPMM, q)
+        for _ in range(2):
+            out = torch.full((q.M, q.N), float("nan"), device="cuda")
+            b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=q.K, out=out, workspace=ws, algo=TILE)
+            assert b.device_status(ws) == 0
+            gate(out, ref, T, "spmm, balanced partition, NaN in an unreferenced row of D")
+    finally:
+        b.debug_force_partition(0)
 
 
 def test_tile_accuracy_on_same_sign_data_and_long_rows(b):
