@@ -13,11 +13,25 @@ namespace b2sp {
 constexpr int kSlabTileRows = 128;   // rows of an output tile (= kFusedRows)
 
 // The balanced partition deals the granules of all row tiles evenly to groups of CTAs: group c of n gets granules
-// [c * G / n, (c + 1) * G / n) of G.  The group that holds granule g: the last one whose range starts at or before g.
-__host__ __device__ inline long long balanced_group_of(long long g, long long gtot, long long groups)
-{
-    return ((g + 1) * groups - 1) / gtot;
-}
+// [c * G / n, (c + 1) * G / n) of G.  In 32-bit arithmetic throughout (G < 2^31, n a few hundred at most): 64-bit
+// divisions are calls of a library routine, and a call in the tile kernel cost it 9% of its speed.
+struct Balance {
+    int gtot, groups, q, r;   // G, n, G / n, G % n
+    __host__ __device__ Balance(int gtot_, int groups_) : gtot(gtot_), groups(groups_), q(gtot_ / groups_), r(gtot_ % groups_) {}
+    // first granule of group c (c = groups gives G): floor(c * G / n) = c * q + floor(c * r / n)
+    __host__ __device__ int start(int c) const { return c * q + c * r / groups; }
+    // the group that holds granule g: the last one whose range starts at or before g
+    __host__ __device__ int group_of(int g) const
+    {
+        int c = (int)((float)g * (float)groups / (float)gtot);   // within one or two of the answer
+        c = c < 0 ? 0 : c >= groups ? groups - 1 : c;
+        while (c > 0 && start(c) > g) --c;
+        while (c + 1 < groups && start(c + 1) <= g) ++c;
+        return c;
+    }
+    // how many groups share the tile whose granules are [first, first + gpt)
+    __host__ __device__ int groups_of_tile(int first, int gpt) const { return group_of(first + gpt - 1) - group_of(first) + 1; }
+};
 
 struct SlabSumArgs {
     const float *slabs;        // problem p, slab k: slabs + (p * KS + k) * slab, rows ld apart
@@ -47,11 +61,7 @@ __global__ void __launch_bounds__(256) slab_sum_kernel(const SlabSumArgs a)
         const long long pr = e / n4;
         const int r = (int)(pr % a.M), p = (int)(pr / a.M);
         int cnt = a.KS;
-        if (a.bal_ctas) {
-            const long long unit = (long long)p * a.Mt + r / kSlabTileRows, gtot = (long long)a.batch * a.Mt * a.gpt;
-            const int groups = a.bal_ctas / a.Nt;
-            cnt = (int)(balanced_group_of(unit * a.gpt + a.gpt - 1, gtot, groups) - balanced_group_of(unit * a.gpt, gtot, groups)) + 1;
-        }
+        if (a.bal_ctas) cnt = Balance(a.batch * a.Mt * a.gpt, a.bal_ctas / a.Nt).groups_of_tile((p * a.Mt + r / kSlabTileRows) * a.gpt, a.gpt);
         const float *src = a.slabs + (long long)p * a.KS * a.slab + (long long)r * a.ld + n;
         // (the first four slabs' loads in flight together)
         float4 v[4];

@@ -121,21 +121,25 @@ int pick_balanced(long long units, int nt, int blocks, int ks, int *slabs)
     const int forced = g_forced_partition.load(std::memory_order_relaxed);   // b2sp_debug_force_partition
     if (forced == 1 || blocks % kFusedFlushBlocks != 0 || nt > kSMs) return 0;
     const long long gpt = blocks / kFusedFlushBlocks, gtot = units * gpt;
+    if (gtot >= 0x7fffffffll / kSMs) return 0;   // (the partition's arithmetic is 32-bit)
     const long long groups = gtot < kSMs / nt ? gtot : kSMs / nt;
     const long long gmax = (gtot + groups - 1) / groups;
     if ((gmax + gpt - 2) / gpt + 1 > kFusedMaxSegs) return 0;   // a CTA would touch too many row tiles
     if (forced != 2) {
         // Worth it when the longest CTA gets clearly shorter than in the plain partition (whose CTAs come in waves).
-        // Measured on SPMM: the time falls by about 0.6 of what the lengths promise (more CTAs at work slow each
-        // other down), and slabs where the plain partition writes straight into O (one K split) cost a few percent:
-        // at 7/8 of the length 8192^2 x 128 gains 4%, x 256 (one K split) 0.5%, x 512 (one K split, two waves) 3%.
+        // Measured: the time falls by about 0.6 of what the lengths promise (more CTAs at work slow each other down,
+        // and the balanced FusedMM kernel is a few percent slower per block), and slabs where the plain partition writes
+        // straight into O (one K split) cost a few percent.  At 7/8 of the length: 8192^2 x 128 SPMM -7%, FusedMM -3%;
+        // x 256 (one K split) -4% / -1%; 32768 x 8192 x 128 (one K split, two waves) -3% / -5%.  At 2/3 (24576 x 8192,
+        // 192 tiles): -27% / -26%.  At equal length it loses 6-14%.
         const long long plain = (units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks);
         if (gmax * kFusedFlushBlocks * 100 > plain * (ks > 1 ? 94 : 88)) return 0;
     }
     int most = 1;
+    const Balance balance((int)gtot, (int)groups);
     for (long long u = 0; u < units; ++u) {
-        const long long n = balanced_group_of(u * gpt + gpt - 1, gtot, groups) - balanced_group_of(u * gpt, gtot, groups) + 1;
-        if (n > most) most = (int)n;
+        const int n = balance.groups_of_tile((int)(u * gpt), (int)gpt);
+        if (n > most) most = n;
     }
     *slabs = most < 2 ? 2 : most;   // (the kernel reads "one slab" as "straight into the output")
     return (int)(groups * nt);
@@ -226,7 +230,7 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     size_t win_bytes = sizeof(int2) * (size_t)batch * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
-    if (fused && Kd == 0 && batch == 1) {   // (SPMM)
+    if (fused && batch == 1) {   // (FusedMM and SPMM on one problem)
         int slabs = 0;
         p.bal_ctas = pick_balanced(p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, &slabs);
         if (p.bal_ctas) p.KS = slabs;
@@ -305,10 +309,16 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
         if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
         return launch_fused_tile<128, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
     }
-    if constexpr (MODE == kModeSpmm) {
+    if constexpr (MODE != kModeSddmm) {
         if (a.bal_ctas > 0) {
-            if (exact) return launch_fused_tile<32, kModeSpmm, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
-            return launch_fused_tile<32, kModeSpmm, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
+            if (exact) {
+                if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
+                if (kdp == 64) return launch_fused_tile<64, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
+                return launch_fused_tile<128, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
+            }
+            if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
+            if (kdp == 64) return launch_fused_tile<64, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
+            return launch_fused_tile<128, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
         }
     }
     if (exact) {

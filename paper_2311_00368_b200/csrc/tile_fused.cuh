@@ -61,7 +61,7 @@ constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 // ... segment writes slab 0, 1, ...).  The CTAs of a group work on the same blocks of S at the same time, so S is
 // fetched from memory once per group.
 constexpr int kFusedMaxSegs = 4;
-// (balanced_group_of, in slab_sum.cuh, tells which group holds a granule.)
+// (struct Balance, in slab_sum.cuh, holds the arithmetic.)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
@@ -148,139 +148,30 @@ struct FusedCfg {
     // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
     // chunk of blocks while the previous partial sum is flushed.
     static constexpr int NOB = SPMM ? 2 : 1;
-    static constexpr bool BALANCED = SPMM;   // the mode knows the balanced partition
+    static constexpr bool BALANCED = FUSED;   // the mode knows the balanced partition (FusedMM, SPMM)
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
 
-// PART: how the work is dealt to CTAs.  kPartTiles: every CTA has one output tile and one of its KS equal K splits.
-// kPartBatched: the same over several problems (FusedTileArgs::batch) -- a template parameter because without it the
-// problem index is the constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to
-// spare).  kPartBalanced: the balanced partition (see kFusedMaxSegs); a template parameter too: with the choice made
-// at run time the SPMM kernel was 5% slower on either partition.
-constexpr int kPartTiles = 0, kPartBatched = 1, kPartBalanced = 2;
-template <int KDP, int MODE, int PART = kPartTiles, bool EXACT = false>
-__global__ void __launch_bounds__((FusedCfg<KDP, MODE, EXACT>::THREADS), 1)
-fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
-                  const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
-                  const __grid_constant__ CUtensorMap tm_out, const FusedTileArgs a)
+// One thread's row (`row` of the tile, tensor-memory lane address lane_addr) of the A tile that begins at row tm0 of
+// problem tprob: the 16-column groups first, first + step, ... are split into tf32 hi (tensor memory) and lo (tensor
+// memory for SDDMM, shared memory at alo_smem for FusedMM; none for operands exact in tf32).
+template <int KDP, int MODE, bool EXACT>
+__device__ __forceinline__ void load_a_tile_impl(const void *A, long long lda, long long stride_A, int M, int Kd, uint32_t tmem,
+                                                 uint32_t lane_addr, uint32_t alo_smem, int row, int tm0, int tprob, int first, int step)
 {
     using Cfg = FusedCfg<KDP, MODE, EXACT>;
-    constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
-    constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
-    constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
-    extern __shared__ uint8_t smem_raw[];
-    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
-    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    const uint32_t ring = smem_base;                               // RING chunks of 32 KB
-    const uint32_t alo_smem = smem_base + RING * kFusedChunk;      // FusedMM: A_lo, K-major, 16 KB per 32 k
-    const uint32_t aux = alo_smem + Cfg::ALO_BYTES;
-    auto full = [&](int s) { return aux + 8u * s; };
-    auto empty = [&](int s) { return aux + 8u * (RING + s); };
-    auto p_full = [&](int b) { return aux + 8u * (2 * RING + b); };
-    auto p_free = [&](int b) { return aux + 8u * (2 * RING + 2 + b); };
-    auto pp_full = [&](int b) { return aux + 8u * (2 * RING + 4 + b); };
-    auto pp_free = [&](int b) { return aux + 8u * (2 * RING + 6 + b); };
-    constexpr int NSLOT = Cfg::SLOTS, NH = Cfg::HELPERS, NOB = Cfg::NOB;
-    auto o_full = [&](int b) { return aux + 8u * (b == 0 ? 2 * RING + 8 : 2 * RING + 11 + 2 * NSLOT); };
-    auto sl_full = [&](int s) { return aux + 8u * (2 * RING + 9 + s); };
-    auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
-    auto o_free = [&](int b) { return aux + 8u * (2 * RING + 9 + 2 * NSLOT + b); };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 12 + 2 * NSLOT));
-    const uint32_t helper_tabs = aux + 1024, slots = aux + 1024 + kFusedMaxHelpers * 256;
-    const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
+    constexpr bool FUSED = Cfg::FUSED;
+    struct { const void *A; long long lda, stride_A; int M, Kd; } a = {A, lda, stride_A, M, Kd};
 
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    constexpr bool BATCHED = PART == kPartBatched, bal = PART == kPartBalanced;
-    static_assert(!bal || Cfg::BALANCED, "this mode does not know the balanced partition");
-    const int prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;            // problem of the batch
-    const int cta = BATCHED ? blockIdx.x % a.ctas_per_problem : blockIdx.x;
-    const int ks = cta % a.KS;
-    const int tile = cta / a.KS;
-    const int nt = tile % a.Nt, mt = tile / a.Nt;
-    const int nblk_all = (a.Wk + WPB - 1) / WPB;
-    const int m0 = mt * kFusedRows;
-    const int tiles_pp = a.tiles_pp;                             // output tiles per problem
-    const int krow0 = prob * a.Kp;                               // first row of this problem in the stacked operand copies
-    // Balanced partition: this CTA's granules [g0, g1) of the batch's units * gpt, and its segments (one per
-    // output tile it touches) in shared memory, read by the roles through seg_at().
-    // segment records of eight ints (first block counted from the CTA's first, first row of the tile, column tile,
-    // first block within the tile's row of blocks, slab, problem, -, -); their number at segtab - 8
-    const uint32_t segtab = aux + 896;
-    constexpr uint32_t kSegStart = 0, kSegM0 = 4, kSegNt = 8, kSegBt0 = 12, kSegOrd = 16, kSegProb = 20;
-    const int gpt = nblk_all / kFusedFlushBlocks;
-    const int groups = bal ? a.bal_ctas / a.Nt : 1, grp = (int)blockIdx.x / a.Nt;   // (CTA blockIdx.x: group grp, column tile blockIdx.x % Nt)
-    const int mtiles = tiles_pp / a.Nt;                                               // row tiles per problem
-    const long long gtot = (long long)a.batch * mtiles * gpt;
-    const long long g0 = bal ? grp * gtot / groups : 0, g1 = bal ? (grp + 1ll) * gtot / groups : 0;
-    const int b0 = bal ? 0 : (int)((long long)nblk_all * ks / a.KS);
-    const int nblk = bal ? (int)(g1 - g0) * kFusedFlushBlocks : (int)((long long)nblk_all * (ks + 1) / a.KS) - b0;
-    if (bal && threadIdx.x == 0) {
-        int n = 0;
-        for (long long g = g0; g < g1 && n < kFusedMaxSegs; ++n) {
-            const int unit = (int)(g / gpt);                    // problem * row tiles + row tile
-            const long long gfirst = (long long)unit * gpt;
-            const uint32_t rec = segtab + n * 32;
-            ptx::sts32(rec + kSegStart, (uint32_t)((int)(g - g0) * kFusedFlushBlocks));
-            ptx::sts32(rec + kSegM0, (uint32_t)(unit % mtiles * kFusedRows));
-            ptx::sts32(rec + kSegNt, (uint32_t)((int)blockIdx.x % a.Nt));
-            ptx::sts32(rec + kSegBt0, (uint32_t)((int)(g - gfirst) * kFusedFlushBlocks));
-            ptx::sts32(rec + kSegOrd, (uint32_t)(grp - (int)balanced_group_of(gfirst, gtot, groups)));
-            ptx::sts32(rec + kSegProb, (uint32_t)(unit / mtiles));
-            g = gfirst + gpt < g1 ? gfirst + gpt : g1;
-        }
-        ptx::sts32(segtab - 8, (uint32_t)n);
-    }
-    // the record (shared-memory address) of the segment that holds block blk of this CTA, and a field of a record
-    auto seg_at = [&](int blk) -> uint32_t {
-        const int n = (int)ptx::lds32(segtab - 8);
-        uint32_t rec = segtab;
-        for (int i = 1; i < n; ++i) rec += blk >= (int)ptx::lds32(segtab + i * 32) ? 32u : 0u;
-        return rec;
-    };
-    auto seg_f = [&](uint32_t rec, uint32_t field) -> int { return (int)ptx::lds32(rec + field); };
-
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
-        for (int b = 0; b < 2; ++b) {
-            ptx::mbar_init(p_full(b), 1);
-            ptx::mbar_init(p_free(b), FUSED ? 4 * Cfg::PSETS : 4);
-            ptx::mbar_init(pp_full(b), 4);
-            ptx::mbar_init(pp_free(b), 1);
-        }
-        for (int b = 0; b < NOB; ++b) { ptx::mbar_init(o_full(b), 1); ptx::mbar_init(o_free(b), 4); }
-        for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(sl_full(s), 1); ptx::mbar_init(sl_empty(s), 1); }
-        ptx::fence_mbar_init();
-    }
-    if (warp == 1) {
-        __syncwarp();
-        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
-        ptx::tmem_relinquish();
-    }
-    ptx::tc_fence_before_sync();
-    __syncthreads();
-    ptx::tc_fence_after_sync();
-    const uint32_t tmem = *tmem_slot;
-    bool failed = false;
-
-    // ---- A tile -> TMEM (hi, and lo for SDDMM) / shared memory (lo for FusedMM); thread = row ----
-    // A warp reaches the tensor-memory lanes of quarter warp % 4: all warps of a quarter but the MMA and the
-    // TMA warp share the tile's 16-column groups.
-    const int q = warp & 3;                 // TMEM lane quarter
-    const int row = q * 32 + lane;          // row inside the tile
-    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-    constexpr int NWARP = Cfg::THREADS / 32;
-    const int pro_n = q == 1 ? NWARP / 4 - 2 : NWARP / 4;                            // warps of this quarter that take part
-    const int pro_i = q == 1 ? (warp == 5 ? 0 : (warp >> 2) - 2) : (warp >> 2);      // ... and this warp's place among them
-    if (!SPMM && warp != 1 && warp != kFusedTmaWarp) {
-        const int grow = m0 + row;
-        const long long aoff = prob * a.stride_A + (long long)(grow < a.M ? grow : 0) * a.lda;
+        const int grow = tm0 + row;
+        const long long aoff = tprob * a.stride_A + (long long)(grow < a.M ? grow : 0) * a.lda;
         const float *arow = static_cast<const float *>(a.A) + aoff;
         const unsigned short *arow16 = static_cast<const unsigned short *>(a.A) + aoff;
         const bool vec = (a.lda & 3) == 0 && (a.stride_A & 3) == 0 && (reinterpret_cast<uintptr_t>(a.A) & 15) == 0 &&
                          (!EXACT || (a.lda & 7) == 0);   // (16-byte loads of eight bf16)
 #pragma unroll 1
-        for (int c = pro_i * 16; c < KDP; c += pro_n * 16) {
+        for (int c = first * 16; c < KDP; c += step * 16) {
             uint32_t hi[16], lo[16];
             float v[16];
 #pragma unroll
@@ -340,6 +231,140 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         ptx::tmem_st_wait();
         if (FUSED) ptx::fence_proxy_async_smem();
     }
+
+// The same as a function of its own, for the reload at the end of a segment of the balanced partition: it runs once per
+// segment, and its code stays out of the processors' loop.
+template <int KDP, int MODE, bool EXACT>
+__device__ __noinline__ void reload_a_tile(const void *A, long long lda, long long stride_A, int M, int Kd, uint32_t tmem,
+                                           uint32_t lane_addr, uint32_t alo_smem, int row, int tm0, int tprob)
+{
+    load_a_tile_impl<KDP, MODE, EXACT>(A, lda, stride_A, M, Kd, tmem, lane_addr, alo_smem, row, tm0, tprob, 0, 1);
+}
+
+// PART: how the work is dealt to CTAs.  kPartTiles: every CTA has one output tile and one of its KS equal K splits.
+// kPartBatched: the same over several problems (FusedTileArgs::batch) -- a template parameter because without it the
+// problem index is the constant 0 and the kernel is exactly the single-problem one (the SDDMM mode has no registers to
+// spare).  kPartBalanced: the balanced partition (see kFusedMaxSegs); a template parameter too: with the choice made
+// at run time the SPMM kernel was 5% slower on either partition.
+constexpr int kPartTiles = 0, kPartBatched = 1, kPartBalanced = 2;
+template <int KDP, int MODE, int PART = kPartTiles, bool EXACT = false>
+__global__ void __launch_bounds__((FusedCfg<KDP, MODE, EXACT>::THREADS), 1)
+fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_constant__ CUtensorMap tm_blo,
+                  const __grid_constant__ CUtensorMap tm_dhi, const __grid_constant__ CUtensorMap tm_dlo,
+                  const __grid_constant__ CUtensorMap tm_out, const FusedTileArgs a)
+{
+    using Cfg = FusedCfg<KDP, MODE, EXACT>;
+    constexpr bool FUSED = Cfg::FUSED, SPMM = Cfg::SPMM;
+    constexpr int RING = Cfg::RING, NCH_B = Cfg::NCH_B;
+    constexpr int WPB = kFusedBlk / kFusedW;   // windows per block
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    const uint32_t ring = smem_base;                               // RING chunks of 32 KB
+    const uint32_t alo_smem = smem_base + RING * kFusedChunk;      // FusedMM: A_lo, K-major, 16 KB per 32 k
+    const uint32_t aux = alo_smem + Cfg::ALO_BYTES;
+    auto full = [&](int s) { return aux + 8u * s; };
+    auto empty = [&](int s) { return aux + 8u * (RING + s); };
+    auto p_full = [&](int b) { return aux + 8u * (2 * RING + b); };
+    auto p_free = [&](int b) { return aux + 8u * (2 * RING + 2 + b); };
+    auto pp_full = [&](int b) { return aux + 8u * (2 * RING + 4 + b); };
+    auto pp_free = [&](int b) { return aux + 8u * (2 * RING + 6 + b); };
+    constexpr int NSLOT = Cfg::SLOTS, NH = Cfg::HELPERS, NOB = Cfg::NOB;
+    auto o_full = [&](int b) { return aux + 8u * (b == 0 ? 2 * RING + 8 : 2 * RING + 11 + 2 * NSLOT); };
+    auto sl_full = [&](int s) { return aux + 8u * (2 * RING + 9 + s); };
+    auto sl_empty = [&](int s) { return aux + 8u * (2 * RING + 9 + NSLOT + s); };
+    auto o_free = [&](int b) { return aux + 8u * (2 * RING + 9 + 2 * NSLOT + b); };
+    const uint32_t a_ready = aux + 880;   // balanced FusedMM: the A tile of the next segment is in place (four processor warps)
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_gen + (aux - smem_base) + 8 * (2 * RING + 12 + 2 * NSLOT));
+    const uint32_t helper_tabs = aux + 1024, slots = aux + 1024 + kFusedMaxHelpers * 256;
+    const uint32_t flush_stage = slots + NSLOT * Cfg::SLOT_BYTES;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr bool BATCHED = PART == kPartBatched, bal = PART == kPartBalanced;
+    static_assert(!bal || Cfg::BALANCED, "this mode does not know the balanced partition");
+    const int prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;            // problem of the batch
+    const int cta = BATCHED ? blockIdx.x % a.ctas_per_problem : blockIdx.x;
+    const int ks = cta % a.KS;
+    const int tile = cta / a.KS;
+    const int nt = tile % a.Nt, mt = tile / a.Nt;
+    const int nblk_all = (a.Wk + WPB - 1) / WPB;
+    const int m0 = mt * kFusedRows;
+    const int tiles_pp = a.tiles_pp;                             // output tiles per problem
+    const int krow0 = prob * a.Kp;                               // first row of this problem in the stacked operand copies
+    // Balanced partition: this CTA's granules [g0, g1) of the batch's units * gpt, and its segments (one per
+    // output tile it touches) in shared memory, read by the roles through seg_at().
+    // segment records of eight ints (first block counted from the CTA's first, first row of the tile, column tile,
+    // first block within the tile's row of blocks, slab, problem, -, -); their number at segtab - 8
+    const uint32_t segtab = aux + 896;
+    constexpr uint32_t kSegStart = 0, kSegM0 = 4, kSegNt = 8, kSegBt0 = 12, kSegOrd = 16, kSegProb = 20;
+    const int gpt = nblk_all / kFusedFlushBlocks;
+    const int grp = (int)blockIdx.x / a.Nt;                        // (CTA blockIdx.x: group grp, column tile blockIdx.x % Nt)
+    const int mtiles = tiles_pp / a.Nt;                            // row tiles per problem
+    const Balance balance(bal ? a.batch * mtiles * gpt : 1, bal ? a.bal_ctas / a.Nt : 1);
+    const int g0 = bal ? balance.start(grp) : 0, g1 = bal ? balance.start(grp + 1) : 0;
+    const int b0 = bal ? 0 : (int)((long long)nblk_all * ks / a.KS);
+    const int nblk = bal ? (g1 - g0) * kFusedFlushBlocks : (int)((long long)nblk_all * (ks + 1) / a.KS) - b0;
+    if (bal && threadIdx.x == 0) {
+        int n = 0;
+        for (int g = g0; g < g1 && n < kFusedMaxSegs; ++n) {
+            const int unit = g / gpt;                    // problem * row tiles + row tile
+            const int gfirst = unit * gpt;
+            const uint32_t rec = segtab + n * 32;
+            ptx::sts32(rec + kSegStart, (uint32_t)((g - g0) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegM0, (uint32_t)(unit % mtiles * kFusedRows));
+            ptx::sts32(rec + kSegNt, (uint32_t)((int)blockIdx.x % a.Nt));
+            ptx::sts32(rec + kSegBt0, (uint32_t)((g - gfirst) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegOrd, (uint32_t)(grp - balance.group_of(gfirst)));
+            ptx::sts32(rec + kSegProb, (uint32_t)(unit / mtiles));
+            g = gfirst + gpt < g1 ? gfirst + gpt : g1;
+        }
+        ptx::sts32(segtab - 8, (uint32_t)n);
+    }
+    // the record (shared-memory address) of the segment that holds block blk of this CTA, and a field of a record
+    auto seg_at = [&](int blk) -> uint32_t {
+        const int n = (int)ptx::lds32(segtab - 8);
+        uint32_t rec = segtab;
+        for (int i = 1; i < n; ++i) rec += blk >= (int)ptx::lds32(segtab + i * 32) ? 32u : 0u;
+        return rec;
+    };
+    auto seg_f = [&](uint32_t rec, uint32_t field) -> int { return (int)ptx::lds32(rec + field); };
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < RING; ++s) { ptx::mbar_init(full(s), 1); ptx::mbar_init(empty(s), 1); }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(p_full(b), 1);
+            ptx::mbar_init(p_free(b), FUSED ? 4 * Cfg::PSETS : 4);
+            ptx::mbar_init(pp_full(b), 4);
+            ptx::mbar_init(pp_free(b), 1);
+        }
+        for (int b = 0; b < NOB; ++b) { ptx::mbar_init(o_full(b), 1); ptx::mbar_init(o_free(b), 4); }
+        for (int s = 0; s < NSLOT; ++s) { ptx::mbar_init(sl_full(s), 1); ptx::mbar_init(sl_empty(s), 1); }
+        ptx::mbar_init(a_ready, 4);
+        ptx::fence_mbar_init();
+    }
+    if (warp == 1) {
+        __syncwarp();
+        ptx::tmem_alloc(ptx::smem_u32(const_cast<uint32_t *>(tmem_slot)), 512);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem = *tmem_slot;
+    bool failed = false;
+
+    // ---- A tile -> TMEM (hi, and lo for SDDMM) / shared memory (lo for FusedMM); thread = row ----
+    // A warp reaches the tensor-memory lanes of quarter warp % 4: all warps of a quarter but the MMA and the
+    // TMA warp share the tile's 16-column groups.
+    const int q = warp & 3;                 // TMEM lane quarter
+    const int row = q * 32 + lane;          // row inside the tile
+    const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+    constexpr int NWARP = Cfg::THREADS / 32;
+    const int pro_n = q == 1 ? NWARP / 4 - 2 : NWARP / 4;                            // warps of this quarter that take part
+    const int pro_i = q == 1 ? (warp == 5 ? 0 : (warp >> 2) - 2) : (warp >> 2);      // ... and this warp's place among them
+    if (!SPMM && warp != 1 && warp != kFusedTmaWarp)
+        load_a_tile_impl<KDP, MODE, EXACT>(a.A, a.lda, a.stride_A, a.M, a.Kd, tmem, lane_addr, alo_smem, row, bal ? (int)ptx::lds32(segtab + kSegM0) : m0,
+                                           bal ? (int)ptx::lds32(segtab + kSegProb) : prob, pro_i, pro_n);
     ptx::tc_fence_before_sync();
     __syncthreads();
     ptx::tc_fence_after_sync();
@@ -482,17 +507,21 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             // Chunk order = the order the MMA thread consumes them: B(0); then per block b:
             // D(b,0) D(b,1) | B(b+1) | D(b,2) D(b,3)   (SDDMM: B chunks only; last block of a chunk: B(b+1) last).
             int c = 0;
+            // first row of the CTA's block 0 in the stacked operand copies, column tile, and (balanced partition) the
+            // block at which the next segment begins
+            int seg_col0 = krow0 + b0 * kFusedBlk, ntile = nt, seg_end = bal ? 0 : nblk;
             auto put = [&](bool is_b, int blk, int i) -> bool {
                 const int s = c % RING;
                 if (c >= RING && !ptx::mbar_wait(empty(s), ((c / RING) - 1) & 1)) return false;
                 if (c == a.debug_drop_chunk) { ++c; return true; }   // (test hook: nobody will ever complete this chunk's barrier)
                 const uint32_t dst = ring + s * kFusedChunk;
-                int col0 = krow0 + (b0 + blk) * kFusedBlk, ntile = nt;
-                if (bal) {
+                if (bal && blk >= seg_end) {   // a later segment than the one before (the blocks come in increasing order)
                     const uint32_t sg = seg_at(blk);
-                    col0 = seg_f(sg, kSegProb) * a.Kp + (seg_f(sg, kSegBt0) + blk - seg_f(sg, kSegStart)) * kFusedBlk;
+                    seg_col0 = seg_f(sg, kSegProb) * a.Kp + (seg_f(sg, kSegBt0) - seg_f(sg, kSegStart)) * kFusedBlk;
                     ntile = seg_f(sg, kSegNt);
+                    seg_end = sg + 32 < segtab + 32 * (uint32_t)ptx::lds32(segtab - 8) ? seg_f(sg + 32, kSegStart) : nblk;
                 }
+                const int col0 = seg_col0 + blk * kFusedBlk;
                 ptx::mbar_arrive_expect_tx(full(s), (is_b ? kFusedChunk : 2 * kFusedW * a.NT * 4) / (EXACT ? 2 : 1));   // hi (+ lo)
                 if (is_b) {   // B rows col0..col0+127, k group i
                     ptx::tma_load_3d(dst, &tm_bhi, full(s), 0, col0, i);
@@ -531,10 +560,19 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
             // of three; the flush adds the two halves.
             const bool cat = !EXACT && a.NT == 64;
             int c = 0, ppu = 0;   // chunk counter, P' buffer uses so far
+            // balanced partition: the next segment whose A tile GEMM1 will need, and its first block
+            int a_seg = 1, a_next = (bal && !SPMM && (int)ptx::lds32(segtab - 8) > 1) ? (int)ptx::lds32(segtab + 32 + kSegStart) : -1;
             auto gemm1 = [&](int b) -> bool {   // P = A_tile * B_block^T over NCH_B chunks
                 const int pb = FUSED ? 0 : (b & 1);
                 const int puse = FUSED ? b : (b >> 1);
                 if (puse > 0 && !ptx::mbar_wait(p_free(pb), (puse - 1) & 1)) return false;   // P drained?
+                if (bal && !SPMM && b == a_next) {
+                    // first block of a new segment: the processors have put the next row tile of A in place
+                    if (!ptx::mbar_wait(a_ready, (a_seg - 1) & 1)) return false;
+                    ptx::tc_fence_after_sync();
+                    ++a_seg;
+                    a_next = a_seg < (int)ptx::lds32(segtab - 8) ? (int)ptx::lds32(segtab + a_seg * 32 + kSegStart) : -1;
+                }
                 const uint32_t pacc = tmem + Cfg::COL_P + pb * kFusedBlk;
                 for (int i = 0; i < NCH_B; ++i, ++c) {
                     const int s = c % RING;
@@ -627,7 +665,11 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         const int nwin = nblk * WPB;
         constexpr int PSETS = Cfg::PSETS;
         const int pset = warp >= 16 ? 1 : 0;   // which set of processor warps this one belongs to
-        for (int it = FUSED ? pset : 0; it < nwin; it += FUSED ? PSETS : 1) {
+        // (balanced FusedMM: one round per segment, it_end = first window of the next segment; otherwise a single round)
+        int it = FUSED ? pset : 0;
+        int it_end = (bal && !SPMM && (int)ptx::lds32(segtab - 8) > 1) ? (int)ptx::lds32(segtab + 32 + kSegStart) * WPB : nwin;
+        for (;;) {
+        for (; it < it_end; it += FUSED ? PSETS : 1) {
             const int blk = it / WPB, w = it % WPB;
             // FusedMM / SPMM: one item (32 rows) per processor warp and window.  SDDMM: two items of 16 rows,
             // lanes 0-15 and lanes 16-31 each with their own slot.
@@ -735,6 +777,19 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
                 __syncwarp();
                 if ((lane & 15) == 0) ptx::mbar_arrive(sl_full(s));
             }
+        }
+        if (failed || it_end >= nwin) break;
+        // End of a segment of the balanced partition.  GEMM1 of its last block is complete (both sets have read its
+        // result), so the A tile makes way for the next segment's: the first set of processors loads it (the second one
+        // is flushing O meanwhile), and GEMM1 of the next block waits for its four warps.
+        const uint32_t next = seg_at(it_end / WPB);   // the segment that begins there
+        if (pset == 0) {
+            reload_a_tile<KDP, MODE, EXACT>(a.A, a.lda, a.stride_A, a.M, a.Kd, tmem, lane_addr, alo_smem, row, seg_f(next, kSegM0), seg_f(next, kSegProb));
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(a_ready);
+        }
+        it_end = next + 32 < segtab + 32 * (uint32_t)ptx::lds32(segtab - 8) ? seg_f(next + 32, kSegStart) * WPB : nwin;
         }
     } else if (Cfg::DEDICATED_FLUSH && warp >= Cfg::FLUSH_WARP0) {
         // ---------------- flusher warps (SPMM): take every chunk's partial sum out of tensor memory ----------------

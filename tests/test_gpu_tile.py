@@ -310,44 +310,55 @@ def _k_split_epilogues(b, ks, width):
         assert torch.equal(again, out.contiguous()), f"{name}: two runs differ ({ks} K splits)"
 
 
-@pytest.mark.parametrize("M,K,N,kind", [
-    (256, 512, 128, "uniform"),      # two row tiles, one granule each
-    (1000, 2048, 200, "uniform"),    # ragged last row tile, two column tiles (CTAs in groups of two), ragged width
-    (130, 4096, 300, "powerlaw"),    # three column tiles: 49 groups of three CTAs, eight granules per row tile
-    (5000, 512, 128, "uniform"),     # 40 row tiles of one granule: several whole tiles per CTA
-    (2049, 1536, 96, "band"),        # 17 row tiles of three granules: segments begin and end inside tiles
-    (700, 8192, 64, "uniform"),      # six row tiles of sixteen granules, one per CTA: sixteen slabs per tile
+@pytest.mark.parametrize("M,K,Kd,N,kind,density", [
+    (256, 512, 32, 128, "uniform", 0.15),      # two row tiles, one granule each
+    (1000, 2048, 128, 200, "uniform", 0.15),   # ragged last row tile, two column tiles (CTAs in groups of two), ragged width
+    (130, 4096, 100, 300, "powerlaw", 0.15),   # three column tiles: 49 groups of three CTAs (FusedMM: two phases at this width)
+    (700, 8192, 64, 64, "uniform", 0.15),      # six row tiles of sixteen granules, one per CTA: sixteen slabs per tile
+    (6400, 2048, 64, 128, "uniform", 0.05),    # 200 granules on 148 CTAs: one or two each, segments end inside row tiles
+    (25600, 512, 128, 64, "uniform", 0.05),    # 200 row tiles of one granule: CTAs with two whole tiles (two A tiles)
+    (20000, 1024, 32, 200, "powerlaw", 0.04),  # 157 row tiles of two granules, groups of two CTAs: up to three segments
+    (9000, 1536, 128, 128, "band", 0.05),      # 71 row tiles of three granules
 ])
-def test_balanced_partition_matches_plain(b, M, K, N, kind):
-    """SPMM on the balanced partition (granules of all row tiles dealt evenly to the CTAs, a slab per segment, the
-    slab-sum kernel behind) against the oracle, for bfloat16 operands too, on an output whose rows are padded and held
-    NaNs; twice, bit-equal; and the plain partition on the same workspace size rules afterwards."""
-    p = W.small_random(4300 + M, M, K, 0.15, 32, N, kind=kind)
+def test_balanced_partition_matches_plain(b, M, K, Kd, N, kind, density):
+    """SPMM and FusedMM on the balanced partition (granules of all row tiles dealt evenly to the CTAs, a slab per segment,
+    the slab-sum kernel behind; FusedMM reloads its A tile between segments) against the oracle, for bfloat16 operands
+    too, on an output whose rows are padded and held NaNs; twice, bit-equal; and the plain partition the same way."""
+    p = W.small_random(4300 + M, M, K, density, Kd, N, kind=kind)
     d = DevProblem(p)
-    ref, T = oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D)
-    D16 = d.D.to(torch.bfloat16)
-    ref16, T16 = oracle.spmm(p.row_ptr, p.col_idx, p.values, D16.float().cpu().numpy())
-    outs = {}
+    A16, B16, D16 = (t.to(torch.bfloat16) for t in (d.A, d.B, d.D))
+    h = lambda t: t.float().cpu().numpy()
+    calls = {
+        "spmm": (oracle.spmm(p.row_ptr, p.col_idx, p.values, p.D), oracle.spmm(p.row_ptr, p.col_idx, p.values, h(D16)),
+                 lambda o, ws, algo: b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=o, workspace=ws, algo=algo),
+                 lambda o, ws, algo: b.spmm(d.row_ptr, d.col_idx, d.values, D16, K=p.K, out=o, workspace=ws, algo=algo, dtype=torch.bfloat16),
+                 b.OP_SPMM),
+        "fusedmm": (oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D),
+                    oracle.fusedmm(p.row_ptr, p.col_idx, p.values, h(A16), h(B16), h(D16)),
+                    lambda o, ws, algo: b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=o, workspace=ws, algo=algo),
+                    lambda o, ws, algo: b.fusedmm(d.row_ptr, d.col_idx, d.values, A16, B16, D16, out=o, workspace=ws, algo=algo, dtype=torch.bfloat16),
+                    b.OP_FUSEDMM),
+    }
     for part in (2, 1):
         b.debug_force_partition(part)
         try:
-            ws = _ws(b, b.OP_SPMM, p)
+            ws = _ws(b, b.OP_FUSEDMM, p)
             b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
-            for pad in (4, 3):
-                padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
-                out = padded[:, :p.N]
-                b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=out, workspace=ws, algo=PREPARED)
-                assert b.last_algo(b.OP_SPMM) == TILE and b.device_status(ws) == 0
-                gate(out, ref, T, f"spmm partition {part}, rows padded by {pad}")
-                assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
-            again = torch.full((p.M, p.N), float("nan"), device="cuda")
-            b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=again, workspace=ws, algo=TILE)
-            assert torch.equal(again, out.contiguous()), f"two runs differ (partition {part})"
-            outs[part] = again
-            o16 = torch.full((p.M, p.N), float("nan"), device="cuda")
-            b.spmm(d.row_ptr, d.col_idx, d.values, D16, K=p.K, out=o16, workspace=ws, algo=TILE, dtype=torch.bfloat16)
-            assert b.device_status(ws) == 0
-            gate(o16, ref16, T16, f"spmm bf16 partition {part}")
+            for name, ((ref, T), (ref16, T16), call, call16, op) in calls.items():
+                for pad in (4, 3):
+                    padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
+                    out = padded[:, :p.N]
+                    call(out, ws, PREPARED)
+                    assert b.last_algo(op) == TILE and b.device_status(ws) == 0
+                    gate(out, ref, T, f"{name} partition {part}, rows padded by {pad}")
+                    assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
+                again = torch.full((p.M, p.N), float("nan"), device="cuda")
+                call(again, ws, TILE)
+                assert torch.equal(again, out.contiguous()), f"{name}: two runs differ (partition {part})"
+                o16 = torch.full((p.M, p.N), float("nan"), device="cuda")
+                call16(o16, ws, TILE)
+                assert b.device_status(ws) == 0
+                gate(o16, ref16, T16, f"{name} bf16 partition {part}")
         finally:
             b.debug_force_partition(0)
     assert d.pattern_untouched()
