@@ -116,7 +116,7 @@ int pick_split(int base_tiles, int blocks)
 // of `nt` column tiles: groups of nt CTAs, the 4-block flush granules of all row tiles dealt evenly to the groups,
 // one CTA per SM.  Returns the number of CTAs (0: the plain partition, tiles x K splits, stays) and the slabs a tile
 // needs (= the most groups that share a row tile).
-int pick_balanced(long long units, int nt, int blocks, int ks, int *slabs)
+int pick_balanced(long long units, int nt, int blocks, int ks, bool spmm, int *slabs)
 {
     const int forced = g_forced_partition.load(std::memory_order_relaxed);   // b2sp_debug_force_partition
     if (forced == 1 || blocks % kFusedFlushBlocks != 0 || nt > kSMs) return 0;
@@ -133,7 +133,7 @@ int pick_balanced(long long units, int nt, int blocks, int ks, int *slabs)
         // x 256 (one K split) -4% / -1%; 32768 x 8192 x 128 (one K split, two waves) -3% / -5%.  At 2/3 (24576 x 8192,
         // 192 tiles): -27% / -26%.  At equal length it loses 6-14%.
         const long long plain = (units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks);
-        if (gmax * kFusedFlushBlocks * 100 > plain * (ks > 1 ? 94 : 88)) return 0;
+        if (gmax * kFusedFlushBlocks * 100 > plain * (ks == 1 ? 88 : spmm ? 94 : 90)) return 0;
     }
     int most = 1;
     const Balance balance((int)gtot, (int)groups);
@@ -232,7 +232,7 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
     if (fused && batch == 1) {   // (FusedMM and SPMM on one problem)
         int slabs = 0;
-        p.bal_ctas = pick_balanced(p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, &slabs);
+        p.bal_ctas = pick_balanced(p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, Kd == 0, &slabs);
         if (p.bal_ctas) p.KS = slabs;
     }
     size_t off = align_up(base_off, 1024);

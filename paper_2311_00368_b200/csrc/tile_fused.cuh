@@ -302,8 +302,8 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     const int mtiles = tiles_pp / a.Nt;                            // row tiles per problem
     const Balance balance(bal ? a.batch * mtiles * gpt : 1, bal ? a.bal_ctas / a.Nt : 1);
     const int g0 = bal ? balance.start(grp) : 0, g1 = bal ? balance.start(grp + 1) : 0;
-    const int b0 = bal ? 0 : (int)((long long)nblk_all * ks / a.KS);
-    const int nblk = bal ? (g1 - g0) * kFusedFlushBlocks : (int)((long long)nblk_all * (ks + 1) / a.KS) - b0;
+    const int b0 = bal ? 0 : nblk_all * ks / a.KS;   // (32-bit: at most 6 k blocks, 32 splits)
+    const int nblk = bal ? (g1 - g0) * kFusedFlushBlocks : nblk_all * (ks + 1) / a.KS - b0;
     if (bal && threadIdx.x == 0) {
         int n = 0;
         for (int g = g0; g < g1 && n < kFusedMaxSegs; ++n) {
