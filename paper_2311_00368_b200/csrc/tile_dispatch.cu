@@ -230,9 +230,9 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     size_t win_bytes = sizeof(int2) * (size_t)batch * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
-    if (fused && batch == 1) {   // (FusedMM and SPMM on one problem)
+    if (fused && (long long)batch * nnz < 0x7fffffffll) {   // (FusedMM and SPMM; positions in a batch's stacked values are ints)
         int slabs = 0;
-        p.bal_ctas = pick_balanced(p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, Kd == 0, &slabs);
+        p.bal_ctas = pick_balanced((long long)batch * p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, Kd == 0, &slabs);
         if (p.bal_ctas) p.KS = slabs;
     }
     size_t off = align_up(base_off, 1024);
@@ -299,16 +299,6 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
-        if (exact) {
-            if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-            if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-            return launch_fused_tile<128, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-        }
-        if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-    }
     if constexpr (MODE != kModeSddmm) {
         if (a.bal_ctas > 0) {
             if (exact) {
@@ -320,6 +310,16 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
             if (kdp == 64) return launch_fused_tile<64, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
             return launch_fused_tile<128, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
         }
+    }
+    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
+        if (exact) {
+            if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
+            if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
+            return launch_fused_tile<128, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
+        }
+        if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
     }
     if (exact) {
         if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);

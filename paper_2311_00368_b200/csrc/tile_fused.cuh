@@ -813,18 +813,24 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
         const int2 *win = a.win + (size_t)prob * a.M * a.Wk;               // window table
         float *out_values = a.out + prob * a.stride_O;                     // and (SDDMM) output values
         // (balanced partition: the tile and the first window of the segment that holds the items load_rec is asked
-        // for, which come in increasing order; single problem, so `win` and `s_values` are the problem's)
-        int seg_m0 = m0, seg_w0 = wbase, seg_end = bal ? 0 : nitems;
+        // for, which come in increasing order; in a batch also the problem's window table and the offset of its stored
+        // values, which goes into the records' positions)
+        int seg_m0 = m0, seg_w0 = wbase, seg_end = bal ? 0 : nitems, seg_pos0 = 0;
         auto load_rec = [&](int jj) {   // lane = row: window record of one row of item jj
             int2 r = make_int2(0, 0);
             if (bal && jj >= seg_end && jj < nitems) {   // the item is in a later segment than the one before: read its record
                 const uint32_t sg = seg_at(jj / (IPW * WPB));
                 seg_m0 = seg_f(sg, kSegM0);
                 seg_w0 = (seg_f(sg, kSegBt0) - seg_f(sg, kSegStart)) * WPB;
+                if (a.batch > 1) {   // the segment's problem: its window table, and where its stored values begin
+                    win = a.win + (size_t)seg_f(sg, kSegProb) * a.M * a.Wk;
+                    seg_pos0 = seg_f(sg, kSegProb) * (int)a.stride_sv;
+                }
                 seg_end = sg + 32 < segtab + 32 * (uint32_t)ptx::lds32(segtab - 8) ? seg_f(sg + 32, kSegStart) * (IPW * WPB) : nitems;
             }
             const int hrow = seg_m0 + (jj % IPW) * IR + lane, wglob = seg_w0 + jj / IPW;
             if (jj < nitems && lane < IR && hrow < a.M && wglob < a.Wk) r = __ldg(win + (size_t)hrow * a.Wk + wglob);
+            if (bal) r.x += seg_pos0;
             return r;
         };
         // the records of the next two items are in flight while an item is processed

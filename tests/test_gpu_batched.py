@@ -111,6 +111,43 @@ def test_batch_with_several_k_splits(b, ks):
         b.debug_force_k_splits(0)
 
 
+@pytest.mark.parametrize("nb,M,K,Kd,N", [
+    (3, 300, 1024, 48, 100),     # three row tiles of two granules per problem
+    (5, 4100, 1024, 64, 64),     # 33 row tiles per problem: 330 granules on 148 CTAs, segments run from one problem into the next
+    (2, 1500, 2048, 128, 200),   # two column tiles: groups of two CTAs
+])
+def test_batch_on_the_balanced_partition(b, nb, M, K, Kd, N):
+    """The granules of all problems' row tiles dealt evenly to the CTAs: a segment names its problem (window table,
+    stored values, operand rows, slab, output).  Against the oracle, NULL values and a shared pattern too, twice
+    bit-equal, and the plain partition the same way."""
+    probs = [W.small_random(5600 + 7 * i + M, M, K, d, Kd, N) for i, d in zip(range(nb), (0.06, 0.03, 0.1, 0.05, 0.08))]
+    s = Stacked(probs)
+    refs_null = [oracle.fusedmm(p.row_ptr, p.col_idx, None, p.A, p.B, p.D) for p in probs]
+    for part in (2, 1):
+        b.debug_force_partition(part)
+        try:
+            ws = s.workspace(b)
+            padded = torch.full((s.nb, s.M + 3, s.N + 12), float("nan"), device="cuda")
+            out = padded[:, :s.M, :s.N]
+            run(b, s, TILE, ws, TILE, f"partition {part}", out=out)
+            s.check(out, f"batched, partition {part}")
+            assert torch.isnan(padded[:, s.M:, :]).all() and torch.isnan(padded[:, :, s.N:]).all(), "padding written"
+            b.prepare_pattern_batched(s.row_ptr, s.col_idx, K, ws)
+            again = run(b, s, PREPARED, ws, TILE, f"partition {part}, prepared")
+            assert torch.equal(again, out.contiguous()), "two runs differ"
+            s.check(run(b, s, TILE, ws, TILE, "NULL values", values=False), f"batched, partition {part}, NULL values", refs_null)
+            # one pattern for all problems (stride 0), operands per problem
+            p0 = probs[0]
+            t = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+            shared = [oracle.fusedmm(p0.row_ptr, p0.col_idx, p0.values, p.A, p.B, p.D) for p in probs]
+            o2 = torch.full((s.nb, s.M, s.N), float("nan"), device="cuda")
+            b.fusedmm_batched(t(p0.row_ptr), t(p0.col_idx), t(p0.values), s.A, s.B, s.D, out=o2, workspace=ws, algo=TILE)
+            assert b.last_algo(b.OP_FUSEDMM) == TILE and b.device_status(ws) == 0
+            s.check(o2, f"batched, partition {part}, shared pattern", shared)
+        finally:
+            b.debug_force_partition(0)
+
+
 def test_shared_pattern_and_shared_operands(b):
     """Stride 0: one pattern (1-D CSR arrays) and one D for all problems, A and B per problem."""
     p0 = W.small_random(5200, 260, 640, 0.2, 64, 128)
