@@ -113,27 +113,29 @@ int pick_split(int base_tiles, int blocks)
 }
 
 // The balanced partition (see tile_fused.cuh) of `units` row tiles of `blocks` 128-column blocks each, for an output
-// of `nt` column tiles: groups of nt CTAs, the 4-block flush granules of all row tiles dealt evenly to the groups,
-// one CTA per SM.  Returns the number of CTAs (0: the plain partition, tiles x K splits, stays) and the slabs a tile
-// needs (= the most groups that share a row tile).
-int pick_balanced(long long units, int nt, int blocks, int ks, bool spmm, int *slabs)
+// of `nt` column tiles: groups of nt CTAs, the granules of all row tiles (4-block flush granules; single blocks for
+// SDDMM) dealt evenly to the groups, one CTA per SM.  Returns the number of CTAs (0: the plain partition, tiles x K
+// splits, stays) and the slabs a tile needs (= the most groups that share a row tile).
+int pick_balanced(long long units, int nt, int blocks, int ks, int mode, int *slabs)
 {
     const int forced = g_forced_partition.load(std::memory_order_relaxed);   // b2sp_debug_force_partition
-    if (forced == 1 || blocks % kFusedFlushBlocks != 0 || nt > kSMs) return 0;
-    const long long gpt = blocks / kFusedFlushBlocks, gtot = units * gpt;
+    const int gran = mode == kModeSddmm ? 1 : kFusedFlushBlocks;            // SDDMM accumulates nothing across blocks
+    if (forced == 1 || blocks % gran != 0 || nt > kSMs) return 0;
+    const long long gpt = blocks / gran, gtot = units * gpt;
     if (gtot >= 0x7fffffffll / kSMs) return 0;   // (the partition's arithmetic is 32-bit)
     const long long groups = gtot < kSMs / nt ? gtot : kSMs / nt;
     const long long gmax = (gtot + groups - 1) / groups;
     if ((gmax + gpt - 2) / gpt + 1 > kFusedMaxSegs) return 0;   // a CTA would touch too many row tiles
     if (forced != 2) {
         // Worth it when the longest CTA gets clearly shorter than in the plain partition (whose CTAs come in waves).
-        // Measured: the time falls by about 0.6 of what the lengths promise (more CTAs at work slow each other down,
-        // and the balanced FusedMM kernel is a few percent slower per block), and slabs where the plain partition writes
-        // straight into O (one K split) cost a few percent.  At 7/8 of the length: 8192^2 x 128 SPMM -7%, FusedMM -3%;
-        // x 256 (one K split) -4% / -1%; 32768 x 8192 x 128 (one K split, two waves) -3% / -5%.  At 2/3 (24576 x 8192,
-        // 192 tiles): -27% / -26%.  At equal length it loses 6-14%.
-        const long long plain = (units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks);
-        if (gmax * kFusedFlushBlocks * 100 > plain * (ks == 1 ? 88 : spmm ? 94 : 90)) return 0;
+        // A CTA that goes on into the next row tile reloads its A tile (FusedMM, SDDMM: about a block and a half of
+        // time).  Measured: the time falls by about 0.6 of what the lengths promise (more CTAs at work slow each other
+        // down), and slabs where the plain partition writes straight into O (one K split) cost a few percent.  At 7/8 of
+        // the length: 8192^2 x 128 SPMM -7%, FusedMM -3%, SDDMM -3%; x 256 (one K split) SPMM -4%, FusedMM -1%; 4096^2
+        // SDDMM (8 -> 7 blocks per CTA) +3%.  At 2/3 (24576 x 8192, 192 row tiles): -27% / -26% / -27%.
+        const long long plain2 = 2 * ((units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks));
+        const long long mine2 = 2 * gmax * gran + (mode == kModeSpmm ? 0 : 3);
+        if (mine2 * 100 > plain2 * (mode == kModeSddmm || ks > 1 ? 94 : 90)) return 0;
     }
     int most = 1;
     const Balance balance((int)gtot, (int)groups);
@@ -230,10 +232,10 @@ FusedPlan plan_fused_tile(int M, int K, int Kd, int N, long long nnz, size_t bas
     size_t win_bytes = sizeof(int2) * (size_t)batch * (size_t)M * (size_t)p.Wk;
     if (win_bytes > (size_t)2 << 30 || p.Wk > kMasksMaxWk) return p;
     p.KS = pick_split(batch * p.Mt * p.Nt, p.Kp / kFusedBlk);
-    if (fused && (long long)batch * nnz < 0x7fffffffll) {   // (FusedMM and SPMM; positions in a batch's stacked values are ints)
+    if ((long long)batch * nnz < 0x7fffffffll) {   // (positions in a batch's stacked values are ints)
         int slabs = 0;
-        p.bal_ctas = pick_balanced((long long)batch * p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, Kd == 0, &slabs);
-        if (p.bal_ctas) p.KS = slabs;
+        p.bal_ctas = pick_balanced((long long)batch * p.Mt, p.Nt, p.Kp / kFusedBlk, p.KS, !fused ? kModeSddmm : Kd == 0 ? kModeSpmm : kModeFused, &slabs);
+        if (p.bal_ctas) p.KS = fused ? slabs : 1;   // (SDDMM has no partial outputs)
     }
     size_t off = align_up(base_off, 1024);
     p.off_win = off;
@@ -299,7 +301,7 @@ b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const C
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    if constexpr (MODE != kModeSddmm) {
+    {
         if (a.bal_ctas > 0) {
             if (exact) {
                 if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);

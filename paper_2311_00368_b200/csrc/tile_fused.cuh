@@ -55,11 +55,13 @@ constexpr int kFusedNT = 128;       // most O columns per CTA (UMMA N of GEMM2);
 constexpr int kFusedFlushBlocks = 4;
 constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 // The balanced partition (FusedTileArgs::bal_ctas): the CTAs form groups of Nt (one CTA per column tile of O), and
-// the 4-block flush granules of all row tiles, in the order (problem, row tile, granule), are dealt evenly to the
-// groups -- group c of n gets granules [c * G / n, (c + 1) * G / n) of G -- so a CTA may finish one output tile and go
-// on with the next row tile's: at most kFusedMaxSegs segments, each with a slab of its own (the tile's first, second,
-// ... segment writes slab 0, 1, ...).  The CTAs of a group work on the same blocks of S at the same time, so S is
-// fetched from memory once per group.
+// the granules of all row tiles -- the 4-block flush granules of FusedMM / SPMM, single blocks for SDDMM -- in the order
+// (problem, row tile, granule) are dealt evenly to the groups: group c of n gets granules [c * G / n, (c + 1) * G / n)
+// of G.  So a CTA may finish one output tile and go on with the next row tile's: at most kFusedMaxSegs segments, each
+// (FusedMM / SPMM) with a slab of its own (the tile's first, second, ... segment writes slab 0, 1, ...); between
+// segments FusedMM and SDDMM reload their A tile.  The CTAs of a group work on the same blocks of S at the same time,
+// so S is fetched from memory once per group.
+// (struct Balance, in slab_sum.cuh, holds the arithmetic.)
 constexpr int kFusedMaxSegs = 4;
 // (struct Balance, in slab_sum.cuh, holds the arithmetic.)
 
@@ -148,7 +150,8 @@ struct FusedCfg {
     // SPMM has tensor memory to spare: two O accumulators, so that the tensor core works on the next
     // chunk of blocks while the previous partial sum is flushed.
     static constexpr int NOB = SPMM ? 2 : 1;
-    static constexpr bool BALANCED = FUSED;   // the mode knows the balanced partition (FusedMM, SPMM)
+    // the balanced partition deals granules of this many blocks: the flush granules of FusedMM / SPMM, single blocks for SDDMM
+    static constexpr int GRAN = FUSED ? kFusedFlushBlocks : 1;
     static constexpr uint32_t COL_O = 0, COL_P = FUSED ? 128 : 0, COL_PP = 256;
     static constexpr uint32_t COL_AHI = FUSED ? 384 : 256, COL_ALO = 384;
 };
@@ -281,7 +284,6 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr bool BATCHED = PART == kPartBatched, bal = PART == kPartBalanced;
-    static_assert(!bal || Cfg::BALANCED, "this mode does not know the balanced partition");
     const int prob = BATCHED ? blockIdx.x / a.ctas_per_problem : 0;            // problem of the batch
     const int cta = BATCHED ? blockIdx.x % a.ctas_per_problem : blockIdx.x;
     const int ks = cta % a.KS;
@@ -297,23 +299,24 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
     // first block within the tile's row of blocks, slab, problem, -, -); their number at segtab - 8
     const uint32_t segtab = aux + 896;
     constexpr uint32_t kSegStart = 0, kSegM0 = 4, kSegNt = 8, kSegBt0 = 12, kSegOrd = 16, kSegProb = 20;
-    const int gpt = nblk_all / kFusedFlushBlocks;
+    constexpr int GRAN = Cfg::GRAN;
+    const int gpt = nblk_all / GRAN;
     const int grp = (int)blockIdx.x / a.Nt;                        // (CTA blockIdx.x: group grp, column tile blockIdx.x % Nt)
     const int mtiles = tiles_pp / a.Nt;                            // row tiles per problem
     const Balance balance(bal ? a.batch * mtiles * gpt : 1, bal ? a.bal_ctas / a.Nt : 1);
     const int g0 = bal ? balance.start(grp) : 0, g1 = bal ? balance.start(grp + 1) : 0;
     const int b0 = bal ? 0 : nblk_all * ks / a.KS;   // (32-bit: at most 6 k blocks, 32 splits)
-    const int nblk = bal ? (g1 - g0) * kFusedFlushBlocks : nblk_all * (ks + 1) / a.KS - b0;
+    const int nblk = bal ? (g1 - g0) * GRAN : nblk_all * (ks + 1) / a.KS - b0;
     if (bal && threadIdx.x == 0) {
         int n = 0;
         for (int g = g0; g < g1 && n < kFusedMaxSegs; ++n) {
             const int unit = g / gpt;                    // problem * row tiles + row tile
             const int gfirst = unit * gpt;
             const uint32_t rec = segtab + n * 32;
-            ptx::sts32(rec + kSegStart, (uint32_t)((g - g0) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegStart, (uint32_t)((g - g0) * GRAN));
             ptx::sts32(rec + kSegM0, (uint32_t)(unit % mtiles * kFusedRows));
             ptx::sts32(rec + kSegNt, (uint32_t)((int)blockIdx.x % a.Nt));
-            ptx::sts32(rec + kSegBt0, (uint32_t)((g - gfirst) * kFusedFlushBlocks));
+            ptx::sts32(rec + kSegBt0, (uint32_t)((g - gfirst) * GRAN));
             ptx::sts32(rec + kSegOrd, (uint32_t)(grp - balance.group_of(gfirst)));
             ptx::sts32(rec + kSegProb, (uint32_t)(unit / mtiles));
             g = gfirst + gpt < g1 ? gfirst + gpt : g1;

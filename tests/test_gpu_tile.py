@@ -321,9 +321,10 @@ def _k_split_epilogues(b, ks, width):
     (9000, 1536, 128, 128, "band", 0.05),      # 71 row tiles of three granules
 ])
 def test_balanced_partition_matches_plain(b, M, K, Kd, N, kind, density):
-    """SPMM and FusedMM on the balanced partition (granules of all row tiles dealt evenly to the CTAs, a slab per segment,
-    the slab-sum kernel behind; FusedMM reloads its A tile between segments) against the oracle, for bfloat16 operands
-    too, on an output whose rows are padded and held NaNs; twice, bit-equal; and the plain partition the same way."""
+    """SPMM, SDDMM and FusedMM on the balanced partition (granules of all row tiles dealt evenly to the CTAs; SPMM and
+    FusedMM: a slab per segment, the slab-sum kernel behind; FusedMM and SDDMM reload their A tile between segments)
+    against the oracle, for bfloat16 operands too, on an output whose rows are padded and held NaNs; twice, bit-equal; and
+    the plain partition the same way."""
     p = W.small_random(4300 + M, M, K, density, Kd, N, kind=kind)
     d = DevProblem(p)
     A16, B16, D16 = (t.to(torch.bfloat16) for t in (d.A, d.B, d.D))
@@ -333,6 +334,10 @@ def test_balanced_partition_matches_plain(b, M, K, Kd, N, kind, density):
                  lambda o, ws, algo: b.spmm(d.row_ptr, d.col_idx, d.values, d.D, K=p.K, out=o, workspace=ws, algo=algo),
                  lambda o, ws, algo: b.spmm(d.row_ptr, d.col_idx, d.values, D16, K=p.K, out=o, workspace=ws, algo=algo, dtype=torch.bfloat16),
                  b.OP_SPMM),
+        "sddmm": (oracle.sddmm(p.row_ptr, p.col_idx, p.values, p.A, p.B), oracle.sddmm(p.row_ptr, p.col_idx, p.values, h(A16), h(B16)),
+                  lambda o, ws, algo: b.sddmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, out=o, workspace=ws, algo=algo),
+                  lambda o, ws, algo: b.sddmm(d.row_ptr, d.col_idx, d.values, A16, B16, out=o, workspace=ws, algo=algo, dtype=torch.bfloat16),
+                  b.OP_SDDMM),
         "fusedmm": (oracle.fusedmm(p.row_ptr, p.col_idx, p.values, p.A, p.B, p.D),
                     oracle.fusedmm(p.row_ptr, p.col_idx, p.values, h(A16), h(B16), h(D16)),
                     lambda o, ws, algo: b.fusedmm(d.row_ptr, d.col_idx, d.values, d.A, d.B, d.D, out=o, workspace=ws, algo=algo),
@@ -345,17 +350,22 @@ def test_balanced_partition_matches_plain(b, M, K, Kd, N, kind, density):
             ws = _ws(b, b.OP_FUSEDMM, p)
             b.prepare_pattern(d.row_ptr, d.col_idx, p.K, ws)
             for name, ((ref, T), (ref16, T16), call, call16, op) in calls.items():
+                shape = (p.nnz,) if name == "sddmm" else (p.M, p.N)
                 for pad in (4, 3):
-                    padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
-                    out = padded[:, :p.N]
+                    if name == "sddmm":
+                        out = torch.full(shape, float("nan"), device="cuda")
+                    else:
+                        padded = torch.full((p.M, p.N + pad), float("nan"), device="cuda")
+                        out = padded[:, :p.N]
                     call(out, ws, PREPARED)
                     assert b.last_algo(op) == TILE and b.device_status(ws) == 0
                     gate(out, ref, T, f"{name} partition {part}, rows padded by {pad}")
-                    assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
-                again = torch.full((p.M, p.N), float("nan"), device="cuda")
+                    if name != "sddmm":
+                        assert torch.isnan(padded[:, p.N:]).all(), "the padding of the output rows was written"
+                again = torch.full(shape, float("nan"), device="cuda")
                 call(again, ws, TILE)
                 assert torch.equal(again, out.contiguous()), f"{name}: two runs differ (partition {part})"
-                o16 = torch.full((p.M, p.N), float("nan"), device="cuda")
+                o16 = torch.full(shape, float("nan"), device="cuda")
                 call16(o16, ws, TILE)
                 assert b.device_status(ws) == 0
                 gate(o16, ref16, T16, f"{name} bf16 partition {part}")
