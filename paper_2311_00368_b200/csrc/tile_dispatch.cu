@@ -135,7 +135,10 @@ int pick_balanced(long long units, int nt, int blocks, int ks, int mode, int *sl
         // SDDMM (8 -> 7 blocks per CTA) +3%.  At 2/3 (24576 x 8192, 192 row tiles): -27% / -26% / -27%.
         const long long plain2 = 2 * ((units * nt * ks + kSMs - 1) / kSMs * ((blocks + ks - 1) / ks));
         const long long mine2 = 2 * gmax * gran + (mode == kModeSpmm ? 0 : 3);
-        if (mine2 * 100 > plain2 * (mode == kModeSddmm || ks > 1 ? 94 : 90)) return 0;
+        // (SPMM on one column tile: slabs where there were none cost more than 1/8 of the length buys -- 16384 x 4096 x 128,
+        // cache-warm: +4%)
+        const int percent = mode == kModeSddmm || ks > 1 ? 94 : mode == kModeSpmm && nt == 1 ? 86 : 90;
+        if (mine2 * 100 > plain2 * percent) return 0;
     }
     int most = 1;
     const Balance balance((int)gtot, (int)groups);
@@ -199,7 +202,8 @@ bool tile_profitable(int op, int M, int K, int width, long long nnz)
     // (sub-warps share a row): measured at width 32 on 1k^2 ... 32k x 8k, the cross-over is about 3.5x
     // higher for SPMM, 2x for SDDMM, 2.5x for FusedMM.  With 74 or more row tiles (no K split) the last
     // wave of CTAs is partly empty (96 tiles: 65% of the SMs; 192 tiles: two waves, 65%), which the tile
-    // family pays in full: the cross-over rises by the waves' efficiency against the usual 86%.
+    // family pays in full unless the balanced partition applies: the cross-over rises by the waves' efficiency
+    // against the usual 86%.
     if (M < 256 || K < 256 || width < 16 || nnz <= 0) return false;
     const double cells = (double)M * (double)K;
     const double density = (double)nnz / cells;
@@ -209,7 +213,12 @@ bool tile_profitable(int op, int M, int K, int width, long long nnz)
     const int tiles = (M + kFusedRows - 1) / kFusedRows;
     if (tiles >= kSMs / 2 && width <= kFusedNT) {
         const int waves = (tiles + kSMs - 1) / kSMs;
-        const double eff = (double)tiles / ((double)waves * kSMs);
+        double eff = (double)tiles / ((double)waves * kSMs);
+        // (the balanced partition, where the planner takes it, wins back about 0.6 of what the waves lose)
+        int slabs = 0;
+        const int blocks = (K + kFusedBlk - 1) / kFusedBlk;
+        if (pick_balanced(tiles, 1, blocks, pick_split(tiles, blocks), op == B2SP_OP_SDDMM ? kModeSddmm : op == B2SP_OP_SPMM ? kModeSpmm : kModeFused, &slabs))
+            eff += 0.6 * (1.0 - eff);
         const double factor = 0.86 / eff;
         crossover *= factor < 1.0 ? 1.0 : factor > 1.35 ? 1.35 : factor;
     }
