@@ -732,6 +732,17 @@ def main():
     probe_gflops = b.probe_fp32_peak(4096, device)
     roof["fp32_fma_probe"] = {"tflops": probe_gflops / 1e3, "achieved_over_probe": fl[dom] / dom_ms / 1e6 / probe_gflops,
                               "how": "b2sp_probe_fp32_peak: 8 FMA chains x 2048 threads x every SM, CUDA events, best of 10"}
+    # second resource of the dense-tile kernels: the B / D operand tiles every CTA streams from L2 into shared memory
+    # (tf32 hi + lo, 8 bytes per element, once per 128-row tile and 128-column block of S), against the rate at which
+    # the SMs can pull 32 KB chunks out of L2 right now
+    if algos[dom] == "tile":
+        per_sm, total = b.probe_l2_pull(device)
+        row_tiles, blocks = -(-p.M // 128), -(-p.K // 128)
+        widths = {"spmm": p.N, "sddmm": p.Kd, "fusedmm": p.Kd + p.N}[dom]
+        stream_bytes = row_tiles * blocks * 128 * (-(-widths // 32) * 32) * 8
+        roof["l2_operand_stream"] = {"bytes_per_launch": stream_bytes, "gbs": stream_bytes / dom_ms / 1e6,
+                                     "probe_gbs": total, "probe_gbs_per_sm": per_sm, "frac_of_probe": stream_bytes / dom_ms / 1e6 / total,
+                                     "how": "b2sp_probe_l2_pull: cp.async.bulk of 32 KB chunks, three in flight per SM, every SM, best of 5"}
     roof["traffic"] = MEASURED_TRAFFIC_BYTES.get((args.workload, algos[dom]))
     roof["traffic_source"] = ("one ncu capture of this kernel on this workload (dram__bytes_read.sum + dram__bytes_write.sum, "
                               "summary under profiles/), not measured in this run" if roof["traffic"] else None)

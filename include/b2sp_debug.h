@@ -23,6 +23,18 @@ extern "C" {
 b2sp_status b2sp_probe_fp32_peak(int iters, float *scratch, double *gflops_host, void *stream);
 
 /*
+ * The rate at which the SMs of the current device pull 32 KB operand chunks out of L2 into shared memory with bulk
+ * asynchronous copies (`cp.async.bulk`, three in flight per SM, one CTA per SM, all SMs at once; best of 5 launches
+ * timed with CUDA events), in GB/s per SM and for the whole GPU.  The dense-tile kernels stream their B / D operand
+ * tiles this way; the numbers say how much of that path they use.
+ * `scratch` = DEVICE buffer of `scratch_bytes` >= 1 MiB + 16 bytes, 16-byte aligned; its first 16 bytes are
+ * overwritten, up to 16 MiB of the rest are read (any contents).  `gbs_per_sm_host`, `gbs_total_host` = HOST pointers
+ * for the results.  Synchronises `stream`.  B2SP_ERR_INVALID_ARG, B2SP_ERR_CUDA; B2SP_ERR_TIMEOUT if a copy did not
+ * land within the kernel's bounded wait.
+ */
+b2sp_status b2sp_probe_l2_pull(void *scratch, size_t scratch_bytes, double *gbs_per_sm_host, double *gbs_total_host, void *stream);
+
+/*
  * Which kernel family the most recent call of the given op (B2SP_OP_*) on this host thread resolved
  * B2SP_ALGO_AUTO (or its explicit request) to: one of B2SP_ALGO_ROW, _ROW_NAT, _TILE; -1 if the
  * op has not been called.  Number of kernels that call enqueued: b2sp_last_launches(op).

@@ -74,6 +74,8 @@ lib.b2sp_validate_csr.restype = _i
 lib.b2sp_validate_csr.argtypes = [_i, _i, _ll, _vp, _vp, _vp, _sz, _vp]
 lib.b2sp_probe_fp32_peak.restype = _i
 lib.b2sp_probe_fp32_peak.argtypes = [_i, _vp, ctypes.POINTER(ctypes.c_double), _vp]
+lib.b2sp_probe_l2_pull.restype = _i
+lib.b2sp_probe_l2_pull.argtypes = [_vp, ctypes.c_size_t, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double), _vp]
 lib.b2sp_device_status.restype = _i
 lib.b2sp_device_status.argtypes = [_vp, _vp]
 lib.b2sp_last_algo.restype = _i
@@ -152,6 +154,15 @@ def probe_fp32_peak(iters: int = 4096, device=None) -> float:
     out = ctypes.c_double(0.0)
     _check(lib.b2sp_probe_fp32_peak(iters, _ptr(scratch), ctypes.byref(out), _stream()), "b2sp_probe_fp32_peak")
     return float(out.value)
+
+
+def probe_l2_pull(device=None):
+    """b2sp_probe_l2_pull: (GB/s per SM, GB/s of the whole GPU) of 32 KB bulk copies from L2 into shared memory (synchronises)."""
+    scratch = torch.zeros((17 << 20) + 64, dtype=torch.uint8, device=device or "cuda")
+    per_sm, total = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib.b2sp_probe_l2_pull(_ptr(scratch), scratch.numel(), ctypes.byref(per_sm), ctypes.byref(total), _stream()),
+           "b2sp_probe_l2_pull")
+    return float(per_sm.value), float(total.value)
 
 
 def last_algo(op: int) -> int:

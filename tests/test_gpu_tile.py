@@ -538,3 +538,13 @@ def test_a_wait_that_runs_out_is_reported_and_the_gpu_stays_usable(b):
     fused_tile_check(b, p)
     ref, T = oracle.spmm(big.row_ptr, big.col_idx, big.values, big.D)
     gate(b.spmm_host(t(big.row_ptr), t(big.col_idx), t(big.values), t(big.D), hO), ref, T, "spmm_host after the hook")
+
+
+def test_l2_pull_probe(b):
+    """The measurement aid behind bench.py's `roofline.l2_operand_stream`: a plausible rate, and the argument checks."""
+    per_sm, total = b.probe_l2_pull()
+    assert 20.0 < per_sm < 500.0 and 50.0 * per_sm < total < 400.0 * per_sm
+    import ctypes
+    small = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    x, y = ctypes.c_double(), ctypes.c_double()
+    assert b.lib.b2sp_probe_l2_pull(small.data_ptr(), small.numel(), ctypes.byref(x), ctypes.byref(y), None) == 1
