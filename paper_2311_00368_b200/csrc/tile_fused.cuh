@@ -374,7 +374,7 @@ fused_tile_kernel(const __grid_constant__ CUtensorMap tm_bhi, const __grid_const
 
     // Everything above (barriers, tensor memory, the A tile: none of it written by the kernel before) ran
     // while the operand-split kernel, whose programmatic dependent this grid is, was still at work.  Its tf32
-    // copies and its verdict on a prepared table are needed from here on.  After it the flags are final (the
+    // copies and its check of a prepared table are needed from here on.  After it the flags are final (the
     // pre-pass or that kernel's signature check wrote them), so the gated row kernel launched behind this
     // grid may run beside it.
     ptx::wait_for_primary_grid();
