@@ -53,6 +53,7 @@ __global__ void __launch_bounds__(128, 1) l2_pull_kernel(const char *src, size_t
         const size_t nchunks = bytes / kPullChunk;
         size_t pos = (size_t)blockIdx.x * 977 % nchunks;
         bool gave_up = false;
+        int drain = kPullDepth - 1;   // after a wait has run out: this many more waits, for the copies still in flight
         for (int it = 0; it < iters + kPullDepth; ++it) {
             const int s = it % kPullDepth;
             if (it >= kPullDepth) {
@@ -63,7 +64,11 @@ __global__ void __launch_bounds__(128, 1) l2_pull_kernel(const char *src, size_t
                                  : "=r"(done) : "r"(shared_addr(&bar[s])), "r"(parity) : "memory");
                 if (!done) gave_up = true;
             }
-            if (it < iters && !gave_up) {
+            if (gave_up) {
+                if (drain-- <= 0) break;
+                continue;
+            }
+            if (it < iters) {
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(shared_addr(&bar[s])), "r"(kPullChunk) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                              ::"r"(shared_addr(buf + (size_t)s * kPullChunk)), "l"(src + pos * kPullChunk), "r"(kPullChunk),
