@@ -87,3 +87,42 @@ def test_random_shapes_every_entry_point(seed):
     rng = np.random.default_rng(seed)
     for _ in range(25):
         _one_case(b, rng)
+
+
+def test_random_large_shapes_on_the_balanced_partition():
+    """Seeded shapes with tens to hundreds of row tiles, the dense-tile planner pinned to the balanced partition (several
+    segments per CTA, groups of CTAs for wide outputs, A tiles reloaded between segments; where the number of blocks is
+    not a multiple of four, FusedMM and SPMM keep the plain partition and SDDMM deals single blocks): the three ops on a
+    prepared table against the oracle, every element."""
+    assert torch.cuda.is_available()
+    from paper_2311_00368_b200 import binding as b
+    dev = lambda x: torch.from_numpy(np.ascontiguousarray(x)).cuda()
+    rng = np.random.default_rng(7)
+    b.debug_force_partition(2)
+    try:
+        for _ in range(6):
+            M, K = int(rng.integers(2000, 40000)), int(rng.choice([512, 640, 1024, 1536, 2048, 2500, 4096]))
+            Kd, N = int(rng.choice([32, 64, 100, 128])), int(rng.choice([32, 64, 128, 200, 256]))
+            dens, kind = float(rng.choice([0.02, 0.04, 0.06])), str(rng.choice(["uniform", "powerlaw"]))
+            p = W.small_random(int(rng.integers(1 << 30)), M, K, dens, Kd, N, kind=kind)
+            use_bf, null = bool(rng.integers(0, 2)), bool(rng.random() < 0.25)
+            what = f"M={M} K={K} Kd={Kd} N={N} d={dens} {kind} bf16={use_bf} null={null}"
+            A, B, D, dt, cvt = p.A, p.B, p.D, torch.float32, dev
+            if use_bf:
+                A, B, D = (torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).float().numpy() for x in (A, B, D))
+                dt, cvt = torch.bfloat16, (lambda x: dev(x).to(torch.bfloat16))
+            rp, ci, v, dA, dB, dD = dev(p.row_ptr), dev(p.col_idx), dev(p.values), cvt(A), cvt(B), cvt(D)
+            ws = torch.empty(max(max(b.workspace_bytes(o, M, K, Kd, N, p.nnz) for o in range(3)), 1 << 20), dtype=torch.uint8, device="cuda")
+            b.prepare_pattern(rp, ci, K, ws)
+            sv, hv = (None, None) if null else (v, p.values)
+            got = {"spmm": b.spmm(rp, ci, v, dD, K=K, workspace=ws, algo=4, dtype=dt),
+                   "sddmm": b.sddmm(rp, ci, sv, dA, dB, workspace=ws, algo=4, dtype=dt),
+                   "fusedmm": b.fusedmm(rp, ci, sv, dA, dB, dD, workspace=ws, algo=4, dtype=dt)}
+            assert b.device_status(ws) == 0, what
+            ref = {"spmm": oracle.spmm(p.row_ptr, p.col_idx, p.values, D), "sddmm": oracle.sddmm(p.row_ptr, p.col_idx, hv, A, B),
+                   "fusedmm": oracle.fusedmm(p.row_ptr, p.col_idx, hv, A, B, D)}
+            for op, out in got.items():
+                ok, ratio = oracle.within_tolerance(out.cpu().numpy(), *ref[op])
+                assert ok, f"{op}: {what}: worst error / allowed = {ratio:.3g}"
+    finally:
+        b.debug_force_partition(0)
