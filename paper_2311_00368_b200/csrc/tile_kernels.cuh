@@ -223,14 +223,24 @@ __device__ __forceinline__ bool split_job(const SplitJob &j)
                      (reinterpret_cast<uintptr_t>(j.X) & (bf16 ? 7 : 15)) == 0;
     const long long rows_all = (long long)j.batch * j.rows_p;
     const long long groups = rows_all * (j.cols_p >> 2);  // float4 groups
+    const bool small = groups < 0x7fffffffll;
     bool bad = false;
     for (long long g = (long long)blockIdx.x * blockDim.x + threadIdx.x; g < groups;
          g += (long long)gridDim.x * blockDim.x) {
         const int q = (int)(g & 7);                 // float4 inside the 32-float group
         const long long rg = g >> 3;                // (column group, stacked row) pair
-        const long long rs = rg % rows_all;
-        const int b = (int)(rs / j.rows_p), r = (int)(rs % j.rows_p);
-        const int c = (int)(rg / rows_all) * 32 + q * 4;
+        int b, r, c;
+        if (small) {   // 32-bit index arithmetic (64-bit divisions are library calls: they were most of this kernel's time)
+            const unsigned rg32 = (unsigned)rg, cg = rg32 / (unsigned)rows_all, rs = rg32 - cg * (unsigned)rows_all;
+            b = j.batch == 1 ? 0 : (int)(rs / (unsigned)j.rows_p);
+            r = (int)(rs - (unsigned)b * (unsigned)j.rows_p);
+            c = (int)cg * 32 + q * 4;
+        } else {
+            const long long rs = rg % rows_all;
+            b = (int)(rs / j.rows_p);
+            r = (int)(rs % j.rows_p);
+            c = (int)(rg / rows_all) * 32 + q * 4;
+        }
         uint32_t h[4] = {0, 0, 0, 0}, l[4] = {0, 0, 0, 0};
         if (r < j.rows && c < j.cols) {
             const long long at = (long long)b * j.batch_stride + (long long)r * j.ld + c;
