@@ -51,18 +51,33 @@ __global__ void __launch_bounds__(256) slab_sum_kernel(const SlabSumArgs a)
     const bool skip = (*reinterpret_cast<const volatile int *>(a.flags) | *reinterpret_cast<const volatile int *>(a.flags + 1)) != 0;
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (skip) return;
-    asm volatile("griddepcontrol.wait;" ::: "memory");                // the tile kernel has completed: the slabs are whole
+    bool waited = false;   // (a thread works out where its first element is before it waits for the tile kernel)
     const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x, nthreads = (long long)gridDim.x * blockDim.x;
     const int n4 = (a.N + 3) >> 2;
     const long long total = (long long)a.batch * a.M * n4;
     const bool vec_out = (a.ldo & 3) == 0 && (a.stride_O & 3) == 0 && (reinterpret_cast<uintptr_t>(a.O) & 15) == 0;
+    const bool small = total < 0x7fffffffll;   // 32-bit index arithmetic (64-bit divisions are library calls)
+    const Balance balance(a.bal_ctas ? a.batch * a.Mt * a.gpt : 1, a.bal_ctas ? a.bal_ctas / a.Nt : 1);
     for (long long e = tid; e < total; e += nthreads) {
-        const int n = (int)(e % n4) * 4;
-        const long long pr = e / n4;
-        const int r = (int)(pr % a.M), p = (int)(pr / a.M);
+        int n, r, p;
+        if (small) {
+            const unsigned e32 = (unsigned)e, pr = e32 / (unsigned)n4;
+            n = (int)(e32 - pr * (unsigned)n4) * 4;
+            p = a.batch == 1 ? 0 : (int)(pr / (unsigned)a.M);
+            r = (int)(pr - (unsigned)p * (unsigned)a.M);
+        } else {
+            n = (int)(e % n4) * 4;
+            const long long pr = e / n4;
+            r = (int)(pr % a.M);
+            p = (int)(pr / a.M);
+        }
         int cnt = a.KS;
-        if (a.bal_ctas) cnt = Balance(a.batch * a.Mt * a.gpt, a.bal_ctas / a.Nt).groups_of_tile((p * a.Mt + r / kSlabTileRows) * a.gpt, a.gpt);
+        if (a.bal_ctas) cnt = balance.groups_of_tile((p * a.Mt + r / kSlabTileRows) * a.gpt, a.gpt);
         const float *src = a.slabs + (long long)p * a.KS * a.slab + (long long)r * a.ld + n;
+        if (!waited) {
+            asm volatile("griddepcontrol.wait;" ::: "memory");   // the tile kernel has completed: the slabs are whole
+            waited = true;
+        }
         // (the first four slabs' loads in flight together)
         float4 v[4];
 #pragma unroll
