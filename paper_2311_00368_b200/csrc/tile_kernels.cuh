@@ -69,7 +69,7 @@ tile_masks_kernel(int M, int K, int Wk, long long nnz, const int *__restrict__ r
     bool bad = false;
     const long long rows_all = (long long)M * sig.batch;
     for (long long rowg = blockIdx.x; rowg < rows_all; rowg += gridDim.x) {
-        const int pb = (int)(rowg / M), row = (int)(rowg % M);
+        const int pb = sig.batch == 1 ? 0 : (int)(rowg / M), row = (int)(rowg - (long long)pb * M);   // (no 64-bit division for a single pattern)
         const int *__restrict__ row_ptr = row_ptr0 + pb * sig.rp_stride;
         const int *__restrict__ col_idx = col_idx0 + pb * sig.nz_stride;
         const bool vec = (reinterpret_cast<uintptr_t>(col_idx) & 15) == 0;
