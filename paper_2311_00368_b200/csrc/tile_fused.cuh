@@ -2,7 +2,8 @@
 // one kernel, three modes.
 //
 // One CTA owns 128 rows of S (= rows of A and O), a range of 128-column blocks of S (4 windows of 32
-// columns each) and, for FusedMM / SPMM, one 128-column tile of O.
+// columns each) and, for FusedMM / SPMM, one 128-column tile of O -- or, on the balanced partition (see
+// kFusedMaxSegs), a run of blocks that may go on from one row tile into the next ones.
 //   * A_tile (128 x Kd) is split into tf32 hi/lo once: A_hi lives in tensor memory for the CTA's
 //     life; A_lo lives in tensor memory too (SDDMM) or in shared memory (FusedMM, where TMEM is
 //     needed for O and P').
@@ -63,13 +64,12 @@ constexpr int kFusedChunk = 32768;  // bytes of one pipeline chunk (hi + lo)
 // so S is fetched from memory once per group.
 // (struct Balance, in slab_sum.cuh, holds the arithmetic.)
 constexpr int kFusedMaxSegs = 4;
-// (struct Balance, in slab_sum.cuh, holds the arithmetic.)
 
 struct FusedTileArgs {
     int M, K, Kd, Kdp, N, Wk, KS, Nt;
     // A batch of `batch` independent problems of the same sizes in one launch: CTA blockIdx.x works on problem
-    // blockIdx.x / ctas_per_problem.  Window tables, tf32 operand copies (rows b*Kp ...), slabs and arrival
-    // counters of the problems are stacked; the caller's arrays are `stride_*` elements apart.
+    // blockIdx.x / ctas_per_problem.  Window tables, tf32 operand copies (rows b*Kp ...) and slabs of the problems
+    // are stacked; the caller's arrays are `stride_*` elements apart.
     int batch, ctas_per_problem, Kp;
     long long stride_sv, stride_A, stride_O;
     int NT;                   // O columns per CTA (UMMA N of GEMM2): 128, or 64 when N <= 64
