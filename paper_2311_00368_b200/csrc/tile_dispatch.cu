@@ -305,41 +305,36 @@ b2sp_status launch_fused_tile(const CUtensorMap &bh, const CUtensorMap &bl, cons
     return cudaGetLastError() == cudaSuccess ? B2SP_OK : B2SP_ERR_CUDA;
 }
 
+// Picks the instantiation: PART from the plan, EXACT from the operand type, KDP from the padded Kd (SPMM has no A / B:
+// only its KDP = 32 instantiation exists).
+template <int MODE, int PART, bool EXACT>
+b2sp_status launch_fused_part(int kdp, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh, const CUtensorMap &dl,
+                              const CUtensorMap &out, const FusedTileArgs &a, int items, cudaStream_t st)
+{
+    if constexpr (MODE == kModeSpmm) {
+        return launch_fused_tile<32, MODE, PART, EXACT>(bh, bl, dh, dl, out, a, items, st);
+    } else {
+        if (kdp == 32) return launch_fused_tile<32, MODE, PART, EXACT>(bh, bl, dh, dl, out, a, items, st);
+        if (kdp == 64) return launch_fused_tile<64, MODE, PART, EXACT>(bh, bl, dh, dl, out, a, items, st);
+        return launch_fused_tile<128, MODE, PART, EXACT>(bh, bl, dh, dl, out, a, items, st);
+    }
+}
+
 template <int MODE>
 b2sp_status launch_fused_kdp(int kdp, bool exact, const CUtensorMap &bh, const CUtensorMap &bl, const CUtensorMap &dh,
                              const CUtensorMap &dl, const CUtensorMap &out, const FusedTileArgs &a, int items,
                              cudaStream_t st)
 {
-    {
-        if (a.bal_ctas > 0) {
-            if (exact) {
-                if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
-                if (kdp == 64) return launch_fused_tile<64, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
-                return launch_fused_tile<128, MODE, kPartBalanced, true>(bh, bl, dh, dl, out, a, items, st);
-            }
-            if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
-            if (kdp == 64) return launch_fused_tile<64, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
-            return launch_fused_tile<128, MODE, kPartBalanced, false>(bh, bl, dh, dl, out, a, items, st);
-        }
+    if (a.bal_ctas > 0)
+        return exact ? launch_fused_part<MODE, kPartBalanced, true>(kdp, bh, bl, dh, dl, out, a, items, st)
+                     : launch_fused_part<MODE, kPartBalanced, false>(kdp, bh, bl, dh, dl, out, a, items, st);
+    if constexpr (MODE == kModeFused) {   // (only FusedMM is offered on batches)
+        if (a.batch > 1)
+            return exact ? launch_fused_part<MODE, kPartBatched, true>(kdp, bh, bl, dh, dl, out, a, items, st)
+                         : launch_fused_part<MODE, kPartBatched, false>(kdp, bh, bl, dh, dl, out, a, items, st);
     }
-    if (MODE == kModeFused && a.batch > 1) {   // (only FusedMM is offered on batches)
-        if (exact) {
-            if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-            if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-            return launch_fused_tile<128, kModeFused, kPartBatched, true>(bh, bl, dh, dl, out, a, items, st);
-        }
-        if (kdp == 32) return launch_fused_tile<32, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, kModeFused, kPartBatched, false>(bh, bl, dh, dl, out, a, items, st);
-    }
-    if (exact) {
-        if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
-        if (kdp == 64) return launch_fused_tile<64, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
-        return launch_fused_tile<128, MODE, kPartTiles, true>(bh, bl, dh, dl, out, a, items, st);
-    }
-    if (MODE == kModeSpmm || kdp == 32) return launch_fused_tile<32, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
-    if (kdp == 64) return launch_fused_tile<64, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
-    return launch_fused_tile<128, MODE, kPartTiles, false>(bh, bl, dh, dl, out, a, items, st);
+    return exact ? launch_fused_part<MODE, kPartTiles, true>(kdp, bh, bl, dh, dl, out, a, items, st)
+                 : launch_fused_part<MODE, kPartTiles, false>(kdp, bh, bl, dh, dl, out, a, items, st);
 }
 
 // Splits (or only checks) up to three dense operands and clears the device status word.
