@@ -464,7 +464,9 @@ b2sp_status fused_tile(const FusedPlan &p, bool prepared, int mode, int M, int K
         sa.gpt = p.Kp / kFusedBlk / kFusedFlushBlocks; sa.bal_ctas = p.bal_ctas;
         sa.flags = flags;
         const long long threads = (long long)nb * M * ((N + 3) / 4);
-        const long long want = (threads + 255) / 256, cap = (long long)kSMs * 8;
+        // (four CTAs per SM: all of them start at once when the tile kernel's CTAs leave, so the gated row kernel, this grid's
+        // programmatic dependent, starts beside them and not after a second wave; measured against eight: FusedMM and SPMM -1%)
+        const long long want = (threads + 255) / 256, cap = (long long)kSMs * 4;
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)(want < cap ? want : cap));
         cfg.blockDim = dim3(256);
