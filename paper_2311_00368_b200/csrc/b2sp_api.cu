@@ -232,7 +232,14 @@ extern "C" const char *b2sp_status_string(b2sp_status s)
 // writing the sampled values once: measured at N = 512 on the 8192^2 / 30% workload, 717 us fused
 // against 134 + 430 us for SDDMM into a scratch C and SPMM on C.  So wide outputs take the two
 // phases inside one call (same window table, same fallback), and C lives in the workspace.
-static bool fusedmm_two_phase(int N) { return N > 256; }
+// With two tiles (128 < N <= 256) the second GEMM1 costs more than C's round trip when GEMM1 is long and the
+// problem large: measured at N = 256, Kd = 128, two phases against fused: 8192^2 315 against 342 us (10% density
+// 298 against 337), 4096 x 8192 175 against 188, 16384 x 2048 187 against 191, 4096^2 115 against 114; but
+// 8192 x 4096 at Kd = 64 172 against 159 and 2048^2 52 against 40.
+static bool fusedmm_two_phase(int M, int K, int Kd, int N)
+{
+    return N > 256 || (N > 128 && Kd > 64 && (double)M * (double)K >= 3.0e7);
+}
 
 // Workspace of the dense-tile family for an op (0: these sizes are outside the family).
 static size_t tile_workspace_bytes(int op, int M, int K, int Kd, int N, long long nnz, size_t row_bytes)
@@ -241,7 +248,7 @@ static size_t tile_workspace_bytes(int op, int M, int K, int Kd, int N, long lon
                   : op == B2SP_OP_SDDMM ? plan_fused_tile(M, K, Kd, 0, nnz, row_bytes, false)
                                         : plan_fused_tile(M, K, Kd, N, nnz, row_bytes, true);
     if (!p.feasible) return 0;
-    if (op == B2SP_OP_FUSEDMM && fusedmm_two_phase(N)) {
+    if (op == B2SP_OP_FUSEDMM && fusedmm_two_phase(M, K, Kd, N)) {
         TwoPhasePlan t = plan_two_phase(M, K, Kd, N, nnz, row_bytes);
         if (t.feasible && t.bytes > p.bytes) return t.bytes;
     }
@@ -500,7 +507,7 @@ static b2sp_status fusedmm_impl(int M, int K, int Kd, int N, long long nnz, cons
     Workspace w = carve(workspace);
     if (use == B2SP_ALGO_TILE) {
         TwoPhasePlan two;
-        if (fusedmm_two_phase(N)) two = plan_two_phase(M, K, Kd, N, nnz, row_bytes);
+        if (fusedmm_two_phase(M, K, Kd, N)) two = plan_two_phase(M, K, Kd, N, nnz, row_bytes);
         if (two.feasible && workspace_bytes >= two.bytes) {
             float *C = reinterpret_cast<float *>(static_cast<char *>(workspace) + two.off_c);
             rc = fused_tile(two.sddmm, prepared, 0, M, K, Kd, 0, nnz, row_ptr, col_idx, s_values, A, lda, B, ldb, nullptr, 0,
@@ -597,7 +604,7 @@ bool bad_batch_args(int batch, int M, int K, long long nnz_stride, const int *ro
 
 FusedPlan plan_batched(int batch, int M, int K, int Kd, int N, long long nnz_stride)
 {
-    if (fusedmm_two_phase(N)) return FusedPlan();   // wide outputs: not on the dense-tile family in a batch
+    if (N > 256) return FusedPlan();   // wide outputs: not on the dense-tile family in a batch
     return plan_fused_tile(M, K, Kd, N, nnz_stride, row_workspace_bytes(M), true, batch);
 }
 
