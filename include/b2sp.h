@@ -148,10 +148,10 @@ b2sp_status b2sp_sddmm(int M, int K, int Kd, long long nnz,
 /*
  * FusedMM, Eq. 3 / Alg. 3 (FusedMM-ROW):  O = (S .* (A * B^T)) * D, i.e. the SDDMM values of a
  * row are consumed by the SPMM sweep of the same row without being written to global memory.
- * (One exception, a measured trade: the dense-tile family with N > 256 would recompute the sampled
- * values once per 128-column tile of O, so it writes them once into the workspace and runs its SPMM
- * stage on them, inside the same call.)  s_values may be NULL (all ones).  Arguments as in the two
- * ops above.
+ * (One exception, a measured trade: the dense-tile family recomputes the sampled values once per
+ * 128-column tile of O, so with N > 256 -- and with 128 < N <= 256 when Kd > 64 and S has at least
+ * 3e7 cells -- it writes them once into the workspace and runs its SPMM stage on them, inside the same
+ * call.)  s_values may be NULL (all ones).  Arguments as in the two ops above.
  */
 b2sp_status b2sp_fusedmm(int M, int K, int Kd, int N, long long nnz,
                          const int *row_ptr, const int *col_idx, const float *s_values,
